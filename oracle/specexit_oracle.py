@@ -1,0 +1,592 @@
+"""CPU oracle for the speculative-exit step.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, step-by-step restatement of what one iteration of signal-guided
+speculative decoding computes (Algorithm 1 of the paper, the body of its loop without
+the target trunk): the draft pass run autoregressively, the extended head of Eq. 1
+(token logits plus the confidence / progress / remaining rows), the activations of
+Eq. 3-5, greedy verification against the target head, and the smoothed, thresholded
+exit decision (Section 3.3, Appendix A.1).  Only the tests, the smoke check and the
+benchmark's CPU-baseline leg may use it; the product never does, and it shares no code
+with the CUDA path.
+
+Arithmetic.  Every contraction and every elementwise step is evaluated in float64 with
+library matmuls as single steps, so a result does not depend on summation order.  Values
+are then rounded to the storage type the method fixes: activations handed from one layer
+to the next are bf16 (via fp32, round-to-nearest-even) at exactly these points -
+x, n1, q, k, v (q and k after the rotation), o, a, n2, m, y, g - and logits, signal
+values, log-probabilities, scores and the smoothed state are fp32.  An argmax is taken on
+the fp32 logits; ties go to the lower index.
+
+Parity status.  The paper prints no numeric example of the draft forward, so that part is
+"parity unpinned" by the paper itself; tests pin it against closed forms, textbook special
+cases, brute force and an independent float64 restatement instead.  The smoothing rule, the
+activations, the threshold logic and the acceptance rule are pinned by hand-worked values
+and invariants (see tests/).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+F64 = torch.float64
+
+# signal activations (Eq. 3-5): sigmoid for confidence/progress; the remaining-length row
+# regresses log(1 + r), so r = exp(z) - 1
+ACT_SIGMOID, ACT_EXPM1, ACT_IDENTITY = 0, 1, 2
+DIR_GT, DIR_LT = 0, 1
+EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
+
+EXEMPT_REL_GAP = 1e-3
+
+
+def bf16r(x: torch.Tensor) -> torch.Tensor:
+    """Round to bf16 the way a kernel holding an fp32 value would; result kept as f64."""
+    return x.to(torch.float32).to(torch.bfloat16).to(F64)
+
+
+def f32r(x: torch.Tensor) -> torch.Tensor:
+    return x.to(torch.float32).to(F64)
+
+
+def linear(x: torch.Tensor, W: torch.Tensor, chunk: int = 8192) -> torch.Tensor:
+    """``x @ W^T`` in float64.  ``x`` is ``[R, K]`` f64, ``W`` is ``[N, K]`` (bf16 storage).
+    ``W`` is widened a slab of rows at a time only to bound memory."""
+    R, N = x.shape[0], W.shape[0]
+    out = torch.empty(R, N, dtype=F64)
+    for n0 in range(0, N, chunk):
+        n1 = min(N, n0 + chunk)
+        out[:, n0:n1] = x @ W[n0:n1].to(F64).t()
+    return out
+
+
+def rmsnorm(x: torch.Tensor, gamma: torch.Tensor, eps: float) -> torch.Tensor:
+    """Root-mean-square normalisation over the last axis, then the gain."""
+    ms = (x * x).mean(dim=-1, keepdim=True)
+    return x * torch.rsqrt(ms + eps) * gamma.to(F64)
+
+
+def rope(x: torch.Tensor, pos: int, theta: float) -> torch.Tensor:
+    """Rotary embedding, rotate-half pairing (i, i + d/2), absolute position ``pos``.
+    ``x`` is ``[heads, d]``."""
+    d = x.shape[-1]
+    half = d // 2
+    i = torch.arange(half, dtype=F64)
+    ang = float(pos) * torch.pow(torch.tensor(theta, dtype=F64), -2.0 * i / d)
+    c, s = torch.cos(ang), torch.sin(ang)
+    x1, x2 = x[..., :half], x[..., half:]
+    return torch.cat([x1 * c - x2 * s, x2 * c + x1 * s], dim=-1)
+
+
+def silu(x: torch.Tensor) -> torch.Tensor:
+    return x / (1.0 + torch.exp(-x))
+
+
+def activate(z: torch.Tensor, act: Sequence[int]) -> torch.Tensor:
+    """Eq. 3-5: map the raw signal rows ``z [..., S]`` to signal values."""
+    out = torch.empty_like(z)
+    for i, a in enumerate(act):
+        zi = z[..., i]
+        if a == ACT_SIGMOID:
+            out[..., i] = 1.0 / (1.0 + torch.exp(-zi))
+        elif a == ACT_EXPM1:
+            out[..., i] = torch.expm1(zi)
+        else:
+            out[..., i] = zi
+    return out
+
+
+def argmax_low(v: torch.Tensor) -> int:
+    """Index of the maximum; the lowest index among equals."""
+    m = v.max()
+    return int(torch.nonzero(v == m)[0, 0])
+
+
+def top_gap(v: torch.Tensor, k: int = 1) -> float:
+    """(k-th largest - (k+1)-th largest) / |largest| on fp32 logits: the deciding margin."""
+    t = torch.topk(v, k + 1).values
+    den = abs(float(t[0]))
+    return float(t[k - 1] - t[k]) / den if den > 0 else 0.0
+
+
+def topk_low(v: torch.Tensor, k: int) -> List[int]:
+    """The k largest entries, larger value first, lower index first among equals."""
+    order = sorted(range(v.numel()), key=lambda i: (-float(v[i]), i)) if v.numel() <= 4096 else None
+    if order is not None:
+        return order[:k]
+    # large vocabularies: take a candidate pool, then order it exactly
+    pool = torch.topk(v, min(v.numel(), k + 32)).indices.tolist()
+    kth = sorted((float(v[i]) for i in pool), reverse=True)[k - 1]
+    pool = torch.nonzero(v >= kth).flatten().tolist()
+    pool.sort(key=lambda i: (-float(v[i]), i))
+    return pool[:k]
+
+
+# --------------------------------------------------------------------------------------
+# paged KV cache
+# --------------------------------------------------------------------------------------
+class PagedKV:
+    """Private copy of a paged bf16 KV cache ``[num_pages, n_kv, page, d]``."""
+
+    def __init__(self, k_pages, v_pages, page_table, cache_len):
+        self.k = k_pages.clone()
+        self.v = v_pages.clone()
+        self.table = page_table.clone()
+        self.len = [int(n) for n in cache_len]
+        self.page = int(k_pages.shape[2])
+        self._prefix: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = {}
+
+    def _loc(self, b: int, slot: int) -> Tuple[int, int]:
+        lp, off = divmod(slot, self.page)
+        if lp >= self.table.shape[1] or int(self.table[b, lp]) < 0:
+            raise IndexError(f"slot {slot} of sequence {b} is beyond its page table")
+        return int(self.table[b, lp]), off
+
+    def write(self, b: int, slot: int, k: torch.Tensor, v: torch.Tensor) -> None:
+        pp, off = self._loc(b, slot)
+        self.k[pp, :, off, :] = k.to(torch.bfloat16)
+        self.v[pp, :, off, :] = v.to(torch.bfloat16)
+
+    def read(self, b: int, slot: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        pp, off = self._loc(b, slot)
+        return self.k[pp, :, off, :].to(F64), self.v[pp, :, off, :].to(F64)
+
+    def prefix(self, b: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        """K, V of slots [0, len[b]) as ``[n_kv, len, d]`` f64 (kept: the prefix is fixed
+        for the whole iteration)."""
+        if b not in self._prefix:
+            n = self.len[b]
+            npg = (n + self.page - 1) // self.page
+            pages = self.table[b, :npg].to(torch.int64)
+            kk = self.k[pages].permute(1, 0, 2, 3).reshape(self.k.shape[1], npg * self.page, -1)
+            vv = self.v[pages].permute(1, 0, 2, 3).reshape(self.v.shape[1], npg * self.page, -1)
+            self._prefix[b] = (kk[:, :n].to(F64), vv[:, :n].to(F64))
+        return self._prefix[b]
+
+
+# --------------------------------------------------------------------------------------
+# the draft model: concat(feature, embedding) -> fc -> one pre-norm decoder layer -> norm
+# -> extended head (Eq. 1)
+# --------------------------------------------------------------------------------------
+@dataclass
+class Row:
+    b: int                 # sequence
+    feat: torch.Tensor     # [H] f64 holding bf16 values: hidden of the previous position
+    tok: int               # token at this position
+    pos: int               # absolute rotary position
+    slot: int              # cache slot its K/V are written to
+    visible: List[int]     # slots beyond the cached prefix it may attend to (incl. its own)
+
+
+@dataclass
+class HeadOut:
+    logits: torch.Tensor   # [R, V] fp32 values in f64
+    z: torch.Tensor        # [R, S] raw signal rows, fp32 values
+    s: torch.Tensor        # [R, S] activated signals, fp32 values
+
+
+class DraftModel:
+    def __init__(self, shape, weights: Dict[str, torch.Tensor], act=(ACT_SIGMOID,) * 3,
+                 target_head: Optional[torch.Tensor] = None):
+        self.sh = shape
+        self.w = weights
+        self.act = tuple(act)
+        # the target's LM head; by default the draft's vocabulary rows
+        self.target_head = target_head if target_head is not None else weights["head"][:shape.V]
+
+    # Eq. 1: one matrix, vocabulary rows first, signal rows last, same hidden state
+    def head(self, g: torch.Tensor) -> HeadOut:
+        V, S = self.sh.V, self.sh.S
+        full = f32r(linear(g, self.w["head"]))
+        z = full[:, V:V + S]
+        return HeadOut(logits=full[:, :V], z=z, s=f32r(activate(z, self.act)))
+
+    def attention(self, kv: PagedKV, row: Row, q: torch.Tensor) -> torch.Tensor:
+        """softmax(q K^T / sqrt(d)) V over the cached prefix and the visible new slots.
+        ``q`` is ``[n_q, d]``; returns ``[n_q, d]``."""
+        sh = self.sh
+        group = sh.n_q // sh.n_kv
+        Kp, Vp = kv.prefix(row.b)
+        extra = [kv.read(row.b, s) for s in row.visible]
+        if extra:
+            Ke = torch.stack([e[0] for e in extra], dim=1)   # [n_kv, E, d]
+            Ve = torch.stack([e[1] for e in extra], dim=1)
+            Kall, Vall = torch.cat([Kp, Ke], dim=1), torch.cat([Vp, Ve], dim=1)
+        else:
+            Kall, Vall = Kp, Vp
+        out = torch.empty(sh.n_q, sh.d, dtype=F64)
+        for h in range(sh.n_q):
+            kvh = h // group
+            sc = (Kall[kvh] @ q[h]) / math.sqrt(sh.d)
+            p = torch.softmax(sc, dim=0)
+            out[h] = p @ Vall[kvh]
+        return out
+
+    def round(self, kv: PagedKV, rows: List[Row]) -> Tuple[torch.Tensor, HeadOut]:
+        """One draft pass over ``rows``; appends their K/V to the cache.  Returns the
+        final-normed hidden ``g [R, H]`` (bf16 values) and the head outputs."""
+        sh, w = self.sh, self.w
+        R = len(rows)
+        toks = torch.tensor([r.tok for r in rows], dtype=torch.int64)
+        u = torch.cat([torch.stack([r.feat for r in rows]), w["embed"][toks].to(F64)], dim=1)
+        x = bf16r(linear(u, w["fc"]))
+        n1 = bf16r(rmsnorm(x, w["norm1"], sh.eps))
+        qkv = linear(n1, w["wqkv"])
+        nq, nk, d = sh.n_q, sh.n_kv, sh.d
+        o = torch.empty(R, nq * d, dtype=F64)
+        qs = []
+        for i, r in enumerate(rows):          # all rows' K/V land first: siblings never see
+            q = qkv[i, :nq * d].view(nq, d)   # each other unless listed in `visible`
+            k = qkv[i, nq * d:(nq + nk) * d].view(nk, d)
+            v = qkv[i, (nq + nk) * d:].view(nk, d)
+            qs.append(bf16r(rope(q, r.pos, sh.theta)))
+            kv.write(r.b, r.slot, bf16r(rope(k, r.pos, sh.theta)), bf16r(v))
+        for i, r in enumerate(rows):
+            o[i] = bf16r(self.attention(kv, r, qs[i])).reshape(-1)
+        a = bf16r(x + linear(o, w["wo"]))
+        n2 = bf16r(rmsnorm(a, w["norm2"], sh.eps))
+        gu = linear(n2, w["wgate_up"])
+        m = bf16r(silu(gu[:, :sh.F]) * gu[:, sh.F:])
+        y = bf16r(a + linear(m, w["wdown"]))
+        g = bf16r(rmsnorm(y, w["normf"], sh.eps))
+        return g, self.head(g)
+
+
+# --------------------------------------------------------------------------------------
+# chain drafting
+# --------------------------------------------------------------------------------------
+@dataclass
+class ChainDraft:
+    cand_tok: torch.Tensor      # [B, K+1] slot 0 = last accepted token, slot j = j-th draft token
+    hidden: torch.Tensor        # [B, K, H] g of round k (bf16 values, f64)
+    slot_signal: torch.Tensor   # [B, K+1, S]; slot j carries the signal computed from the
+    #                             position of slot j's token (round j+1); slot K: NaN
+    gap: torch.Tensor           # [B, K] relative top-2 gap at each draft argmax
+    z: torch.Tensor             # [B, K, S] raw signal rows per round
+
+
+def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, K: int,
+                forced: Optional[Dict[Tuple[int, int], int]] = None) -> ChainDraft:
+    """K autoregressive draft rounds per sequence.  ``forced[(b, k)]`` (k = 1..K) replaces
+    the k-th draft token of sequence b (used to replay a near-tie the other way)."""
+    B, H, S = f0.shape[0], model.sh.H, model.sh.S
+    cand = torch.zeros(B, K + 1, dtype=torch.int64)
+    cand[:, 0] = t0.to(torch.int64)
+    hidden = torch.empty(B, K, H, dtype=F64)
+    sig = torch.full((B, K + 1, S), float("nan"), dtype=F64)
+    zz = torch.empty(B, K, S, dtype=F64)
+    gap = torch.empty(B, K, dtype=F64)
+    feat = f0.to(F64)
+    for k in range(1, K + 1):
+        rows = [Row(b=b, feat=feat[b], tok=int(cand[b, k - 1]), pos=kv.len[b] + k - 1,
+                    slot=kv.len[b] + k - 1,
+                    visible=[kv.len[b] + j for j in range(k)]) for b in range(B)]
+        g, ho = model.round(kv, rows)
+        for b in range(B):
+            tok = argmax_low(ho.logits[b])
+            gap[b, k - 1] = top_gap(ho.logits[b])
+            if forced and (b, k) in forced:
+                tok = int(forced[(b, k)])
+            cand[b, k] = tok
+        hidden[:, k - 1] = g
+        sig[:, k - 1] = ho.s
+        zz[:, k - 1] = ho.z
+        feat = g
+    return ChainDraft(cand, hidden, sig, gap, zz)
+
+
+# --------------------------------------------------------------------------------------
+# tree drafting: top-k children per expanded node, `depth` levels, best `max_nodes` kept
+# --------------------------------------------------------------------------------------
+@dataclass
+class Cand:
+    cid: int          # generation order: depth 1 first, then by expanding row, then by rank
+    depth: int
+    parent: int       # candidate id of the parent, -1 for children of the root
+    tok: int
+    logp: float
+    score: float      # fp32 sum of log-probabilities along the path
+    src_row: int      # drafted row whose head produced it
+    row: int = -1     # drafted row that took it as input (-1: never expanded)
+
+
+@dataclass
+class TreeDraft:
+    cands: List[List[Cand]]         # per sequence, all candidates
+    cand_tok: torch.Tensor          # [B, P] slot 0 = root (last accepted token)
+    parent: torch.Tensor            # [B, P] parent slot, -1 for the root
+    depth: torch.Tensor             # [B, P]
+    slot_row: torch.Tensor          # [B, P] drafted row with this slot's token as input, else -1
+    slot_src_row: torch.Tensor      # [B, P] drafted row whose head produced the slot's token
+    hidden: torch.Tensor            # [B, rows, H]
+    slot_signal: torch.Tensor       # [B, P, S], NaN where the slot was never expanded
+    margins: Dict[Tuple, float] = field(default_factory=dict)  # deciding margin per decision
+    slot_cid: Optional[torch.Tensor] = None
+
+
+def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, depth: int,
+               topk: int, max_nodes: int, override: Optional[Dict[Tuple, List[int]]] = None
+               ) -> TreeDraft:
+    """Tree drafting.  Round 1 drafts the root; round r >= 2 expands the `topk` best
+    candidates of depth r-1 (score = sum of log-probabilities; ties: lower candidate id).
+    After the last round the `max_nodes` best candidates overall are kept and laid out in
+    candidate-id order behind the root.  ``override`` replaces single decisions by the
+    given choice: ``("topk", b, row) -> token ids``, ``("expand", b, depth) -> cand ids``,
+    ``("keep", b) -> cand ids``."""
+    sh = model.sh
+    B, H, S = f0.shape[0], sh.H, sh.S
+    ov = override or {}
+    n_rows = 1 + topk * (depth - 1)
+    P = 1 + max_nodes
+    hidden = torch.empty(B, n_rows, H, dtype=F64)
+    row_sig = torch.full((B, n_rows, S), float("nan"), dtype=F64)
+    cands: List[List[Cand]] = [[] for _ in range(B)]
+    margins: Dict[Tuple, float] = {}
+    row_vis: List[Dict[int, List[int]]] = [dict() for _ in range(B)]
+
+    def emit(b, row, par_cid, par_score, dep, logits):
+        ids = topk_low(logits, topk)
+        margins[("topk", b, row)] = top_gap(logits, topk) if topk < logits.numel() else 1.0
+        if ("topk", b, row) in ov:
+            ids = list(ov[("topk", b, row)])
+        lse = torch.logsumexp(logits, dim=0)
+        for t in ids:
+            lp = f32r(logits[t] - lse)
+            sc = f32r(torch.tensor(par_score, dtype=F64) + lp)
+            cands[b].append(Cand(cid=len(cands[b]), depth=dep, parent=par_cid, tok=int(t),
+                                 logp=float(lp), score=float(sc), src_row=row))
+
+    # round 1: the root row
+    rows = [Row(b=b, feat=f0[b].to(F64), tok=int(t0[b]), pos=kv.len[b], slot=kv.len[b],
+                visible=[kv.len[b]]) for b in range(B)]
+    for b in range(B):
+        row_vis[b][0] = [kv.len[b]]
+    g, ho = model.round(kv, rows)
+    for b in range(B):
+        hidden[b, 0] = g[b]
+        row_sig[b, 0] = ho.s[b]
+        emit(b, 0, -1, 0.0, 1, ho.logits[b])
+
+    for r in range(2, depth + 1):
+        rows, owner = [], []
+        for b in range(B):
+            level = [c for c in cands[b] if c.depth == r - 1]
+            level.sort(key=lambda c: (-c.score, c.cid))
+            if len(level) > topk:
+                den = abs(level[0].score)
+                margins[("expand", b, r - 1)] = (
+                    (level[topk - 1].score - level[topk].score) / den if den > 0 else 0.0)
+            chosen = level[:topk]
+            if ("expand", b, r - 1) in ov:
+                byid = {c.cid: c for c in cands[b]}
+                chosen = [byid[i] for i in ov[("expand", b, r - 1)]]
+            for j, c in enumerate(chosen):
+                rid = 1 + (r - 2) * topk + j
+                c.row = rid
+                vis = list(row_vis[b][c.src_row]) + [kv.len[b] + rid]
+                row_vis[b][rid] = vis
+                rows.append(Row(b=b, feat=hidden[b, c.src_row], tok=c.tok,
+                                pos=kv.len[b] + r - 1, slot=kv.len[b] + rid, visible=vis))
+                owner.append((b, rid, c))
+        g, ho = model.round(kv, rows)
+        for i, (b, rid, c) in enumerate(owner):
+            hidden[b, rid] = g[i]
+            row_sig[b, rid] = ho.s[i]
+            emit(b, rid, c.cid, c.score, r, ho.logits[i])
+
+    cand_tok = torch.zeros(B, P, dtype=torch.int64)
+    parent = torch.full((B, P), -1, dtype=torch.int64)
+    dep = torch.zeros(B, P, dtype=torch.int64)
+    slot_row = torch.full((B, P), -1, dtype=torch.int64)
+    slot_src = torch.full((B, P), -1, dtype=torch.int64)
+    slot_cid = torch.full((B, P), -1, dtype=torch.int64)
+    slot_sig = torch.full((B, P, S), float("nan"), dtype=F64)
+    for b in range(B):
+        ranked = sorted(cands[b], key=lambda c: (-c.score, c.cid))
+        if len(ranked) > max_nodes:
+            den = abs(ranked[0].score)
+            margins[("keep", b)] = ((ranked[max_nodes - 1].score - ranked[max_nodes].score) / den
+                                    if den > 0 else 0.0)
+        keep = sorted(c.cid for c in ranked[:max_nodes])
+        if ("keep", b) in ov:
+            keep = sorted(ov[("keep", b)])
+        slot_of = {-1: 0}
+        cand_tok[b, 0] = int(t0[b])
+        slot_row[b, 0] = 0
+        slot_sig[b, 0] = row_sig[b, 0]
+        for s, cid in enumerate(keep, start=1):
+            c = cands[b][cid]
+            slot_of[cid] = s
+            cand_tok[b, s] = c.tok
+            parent[b, s] = slot_of[c.parent]     # parents precede children in id order
+            dep[b, s] = c.depth
+            slot_row[b, s] = c.row
+            slot_src[b, s] = c.src_row
+            slot_cid[b, s] = cid
+            if c.row >= 0:
+                slot_sig[b, s] = row_sig[b, c.row]
+    return TreeDraft(cands, cand_tok, parent, dep, slot_row, slot_src, hidden, slot_sig, margins,
+                     slot_cid)
+
+
+# --------------------------------------------------------------------------------------
+# verification (Algorithm 1: accept tokens, accept length, recover token)
+# --------------------------------------------------------------------------------------
+@dataclass
+class VerifyOut:
+    target_tok: torch.Tensor   # [B, P]
+    accept_len: torch.Tensor   # [B]
+    path: List[List[int]]      # per sequence: accepted slots, starting with slot 0
+    recover_tok: torch.Tensor  # [B]
+    gap: torch.Tensor          # [B, P] relative top-2 gap of the target argmax
+
+
+def target_argmax(model: DraftModel, target_hidden: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    B, P, H = target_hidden.shape
+    logits = f32r(linear(target_hidden.reshape(B * P, H).to(F64), model.target_head))
+    tok = torch.tensor([argmax_low(logits[i]) for i in range(B * P)], dtype=torch.int64)
+    gap = torch.tensor([top_gap(logits[i]) for i in range(B * P)], dtype=F64)
+    return tok.view(B, P), gap.view(B, P)
+
+
+def accept_chain(cand_tok: Sequence[int], target_tok: Sequence[int]) -> Tuple[int, List[int], int]:
+    """Longest prefix of draft tokens that equal the target's greedy choice one slot
+    earlier; the recover token is the target's choice after the last accepted slot."""
+    K = len(cand_tok) - 1
+    L = 0
+    while L < K and int(cand_tok[L + 1]) == int(target_tok[L]):
+        L += 1
+    return L, list(range(L + 1)), int(target_tok[L])
+
+
+def accept_tree(cand_tok: Sequence[int], parent: Sequence[int], target_tok: Sequence[int]
+                ) -> Tuple[int, List[int], int]:
+    """Walk from the root to the child whose token is the target's greedy choice at the
+    current slot, until there is none."""
+    P = len(cand_tok)
+    cur, path = 0, [0]
+    while True:
+        nxt = [s for s in range(1, P) if int(parent[s]) == cur and int(cand_tok[s]) == int(target_tok[cur])]
+        if not nxt:
+            break
+        cur = nxt[0]
+        path.append(cur)
+    return len(path) - 1, path, int(target_tok[cur])
+
+
+def verify(model: DraftModel, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
+           parent: Optional[torch.Tensor] = None,
+           forced_target: Optional[Dict[Tuple[int, int], int]] = None) -> VerifyOut:
+    tt, gap = target_argmax(model, target_hidden)
+    if forced_target:
+        for (b, j), t in forced_target.items():
+            tt[b, j] = t
+    B = tt.shape[0]
+    L = torch.zeros(B, dtype=torch.int64)
+    rec = torch.zeros(B, dtype=torch.int64)
+    paths = []
+    for b in range(B):
+        if parent is None:
+            l, p, r = accept_chain(cand_tok[b].tolist(), tt[b].tolist())
+        else:
+            l, p, r = accept_tree(cand_tok[b].tolist(), parent[b].tolist(), tt[b].tolist())
+        L[b], rec[b] = l, r
+        paths.append(p)
+    return VerifyOut(tt, L, paths, rec, gap)
+
+
+# --------------------------------------------------------------------------------------
+# exit decision (Section 3.3; Appendix A.1: EWMA x_t = alpha s_t + (1 - alpha) x_{t-1})
+# --------------------------------------------------------------------------------------
+@dataclass
+class ExitCfg:
+    alpha: float = 0.3
+    thr: Tuple[float, float, float] = (0.9, 0.8, 100.0)
+    dir: Tuple[int, int, int] = (DIR_GT, DIR_GT, DIR_LT)
+    enable_mask: int = 0b001           # bit i: signal i takes part (AND over enabled ones)
+    ema_positions: int = EMA_VERIFIED_CONTEXT
+    split_bitmap: Optional[torch.Tensor] = None   # int32 words, bit t%32 of word t//32; None = all
+    stop_think_token: int = 0
+
+
+@dataclass
+class ExitState:
+    x: torch.Tensor          # [B, S] smoothed signals (fp32 values)
+    n_updates: torch.Tensor  # [B]
+    thinking: torch.Tensor   # [B] 1 while inside the reasoning phase
+
+    @staticmethod
+    def fresh(B: int, S: int = 3) -> "ExitState":
+        return ExitState(torch.zeros(B, S, dtype=F64), torch.zeros(B, dtype=torch.int64),
+                         torch.ones(B, dtype=torch.int64))
+
+    def clone(self) -> "ExitState":
+        return ExitState(self.x.clone(), self.n_updates.clone(), self.thinking.clone())
+
+
+def is_split(cfg: ExitCfg, tok: int) -> bool:
+    if cfg.split_bitmap is None:
+        return True
+    word = int(cfg.split_bitmap[tok // 32]) & 0xFFFFFFFF
+    return bool((word >> (tok % 32)) & 1)
+
+
+def thresholds_pass(cfg: ExitCfg, x: torch.Tensor) -> bool:
+    """AND over the enabled signals; 'greater than' / 'less than' are strict."""
+    x32 = x.to(torch.float32)
+    for i in range(x.numel()):
+        if not (cfg.enable_mask >> i) & 1:
+            continue
+        thr = torch.tensor(cfg.thr[i], dtype=torch.float32)
+        ok = bool(x32[i] > thr) if cfg.dir[i] == DIR_GT else bool(x32[i] < thr)
+        if not ok:
+            return False
+    return True
+
+
+def ewma(cfg: ExitCfg, x: torch.Tensor, n_updates: int, s: torch.Tensor) -> torch.Tensor:
+    """One smoothing step in fp32 storage; the first sample initialises the state."""
+    if n_updates == 0:
+        return f32r(s)
+    a = float(torch.tensor(cfg.alpha, dtype=torch.float32))   # alpha as the fp32 the kernel holds
+    return f32r(a * s + (1.0 - a) * x)
+
+
+@dataclass
+class ExitOut:
+    exit_flag: torch.Tensor       # [B]
+    accept_len: torch.Tensor      # [B] after truncation
+    recover_tok: torch.Tensor     # [B] after substitution
+    smoothed: torch.Tensor        # [B, S]
+
+
+def exit_update(cfg: ExitCfg, state: ExitState, slot_signal: torch.Tensor, cand_tok: torch.Tensor,
+                paths: List[List[int]], accept_len: torch.Tensor, recover_tok: torch.Tensor) -> ExitOut:
+    """Walk the accepted slots in path order.  Each slot that carries a signal updates the
+    smoothed state; the first slot whose token is a step-split token while the smoothed
+    signals pass the thresholds ends the reasoning phase: the accepted length is cut at
+    that slot and the recover token becomes the stop-think token.  ``state`` is updated
+    in place; a sequence that is no longer thinking is left untouched."""
+    B = len(paths)
+    ef = torch.zeros(B, dtype=torch.int64)
+    Lo = accept_len.clone().to(torch.int64)
+    ro = recover_tok.clone().to(torch.int64)
+    for b in range(B):
+        if int(state.thinking[b]) == 0:
+            continue
+        L = int(accept_len[b])
+        for idx in range(L + 1):
+            slot = paths[b][idx]
+            sig = slot_signal[b, slot]
+            if cfg.ema_positions == EMA_VERIFIED_CONTEXT or idx == 0:
+                if bool(torch.isnan(sig).any()):
+                    break                     # never drafted from this slot: nothing new to smooth
+                state.x[b] = ewma(cfg, state.x[b], int(state.n_updates[b]), sig)
+                state.n_updates[b] += 1
+            if is_split(cfg, int(cand_tok[b, slot])) and thresholds_pass(cfg, state.x[b]):
+                ef[b], Lo[b], ro[b] = 1, idx, cfg.stop_think_token
+                state.thinking[b] = 0
+                break
+    return ExitOut(ef, Lo, ro, state.x.clone())

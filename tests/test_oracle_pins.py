@@ -1,0 +1,634 @@
+"""Pins for the CPU oracle: hand-worked values, closed forms, textbook special cases,
+invariants and brute force.  None of these re-types the oracle's own formula: each expected
+value is derived independently (by hand, by a closed form, by enumeration, or by numpy)."""
+import itertools
+import math
+import os
+import random
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import specexit_oracle as orc
+from paper_2509_24248_b200 import synth
+from tests import harness
+
+F64 = torch.float64
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append(line.split())
+    return out
+
+
+# ---------------------------------------------------------------- EWMA (Appendix A.1)
+def test_ewma_hand_worked_values():
+    rows = [(float(a), float(s), float(x)) for a, s, x in _rows("ewma_worked.txt")]
+    # first block: alpha 0.3, first sample initialises
+    cfg = orc.ExitCfg(alpha=0.3)
+    x, n = torch.zeros(1, dtype=F64), 0
+    for a, s, want in rows[:3]:
+        x = orc.ewma(cfg, x, n, torch.tensor([s], dtype=F64))
+        n += 1
+        assert abs(float(x) - want) < 1e-6
+    # second block: the paper's alpha 0.1, state seeded with 0.5 (n_updates > 0)
+    cfg = orc.ExitCfg(alpha=0.1)
+    x, n = torch.tensor([0.5], dtype=F64), 1
+    for a, s, want in rows[3:]:
+        x = orc.ewma(cfg, x, n, torch.tensor([s], dtype=F64))
+        n += 1
+        assert abs(float(x) - want) < 1e-6
+
+
+@pytest.mark.parametrize("alpha", [0.1, 0.3, 0.75])
+def test_ewma_closed_form_constant_signal(alpha):
+    cfg = orc.ExitCfg(alpha=alpha)
+    c, x0 = 0.8, 0.1
+    x = torch.tensor([x0], dtype=F64)
+    for n in range(1, 30):
+        x = orc.ewma(cfg, x, n, torch.tensor([c], dtype=F64))
+        assert abs(float(x) - (c + (1 - alpha) ** n * (x0 - c))) < 1e-5
+    # first-sample initialisation keeps a constant signal constant
+    x = orc.ewma(cfg, torch.zeros(1, dtype=F64), 0, torch.tensor([c], dtype=F64))
+    assert abs(float(x) - c) < 1e-7
+
+
+# ---------------------------------------------------------------- activations (Eq. 3-5)
+def test_activations():
+    z = torch.tensor([[0.0, math.log(3.0), math.log(101.0)]], dtype=F64)
+    s = orc.activate(z, (orc.ACT_SIGMOID, orc.ACT_SIGMOID, orc.ACT_EXPM1))
+    assert abs(float(s[0, 0]) - 0.5) < 1e-12          # sigmoid(0) = 1/2
+    assert abs(float(s[0, 1]) - 0.75) < 1e-12         # sigmoid(ln 3) = 3/4
+    assert abs(float(s[0, 2]) - 100.0) < 1e-9         # head regresses log(1+r): r = 100
+    s = orc.activate(z, (orc.ACT_IDENTITY,) * 3)
+    assert torch.equal(s, z)
+
+
+# ---------------------------------------------------------------- exit decision (Alg. 1, Sec. 3.3)
+def _exit_once(cfg, sig_conf, toks, L, state=None, S=3):
+    P = len(toks)
+    ss = torch.full((1, P, S), float("nan"), dtype=F64)
+    for j, c in enumerate(sig_conf):
+        if c is not None:
+            ss[0, j] = torch.tensor([c, 0.5, 0.5], dtype=F64)
+    st = state if state is not None else orc.ExitState.fresh(1, S)
+    out = orc.exit_update(cfg, st, ss, torch.tensor([toks]), [list(range(P))],
+                          torch.tensor([L]), torch.tensor([99]))
+    return out, st
+
+
+def test_exit_hand_worked_scenario():
+    # x: 0.5 ; 0.3*0.95+0.7*0.5 = 0.635 ; 0.3*0.99+0.7*0.635 = 0.7415   (alpha 0.3)
+    cfg = orc.ExitCfg(alpha=0.3, thr=(0.6, 0, 0), enable_mask=1, stop_think_token=42)
+    out, st = _exit_once(cfg, [0.5, 0.95, 0.99, None], [10, 11, 12, 13], L=3)
+    assert int(out.exit_flag[0]) == 1 and int(out.accept_len[0]) == 1
+    assert int(out.recover_tok[0]) == 42 and int(st.thinking[0]) == 0
+    assert abs(float(out.smoothed[0, 0]) - 0.635) < 1e-6 and int(st.n_updates[0]) == 2
+    # only token 12 is a step-split token: exit moves to slot 2 with x = 0.7415
+    bm = torch.zeros(1, dtype=torch.int32)
+    bm[0] = 1 << 12
+    cfg2 = orc.ExitCfg(alpha=0.3, thr=(0.6, 0, 0), enable_mask=1, stop_think_token=42, split_bitmap=bm)
+    out, st = _exit_once(cfg2, [0.5, 0.95, 0.99, None], [10, 11, 12, 13], L=3)
+    assert int(out.exit_flag[0]) == 1 and int(out.accept_len[0]) == 2
+    assert abs(float(out.smoothed[0, 0]) - 0.7415) < 1e-6
+    # the draft stopped at slot 1: slot 2 is outside the accepted prefix, no exit
+    out, st = _exit_once(cfg2, [0.5, 0.95, 0.99, None], [10, 11, 12, 13], L=1)
+    assert int(out.exit_flag[0]) == 0 and int(out.accept_len[0]) == 1 and int(out.recover_tok[0]) == 99
+    assert int(st.thinking[0]) == 1 and int(st.n_updates[0]) == 2
+    # threshold higher than anything reached
+    cfg3 = orc.ExitCfg(alpha=0.3, thr=(0.75, 0, 0), enable_mask=1, stop_think_token=42)
+    out, st = _exit_once(cfg3, [0.5, 0.95, 0.99, None], [10, 11, 12, 13], L=3)
+    assert int(out.exit_flag[0]) == 0 and int(out.accept_len[0]) == 3
+    assert int(st.n_updates[0]) == 3      # slot 3 carries no signal: smoothing stops there
+
+
+def test_exit_first_only_mode_and_and_combination():
+    # paper-literal: only the signal of the last accepted token (slot 0) is smoothed
+    cfg = orc.ExitCfg(alpha=0.3, thr=(0.6, 0, 0), enable_mask=1, stop_think_token=1,
+                      ema_positions=orc.EMA_FIRST_ONLY)
+    out, st = _exit_once(cfg, [0.5, 0.95, 0.99, None], [10, 11, 12, 13], L=3)
+    assert int(out.exit_flag[0]) == 0 and int(st.n_updates[0]) == 1
+    assert abs(float(out.smoothed[0, 0]) - 0.5) < 1e-7
+    # SpecExit*-style: conf > .8 AND prog > .3 AND rem < 200 ; signals (c, .5, .5)
+    cfg = orc.ExitCfg(alpha=1.0, thr=(0.8, 0.3, 200.0), dir=(orc.DIR_GT, orc.DIR_GT, orc.DIR_LT),
+                      enable_mask=0b111, stop_think_token=1)
+    out, _ = _exit_once(cfg, [0.9], [3], L=0)
+    assert int(out.exit_flag[0]) == 1
+    cfg = orc.ExitCfg(alpha=1.0, thr=(0.8, 0.6, 200.0), dir=(orc.DIR_GT, orc.DIR_GT, orc.DIR_LT),
+                      enable_mask=0b111, stop_think_token=1)
+    out, _ = _exit_once(cfg, [0.9], [3], L=0)
+    assert int(out.exit_flag[0]) == 0           # progress 0.5 is not > 0.6
+    cfg = orc.ExitCfg(alpha=1.0, thr=(0.8, 0.3, 0.4), dir=(orc.DIR_GT, orc.DIR_GT, orc.DIR_LT),
+                      enable_mask=0b111, stop_think_token=1)
+    out, _ = _exit_once(cfg, [0.9], [3], L=0)
+    assert int(out.exit_flag[0]) == 0           # remaining 0.5 is not < 0.4
+    # strictness: "greater than 0.9" is false at exactly 0.9 (fp32 compare)
+    cfg = orc.ExitCfg(alpha=1.0, thr=(0.5, 0, 0), enable_mask=1, stop_think_token=1)
+    out, _ = _exit_once(cfg, [0.5], [3], L=0)
+    assert int(out.exit_flag[0]) == 0
+
+
+def test_exit_invariants_random():
+    rng = random.Random(5)
+    for trial in range(200):
+        K = rng.randint(1, 6)
+        L = rng.randint(0, K)
+        conf = [rng.random() for _ in range(K)] + [None]
+        toks = [rng.randrange(64) for _ in range(K + 1)]
+        bm = torch.tensor([rng.getrandbits(31), rng.getrandbits(31)], dtype=torch.int32)
+        prev_flag = 1
+        for thr in [0.0, 0.2, 0.4, 0.6, 0.8, 1.0]:
+            cfg = orc.ExitCfg(alpha=0.3, thr=(thr, 0, 0), enable_mask=1, stop_think_token=5,
+                              split_bitmap=bm)
+            out, st = _exit_once(cfg, conf, toks, L)
+            flag = int(out.exit_flag[0])
+            assert flag <= prev_flag                      # monotone in a "greater than" threshold
+            prev_flag = flag
+            assert 0 <= int(out.accept_len[0]) <= L <= K
+            if flag:
+                assert int(out.recover_tok[0]) == 5 and int(st.thinking[0]) == 0
+                assert orc.is_split(cfg, toks[int(out.accept_len[0])])
+            else:
+                assert int(out.recover_tok[0]) == 99 and int(out.accept_len[0]) == L
+        # an empty split set never exits
+        cfg = orc.ExitCfg(alpha=0.3, thr=(0.0, 0, 0), enable_mask=1,
+                          split_bitmap=torch.zeros(2, dtype=torch.int32))
+        out, _ = _exit_once(cfg, conf, toks, L)
+        assert int(out.exit_flag[0]) == 0
+        # a sequence that left the reasoning phase is frozen
+        st = orc.ExitState.fresh(1)
+        st.thinking[0] = 0
+        st.x[0] = torch.tensor([0.1, 0.2, 0.3], dtype=F64)
+        before = st.clone()
+        cfg = orc.ExitCfg(alpha=0.3, thr=(0.0, 0, 0), enable_mask=1)
+        out, st = _exit_once(cfg, conf, toks, L, state=st)
+        assert int(out.exit_flag[0]) == 0 and int(out.accept_len[0]) == L
+        assert torch.equal(st.x, before.x) and torch.equal(st.n_updates, before.n_updates)
+
+
+def test_exit_lt_direction_monotone():
+    for thr_lo, thr_hi in [(10.0, 50.0), (50.0, 150.0)]:
+        flags = []
+        for thr in (thr_lo, thr_hi):
+            cfg = orc.ExitCfg(alpha=1.0, thr=(0, 0, thr), dir=(orc.DIR_GT, orc.DIR_GT, orc.DIR_LT),
+                              enable_mask=0b100)
+            ss = torch.tensor([[[0.5, 0.5, 40.0]]], dtype=F64)
+            out = orc.exit_update(cfg, orc.ExitState.fresh(1), ss, torch.tensor([[1]]), [[0]],
+                                  torch.tensor([0]), torch.tensor([9]))
+            flags.append(int(out.exit_flag[0]))
+        assert flags[0] <= flags[1]                        # non-decreasing in a "less than" threshold
+    assert flags == [1, 1]
+
+
+# ---------------------------------------------------------------- acceptance (Alg. 1)
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 5, 6])
+def test_accept_chain_brute_force(K):
+    for bits in itertools.product("01", repeat=K):
+        pattern = "".join(bits)
+        cand = [7] + [100 + j for j in range(1, K + 1)]
+        target = [(cand[j + 1] if pattern[j] == "1" else 999) for j in range(K)] + [555]
+        L, path, rec = orc.accept_chain(cand, target)
+        want = pattern.find("0") if "0" in pattern else K          # length of the all-ones prefix
+        assert L == want and path == list(range(want + 1)) and rec == target[want] and L <= K
+
+
+def test_accept_tree_brute_force():
+    rng = random.Random(3)
+    for trial in range(300):
+        P = rng.randint(1, 12)
+        parent = [-1] + [rng.randrange(s) for s in range(1, P)]
+        tok = [0] * P
+        for s in range(1, P):       # siblings carry distinct tokens, as top-k children do
+            used = {tok[c] for c in range(1, s) if parent[c] == parent[s]}
+            tok[s] = rng.choice([t for t in range(12) if t not in used])
+        target = [rng.randrange(4) for _ in range(P)]
+        # enumerate every root path, keep the fully accepted ones
+        accepted = []
+        for s in range(P):
+            chain = [s]
+            while parent[chain[-1]] >= 0:
+                chain.append(parent[chain[-1]])
+            chain.reverse()
+            if all(tok[chain[i]] == target[chain[i - 1]] for i in range(1, len(chain))):
+                accepted.append(chain)
+        best = max(len(c) for c in accepted)
+        longest = [c for c in accepted if len(c) == best]
+        assert len(longest) == 1
+        L, path, rec = orc.accept_tree(tok, parent, target)
+        assert path == longest[0] and L == best - 1 and rec == target[path[-1]]
+
+
+# ---------------------------------------------------------------- building blocks: textbook cases
+def test_rmsnorm_constant_vector_and_scaling():
+    g = torch.tensor([1.0, 2.0, -1.0, 0.5], dtype=F64)
+    out = orc.rmsnorm(torch.full((1, 4), -3.0, dtype=F64), g, 0.0)
+    assert torch.allclose(out, -g.view(1, 4))
+    x = torch.randn(3, 16, dtype=F64)
+    a = orc.rmsnorm(x, torch.ones(16, dtype=F64), 0.0)
+    assert torch.allclose((a * a).mean(dim=1), torch.ones(3, dtype=F64))         # unit RMS
+    assert torch.allclose(orc.rmsnorm(5.0 * x, torch.ones(16, dtype=F64), 0.0), a)  # scale-free
+    # eps enters under the root: x = (2, 2), eps = 5 -> 2 / sqrt(4 + 5) = 2/3
+    out = orc.rmsnorm(torch.tensor([[2.0, 2.0]], dtype=F64), torch.ones(2, dtype=F64), 5.0)
+    assert torch.allclose(out, torch.full((1, 2), 2.0 / 3.0, dtype=F64))
+
+
+def test_rope_rotation_values_and_properties():
+    # d = 2: one pair, frequency theta^0 = 1: (1, 0) at position 1 -> (cos 1, sin 1)
+    out = orc.rope(torch.tensor([[1.0, 0.0]], dtype=F64), 1, 10000.0)
+    assert torch.allclose(out, torch.tensor([[0.5403023058681398, 0.8414709848078965]], dtype=F64))
+    # d = 4, theta = 1e4: pairs (0,2) at frequency 1 and (1,3) at 1e4^(-2/4) = 0.01
+    out = orc.rope(torch.tensor([[0.0, 1.0, 0.0, 0.0]], dtype=F64), 100, 10000.0)
+    assert torch.allclose(out, torch.tensor([[0.0, math.cos(1.0), 0.0, math.sin(1.0)]], dtype=F64))
+    out = orc.rope(torch.tensor([[1.0, 0.0, 0.0, 0.0]], dtype=F64), 3, 10000.0)
+    assert torch.allclose(out, torch.tensor([[math.cos(3.0), 0.0, math.sin(3.0), 0.0]], dtype=F64))
+    q, k = torch.randn(2, 32, dtype=F64), torch.randn(2, 32, dtype=F64)
+    assert torch.allclose(orc.rope(q, 0, 1e6), q)                                   # identity at 0
+    assert torch.allclose(orc.rope(q, 977, 1e6).norm(dim=1), q.norm(dim=1))         # an isometry
+    d1 = (orc.rope(q, 40, 1e6) * orc.rope(k, 33, 1e6)).sum()
+    d2 = (orc.rope(q, 1007, 1e6) * orc.rope(k, 1000, 1e6)).sum()
+    assert abs(float(d1 - d2)) < 1e-9                                               # relative only
+
+
+def test_silu_values():
+    x = torch.tensor([0.0, math.log(3.0), -math.log(3.0)], dtype=F64)
+    want = torch.tensor([0.0, 0.75 * math.log(3.0), -0.25 * math.log(3.0)], dtype=F64)
+    assert torch.allclose(orc.silu(x), want)
+
+
+def _mini_model(H=8, n_q=2, n_kv=1, d=4, F=8, V=5, S=1, page=4, eps=1e-12, theta=1e4):
+    sh = synth.ModelShape(H=H, n_q=n_q, n_kv=n_kv, d=d, F=F, V=V, S=S, eps=eps, theta=theta, page=page)
+    z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16)
+    w = {"embed": z(V, H), "fc": z(H, 2 * H), "norm1": torch.ones(H, dtype=torch.bfloat16),
+         "norm2": torch.ones(H, dtype=torch.bfloat16), "normf": torch.ones(H, dtype=torch.bfloat16),
+         "wqkv": z(sh.qkv_rows, H), "wo": z(H, n_q * d), "wgate_up": z(2 * F, H), "wdown": z(H, F),
+         "head": z(V + S, H)}
+    w["fc"][:, :H] = torch.eye(H, dtype=torch.bfloat16)       # x = feature
+    return sh, w
+
+
+def _mini_kv(sh, n, kval=None, vval=None, extra=4, seed=0):
+    lens = torch.tensor([n], dtype=torch.int32)
+    kv = synth.make_kv(sh, lens, extra, seed, poison_tail=True)
+    if kval is not None:
+        kv["k_pages"][:] = kval
+    if vval is not None:
+        kv["v_pages"][:] = vval
+    return orc.PagedKV(kv["k_pages"], kv["v_pages"], kv["page_table"], kv["cache_len"])
+
+
+def test_one_token_hand_example():
+    g = {r[0]: [float(v) for v in r[1:]] for r in _rows("one_token_example.txt")}
+    sh, w = _mini_model(H=2, n_q=1, n_kv=1, d=2, F=2, V=3, S=1)
+    w["head"][:] = torch.tensor([[1, 0], [0, 1], [1, 1], [1, -1]], dtype=torch.bfloat16)
+    w["wqkv"][:] = 0.37                                     # attention runs, W_o = 0 discards it
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    kv = _mini_kv(sh, 3)
+    d = orc.draft_chain(model, kv, torch.tensor([[3.0, 4.0]], dtype=torch.bfloat16),
+                        torch.tensor([1]), K=1)
+    assert torch.allclose(d.hidden[0, 0], torch.tensor(g["g_bf16"], dtype=F64), atol=0, rtol=0)
+    assert (d.hidden[0, 0] - torch.tensor(g["g_exact"], dtype=F64)).abs().max() < 4e-3
+    assert int(d.cand_tok[0, 1]) == int(g["token"][0])
+    assert abs(float(d.z[0, 0, 0]) - g["z_bf16"][0]) < 1e-7
+    assert abs(float(d.slot_signal[0, 0, 0]) - g["sigmoid_bf16"][0]) < 1e-6
+    assert abs(float(d.slot_signal[0, 0, 0]) - g["sigmoid_exact"][0]) < 2e-3
+    assert bool(torch.isnan(d.slot_signal[0, 1]).all())     # slot K was never drafted from
+
+
+def test_layer_residual_only_closed_form():
+    # W_o = 0 and W_down = 0: the layer adds nothing, g = RMSNorm(feature) * gain
+    sh, w = _mini_model()
+    w["wqkv"][:] = 0.25
+    w["wgate_up"][:] = 0.5
+    w["normf"][:] = torch.tensor([1, 2, 1, 2, 1, 2, 1, 2], dtype=torch.bfloat16)
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    f = torch.tensor([[1, -1, 2, -2, 1, -1, 2, -2]], dtype=torch.bfloat16)
+    g, _ = model.round(_mini_kv(sh, 5), [orc.Row(0, f[0].to(F64), 0, 5, 5, [5])])
+    rms = math.sqrt(2.5)
+    want = torch.tensor([1, -2, 2, -4, 1, -2, 2, -4], dtype=F64) / rms
+    assert (g[0] - want).abs().max() < 8e-3 * want.abs().max()
+
+
+def test_attention_uniform_scores_closed_form():
+    # W_qkv = 0: q = k_new = v_new = 0, every score is 0, softmax is uniform over the n cached
+    # entries plus the row's own new (zero) entry: o = n/(n+1) * c.  W_o = permutation, so
+    # a = x + perm(o); W_down = 0; no final gain.
+    sh, w = _mini_model()
+    n, c = 7, 2.0
+    perm = [3, 0, 1, 2, 7, 4, 5, 6]                        # (W_o o)[i] = o[perm[i]]: not an involution
+    for i, p in enumerate(perm):
+        w["wo"][i, p] = 1.0
+    kv = _mini_kv(sh, n)
+    kv.v[:] = torch.arange(4, dtype=torch.bfloat16) + c    # v[dim j] = c + j for every cached slot
+    kv.v[:] = torch.where(torch.isnan(kv.k), torch.full_like(kv.v, float("nan")), kv.v)
+    f = torch.tensor([[1, 2, 3, 4, 5, 6, 7, 8]], dtype=torch.bfloat16)
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    g, _ = model.round(kv, [orc.Row(0, f[0].to(F64), 0, n, n, [n])])
+    o = np.array([(c + j) * n / (n + 1) for j in range(4)] * 2)    # both q heads share the kv head
+    a = np.arange(1, 9, dtype=np.float64) + o[perm]
+    want = a / math.sqrt((a * a).mean())
+    assert np.abs(g[0].numpy() - want).max() < 1e-2 * np.abs(want).max()
+
+
+def test_attention_textbook_cases():
+    sh, w = _mini_model(n_q=4, n_kv=2, d=4, H=16)
+    model = orc.DraftModel(sh, w)
+    # (a) all keys equal -> plain mean of V ; GQA: q heads 0,1 read kv head 0, heads 2,3 kv head 1
+    kv = _mini_kv(sh, 6, kval=1.0)
+    kv.v[:, 0] = 10.0
+    kv.v[:, 1] = 20.0
+    kv.len = [6]
+    row = orc.Row(0, None, 0, 0, 0, [])
+    out = model.attention(kv, row, torch.randn(4, 4, dtype=F64))
+    assert torch.allclose(out[:2], torch.full((2, 4), 10.0, dtype=F64))
+    assert torch.allclose(out[2:], torch.full((2, 4), 20.0, dtype=F64))
+    # (b) one cached entry -> exactly its V
+    kv = _mini_kv(sh, 1)
+    out = model.attention(kv, row, torch.randn(4, 4, dtype=F64))
+    assert torch.allclose(out[0], kv.prefix(0)[1][0, 0])
+    # (c) adding one vector to every key shifts all scores alike: output unchanged
+    kv = _mini_kv(sh, 9, seed=4)
+    q = torch.randn(4, 4, dtype=F64)
+    base = model.attention(kv, row, q)
+    kv2 = _mini_kv(sh, 9, seed=4)
+    kv2.k[:] = (kv2.k.to(torch.float32) + 0.5).to(torch.bfloat16)
+    kv3 = orc.PagedKV(kv2.k, kv2.v, kv2.table, kv2.len)
+    # bf16 re-rounding of the shifted keys perturbs slightly; compare against the definition
+    Kp, Vp = kv3.prefix(0)
+    for h in range(4):
+        sc = (Kp[h // 2] @ q[h]) / 2.0                       # sqrt(d) = 2
+        e = np.exp(sc.numpy() - sc.numpy().max())
+        want = (e / e.sum()) @ Vp[h // 2].numpy()
+        assert np.abs(model.attention(kv3, row, q)[h].numpy() - want).max() < 1e-12
+    # (d) a dominant key wins: q = 50 * k_3 -> output ~ v_3
+    Kp, Vp = kv.prefix(0)
+    q = torch.stack([50.0 * Kp[0, 3], 50.0 * Kp[0, 3], 50.0 * Kp[1, 3], 50.0 * Kp[1, 3]])
+    out = model.attention(kv, row, q)
+    sc = (Kp[0] @ q[0]) / 2.0
+    if float(sc[3] - torch.cat([sc[:3], sc[4:]]).max()) > 30:
+        assert torch.allclose(out[0], Vp[0, 3], atol=1e-9)
+    # (e) visible extra slots enter, invisible ones do not
+    kv = _mini_kv(sh, 4, kval=1.0, vval=1.0)
+    kv.write(0, 4, torch.ones(2, 4), torch.full((2, 4), 6.0))
+    kv.write(0, 5, torch.ones(2, 4), torch.full((2, 4), 600.0))
+    out = model.attention(kv, orc.Row(0, None, 0, 0, 0, [4]), torch.randn(4, 4, dtype=F64))
+    assert torch.allclose(out, torch.full((4, 4), 2.0, dtype=F64))    # (4*1 + 6)/5
+
+
+def test_mlp_closed_form_with_permutations():
+    # W_o = 0; gate = n2[pg], up = n2[pu]; y = a + (silu(gate)*up)[pd]; distinct non-involutive perms
+    sh, w = _mini_model()
+    pg = [1, 2, 3, 4, 5, 6, 7, 0]
+    pu = [2, 3, 4, 5, 6, 7, 0, 1]
+    pd = [5, 6, 7, 0, 1, 2, 3, 4]
+    for i in range(8):
+        w["wgate_up"][i, pg[i]] = 1.0
+        w["wgate_up"][8 + i, pu[i]] = 1.0
+        w["wdown"][i, pd[i]] = 1.0
+    f = np.array([1, -2, 3, -4, 0.5, 1.5, -0.5, 2], dtype=np.float64)
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    g, _ = model.round(_mini_kv(sh, 3), [orc.Row(0, torch.tensor(f, dtype=F64), 0, 3, 3, [3])])
+    n2 = f / math.sqrt((f * f).mean())
+    gate, up = n2[pg], n2[pu]
+    m = gate / (1 + np.exp(-gate)) * up
+    y = f + m[pd]
+    want = y / math.sqrt((y * y).mean())
+    assert np.abs(g[0].numpy() - want).max() < 1e-2 * np.abs(want).max()
+
+
+def test_fc_takes_feature_first_then_embedding():
+    # x = W_fc [f ; E[t]] with W_fc = [0 | I]: x is the embedding row of the token
+    sh, w = _mini_model()
+    w["fc"][:] = 0
+    w["fc"][:, 8:] = torch.eye(8, dtype=torch.bfloat16)
+    w["embed"][3] = torch.tensor([2, 0, 0, 0, 0, 0, 0, 2], dtype=torch.bfloat16)
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    g, _ = model.round(_mini_kv(sh, 3), [orc.Row(0, torch.full((8,), 9.0, dtype=F64), 3, 3, 3, [3])])
+    assert torch.allclose(g[0], torch.tensor([2, 0, 0, 0, 0, 0, 0, 2], dtype=F64), atol=1e-2)
+
+
+def test_paging_layout_invariance():
+    # the same logical cache under page sizes 16 / 64 / 128 and shuffled tables: same result
+    base = harness.tiny_workload(B=1, len_lo=37, len_hi=37)
+    outs = []
+    logical = None
+    for page, seed in [(16, 1), (64, 2), (128, 3)]:
+        wl = synth.Workload(**{**base.__dict__, "shape": synth.ModelShape(
+            **{**base.shape.__dict__, "page": page})})
+        case = harness.build_case(wl)
+        kvd = synth.make_kv(wl.shape, case.kv["cache_len"], wl.draft_rows, seed, poison_tail=True)
+        n = 37
+        gk = torch.randn(n, wl.shape.n_kv, wl.shape.d, generator=torch.Generator().manual_seed(9)).to(torch.bfloat16)
+        gv = torch.randn(n, wl.shape.n_kv, wl.shape.d, generator=torch.Generator().manual_seed(10)).to(torch.bfloat16)
+        for s in range(n):
+            pp = int(kvd["page_table"][0, s // page])
+            kvd["k_pages"][pp, :, s % page] = gk[s]
+            kvd["v_pages"][pp, :, s % page] = gv[s]
+        kv = orc.PagedKV(kvd["k_pages"], kvd["v_pages"], kvd["page_table"], kvd["cache_len"])
+        d = orc.draft_chain(harness.oracle_model(case), kv, case.f0, case.t0, wl.K)
+        outs.append(d)
+    for d in outs[1:]:
+        assert torch.equal(d.cand_tok, outs[0].cand_tok)
+        assert torch.equal(d.hidden, outs[0].hidden)
+
+
+# ---------------------------------------------------------------- extended head (Eq. 1)
+def test_head_against_numpy_scan_ties_and_concat():
+    torch.manual_seed(0)
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=4096)
+    w = {"head": (torch.randn(sh.V + 3, sh.H) * 0.02).to(torch.bfloat16)}
+    g = torch.randn(5, sh.H).to(torch.bfloat16).to(F64)
+    model = orc.DraftModel(sh, w)
+    ho = model.head(g)
+    Wn = w["head"].to(torch.float64).numpy()
+    for r in range(5):
+        dense = Wn @ g[r].numpy()
+        best, arg = -np.inf, -1
+        for i in range(sh.V):                     # linear scan, strict '>' keeps the lower index
+            v = np.float32(dense[i])
+            if v > best:
+                best, arg = v, i
+        assert orc.argmax_low(ho.logits[r]) == arg
+        # Eq. 1: the signal outputs are the last rows of the same product
+        sep = w["head"][sh.V:].to(F64) @ g[r]
+        assert torch.allclose(ho.z[r], sep.to(torch.float32).to(F64))
+        assert torch.allclose(ho.s[r], (1 / (1 + torch.exp(-ho.z[r]))).to(torch.float32).to(F64))
+    # duplicated best row at a lower and a higher index: the lower one wins
+    w2 = {"head": w["head"].clone()}
+    a = orc.argmax_low(ho.logits[0])
+    lo, hi = (5, 4000) if a not in (5, 4000) else (6, 4001)
+    w2["head"][lo] = w2["head"][a]
+    w2["head"][hi] = w2["head"][a]
+    ho2 = orc.DraftModel(sh, w2).head(g[:1])
+    assert orc.argmax_low(ho2.logits[0]) == min(lo, a)
+    assert orc.top_gap(ho2.logits[0]) == 0.0
+    # signal rows never take part in the argmax: make them huge
+    w3 = {"head": w["head"].clone()}
+    w3["head"][sh.V:] = 50.0 * torch.sign(g[0]).to(torch.bfloat16)
+    ho3 = orc.DraftModel(sh, w3).head(g[:1])
+    assert orc.argmax_low(ho3.logits[0]) == a and ho3.logits.shape[1] == sh.V
+
+
+def test_topk_low_order_and_large_vocab_path():
+    v = torch.tensor([1.0, 3.0, 3.0, 2.0, 3.0, 0.0], dtype=F64)
+    assert orc.topk_low(v, 4) == [1, 2, 4, 3]
+    torch.manual_seed(1)
+    big = torch.randn(10000, dtype=F64).to(torch.float32).to(F64)
+    big[77] = big[9000] = big.max() + 1
+    got = orc.topk_low(big, 8)
+    want = sorted(range(10000), key=lambda i: (-float(big[i]), i))[:8]
+    assert got == want and got[:2] == [77, 9000]
+
+
+# ---------------------------------------------------------------- tree drafting
+def _tree_case(topk, depth, nodes, B=2, V=40):
+    sh = synth.ModelShape(H=32, n_q=2, n_kv=1, d=16, F=48, V=V, page=16)
+    wl = synth.Workload("t", sh, B=B, mode=synth.TREE, K=depth, topk=topk, max_nodes=nodes,
+                        len_lo=9, len_hi=30, seed=21)
+    return harness.build_case(wl)
+
+
+def test_tree_invariants():
+    case = _tree_case(topk=3, depth=4, nodes=14)
+    wl = case.wl
+    model = harness.oracle_model(case)
+    model.w = {k: (v.to(torch.float32) * (25.0 if k in ("head",) else 1.0)).to(torch.bfloat16)
+               for k, v in case.weights.items()}            # spread the logits a little
+    t = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
+    for b in range(wl.B):
+        cs = t.cands[b]
+        assert len(cs) == 3 + 3 * 9
+        for c in cs:
+            assert c.logp <= 0.0
+            if c.parent >= 0:
+                assert c.score <= cs[c.parent].score + 1e-7      # scores fall along a path
+                assert cs[c.parent].row == c.src_row              # produced by its parent's row
+        kept = {int(x) for x in t.slot_cid[b, 1:]}
+        assert len(kept) == wl.max_nodes
+        for cid in kept:
+            assert cs[cid].parent < 0 or cs[cid].parent in kept   # ancestor-closed
+        for s in range(1, wl.P):
+            p = int(t.parent[b, s])
+            assert 0 <= p < s and int(t.depth[b, s]) == int(t.depth[b, p]) + 1
+        worst_kept = min(cs[c].score for c in kept)
+        assert all(c.score <= worst_kept for c in cs if c.cid not in kept)
+        # children of one parent carry distinct tokens
+        for p in range(wl.P):
+            ch = [int(t.cand_tok[b, s]) for s in range(1, wl.P) if int(t.parent[b, s]) == p]
+            assert len(ch) == len(set(ch))
+
+
+def test_tree_logprobs_sum_to_one_over_full_vocab():
+    case = _tree_case(topk=8, depth=1, nodes=8, B=1, V=8)
+    wl = case.wl
+    t = orc.draft_tree(harness.oracle_model(case), harness.oracle_kv(case), case.f0, case.t0,
+                       1, 8, 8)
+    assert abs(sum(math.exp(c.logp) for c in t.cands[0]) - 1.0) < 1e-6
+    assert sorted(c.tok for c in t.cands[0]) == list(range(8))
+
+
+def test_tree_top1_degenerates_to_chain():
+    case = _tree_case(topk=1, depth=4, nodes=4)
+    wl = case.wl
+    model = harness.oracle_model(case)
+    t = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, 4, 1, 4)
+    c = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 4)
+    assert torch.equal(t.cand_tok, c.cand_tok)
+    assert torch.equal(t.hidden, c.hidden)
+    assert torch.equal(t.slot_signal[:, :4], c.slot_signal[:, :4])
+    assert torch.equal(t.parent[:, 1:], torch.arange(4).repeat(wl.B, 1))
+
+
+# ---------------------------------------------------------------- whole forward vs an independent restatement
+def _np_forward(case, f, tok, b, n_extra_k, n_extra_v):
+    """float64 numpy restatement of one draft position without any intermediate rounding,
+    written against the logical (un-paged) cache."""
+    sh, w = case.wl.shape, {k: v.to(torch.float64).numpy() for k, v in case.weights.items()}
+    page = sh.page
+    n = int(case.kv["cache_len"][b])
+    K = np.zeros((n, sh.n_kv, sh.d))
+    Vv = np.zeros((n, sh.n_kv, sh.d))
+    for s in range(n):
+        pp = int(case.kv["page_table"][b, s // page])
+        K[s] = case.kv["k_pages"][pp, :, s % page].to(torch.float64).numpy()
+        Vv[s] = case.kv["v_pages"][pp, :, s % page].to(torch.float64).numpy()
+    K = np.concatenate([K] + n_extra_k, axis=0) if n_extra_k else K
+    Vv = np.concatenate([Vv] + n_extra_v, axis=0) if n_extra_v else Vv
+    pos = K.shape[0]
+    u = np.concatenate([f, w["embed"][tok]])
+    x = w["fc"] @ u
+
+    def norm(v, g):
+        return v / np.sqrt((v ** 2).mean() + sh.eps) * g
+
+    def rot(v):
+        out = v.copy()
+        h = sh.d // 2
+        for i in range(h):
+            ang = pos * sh.theta ** (-2.0 * i / sh.d)
+            out[:, i] = v[:, i] * math.cos(ang) - v[:, i + h] * math.sin(ang)
+            out[:, i + h] = v[:, i + h] * math.cos(ang) + v[:, i] * math.sin(ang)
+        return out
+
+    qkv = w["wqkv"] @ norm(x, w["norm1"])
+    q = rot(qkv[:sh.n_q * sh.d].reshape(sh.n_q, sh.d))
+    k = rot(qkv[sh.n_q * sh.d:(sh.n_q + sh.n_kv) * sh.d].reshape(sh.n_kv, sh.d))
+    v = qkv[(sh.n_q + sh.n_kv) * sh.d:].reshape(sh.n_kv, sh.d)
+    K = np.concatenate([K, k[None]], axis=0)
+    Vv = np.concatenate([Vv, v[None]], axis=0)
+    o = np.zeros((sh.n_q, sh.d))
+    for h in range(sh.n_q):
+        kvh = h // (sh.n_q // sh.n_kv)
+        sc = K[:, kvh] @ q[h] / math.sqrt(sh.d)
+        p = np.exp(sc - sc.max())
+        o[h] = (p / p.sum()) @ Vv[:, kvh]
+    a = x + w["wo"] @ o.reshape(-1)
+    gu = w["wgate_up"] @ norm(a, w["norm2"])
+    gate, up = gu[:sh.F], gu[sh.F:]
+    y = a + w["wdown"] @ (gate / (1 + np.exp(-gate)) * up)
+    g = norm(y, w["normf"])
+    return g, w["head"] @ g, k[None], v[None]
+
+
+def test_full_forward_against_float64_restatement():
+    wl = synth.workload("C0")
+    case = harness.build_case(wl)
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 2)
+    f = case.f0[0].to(torch.float64).numpy()
+    g1, logits1, k1, v1 = _np_forward(case, f, int(case.t0[0]), 0, [], [])
+    rel = np.linalg.norm(d.hidden[0, 0].numpy() - g1) / np.linalg.norm(g1)
+    assert rel < 1e-2
+    assert int(np.argmax(logits1[:wl.shape.V])) == int(d.cand_tok[0, 1]) or float(d.gap[0, 0]) < 5e-2
+    s1 = 1 / (1 + np.exp(-logits1[wl.shape.V:]))
+    assert np.abs(s1 - d.slot_signal[0, 0].numpy()).max() < 5e-3
+    # second position: attends to the first position's fresh K/V as well
+    g2, _, _, _ = _np_forward(case, g1, int(d.cand_tok[0, 1]), 0, [k1], [v1])
+    rel = np.linalg.norm(d.hidden[0, 1].numpy() - g2) / np.linalg.norm(g2)
+    assert rel < 2e-2
+
+
+def test_chain_iteration_end_to_end_properties():
+    wl = harness.tiny_workload(B=3, K=4)
+    case = harness.build_case(wl)
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    th = harness.chain_target_hidden(case, d)
+    v = orc.verify(model, th, d.cand_tok)
+    assert bool((v.accept_len <= wl.K).all()) and bool((v.accept_len >= 0).all())
+    # zero noise: the target hidden IS the draft hidden, so every draft token is accepted
+    case0 = harness.Case(wl, case.weights, case.kv, case.f0, case.t0, torch.zeros(wl.B))
+    v0 = orc.verify(model, harness.chain_target_hidden(case0, d), d.cand_tok)
+    assert bool((v0.accept_len == wl.K).all())
+    # forcing a draft token changes everything after it and nothing before it
+    alt = (int(d.cand_tok[1, 2]) + 1) % wl.shape.V
+    d2 = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, forced={(1, 2): alt})
+    assert torch.equal(d2.hidden[1, :2], d.hidden[1, :2]) and int(d2.cand_tok[1, 2]) == alt
+    assert not torch.equal(d2.hidden[1, 2], d.hidden[1, 2])
+    assert torch.equal(d2.hidden[0], d.hidden[0])
