@@ -1,0 +1,235 @@
+/*
+ * specexit.h - C ABI of the speculative-exit step on one B200 (sm_100a).
+ *
+ * One iteration of signal-guided speculative decoding (the body of the loop of
+ * Algorithm 1, without the target model's trunk):
+ *
+ *   draft K positions (chain) or a top-k tree with a one-layer draft model whose LM head
+ *   carries three extra rows (Eq. 1: confidence, progress, remaining length)
+ *     -> verify with the target LM head, greedy acceptance (Algorithm 1, "accept tokens,
+ *        accept length, recover token")
+ *     -> smooth the signals (Appendix A.1, EWMA) and threshold them at step-split tokens
+ *        (Section 3.3, "Stopping Conditions"); on exit the accepted length is cut at the
+ *        split token and the recover token becomes the stop-think token.
+ *
+ * Conventions for every entry point
+ *   - Pointers named *_d are DEVICE pointers, 16-byte aligned, owned by the caller, and
+ *     borrowed until the enqueued work has finished.  Everything else is host memory.
+ *   - All work is enqueued on the given stream; no entry point synchronises, allocates
+ *     device memory or frees it (sx_create / sx_destroy only touch host memory).
+ *   - Host-detectable problems (NULL, unsupported shape, workspace too small) return a
+ *     negative sx_status and launch nothing.  Problems only the device can see (a page
+ *     table too short for a write, a token id outside the vocabulary, a bounded wait that
+ *     ran out) are written to *status_d (the smallest code wins); kernels then skip the
+ *     offending access and never trap.  *status_d must be zeroed by the caller before the
+ *     first call and may be shared by several calls; outputs are unspecified when it is
+ *     non-zero.
+ *   - Matrices are bf16, row-major [out, in].  Activations handed between layers are
+ *     bf16; accumulation, normalisation, softmax, rotary and signal math are fp32.
+ *   - One sx_ctx per stream: a context is not thread-safe.
+ */
+#ifndef SPECEXIT_H
+#define SPECEXIT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t sx_status;
+enum {
+  SX_OK = 0,
+  SX_ERR_INVALID_ARG = -1,
+  SX_ERR_UNSUPPORTED = -2,
+  SX_ERR_CAPACITY = -3,    /* page table too short / token id out of range (device) */
+  SX_ERR_WORKSPACE = -4,
+  SX_ERR_CUDA = -5,
+  SX_ERR_TIMEOUT = -6      /* a bounded device-side wait expired */
+};
+
+enum { SX_MODE_CHAIN = 0, SX_MODE_TREE = 1 };
+enum { SX_ACT_SIGMOID = 0, SX_ACT_EXPM1 = 1, SX_ACT_IDENTITY = 2 };   /* Eq. 3-5 */
+enum { SX_DIR_GT = 0, SX_DIR_LT = 1 };                                 /* Appendix A.1 thresholds */
+enum { SX_EMA_VERIFIED_CONTEXT = 0, SX_EMA_FIRST_ONLY = 1 };
+
+#define SX_MAX_SIGNALS 3
+#define SX_MAX_TOPK 8
+#define SX_MAX_TREE_ROWS 64   /* drafted rows per sequence in one iteration (ancestor mask is 64 bit) */
+#define SX_MAX_VERIFY_SLOTS 64
+
+/* Shape of the draft model: concat(feature, embedding) -> fc 2H->H -> one pre-norm decoder
+ * layer (RMSNorm, grouped-query attention with rotary positions over a paged KV cache,
+ * SwiGLU) -> final RMSNorm -> extended head (Eq. 1). */
+typedef struct {
+  int32_t H, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+  int32_t n_signals;                /* rows appended to the LM head, <= SX_MAX_SIGNALS */
+  float rms_eps, rope_theta;
+  int32_t page_size;                /* KV slots per page */
+  int32_t act[SX_MAX_SIGNALS];      /* activation of each signal row */
+} sx_model_cfg;
+
+typedef struct {
+  const void *embed_d;        /* [vocab, H] */
+  const void *fc_d;           /* [H, 2H]: columns 0..H-1 take the feature, H..2H-1 the embedding */
+  const void *norm1_d;        /* [H] gain before attention */
+  const void *wqkv_d;         /* [(n_q + 2 n_kv) * head_dim, H]: q rows, then k rows, then v rows */
+  const void *wo_d;           /* [H, n_q * head_dim] */
+  const void *norm2_d;        /* [H] gain before the MLP */
+  const void *wgate_up_d;     /* [2 * ffn, H]: gate rows, then up rows */
+  const void *wdown_d;        /* [H, ffn] */
+  const void *normf_d;        /* [H] final gain */
+  const void *head_d;         /* [vocab + n_signals, H]: Eq. 1, vocabulary rows first, signal rows last */
+  const void *target_head_d;  /* [vocab, H] target LM head; may alias head_d */
+} sx_weights;
+
+/* Paged KV cache of the draft layer.  Slot s of sequence b lives in physical page
+ * page_table_d[b * max_pages + s / page_size] at offset s % page_size.  K is stored rotated. */
+typedef struct {
+  int32_t batch;
+  const int32_t *cache_len_d;   /* [batch] valid slots per sequence (not advanced by this library) */
+  const int32_t *page_table_d;  /* [batch, max_pages] */
+  int32_t max_pages;
+  int32_t num_pages;            /* physical pages in k_pages_d / v_pages_d */
+  void *k_pages_d;              /* [num_pages, n_kv, page_size, head_dim] bf16 */
+  void *v_pages_d;
+} sx_kv;
+
+typedef struct {
+  int32_t mode;        /* SX_MODE_CHAIN | SX_MODE_TREE */
+  int32_t K;           /* chain length, or tree depth */
+  int32_t topk;        /* tree: children per expanded node (<= SX_MAX_TOPK); chain: 1 */
+  int32_t max_nodes;   /* tree: nodes kept for verification, root excluded (< SX_MAX_VERIFY_SLOTS) */
+} sx_draft_cfg;
+
+/* Exit rule.  Signal i passes when smoothed_i > thr[i] (SX_DIR_GT) or < thr[i] (SX_DIR_LT),
+ * both strict; the enabled signals are AND-combined ("all the signals exceed a predefined
+ * threshold", case study of the appendix). */
+typedef struct {
+  float alpha;                       /* EWMA factor: x <- alpha * s + (1 - alpha) * x */
+  float thr[SX_MAX_SIGNALS];
+  int32_t dir[SX_MAX_SIGNALS];
+  uint32_t enable_mask;              /* bit i: signal i takes part */
+  int32_t ema_positions;             /* which accepted slots feed the EWMA */
+  const uint32_t *split_bitmap_d;    /* vocab bits, bit (t % 32) of word t / 32; NULL: every token splits */
+  int32_t stop_think_token;
+} sx_exit_cfg;
+
+/* Per-sequence state carried across iterations (device, caller-owned). */
+typedef struct {
+  float *x_d;            /* [batch, n_signals] smoothed signals */
+  int32_t *n_updates_d;  /* [batch] samples folded in so far; 0 -> the next sample initialises x */
+  int32_t *thinking_d;   /* [batch] 1 while inside the reasoning phase */
+} sx_exit_state;
+
+/* Outputs of one iteration; P = K + 1 (chain) or 1 + max_nodes (tree); rows = K (chain) or
+ * 1 + topk * (K - 1) (tree).  Slot 0 is the last accepted token. */
+typedef struct {
+  int32_t *cand_tok_d;         /* [B, P] tokens laid out for verification */
+  int32_t *parent_d;           /* [B, P] parent slot (-1 for slot 0); chain: j - 1 */
+  int32_t *depth_d;            /* [B, P] */
+  int32_t *slot_row_d;         /* [B, P] drafted row that took the slot's token as input, or -1 */
+  int32_t *slot_src_row_d;     /* [B, P] drafted row whose head produced the slot's token, -1 for slot 0 */
+  void *hidden_d;              /* [B, rows, H] bf16 final-normed hidden of every drafted row */
+  float *slot_signal_d;        /* [B, P, n_signals]; NaN where the slot was never drafted from */
+  int32_t *target_tok_d;       /* [B, P] target argmax per slot */
+  int32_t *accept_len_d;       /* [B] accepted draft tokens before the exit rule */
+  int32_t *path_d;             /* [B, K + 1] accepted slots in order, path[0] = 0, unused = -1 */
+  int32_t *recover_tok_d;      /* [B] */
+  int32_t *exit_flag_d;        /* [B] */
+  int32_t *accept_len_out_d;   /* [B] after truncation at the split token */
+  int32_t *recover_tok_out_d;  /* [B] stop_think_token where exit_flag = 1 */
+  float *smoothed_d;           /* [B, n_signals] */
+  /* optional (may be NULL), tree mode: every candidate generated, in generation order
+   * (depth 1: ids [0, topk); depth r >= 2: topk + (r-2) topk^2 + j topk + t for the t-th child
+   * of the j-th expanded row), NC = topk + (K - 1) topk^2 per sequence */
+  int32_t *tree_cand_tok_d;    /* [B, NC] */
+  float *tree_cand_score_d;    /* [B, NC] sum of log-probabilities along the path (fp32) */
+  int32_t *tree_cand_row_d;    /* [B, NC] drafted row that expanded the candidate, or -1 */
+} sx_iter_out;
+
+typedef struct sx_ctx sx_ctx;
+
+/* Build a host-side plan for the given shapes.  Weight pointers are recorded, not copied.
+ * Fails with SX_ERR_UNSUPPORTED for shapes the kernels do not cover (H, head_dim, ffn not
+ * multiples of 8; head_dim > 256 or not a power of two; group size > 8; topk, rows or slots
+ * beyond the SX_MAX_* limits). */
+sx_status sx_create(const sx_model_cfg *model, const sx_weights *weights, int32_t max_batch,
+                    const sx_draft_cfg *draft, int32_t max_verify_rows, sx_ctx **out);
+void sx_destroy(sx_ctx *ctx);
+/* Bytes of scratch (device, 256-byte aligned) every compute call needs for this plan. */
+size_t sx_workspace_bytes(const sx_ctx *ctx);
+const char *sx_strerror(sx_status s);
+/* Kernels launched by this context since it was created (host-side counter). */
+int64_t sx_launch_count(const sx_ctx *ctx);
+
+/* One draft round for R rows (Algorithm 1, "generate candidate tokens with M_d"; Eq. 1 and
+ * Eq. 3-5 for the head).  Chain mode: round k = 1..K, R = batch, row b sits at position
+ * cache_len[b] + k - 1 and sees the cache plus the k - 1 rows drafted before it.  Tree mode:
+ * round 1 drafts the root (R = batch); round r >= 2 drafts R = batch * topk rows, row
+ * b * topk + j at position cache_len[b] + r - 1, stored in slot cache_len[b] + 1 +
+ * (r - 2) * topk + j, attending to the cache plus the drafted rows whose bit is set in
+ * row_mask_d[row] (bit i = drafted row i of the same sequence; the own bit included).
+ * The rows' K/V are written into the cache at those slots; cache_len is not advanced.
+ *   feat_d        [R, H] bf16   hidden state of the previous position
+ *   tok_d         [R]           token at this position
+ *   row_mask_d    [R] or NULL   tree rounds >= 2 only
+ *   hidden_out_d  [R, H] bf16   final-normed hidden (feeds the head and the next round)
+ *   tok_out_d     [R, topk]     chain: argmax (topk = 1); tree: the topk best ids, best first,
+ *                               lower id first among equal logits
+ *   logp_out_d    [R, topk]     tree: log-probabilities of those ids; may be NULL in chain mode
+ *   signals_out_d [R, n_signals] activated signal values */
+sx_status sx_draft_step(sx_ctx *ctx, const sx_kv *kv, int32_t round, int32_t R, const void *feat_d,
+                        const int32_t *tok_d, const uint64_t *row_mask_d, void *hidden_out_d,
+                        int32_t *tok_out_d, float *logp_out_d, float *signals_out_d, void *ws_d,
+                        size_t ws_bytes, int32_t *status_d, void *stream);
+
+/* Target LM head with a fused argmax over batch * P given hidden states, then greedy
+ * acceptance (Algorithm 1, "accept tokens t_acpt, accept length l_acpt, recover token t_rec").
+ * Chain (parent_d = NULL): the longest prefix with cand[j] = target[j - 1].  Tree: walk from
+ * slot 0 to the child whose token is the target's choice at the current slot.
+ *   path_d [batch, path_stride] receives the accepted slots (path[0] = 0, rest -1). */
+sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hidden_d,
+                    const int32_t *cand_tok_d, const int32_t *parent_d, int32_t *target_tok_d,
+                    int32_t *accept_len_d, int32_t *path_d, int32_t path_stride,
+                    int32_t *recover_tok_d, void *ws_d, size_t ws_bytes, int32_t *status_d,
+                    void *stream);
+
+/* Exit decision (Section 3.3; Appendix A.1).  Walks path slots 0..accept_len; each slot that
+ * carries a signal updates the EWMA (all of them, or only the first, per ema_positions); the
+ * first slot whose token is a step-split token while the smoothed signals pass ends the
+ * reasoning phase.  Sequences with thinking = 0 are passed through unchanged. */
+sx_status sx_exit_update(sx_ctx *ctx, int32_t batch, int32_t P, const sx_exit_cfg *cfg,
+                         const sx_exit_state *state, const float *slot_signal_d,
+                         const int32_t *cand_tok_d, const int32_t *path_d, int32_t path_stride,
+                         const int32_t *accept_len_d, const int32_t *recover_tok_d,
+                         int32_t *exit_flag_d, int32_t *accept_len_out_d,
+                         int32_t *recover_tok_out_d, float *smoothed_out_d, int32_t *status_d,
+                         void *stream);
+
+/* The whole iteration in one enqueue: all draft rounds, (tree) candidate selection and
+ * layout, verification and the exit decision.  target_hidden_d [B, P, H] stands in for the
+ * target trunk's output at the verify slots; it is read only after the draft has finished. */
+sx_status sx_spec_exit_iter(sx_ctx *ctx, const sx_kv *kv, const sx_exit_cfg *cfg,
+                            const sx_exit_state *state, const void *feat0_d, const int32_t *tok0_d,
+                            const void *target_hidden_d, const sx_iter_out *out, void *ws_d,
+                            size_t ws_bytes, int32_t *status_d, void *stream);
+
+/* Same iteration with HOST buffers for the per-iteration inputs (feature, token, target
+ * hiddens) and the per-iteration results (accepted length, recover token, exit flag, smoothed
+ * signals): copies them in, runs sx_spec_exit_iter, copies the results out and synchronises
+ * the stream.  Staging buffers are the device arrays in `out` and `stage_*_d`. */
+sx_status sx_spec_exit_iter_host(sx_ctx *ctx, const sx_kv *kv, const sx_exit_cfg *cfg,
+                                 const sx_exit_state *state, const void *feat0_h,
+                                 const int32_t *tok0_h, const void *target_hidden_h,
+                                 void *stage_feat0_d, int32_t *stage_tok0_d,
+                                 void *stage_target_hidden_d, const sx_iter_out *out,
+                                 int32_t *accept_len_out_h, int32_t *recover_tok_out_h,
+                                 int32_t *exit_flag_h, float *smoothed_h, void *ws_d,
+                                 size_t ws_bytes, int32_t *status_d, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECEXIT_H */

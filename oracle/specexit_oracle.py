@@ -268,9 +268,10 @@ class ChainDraft:
 
 
 def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, K: int,
-                forced: Optional[Dict[Tuple[int, int], int]] = None) -> ChainDraft:
+                forced: Optional[Dict[Tuple[int, int], int]] = None, chooser=None) -> ChainDraft:
     """K autoregressive draft rounds per sequence.  ``forced[(b, k)]`` (k = 1..K) replaces
-    the k-th draft token of sequence b (used to replay a near-tie the other way)."""
+    the k-th draft token of sequence b (used to replay a near-tie the other way);
+    ``chooser("tok", (b, k), logits, 1, [tok]) -> [tok]`` may do the same on the fly."""
     B, H, S = f0.shape[0], model.sh.H, model.sh.S
     cand = torch.zeros(B, K + 1, dtype=torch.int64)
     cand[:, 0] = t0.to(torch.int64)
@@ -289,6 +290,8 @@ def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tens
             gap[b, k - 1] = top_gap(ho.logits[b])
             if forced and (b, k) in forced:
                 tok = int(forced[(b, k)])
+            if chooser is not None:
+                tok = int(chooser("tok", (b, k), ho.logits[b], 1, [tok])[0])
             cand[b, k] = tok
         hidden[:, k - 1] = g
         sig[:, k - 1] = ho.s
@@ -327,14 +330,16 @@ class TreeDraft:
 
 
 def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, depth: int,
-               topk: int, max_nodes: int, override: Optional[Dict[Tuple, List[int]]] = None
-               ) -> TreeDraft:
+               topk: int, max_nodes: int, override: Optional[Dict[Tuple, List[int]]] = None,
+               chooser=None) -> TreeDraft:
     """Tree drafting.  Round 1 drafts the root; round r >= 2 expands the `topk` best
     candidates of depth r-1 (score = sum of log-probabilities; ties: lower candidate id).
     After the last round the `max_nodes` best candidates overall are kept and laid out in
     candidate-id order behind the root.  ``override`` replaces single decisions by the
     given choice: ``("topk", b, row) -> token ids``, ``("expand", b, depth) -> cand ids``,
-    ``("keep", b) -> cand ids``."""
+    ``("keep", b) -> cand ids``.  ``chooser(kind, key, values, k, default) -> choice`` is
+    asked at every decision instead (values: the row's logits for "topk", else a list of
+    (cand id, score)); it lets a test adopt another implementation's choice at a near-tie."""
     sh = model.sh
     B, H, S = f0.shape[0], sh.H, sh.S
     ov = override or {}
@@ -351,6 +356,8 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
         margins[("topk", b, row)] = top_gap(logits, topk) if topk < logits.numel() else 1.0
         if ("topk", b, row) in ov:
             ids = list(ov[("topk", b, row)])
+        if chooser is not None:
+            ids = list(chooser("topk", (b, row), logits, topk, ids))
         lse = torch.logsumexp(logits, dim=0)
         for t in ids:
             lp = f32r(logits[t] - lse)
@@ -382,6 +389,11 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
             if ("expand", b, r - 1) in ov:
                 byid = {c.cid: c for c in cands[b]}
                 chosen = [byid[i] for i in ov[("expand", b, r - 1)]]
+            if chooser is not None:
+                byid = {c.cid: c for c in cands[b]}
+                pick = chooser("expand", (b, r - 1), [(c.cid, c.score) for c in level], topk,
+                               [c.cid for c in chosen])
+                chosen = [byid[i] for i in pick]
             for j, c in enumerate(chosen):
                 rid = 1 + (r - 2) * topk + j
                 c.row = rid
@@ -412,6 +424,8 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
         keep = sorted(c.cid for c in ranked[:max_nodes])
         if ("keep", b) in ov:
             keep = sorted(ov[("keep", b)])
+        if chooser is not None:
+            keep = sorted(chooser("keep", (b,), [(c.cid, c.score) for c in ranked], max_nodes, keep))
         slot_of = {-1: 0}
         cand_tok[b, 0] = int(t0[b])
         slot_row[b, 0] = 0

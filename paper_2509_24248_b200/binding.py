@@ -1,0 +1,314 @@
+"""ctypes binding of libspecexit.so: argument marshalling only.
+
+Every step of the speculative-exit iteration runs inside the library's CUDA kernels; torch is
+used here for device buffers and streams.  There is no fallback: if the library cannot be
+loaded, or a call returns an error, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import torch
+
+from . import synth
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspecexit.so")
+
+SX_MAX_SIGNALS = 3
+MODE_CHAIN, MODE_TREE = 0, 1
+ACT_SIGMOID, ACT_EXPM1, ACT_IDENTITY = 0, 1, 2
+DIR_GT, DIR_LT = 0, 1
+EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
+
+EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
+           "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
+           "sx_spec_exit_iter_host"]
+
+
+class SxError(RuntimeError):
+    pass
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [("H", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
+                ("n_signals", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
+                ("page_size", C.c_int32), ("act", C.c_int32 * SX_MAX_SIGNALS)]
+
+
+class Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("embed_d", "fc_d", "norm1_d", "wqkv_d", "wo_d", "norm2_d",
+                                          "wgate_up_d", "wdown_d", "normf_d", "head_d", "target_head_d")]
+
+
+class KV(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("cache_len_d", C.c_void_p), ("page_table_d", C.c_void_p),
+                ("max_pages", C.c_int32), ("num_pages", C.c_int32), ("k_pages_d", C.c_void_p),
+                ("v_pages_d", C.c_void_p)]
+
+
+class DraftCfg(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("K", C.c_int32), ("topk", C.c_int32), ("max_nodes", C.c_int32)]
+
+
+class ExitCfg(C.Structure):
+    _fields_ = [("alpha", C.c_float), ("thr", C.c_float * SX_MAX_SIGNALS),
+                ("dir", C.c_int32 * SX_MAX_SIGNALS), ("enable_mask", C.c_uint32),
+                ("ema_positions", C.c_int32), ("split_bitmap_d", C.c_void_p),
+                ("stop_think_token", C.c_int32)]
+
+
+class ExitState(C.Structure):
+    _fields_ = [("x_d", C.c_void_p), ("n_updates_d", C.c_void_p), ("thinking_d", C.c_void_p)]
+
+
+_ITER_FIELDS = ("cand_tok_d", "parent_d", "depth_d", "slot_row_d", "slot_src_row_d", "hidden_d",
+                "slot_signal_d", "target_tok_d", "accept_len_d", "path_d", "recover_tok_d",
+                "exit_flag_d", "accept_len_out_d", "recover_tok_out_d", "smoothed_d",
+                "tree_cand_tok_d", "tree_cand_score_d", "tree_cand_row_d")
+
+
+class IterOut(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _ITER_FIELDS]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the shared library (built in-tree by ``build.py``).  Raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise SxError(f"{LIB_PATH} is missing: run `python -m paper_2509_24248_b200.build` "
+                      "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, sz = C.c_void_p, C.c_int32, C.c_size_t
+    lib.sx_create.restype = i32
+    lib.sx_create.argtypes = [C.POINTER(ModelCfg), C.POINTER(Weights), i32, C.POINTER(DraftCfg), i32,
+                              C.POINTER(vp)]
+    lib.sx_destroy.restype = None
+    lib.sx_destroy.argtypes = [vp]
+    lib.sx_workspace_bytes.restype = sz
+    lib.sx_workspace_bytes.argtypes = [vp]
+    lib.sx_strerror.restype = C.c_char_p
+    lib.sx_strerror.argtypes = [i32]
+    lib.sx_launch_count.restype = C.c_int64
+    lib.sx_launch_count.argtypes = [vp]
+    lib.sx_draft_step.restype = i32
+    lib.sx_draft_step.argtypes = [vp, C.POINTER(KV), i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.sx_verify.restype = i32
+    lib.sx_verify.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
+    lib.sx_exit_update.restype = i32
+    lib.sx_exit_update.argtypes = [vp, i32, i32, C.POINTER(ExitCfg), C.POINTER(ExitState), vp, vp, vp, i32,
+                                   vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.sx_spec_exit_iter.restype = i32
+    lib.sx_spec_exit_iter.argtypes = [vp, C.POINTER(KV), C.POINTER(ExitCfg), C.POINTER(ExitState), vp, vp,
+                                      vp, C.POINTER(IterOut), vp, sz, vp, vp]
+    lib.sx_spec_exit_iter_host.restype = i32
+    lib.sx_spec_exit_iter_host.argtypes = [vp, C.POINTER(KV), C.POINTER(ExitCfg), C.POINTER(ExitState), vp, vp,
+                                           vp, vp, vp, vp, C.POINTER(IterOut), vp, vp, vp, vp, vp, sz, vp, vp]
+    _lib = lib
+    return lib
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        msg = load_library().sx_strerror(code).decode()
+        raise SxError(f"{what} failed: {msg} ({code})")
+
+
+def _p(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+@dataclass
+class ExitParams:
+    alpha: float = 0.3
+    thr: tuple = (0.9, 0.8, 100.0)
+    dir: tuple = (DIR_GT, DIR_GT, DIR_LT)
+    enable_mask: int = 0b001
+    ema_positions: int = EMA_VERIFIED_CONTEXT
+    split_bitmap: Optional[torch.Tensor] = None     # int32 words on the device, or None
+    stop_think_token: int = 0
+
+    def struct(self) -> ExitCfg:
+        c = ExitCfg()
+        c.alpha = self.alpha
+        for i in range(SX_MAX_SIGNALS):
+            c.thr[i] = self.thr[i]
+            c.dir[i] = self.dir[i]
+        c.enable_mask = self.enable_mask
+        c.ema_positions = self.ema_positions
+        c.split_bitmap_d = _p(self.split_bitmap)
+        c.stop_think_token = self.stop_think_token
+        return c
+
+
+class SpecExit:
+    """One context: weights, KV cache, workspace and output buffers for a workload shape."""
+
+    def __init__(self, shape: synth.ModelShape, weights: Dict[str, torch.Tensor], max_batch: int,
+                 mode: int, K: int, topk: int = 1, max_nodes: int = 0,
+                 act=(ACT_SIGMOID, ACT_SIGMOID, ACT_SIGMOID), device: str = "cuda:0",
+                 max_verify_rows: int = 0):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise SxError("a CUDA device is required (there is no CPU fallback)")
+        self.dev = torch.device(device)
+        torch.cuda.set_device(self.dev)
+        self.shape, self.mode, self.K, self.topk, self.max_nodes = shape, mode, K, topk, max_nodes
+        self.max_batch = max_batch
+        self.rows = K if mode == MODE_CHAIN else 1 + topk * (K - 1)
+        self.P = K + 1 if mode == MODE_CHAIN else 1 + max_nodes
+        self.w = {k: (v.to(self.dev).contiguous() if v.device != self.dev else v) for k, v in weights.items()}
+        if "target_head" not in self.w:
+            self.w["target_head"] = self.w["head"]      # rows [0, V) of the shared head
+        mc = ModelCfg(shape.H, shape.n_q, shape.n_kv, shape.d, shape.F, shape.V, shape.S, shape.eps,
+                      shape.theta, shape.page, (C.c_int32 * 3)(*act))
+        ws = Weights(*[self.w[n].data_ptr() for n in ("embed", "fc", "norm1", "wqkv", "wo", "norm2",
+                                                       "wgate_up", "wdown", "normf", "head", "target_head")])
+        dc = DraftCfg(mode, K, topk, max_nodes)
+        h = C.c_void_p()
+        _check(self.lib.sx_create(C.byref(mc), C.byref(ws), max_batch, C.byref(dc), max_verify_rows,
+                                  C.byref(h)), "sx_create")
+        self.h = h
+        self.ws_bytes = int(self.lib.sx_workspace_bytes(h))
+        self.ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device=self.dev)
+        off = (-self.ws.data_ptr()) % 256
+        self.ws_ptr = self.ws.data_ptr() + off
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        self.kv = None
+        self._kv_struct = None
+
+    def close(self) -> None:
+        if getattr(self, "h", None):
+            self.lib.sx_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- buffers -------------------------------------------------------------------------
+    def set_kv(self, kv: Dict[str, torch.Tensor]) -> None:
+        d = self.dev
+        self.kv = {"k_pages": kv["k_pages"].to(d), "v_pages": kv["v_pages"].to(d),
+                   "page_table": kv["page_table"].to(d).contiguous(),
+                   "cache_len": kv["cache_len"].to(d).contiguous()}
+        B = int(self.kv["cache_len"].numel())
+        self.B = B
+        self._kv_struct = KV(B, self.kv["cache_len"].data_ptr(), self.kv["page_table"].data_ptr(),
+                             int(self.kv["page_table"].shape[1]), int(self.kv["k_pages"].shape[0]),
+                             self.kv["k_pages"].data_ptr(), self.kv["v_pages"].data_ptr())
+
+    def new_state(self, B: int) -> Dict[str, torch.Tensor]:
+        return {"x": torch.zeros(B, self.shape.S, dtype=torch.float32, device=self.dev),
+                "n_updates": torch.zeros(B, dtype=torch.int32, device=self.dev),
+                "thinking": torch.ones(B, dtype=torch.int32, device=self.dev)}
+
+    def new_outputs(self, B: int) -> Dict[str, torch.Tensor]:
+        d, P, S = self.dev, self.P, self.shape.S
+        i32 = lambda *s: torch.full(s, -7, dtype=torch.int32, device=d)
+        NC = max(1, self.topk + (self.K - 1) * self.topk * self.topk)
+        return {"tree_cand_tok_d": i32(B, NC), "tree_cand_row_d": i32(B, NC),
+                "tree_cand_score_d": torch.zeros(B, NC, dtype=torch.float32, device=d),
+                "cand_tok_d": i32(B, P), "parent_d": i32(B, P), "depth_d": i32(B, P),
+                "slot_row_d": i32(B, P), "slot_src_row_d": i32(B, P),
+                "hidden_d": torch.zeros(B, self.rows, self.shape.H, dtype=torch.bfloat16, device=d),
+                "slot_signal_d": torch.full((B, P, S), float("nan"), dtype=torch.float32, device=d),
+                "target_tok_d": i32(B, P), "accept_len_d": i32(B), "path_d": i32(B, self.K + 1),
+                "recover_tok_d": i32(B), "exit_flag_d": i32(B), "accept_len_out_d": i32(B),
+                "recover_tok_out_d": i32(B),
+                "smoothed_d": torch.zeros(B, S, dtype=torch.float32, device=d)}
+
+    @staticmethod
+    def _iter_struct(out: Dict[str, torch.Tensor]) -> IterOut:
+        return IterOut(*[out[n].data_ptr() for n in _ITER_FIELDS])
+
+    @staticmethod
+    def _state_struct(st: Dict[str, torch.Tensor]) -> ExitState:
+        return ExitState(st["x"].data_ptr(), st["n_updates"].data_ptr(), st["thinking"].data_ptr())
+
+    def _stream(self) -> int:
+        return torch.cuda.current_stream(self.dev).cuda_stream
+
+    def check_status(self, what: str = "device") -> None:
+        code = int(self.status.item())
+        if code != 0:
+            self.status.zero_()
+            _check(code, what)
+
+    def launch_count(self) -> int:
+        return int(self.lib.sx_launch_count(self.h))
+
+    # ---- entry points (same names as the C ABI) ------------------------------------------------
+    def sx_draft_step(self, round_: int, feat: torch.Tensor, tok: torch.Tensor,
+                      row_mask: Optional[torch.Tensor] = None):
+        R = int(tok.numel())
+        T = self.topk if self.mode == MODE_TREE else 1
+        hid = torch.empty(R, self.shape.H, dtype=torch.bfloat16, device=self.dev)
+        tok_out = torch.empty(R, T, dtype=torch.int32, device=self.dev)
+        logp = torch.empty(R, T, dtype=torch.float32, device=self.dev)
+        sig = torch.empty(R, self.shape.S, dtype=torch.float32, device=self.dev)
+        _check(self.lib.sx_draft_step(self.h, C.byref(self._kv_struct), round_, R, feat.data_ptr(),
+                                      tok.data_ptr(), _p(row_mask), hid.data_ptr(), tok_out.data_ptr(),
+                                      logp.data_ptr(), sig.data_ptr(), self.ws_ptr, self.ws_bytes,
+                                      self.status.data_ptr(), self._stream()), "sx_draft_step")
+        return hid, tok_out, logp, sig
+
+    def sx_verify(self, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
+                  parent: Optional[torch.Tensor] = None, path_stride: Optional[int] = None):
+        B, P = cand_tok.shape
+        ps = path_stride or (self.K + 1)
+        tt = torch.empty(B, P, dtype=torch.int32, device=self.dev)
+        L = torch.empty(B, dtype=torch.int32, device=self.dev)
+        path = torch.empty(B, ps, dtype=torch.int32, device=self.dev)
+        rec = torch.empty(B, dtype=torch.int32, device=self.dev)
+        _check(self.lib.sx_verify(self.h, B, P, target_hidden.data_ptr(), cand_tok.data_ptr(), _p(parent),
+                                  tt.data_ptr(), L.data_ptr(), path.data_ptr(), ps, rec.data_ptr(),
+                                  self.ws_ptr, self.ws_bytes, self.status.data_ptr(), self._stream()),
+               "sx_verify")
+        return tt, L, path, rec
+
+    def sx_exit_update(self, params: ExitParams, state: Dict[str, torch.Tensor], slot_signal: torch.Tensor,
+                       cand_tok: torch.Tensor, path: torch.Tensor, accept_len: torch.Tensor,
+                       recover_tok: torch.Tensor):
+        B, P = cand_tok.shape
+        ef = torch.empty(B, dtype=torch.int32, device=self.dev)
+        Lo = torch.empty(B, dtype=torch.int32, device=self.dev)
+        ro = torch.empty(B, dtype=torch.int32, device=self.dev)
+        sm = torch.empty(B, self.shape.S, dtype=torch.float32, device=self.dev)
+        cfg, st = params.struct(), self._state_struct(state)
+        _check(self.lib.sx_exit_update(self.h, B, P, C.byref(cfg), C.byref(st), slot_signal.data_ptr(),
+                                       cand_tok.data_ptr(), path.data_ptr(), int(path.shape[1]),
+                                       accept_len.data_ptr(), recover_tok.data_ptr(), ef.data_ptr(),
+                                       Lo.data_ptr(), ro.data_ptr(), sm.data_ptr(), self.status.data_ptr(),
+                                       self._stream()), "sx_exit_update")
+        return ef, Lo, ro, sm
+
+    def sx_spec_exit_iter(self, params: ExitParams, state: Dict[str, torch.Tensor], feat0: torch.Tensor,
+                          tok0: torch.Tensor, target_hidden: torch.Tensor, out: Dict[str, torch.Tensor]) -> None:
+        cfg, st, io = params.struct(), self._state_struct(state), self._iter_struct(out)
+        _check(self.lib.sx_spec_exit_iter(self.h, C.byref(self._kv_struct), C.byref(cfg), C.byref(st),
+                                          feat0.data_ptr(), tok0.data_ptr(), target_hidden.data_ptr(),
+                                          C.byref(io), self.ws_ptr, self.ws_bytes, self.status.data_ptr(),
+                                          self._stream()), "sx_spec_exit_iter")
+
+    def sx_spec_exit_iter_host(self, params: ExitParams, state: Dict[str, torch.Tensor], feat0_h: torch.Tensor,
+                               tok0_h: torch.Tensor, target_hidden_h: torch.Tensor, stage: Dict[str, torch.Tensor],
+                               out: Dict[str, torch.Tensor], res_h: Dict[str, torch.Tensor]) -> None:
+        cfg, st, io = params.struct(), self._state_struct(state), self._iter_struct(out)
+        _check(self.lib.sx_spec_exit_iter_host(
+            self.h, C.byref(self._kv_struct), C.byref(cfg), C.byref(st), feat0_h.data_ptr(), tok0_h.data_ptr(),
+            target_hidden_h.data_ptr(), stage["feat0"].data_ptr(), stage["tok0"].data_ptr(),
+            stage["target_hidden"].data_ptr(), C.byref(io), res_h["accept_len"].data_ptr(),
+            res_h["recover_tok"].data_ptr(), res_h["exit_flag"].data_ptr(), res_h["smoothed"].data_ptr(),
+            self.ws_ptr, self.ws_bytes, self.status.data_ptr(), self._stream()), "sx_spec_exit_iter_host")

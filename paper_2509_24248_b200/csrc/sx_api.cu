@@ -1,0 +1,385 @@
+// Host side of the C ABI: argument checks, workspace carve-up and the launch sequence of one
+// speculative-exit iteration.  Nothing here synchronises or allocates device memory.
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "sx_kernels.cuh"
+
+void sx_gemm_init(int device);
+
+struct sx_ctx {
+  SxShape sh;
+  sx_weights w;
+  sx_draft_cfg dc;
+  int max_batch, Rmax, VR, sm_count, device;
+  int rows_per_seq, P, NC;
+  int64_t launches;
+  int max_splits, part_N, attn_max_splits, head_G, head_rows;
+  // workspace offsets (bytes)
+  size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
+      off_tok_rt, off_logp_rt, off_tree, total;
+  // tree sub-offsets relative to off_tree
+  size_t t_tok, t_par, t_src, t_row, t_score, t_rmask, t_selcid, t_seltok, t_fidx, t_hidx, t_nmask, t_rsig;
+};
+
+static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+extern "C" const char *sx_strerror(sx_status s) {
+  switch (s) {
+    case SX_OK: return "ok";
+    case SX_ERR_INVALID_ARG: return "invalid argument";
+    case SX_ERR_UNSUPPORTED: return "shape or mode not supported";
+    case SX_ERR_CAPACITY: return "page table too short or token id out of range";
+    case SX_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case SX_ERR_CUDA: return "CUDA runtime error";
+    case SX_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+static bool pow2(int v) { return v > 0 && (v & (v - 1)) == 0; }
+
+extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32_t max_batch,
+                               const sx_draft_cfg *dc, int32_t max_verify_rows, sx_ctx **out) {
+  if (!m || !w || !dc || !out || max_batch < 1) return SX_ERR_INVALID_ARG;
+  *out = nullptr;
+  const void *ptrs[] = {w->embed_d, w->fc_d, w->norm1_d, w->wqkv_d, w->wo_d, w->norm2_d,
+                        w->wgate_up_d, w->wdown_d, w->normf_d, w->head_d, w->target_head_d};
+  for (const void *p : ptrs)
+    if (!p || ((uintptr_t)p & 15)) return SX_ERR_INVALID_ARG;
+  if (m->H < 8 || m->H % 8 || m->head_dim % 8 || m->ffn % 8 || !pow2(m->head_dim) || m->head_dim > 256 ||
+      m->head_dim < 8)
+    return SX_ERR_UNSUPPORTED;
+  if (m->n_kv_heads < 1 || m->n_q_heads % m->n_kv_heads) return SX_ERR_UNSUPPORTED;
+  const int G = m->n_q_heads / m->n_kv_heads;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8)) return SX_ERR_UNSUPPORTED;
+  if (m->n_signals < 0 || m->n_signals > SX_MAX_SIGNALS || m->vocab < 1 || m->page_size < 1)
+    return SX_ERR_UNSUPPORTED;
+  if (m->H > 16384) return SX_ERR_UNSUPPORTED;
+  if (dc->K < 1) return SX_ERR_INVALID_ARG;
+  sx_ctx *c = new (std::nothrow) sx_ctx();
+  if (!c) return SX_ERR_INVALID_ARG;
+  memset(c, 0, sizeof(*c));
+  c->sh.H = m->H; c->sh.nq = m->n_q_heads; c->sh.nkv = m->n_kv_heads; c->sh.d = m->head_dim;
+  c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.S = m->n_signals; c->sh.page = m->page_size;
+  c->sh.eps = m->rms_eps; c->sh.theta = m->rope_theta;
+  for (int i = 0; i < SX_MAX_SIGNALS; ++i) c->sh.act[i] = m->act[i];
+  c->w = *w;
+  c->dc = *dc;
+  c->max_batch = max_batch;
+  int T = 1;
+  if (dc->mode == SX_MODE_TREE) {
+    T = dc->topk;
+    c->rows_per_seq = 1 + T * (dc->K - 1);
+    c->P = 1 + dc->max_nodes;
+    c->NC = T + (dc->K - 1) * T * T;
+    if (T < 1 || T > SX_MAX_TOPK || T > m->vocab || c->rows_per_seq > SX_MAX_TREE_ROWS ||
+        c->P > SX_MAX_VERIFY_SLOTS || dc->max_nodes < 1 || dc->max_nodes > c->NC) {
+      delete c;
+      return SX_ERR_UNSUPPORTED;
+    }
+  } else if (dc->mode == SX_MODE_CHAIN) {
+    c->rows_per_seq = dc->K;
+    c->P = dc->K + 1;
+    if (dc->K > SX_MAX_TREE_ROWS - 1) { delete c; return SX_ERR_UNSUPPORTED; }
+  } else {
+    delete c;
+    return SX_ERR_INVALID_ARG;
+  }
+  c->Rmax = max_batch * T;
+  c->VR = max_verify_rows > max_batch * c->P ? max_verify_rows : max_batch * c->P;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete c;
+    return SX_ERR_CUDA;
+  }
+  c->device = dev;
+  c->sm_count = prop.multiProcessorCount;
+  sx_gemm_init(dev);
+
+  const SxShape &s = c->sh;
+  const int R = c->Rmax;
+  c->max_splits = 16;
+  c->part_N = s.H;
+  if ((s.nq + 2 * s.nkv) * s.d > c->part_N) c->part_N = (s.nq + 2 * s.nkv) * s.d;
+  if (2 * s.F > c->part_N) c->part_N = 2 * s.F;
+  c->attn_max_splits = 64;
+  c->head_G = 2 * c->sm_count;
+  c->head_rows = R > 256 ? R : 256;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = up256(o + bytes); return at; };
+  c->off_u = take((size_t)R * 2 * s.H * 2);
+  c->off_x = take((size_t)R * s.H * 2);
+  c->off_n = take((size_t)R * s.H * 2);
+  c->off_q = take((size_t)R * s.nq * s.d * 2);
+  c->off_o = take((size_t)R * s.nq * s.d * 2);
+  c->off_a = take((size_t)R * s.H * 2);
+  c->off_m = take((size_t)R * s.F * 2);
+  c->off_g = take((size_t)R * s.H * 2);
+  c->off_part = take((size_t)c->max_splits * R * c->part_N * 4);
+  c->off_attn = take(sx_attn_ws_bytes(s, R, c->attn_max_splits));
+  c->off_hparts = take((size_t)c->head_G * c->head_rows * sizeof(SxHeadPartial));
+  c->off_z = take((size_t)R * SX_MAX_SIGNALS * 4);
+  c->off_tok_rt = take((size_t)R * SX_MAX_TOPK * 4);
+  c->off_logp_rt = take((size_t)R * SX_MAX_TOPK * 4);
+  c->off_tree = o;
+  if (dc->mode == SX_MODE_TREE) {
+    const size_t B = max_batch, NC = c->NC, rows = c->rows_per_seq;
+    size_t base = o;
+    c->t_tok = take(B * NC * 4) - base;
+    c->t_par = take(B * NC * 4) - base;
+    c->t_src = take(B * NC * 4) - base;
+    c->t_row = take(B * NC * 4) - base;
+    c->t_score = take(B * NC * 4) - base;
+    c->t_rmask = take(B * rows * 8) - base;
+    c->t_selcid = take(B * T * 4) - base;
+    c->t_seltok = take(B * T * 4) - base;
+    c->t_fidx = take(B * T * 4) - base;
+    c->t_hidx = take(B * T * 4) - base;
+    c->t_nmask = take(B * T * 8) - base;
+    c->t_rsig = take(B * rows * SX_MAX_SIGNALS * 4) - base;
+  }
+  c->total = o;
+  *out = c;
+  return SX_OK;
+}
+
+extern "C" void sx_destroy(sx_ctx *c) { delete c; }
+extern "C" size_t sx_workspace_bytes(const sx_ctx *c) { return c ? c->total : 0; }
+extern "C" int64_t sx_launch_count(const sx_ctx *c) { return c ? c->launches : 0; }
+
+static sx_status check_ws(const sx_ctx *c, const void *ws, size_t bytes) {
+  if (!ws || ((uintptr_t)ws & 255) || bytes < c->total) return SX_ERR_WORKSPACE;
+  return SX_OK;
+}
+
+static sx_status check_kv(const sx_ctx *c, const sx_kv *kv) {
+  if (!kv || !kv->cache_len_d || !kv->page_table_d || !kv->k_pages_d || !kv->v_pages_d) return SX_ERR_INVALID_ARG;
+  if (kv->batch < 1 || kv->batch > c->max_batch || kv->max_pages < 1 || kv->num_pages < 1) return SX_ERR_INVALID_ARG;
+  if (((uintptr_t)kv->k_pages_d & 15) || ((uintptr_t)kv->v_pages_d & 15)) return SX_ERR_INVALID_ARG;
+  return SX_OK;
+}
+
+static SxTree tree_view(const sx_ctx *c, char *ws) {
+  SxTree t;
+  char *b = ws + c->off_tree;
+  t.T = c->dc.topk; t.D = c->dc.K; t.rows = c->rows_per_seq; t.NC = c->NC; t.max_nodes = c->dc.max_nodes;
+  t.cand_tok = (int32_t *)(b + c->t_tok); t.cand_parent = (int32_t *)(b + c->t_par);
+  t.cand_src_row = (int32_t *)(b + c->t_src); t.cand_row = (int32_t *)(b + c->t_row);
+  t.cand_score = (float *)(b + c->t_score); t.row_mask = (uint64_t *)(b + c->t_rmask);
+  t.sel_cid = (int32_t *)(b + c->t_selcid); t.sel_tok = (int32_t *)(b + c->t_seltok);
+  t.feat_idx = (int32_t *)(b + c->t_fidx); t.hid_idx = (int32_t *)(b + c->t_hidx);
+  t.next_mask = (uint64_t *)(b + c->t_nmask); t.row_sig = (float *)(b + c->t_rsig);
+  return t;
+}
+
+#define SX_TRY(e) do { sx_status _s = (e); if (_s != SX_OK) return _s; } while (0)
+
+// GEMM + its split-K buffer; returns the split count used
+static sx_status gemm(sx_ctx *c, const void *W, int N, int K, const bf16 *X, int R, char *ws, int *splits,
+                      size_t *stride, int32_t *status, cudaStream_t st) {
+  int sp = sx_gemm_pick_splits(N, K, c->sm_count);
+  if (sp > c->max_splits) sp = c->max_splits;
+  *splits = sp;
+  *stride = (size_t)R * N;
+  c->launches += 1;
+  return sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, status, st);
+}
+
+// head over R rows in chunks the kernel can hold; merges into tok/logp/signals
+static sx_status head(sx_ctx *c, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
+                      char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
+                      int32_t *status, cudaStream_t st) {
+  const int cap = sx_head_max_rows(T);
+  SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
+  float *z = (float *)(ws + c->off_z);
+  for (int r0 = 0; r0 < R; r0 += cap) {
+    const int rc = (R - r0 < cap) ? R - r0 : cap;
+    int G = 0;
+    SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
+                          c->head_rows, &G, z, S, c->sm_count, status, st));
+    SxIndex t2 = toi, s2 = si;
+    if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
+    if (s2.idx) s2.idx += r0; else s2.add += r0 * s2.mul;
+    sx_launch_head_finalize(c->sh, rc, parts, G, c->head_rows, T, lse, z, S, tok_out, t2,
+                            logp_out ? logp_out + (size_t)r0 * T : nullptr, sig_out, s2, st);
+    c->launches += 2;
+  }
+  return SX_OK;
+}
+
+static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const bf16 *feat, SxIndex fi,
+                             const int32_t *tok, SxIndex ti, const uint64_t *row_mask, bf16 *hid_user, SxIndex ui,
+                             int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si, char *ws,
+                             int32_t *status, cudaStream_t st) {
+  const SxShape &s = c->sh;
+  bf16 *u = (bf16 *)(ws + c->off_u), *x = (bf16 *)(ws + c->off_x), *n = (bf16 *)(ws + c->off_n);
+  bf16 *q = (bf16 *)(ws + c->off_q), *o = (bf16 *)(ws + c->off_o), *a = (bf16 *)(ws + c->off_a);
+  bf16 *m = (bf16 *)(ws + c->off_m), *g = (bf16 *)(ws + c->off_g);
+  float *part = (float *)(ws + c->off_part);
+  SxRowMap rm;
+  rm.mode = c->dc.mode; rm.round = round; rm.topk = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1; rm.R = R;
+  rm.cache_len = kv->cache_len_d; rm.row_mask = row_mask;
+  int sp; size_t stride;
+  sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
+  SX_TRY(gemm(c, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
+  sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
+  SX_TRY(gemm(c, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
+  sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st);
+  const int nsplit = sx_attn_splits(s, R, kv->max_pages * s.page, c->sm_count);
+  sx_launch_attention(s, rm, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st);
+  SX_TRY(gemm(c, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
+  sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st);
+  SX_TRY(gemm(c, c->w.wgate_up_d, 2 * s.F, s.H, n, R, ws, &sp, &stride, status, st));
+  sx_launch_finish_swiglu(s, R, part, sp, stride, m, st);
+  SX_TRY(gemm(c, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
+  sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
+  c->launches += 8;   // embed, 3 norms, rope, attention x2, swiglu
+  const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
+  SX_TRY(head(c, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, T > 1 ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
+              status, st));
+  return SX_OK;
+}
+
+extern "C" sx_status sx_draft_step(sx_ctx *c, const sx_kv *kv, int32_t round, int32_t R, const void *feat_d,
+                                   const int32_t *tok_d, const uint64_t *row_mask_d, void *hidden_out_d,
+                                   int32_t *tok_out_d, float *logp_out_d, float *signals_out_d, void *ws_d,
+                                   size_t ws_bytes, int32_t *status_d, void *stream) {
+  if (!c || !feat_d || !tok_d || !hidden_out_d || !tok_out_d || !signals_out_d || !status_d) return SX_ERR_INVALID_ARG;
+  SX_TRY(check_kv(c, kv));
+  SX_TRY(check_ws(c, ws_d, ws_bytes));
+  if (((uintptr_t)feat_d & 15) || ((uintptr_t)hidden_out_d & 15)) return SX_ERR_INVALID_ARG;
+  const bool tree = c->dc.mode == SX_MODE_TREE;
+  if (round < 1 || round > c->dc.K) return SX_ERR_INVALID_ARG;
+  const int expect = (tree && round > 1) ? kv->batch * c->dc.topk : kv->batch;
+  if (R != expect) return SX_ERR_INVALID_ARG;
+  if (tree && round > 1 && !row_mask_d) return SX_ERR_INVALID_ARG;
+  if (tree && !logp_out_d) return SX_ERR_INVALID_ARG;
+  const int T = tree ? c->dc.topk : 1;
+  return draft_round(c, kv, round, R, (const bf16 *)feat_d, SxIndex{nullptr, 1, 0}, tok_d, SxIndex{nullptr, 1, 0},
+                     (tree && round > 1) ? row_mask_d : nullptr, (bf16 *)hidden_out_d, SxIndex{nullptr, 1, 0},
+                     tok_out_d, SxIndex{nullptr, T, 0}, logp_out_d, signals_out_d, SxIndex{nullptr, 1, 0},
+                     (char *)ws_d, status_d, (cudaStream_t)stream);
+}
+
+extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *target_hidden_d,
+                               const int32_t *cand_tok_d, const int32_t *parent_d, int32_t *target_tok_d,
+                               int32_t *accept_len_d, int32_t *path_d, int32_t path_stride, int32_t *recover_tok_d,
+                               void *ws_d, size_t ws_bytes, int32_t *status_d, void *stream) {
+  if (!c || !target_hidden_d || !cand_tok_d || !target_tok_d || !accept_len_d || !path_d || !recover_tok_d || !status_d)
+    return SX_ERR_INVALID_ARG;
+  if (batch < 1 || P < 1 || path_stride < 1 || ((uintptr_t)target_hidden_d & 15)) return SX_ERR_INVALID_ARG;
+  if (parent_d && P > SX_MAX_VERIFY_SLOTS) return SX_ERR_UNSUPPORTED;
+  SX_TRY(check_ws(c, ws_d, ws_bytes));
+  cudaStream_t st = (cudaStream_t)stream;
+  SX_TRY(head(c, c->w.target_head_d, c->sh.V, c->sh.V, 0, (const bf16 *)target_hidden_d, batch * P, 1, 0, (char *)ws_d,
+              target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st));
+  sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st);
+  c->launches += 1;
+  return SX_OK;
+}
+
+extern "C" sx_status sx_exit_update(sx_ctx *c, int32_t batch, int32_t P, const sx_exit_cfg *cfg,
+                                    const sx_exit_state *state, const float *slot_signal_d, const int32_t *cand_tok_d,
+                                    const int32_t *path_d, int32_t path_stride, const int32_t *accept_len_d,
+                                    const int32_t *recover_tok_d, int32_t *exit_flag_d, int32_t *accept_len_out_d,
+                                    int32_t *recover_tok_out_d, float *smoothed_out_d, int32_t *status_d, void *stream) {
+  if (!c || !cfg || !state || !slot_signal_d || !cand_tok_d || !path_d || !accept_len_d || !recover_tok_d ||
+      !exit_flag_d || !accept_len_out_d || !recover_tok_out_d || !smoothed_out_d || !status_d)
+    return SX_ERR_INVALID_ARG;
+  if (!state->x_d || !state->n_updates_d || !state->thinking_d || batch < 1 || P < 1 || path_stride < 1)
+    return SX_ERR_INVALID_ARG;
+  if (!(cfg->alpha >= 0.f && cfg->alpha <= 1.f)) return SX_ERR_INVALID_ARG;
+  sx_launch_exit(batch, P, c->sh.S, *cfg, *state, slot_signal_d, cand_tok_d, path_d, path_stride, accept_len_d,
+                 recover_tok_d, exit_flag_d, accept_len_out_d, recover_tok_out_d, smoothed_out_d, c->sh.V, status_d,
+                 (cudaStream_t)stream);
+  c->launches += 1;
+  return SX_OK;
+}
+
+extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit_cfg *cfg, const sx_exit_state *state,
+                                       const void *feat0_d, const int32_t *tok0_d, const void *target_hidden_d,
+                                       const sx_iter_out *o, void *ws_d, size_t ws_bytes, int32_t *status_d,
+                                       void *stream) {
+  if (!c || !cfg || !state || !feat0_d || !tok0_d || !target_hidden_d || !o || !status_d) return SX_ERR_INVALID_ARG;
+  SX_TRY(check_kv(c, kv));
+  SX_TRY(check_ws(c, ws_d, ws_bytes));
+  if (!o->cand_tok_d || !o->hidden_d || !o->slot_signal_d || !o->target_tok_d || !o->accept_len_d || !o->path_d ||
+      !o->recover_tok_d || !o->exit_flag_d || !o->accept_len_out_d || !o->recover_tok_out_d || !o->smoothed_d)
+    return SX_ERR_INVALID_ARG;
+  if (((uintptr_t)feat0_d & 15) || ((uintptr_t)o->hidden_d & 15) || ((uintptr_t)target_hidden_d & 15))
+    return SX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)ws_d;
+  const int B = kv->batch, K = c->dc.K, P = c->P, S = c->sh.S;
+  bf16 *hid = (bf16 *)o->hidden_d;
+  if (c->dc.mode == SX_MODE_CHAIN) {
+    sx_launch_chain_layout(B, K, S, tok0_d, *o, st);
+    c->launches += 1;
+    for (int k = 1; k <= K; ++k) {
+      const bf16 *feat = (k == 1) ? (const bf16 *)feat0_d : hid;
+      SxIndex fi = (k == 1) ? SxIndex{nullptr, 1, 0} : SxIndex{nullptr, K, k - 2};
+      SX_TRY(draft_round(c, kv, k, B, feat, fi, o->cand_tok_d, SxIndex{nullptr, P, k - 1}, nullptr, hid,
+                         SxIndex{nullptr, K, k - 1}, o->cand_tok_d, SxIndex{nullptr, P, k}, nullptr,
+                         o->slot_signal_d, SxIndex{nullptr, P, k - 1}, ws, status_d, st));
+    }
+    SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
+                     K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+  } else {
+    if (!o->parent_d) return SX_ERR_INVALID_ARG;
+    SxTree t = tree_view(c, ws);
+    if (o->tree_cand_tok_d) t.cand_tok = o->tree_cand_tok_d;
+    if (o->tree_cand_score_d) t.cand_score = o->tree_cand_score_d;
+    if (o->tree_cand_row_d) t.cand_row = o->tree_cand_row_d;
+    const int T = t.T, rows = t.rows;
+    int32_t *tok_rt = (int32_t *)(ws + c->off_tok_rt);
+    float *logp_rt = (float *)(ws + c->off_logp_rt);
+    SX_TRY(draft_round(c, kv, 1, B, (const bf16 *)feat0_d, SxIndex{nullptr, 1, 0}, tok0_d, SxIndex{nullptr, 1, 0},
+                       nullptr, hid, SxIndex{nullptr, rows, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt, t.row_sig,
+                       SxIndex{nullptr, rows, 0}, ws, status_d, st));
+    sx_launch_tree_expand(t, B, 1, tok_rt, logp_rt, st);
+    c->launches += 1;
+    for (int r = 2; r <= K; ++r) {
+      SX_TRY(draft_round(c, kv, r, B * T, hid, SxIndex{t.feat_idx, 0, 0}, t.sel_tok, SxIndex{nullptr, 1, 0},
+                         t.next_mask, hid, SxIndex{t.hid_idx, 0, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt,
+                         t.row_sig, SxIndex{t.hid_idx, 0, 0}, ws, status_d, st));
+      sx_launch_tree_expand(t, B, r, tok_rt, logp_rt, st);
+      c->launches += 1;
+    }
+    sx_launch_tree_layout(t, B, S, tok0_d, *o, st);
+    c->launches += 1;
+    SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, o->parent_d, o->target_tok_d, o->accept_len_d,
+                     o->path_d, K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+  }
+  return sx_exit_update(c, B, P, cfg, state, o->slot_signal_d, o->cand_tok_d, o->path_d, K + 1, o->accept_len_d,
+                        o->recover_tok_d, o->exit_flag_d, o->accept_len_out_d, o->recover_tok_out_d, o->smoothed_d,
+                        status_d, stream);
+}
+
+extern "C" sx_status sx_spec_exit_iter_host(sx_ctx *c, const sx_kv *kv, const sx_exit_cfg *cfg,
+                                            const sx_exit_state *state, const void *feat0_h, const int32_t *tok0_h,
+                                            const void *target_hidden_h, void *stage_feat0_d, int32_t *stage_tok0_d,
+                                            void *stage_target_hidden_d, const sx_iter_out *o,
+                                            int32_t *accept_len_out_h, int32_t *recover_tok_out_h, int32_t *exit_flag_h,
+                                            float *smoothed_h, void *ws_d, size_t ws_bytes, int32_t *status_d,
+                                            void *stream) {
+  if (!c || !kv || !feat0_h || !tok0_h || !target_hidden_h || !stage_feat0_d || !stage_tok0_d ||
+      !stage_target_hidden_d || !o || !accept_len_out_h || !recover_tok_out_h || !exit_flag_h || !smoothed_h)
+    return SX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t B = kv->batch, H = c->sh.H;
+  if (cudaMemcpyAsync(stage_feat0_d, feat0_h, B * H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return SX_ERR_CUDA;
+  if (cudaMemcpyAsync(stage_tok0_d, tok0_h, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return SX_ERR_CUDA;
+  if (cudaMemcpyAsync(stage_target_hidden_d, target_hidden_h, B * c->P * H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return SX_ERR_CUDA;
+  SX_TRY(sx_spec_exit_iter(c, kv, cfg, state, stage_feat0_d, stage_tok0_d, stage_target_hidden_d, o, ws_d, ws_bytes,
+                           status_d, stream));
+  cudaMemcpyAsync(accept_len_out_h, o->accept_len_out_d, B * 4, cudaMemcpyDeviceToHost, st);
+  cudaMemcpyAsync(recover_tok_out_h, o->recover_tok_out_d, B * 4, cudaMemcpyDeviceToHost, st);
+  cudaMemcpyAsync(exit_flag_h, o->exit_flag_d, B * 4, cudaMemcpyDeviceToHost, st);
+  cudaMemcpyAsync(smoothed_h, o->smoothed_d, B * c->sh.S * 4, cudaMemcpyDeviceToHost, st);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return SX_ERR_CUDA;
+  return SX_OK;
+}

@@ -1,0 +1,113 @@
+// Shared device-side helpers and host/device structs of the speculative-exit kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/specexit.h"
+
+typedef __nv_bfloat16 bf16;
+
+#define SX_WARP 32
+#define SX_TILE_M 128          // weight rows per GEMM tile
+#define SX_HEAD_PEND 128       // pending top-k entries per row and tile (= SX_TILE_M)
+
+// How the rows of one draft round map to sequences, positions and cache slots.
+struct SxRowMap {
+  int mode;                    // SX_MODE_*
+  int round;                   // 1-based
+  int topk;
+  int R;                       // rows this round
+  const int32_t *cache_len;    // [B]
+  const uint64_t *row_mask;    // [R] tree rounds >= 2, else nullptr
+};
+
+struct SxRowInfo {
+  int b;          // sequence
+  int n;          // cached prefix length
+  int pos;        // rotary position
+  int rel;        // drafted-row index within the sequence (slot = n + rel)
+  uint64_t mask;  // visible drafted rows (own bit included)
+};
+
+__device__ __forceinline__ SxRowInfo sx_row_info(const SxRowMap &m, int r) {
+  SxRowInfo i;
+  if (m.mode == SX_MODE_CHAIN) {
+    i.b = r;
+    i.rel = m.round - 1;
+    i.mask = (i.rel >= 63) ? ~0ull : ((2ull << i.rel) - 1ull);
+  } else if (m.round == 1) {
+    i.b = r;
+    i.rel = 0;
+    i.mask = 1ull;
+  } else {
+    i.b = r / m.topk;
+    i.rel = 1 + (m.round - 2) * m.topk + (r % m.topk);
+    i.mask = m.row_mask[r];
+  }
+  i.n = m.cache_len[i.b];
+  i.pos = i.n + m.round - 1;
+  return i;
+}
+
+__device__ __forceinline__ void sx_set_status(int32_t *status, int32_t code) {
+  if (status) atomicMin(status, code);
+}
+
+// float -> unsigned key with the same order (NaN sorts above +inf; callers never rank NaN)
+__device__ __forceinline__ uint32_t sx_order_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float sx_key_value(uint32_t k) {
+  uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+  return __uint_as_float(u);
+}
+// (value, index) packed so that a larger value wins and, among equal values, the lower index
+__device__ __forceinline__ unsigned long long sx_pack(float v, uint32_t idx) {
+  return ((unsigned long long)sx_order_key(v) << 32) | (unsigned long long)(0xffffffffu - idx);
+}
+__device__ __forceinline__ float sx_pack_value(unsigned long long p) {
+  return sx_key_value((uint32_t)(p >> 32));
+}
+__device__ __forceinline__ uint32_t sx_pack_index(unsigned long long p) {
+  return 0xffffffffu - (uint32_t)(p & 0xffffffffu);
+}
+
+__device__ __forceinline__ float sx_warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float sx_warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ void sx_unpack8(const uint4 &u, float *f) {
+  const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 t = __bfloat1622float2(p[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+__device__ __forceinline__ float sx_round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+__device__ __forceinline__ float sx_activate(float z, int act) {
+  if (act == SX_ACT_SIGMOID) return 1.0f / (1.0f + expf(-z));
+  if (act == SX_ACT_EXPM1) return expm1f(z);
+  return z;
+}
+
+// ----------------------------------------------------------------------------------------
+// Head epilogue state: per-row running top-T (value, index) and log-sum-exp over the
+// vocabulary rows a CTA has seen.  Lives in shared memory; see sx_head_epilogue.cuh.
+// ----------------------------------------------------------------------------------------
+struct SxHeadPartial {       // what a CTA leaves behind for the merge, per row
+  unsigned long long top[SX_MAX_TOPK];   // packed (value, index), best first; 0 = empty
+  float m, l;                            // running max and sum of exp(v - m)
+};

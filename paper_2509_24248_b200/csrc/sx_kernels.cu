@@ -1,0 +1,660 @@
+// Non-GEMM kernels of the speculative-exit step: input staging, split-K finishers fused with
+// RMSNorm / rotary + KV append / SwiGLU, split-K decode attention over the paged cache, the
+// head merge, greedy acceptance, the exit rule and the draft-tree bookkeeping.
+#include <math.h>
+
+#include "sx_kernels.cuh"
+
+__device__ __forceinline__ int sx_index(const SxIndex &x, int r) { return x.idx ? x.idx[r] : r * x.mul + x.add; }
+
+// ---------------------------------------------------------------------------------------
+// u[r] = [ feature(r) ; E[token(r)] ]   (feature first: fc columns 0..H-1 take the feature)
+// ---------------------------------------------------------------------------------------
+__global__ void sx_embed_concat_kernel(int H, int V, const bf16 *feat, SxIndex fi, const int32_t *tok,
+                                       SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status) {
+  const int r = blockIdx.x;
+  int t = tok[sx_index(ti, r)];
+  if (t < 0 || t >= V) {
+    if (threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY);
+    t = 0;
+  }
+  const uint4 *f = reinterpret_cast<const uint4 *>(feat + (size_t)sx_index(fi, r) * H);
+  const uint4 *e = reinterpret_cast<const uint4 *>(embed + (size_t)t * H);
+  uint4 *o = reinterpret_cast<uint4 *>(u + (size_t)r * 2 * H);
+  const int n = H / 8;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    o[i] = f[i];
+    o[n + i] = e[i];
+  }
+}
+
+void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
+                            SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status, cudaStream_t st) {
+  sx_embed_concat_kernel<<<R, 128, 0, st>>>(sh.H, sh.V, feat, fi, tok, ti, embed, u, status);
+}
+
+// ---------------------------------------------------------------------------------------
+// split-K finisher + RMSNorm
+// ---------------------------------------------------------------------------------------
+__global__ void sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t split_stride,
+                                      const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
+                                      bf16 *out_user, SxIndex ui) {
+  extern __shared__ float sx_buf[];
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    float v = 0.f;
+    for (int s = 0; s < splits; ++s) v += part[s * split_stride + (size_t)r * H + i];
+    if (residual) v += __bfloat162float(residual[(size_t)r * H + i]);
+    const bf16 vb = __float2bfloat16_rn(v);
+    if (out_v) out_v[(size_t)r * H + i] = vb;
+    const float vf = __bfloat162float(vb);
+    sx_buf[i] = vf;
+    ss += vf * vf;
+  }
+  ss = sx_warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    t = sx_warp_sum(t);
+    if (threadIdx.x == 0) red[0] = t;
+  }
+  __syncthreads();
+  const float scale = rsqrtf(red[0] / (float)H + eps);
+  bf16 *user = out_user ? out_user + (size_t)sx_index(ui, r) * H : nullptr;
+  for (int i = threadIdx.x; i < H; i += blockDim.x) {
+    const bf16 nb = __float2bfloat16_rn(sx_buf[i] * scale * __bfloat162float(gamma[i]));
+    if (out_n) out_n[(size_t)r * H + i] = nb;
+    if (user) user[i] = nb;
+  }
+}
+
+void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+                           const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
+                           bf16 *out_user, SxIndex ui, cudaStream_t st) {
+  sx_finish_norm_kernel<<<R, 256, sh.H * sizeof(float), st>>>(sh.H, sh.eps, part, splits, split_stride,
+                                                               residual, gamma, out_v, out_n, out_user, ui);
+}
+
+// ---------------------------------------------------------------------------------------
+// split-K finisher of the QKV projection + rotary (rotate-half pairing) + KV append
+// ---------------------------------------------------------------------------------------
+__global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, SxRowMap rm, const float *part,
+                                          int splits, size_t split_stride, bf16 *q_out, sx_kv kv, int page,
+                                          int32_t *status) {
+  const int r = blockIdx.x;
+  const SxRowInfo ri = sx_row_info(rm, r);
+  const int N = (nq + 2 * nkv) * d;
+  const int half = d / 2;
+  const int slot = ri.n + ri.rel;
+  const int lp = slot / page, off = slot % page;
+  int pp = -1;
+  if (lp < kv.max_pages) pp = kv.page_table_d[(size_t)ri.b * kv.max_pages + lp];
+  const bool can_write = (pp >= 0 && pp < kv.num_pages);
+  if (!can_write && threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY);
+  bf16 *kp = reinterpret_cast<bf16 *>(kv.k_pages_d);
+  bf16 *vp = reinterpret_cast<bf16 *>(kv.v_pages_d);
+  const float *row = part + (size_t)r * N;
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    // the angle needs more than fp32 at positions in the tens of thousands
+    const double inv = exp2(-(2.0 * (double)i / (double)d) * log2(theta));
+    double sn, cs;
+    sincos((double)ri.pos * inv, &sn, &cs);
+    const float c = (float)cs, s = (float)sn;
+    for (int h = 0; h < nq + nkv; ++h) {
+      float x1 = 0.f, x2 = 0.f;
+      for (int sp = 0; sp < splits; ++sp) {
+        x1 += row[sp * split_stride + h * d + i];
+        x2 += row[sp * split_stride + h * d + i + half];
+      }
+      const bf16 y1 = __float2bfloat16_rn(x1 * c - x2 * s);
+      const bf16 y2 = __float2bfloat16_rn(x2 * c + x1 * s);
+      if (h < nq) {
+        q_out[(size_t)r * nq * d + h * d + i] = y1;
+        q_out[(size_t)r * nq * d + h * d + i + half] = y2;
+      } else if (can_write) {
+        const size_t base = (((size_t)pp * nkv + (h - nq)) * page + off) * d;
+        kp[base + i] = y1;
+        kp[base + i + half] = y2;
+      }
+    }
+    if (can_write) {
+      for (int h = 0; h < nkv; ++h) {
+        float v1 = 0.f, v2 = 0.f;
+        for (int sp = 0; sp < splits; ++sp) {
+          v1 += row[sp * split_stride + (nq + nkv + h) * d + i];
+          v2 += row[sp * split_stride + (nq + nkv + h) * d + i + half];
+        }
+        const size_t base = (((size_t)pp * nkv + h) * page + off) * d;
+        vp[base + i] = __float2bfloat16_rn(v1);
+        vp[base + i + half] = __float2bfloat16_rn(v2);
+      }
+    }
+  }
+}
+
+void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
+                               size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
+                               cudaStream_t st) {
+  sx_finish_qkv_rope_kernel<<<rm.R, 128, 0, st>>>(sh.nq, sh.nkv, sh.d, (double)sh.theta, rm, part, splits,
+                                                   split_stride, q_out, kv, sh.page, status);
+}
+
+// ---------------------------------------------------------------------------------------
+// split-K finisher of gate/up + SwiGLU
+// ---------------------------------------------------------------------------------------
+__global__ void sx_finish_swiglu_kernel(int F, const float *part, int splits, size_t split_stride, bf16 *m_out) {
+  const int r = blockIdx.y;
+  const float *row = part + (size_t)r * 2 * F;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < F; i += gridDim.x * blockDim.x) {
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      g += row[s * split_stride + i];
+      u += row[s * split_stride + F + i];
+    }
+    const float si = g / (1.0f + expf(-g));
+    m_out[(size_t)r * F + i] = __float2bfloat16_rn(si * u);
+  }
+}
+
+void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+                             bf16 *m_out, cudaStream_t st) {
+  dim3 grid((sh.F + 1023) / 1024, R);
+  if (grid.x < 1) grid.x = 1;
+  sx_finish_swiglu_kernel<<<grid, 256, 0, st>>>(sh.F, part, splits, split_stride, m_out);
+}
+
+// ---------------------------------------------------------------------------------------
+// split-K decode attention over the paged cache.
+// Block = (split, kv head, row).  A key's head_dim spans d/8 lanes (16-byte loads); a warp
+// works on 32/(d/8) keys at once; the G query heads of the group share every K/V load.
+// The last split also takes the visible drafted rows (slots n + bit).
+// Partials: ws_ml[r][hq][split] = (m, l), ws_o[r][hq][split][d] (unnormalised).
+// ---------------------------------------------------------------------------------------
+template <int G>
+__global__ void sx_attn_split_kernel(int nq, int nkv, int d, int page, float scale, SxRowMap rm, const bf16 *q,
+                                     sx_kv kv, int nsplit, float2 *ws_ml, float *ws_o, int32_t *status) {
+  extern __shared__ float sx_sm[];
+  const int split = blockIdx.x, kvh = blockIdx.y, r = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int lpk = d >> 3;                 // lanes per key
+  const int kpw = 32 / lpk;               // keys per warp step
+  const int grp = lane / lpk, sub = lane % lpk;
+  const SxRowInfo ri = sx_row_info(rm, r);
+  const int n = ri.n;
+  const int chunk = (n + nsplit - 1) / nsplit;
+  const int k0 = split * chunk;
+  const int k1 = min(n, k0 + chunk);
+  const int n_extra = (split == nsplit - 1) ? __popcll(ri.mask) : 0;
+  const int total = max(0, k1 - k0) + n_extra;
+
+  float qf[G][8], acc[G][8], m[G], l[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const uint4 qu = *reinterpret_cast<const uint4 *>(q + ((size_t)r * nq + kvh * G + g) * d + sub * 8);
+    sx_unpack8(qu, qf[g]);
+    m[g] = -INFINITY;
+    l[g] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
+  }
+  const bf16 *kp = reinterpret_cast<const bf16 *>(kv.k_pages_d);
+  const bf16 *vp = reinterpret_cast<const bf16 *>(kv.v_pages_d);
+  const int32_t *table = kv.page_table_d + (size_t)ri.b * kv.max_pages;
+  const int step = 4 * kpw;
+  for (int base = 0; base < total; base += step) {
+    const int t = base + warp * kpw + grp;
+    const bool live = t < total;
+    int slot = 0;
+    if (live) {
+      if (t < k1 - k0) {
+        slot = k0 + t;
+      } else {                                   // the (t - (k1-k0))-th set bit of the mask
+        int want = t - max(0, k1 - k0);
+        uint64_t mm = ri.mask;
+        for (int z = 0; z < want; ++z) mm &= mm - 1;
+        slot = n + (__ffsll((long long)mm) - 1);
+      }
+    }
+    bool ok = live;
+    size_t off = 0;
+    if (live) {
+      const int lp = slot / page;
+      int pp = (lp < kv.max_pages) ? table[lp] : -1;
+      if (pp < 0 || pp >= kv.num_pages) { ok = false; sx_set_status(status, SX_ERR_CAPACITY); }
+      else off = (((size_t)pp * nkv + kvh) * page + (slot % page)) * d + sub * 8;
+    }
+    float kf[8], vf[8];
+    if (ok) {
+      sx_unpack8(*reinterpret_cast<const uint4 *>(kp + off), kf);
+      sx_unpack8(*reinterpret_cast<const uint4 *>(vp + off), vf);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { kf[j] = 0.f; vf[j] = 0.f; }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float s = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s = fmaf(qf[g][j], kf[j], s);
+      for (int o = lpk >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      s *= scale;
+      if (ok) {
+        const float mn = fmaxf(m[g], s);
+        const float corr = __expf(m[g] - mn);
+        const float p = __expf(s - mn);
+        l[g] = l[g] * corr + p;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[g][j] = acc[g][j] * corr + p * vf[j];
+        m[g] = mn;
+      }
+    }
+  }
+  // merge the key groups of a warp, then the warps
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    for (int o = lpk; o < 32; o <<= 1) {
+      const float mo = __shfl_xor_sync(0xffffffffu, m[g], o);
+      const float lo = __shfl_xor_sync(0xffffffffu, l[g], o);
+      const float mn = fmaxf(m[g], mo);
+      const float c0 = (m[g] == -INFINITY) ? 0.f : __expf(m[g] - mn);
+      const float c1 = (mo == -INFINITY) ? 0.f : __expf(mo - mn);
+      l[g] = l[g] * c0 + lo * c1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float ao = __shfl_xor_sync(0xffffffffu, acc[g][j], o);
+        acc[g][j] = acc[g][j] * c0 + ao * c1;
+      }
+      m[g] = mn;
+    }
+  }
+  // shared: [4 warps][G][2 + d]
+  float *sm = sx_sm;
+  const int per = 2 + d;
+  if (grp == 0) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float *dst = sm + ((size_t)warp * G + g) * per;
+      if (sub == 0) { dst[0] = m[g]; dst[1] = l[g]; }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) dst[2 + sub * 8 + j] = acc[g][j];
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < G * d; e += blockDim.x) {
+    const int g = e / d, j = e % d;
+    float mm = -INFINITY;
+    for (int w = 0; w < 4; ++w) mm = fmaxf(mm, sm[((size_t)w * G + g) * per]);
+    float ll = 0.f, a = 0.f;
+    for (int w = 0; w < 4; ++w) {
+      const float *src = sm + ((size_t)w * G + g) * per;
+      const float c = (src[0] == -INFINITY) ? 0.f : __expf(src[0] - mm);
+      ll += src[1] * c;
+      a += src[2 + j] * c;
+    }
+    const size_t hq = (size_t)r * nq + kvh * G + g;
+    ws_o[(hq * nsplit + split) * d + j] = a;
+    if (j == 0) ws_ml[hq * nsplit + split] = make_float2(mm, ll);
+  }
+}
+
+__global__ void sx_attn_combine_kernel(int nq, int d, int nsplit, const float2 *ws_ml, const float *ws_o,
+                                       bf16 *o_out) {
+  const size_t hq = (size_t)blockIdx.y * nq + blockIdx.x;
+  float mm = -INFINITY;
+  for (int s = 0; s < nsplit; ++s) mm = fmaxf(mm, ws_ml[hq * nsplit + s].x);
+  float ll = 0.f;
+  for (int s = 0; s < nsplit; ++s) {
+    const float2 t = ws_ml[hq * nsplit + s];
+    if (t.x != -INFINITY) ll += t.y * __expf(t.x - mm);
+  }
+  for (int j = threadIdx.x; j < d; j += blockDim.x) {
+    float a = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+      const float2 t = ws_ml[hq * nsplit + s];
+      if (t.x != -INFINITY) a += ws_o[(hq * nsplit + s) * d + j] * __expf(t.x - mm);
+    }
+    o_out[hq * d + j] = __float2bfloat16_rn(a / ll);
+  }
+}
+
+int sx_attn_splits(const SxShape &sh, int R, int n_cap, int sm_count) {
+  int want = (4 * sm_count + R * sh.nkv - 1) / (R * sh.nkv);
+  int by_len = (n_cap + 255) / 256;
+  int s = want < by_len ? want : by_len;
+  if (s < 1) s = 1;
+  if (s > 64) s = 64;
+  return s;
+}
+
+size_t sx_attn_ws_bytes(const SxShape &sh, int R, int max_splits) {
+  return (size_t)R * sh.nq * max_splits * (sh.d + 2) * sizeof(float);
+}
+
+void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, const bf16 *q, const sx_kv &kv, int nsplit,
+                         float *ws, bf16 *o_out, int32_t *status, cudaStream_t st) {
+  const int R = rm.R;
+  float2 *ws_ml = reinterpret_cast<float2 *>(ws);
+  float *ws_o = ws + (size_t)R * sh.nq * nsplit * 2;
+  const int G = sh.nq / sh.nkv;
+  dim3 grid(nsplit, sh.nkv, R);
+  const size_t smem = (size_t)4 * G * (2 + sh.d) * sizeof(float);
+  const float scale = 1.0f / sqrtf((float)sh.d);
+#define SX_ATTN(GG)                                                                                          \
+  sx_attn_split_kernel<GG><<<grid, 128, smem, st>>>(sh.nq, sh.nkv, sh.d, sh.page, scale, rm, q, kv, nsplit, \
+                                                    ws_ml, ws_o, status)
+  switch (G) {
+    case 1: SX_ATTN(1); break;
+    case 2: SX_ATTN(2); break;
+    case 4: SX_ATTN(4); break;
+    default: SX_ATTN(8); break;
+  }
+#undef SX_ATTN
+  sx_attn_combine_kernel<<<dim3(sh.nq, R), 64, 0, st>>>(sh.nq, sh.d, nsplit, ws_ml, ws_o, o_out);
+}
+
+// ---------------------------------------------------------------------------------------
+// merge of the per-CTA head results: top-T ids (+ log-probabilities), activated signals
+// ---------------------------------------------------------------------------------------
+__global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
+                                        const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
+                                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si) {
+  extern __shared__ unsigned long long sx_cand[];      // [G * T]
+  __shared__ unsigned long long wbest[4];
+  __shared__ float s_lse;
+  const int r = blockIdx.x, tid = threadIdx.x;
+  for (int i = tid; i < G * T; i += blockDim.x) sx_cand[i] = parts[(size_t)(i / T) * part_stride + r].top[i % T];
+  if (tid == 0 && lse) {
+    float mm = -INFINITY;
+    for (int g = 0; g < G; ++g) mm = fmaxf(mm, parts[(size_t)g * part_stride + r].m);
+    float ll = 0.f;
+    for (int g = 0; g < G; ++g) {
+      const SxHeadPartial &p = parts[(size_t)g * part_stride + r];
+      if (p.l > 0.f) ll += p.l * expf(p.m - mm);
+    }
+    s_lse = mm + logf(ll);
+  }
+  __syncthreads();
+  const int tbase = sx_index(toi, r);
+  for (int t = 0; t < T; ++t) {
+    unsigned long long best = 0ull;
+    for (int i = tid; i < G * T; i += blockDim.x) best = max(best, sx_cand[i]);
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if ((tid & 31) == 0) wbest[tid >> 5] = best;
+    __syncthreads();
+    best = max(max(wbest[0], wbest[1]), max(wbest[2], wbest[3]));
+    if (tid == 0) {
+      tok_out[tbase + t] = (int32_t)sx_pack_index(best);
+      if (logp_out) logp_out[(size_t)r * T + t] = lse ? sx_pack_value(best) - s_lse : sx_pack_value(best);
+    }
+    for (int i = tid; i < G * T; i += blockDim.x)
+      if (sx_cand[i] == best) sx_cand[i] = 0ull;       // packed values are unique (index inside)
+    __syncthreads();
+  }
+  if (sig_out && tid < S) {
+    const int a = tid == 0 ? act0 : (tid == 1 ? act1 : act2);
+    sig_out[(size_t)sx_index(si, r) * S + tid] = sx_activate(z[(size_t)r * S + tid], a);
+  }
+}
+
+void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
+                             int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
+                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st) {
+  sx_head_finalize_kernel<<<R, 128, (size_t)G * T * 8, st>>>(parts, G, part_stride, T, lse, z, S, sh.act[0],
+                                                              sh.act[1], sh.act[2], tok_out, toi, logp_out,
+                                                              sig_out, si);
+}
+
+// ---------------------------------------------------------------------------------------
+// chain layout: slot j holds the j-th draft token; the signal of slot j comes from round j+1
+// ---------------------------------------------------------------------------------------
+__global__ void sx_chain_layout_kernel(int B, int K, int S, const int32_t *tok0, sx_iter_out o) {
+  const int P = K + 1;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= B * P) return;
+  const int b = i / P, j = i % P;
+  if (j == 0) o.cand_tok_d[i] = tok0[b];
+  if (o.parent_d) o.parent_d[i] = j - 1;
+  if (o.depth_d) o.depth_d[i] = j;
+  if (o.slot_row_d) o.slot_row_d[i] = (j < K) ? j : -1;
+  if (o.slot_src_row_d) o.slot_src_row_d[i] = j - 1;
+  if (j == K)
+    for (int s = 0; s < S; ++s) o.slot_signal_d[(size_t)i * S + s] = __int_as_float(0x7fc00000);
+}
+
+void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st) {
+  const int n = B * (K + 1);
+  sx_chain_layout_kernel<<<(n + 127) / 128, 128, 0, st>>>(B, K, S, tok0, o);
+}
+
+// ---------------------------------------------------------------------------------------
+// greedy acceptance (Algorithm 1): chain prefix match, or the walk down the tree
+// ---------------------------------------------------------------------------------------
+__global__ void sx_accept_kernel(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
+                                 int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int32_t *c = cand + (size_t)b * P, *t = target + (size_t)b * P;
+  int32_t *pa = path + (size_t)b * path_stride;
+  int L = 0, cur = 0;
+  pa[0] = 0;
+  if (!parent) {
+    while (L < P - 1 && c[L + 1] == t[L]) { ++L; if (L < path_stride) pa[L] = L; }
+    cur = L;
+  } else {
+    const int32_t *par = parent + (size_t)b * P;
+    for (;;) {
+      int nxt = -1;
+      for (int s = 1; s < P; ++s)
+        if (par[s] == cur && c[s] == t[cur]) { nxt = s; break; }
+      if (nxt < 0) break;
+      cur = nxt;
+      ++L;
+      if (L < path_stride) pa[L] = cur;
+    }
+  }
+  for (int j = L + 1; j < path_stride; ++j) pa[j] = -1;
+  accept_len[b] = L;
+  recover[b] = t[cur];
+}
+
+void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
+                      int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st) {
+  sx_accept_kernel<<<(B + 31) / 32, 32, 0, st>>>(B, P, cand, parent, target, accept_len, path, path_stride,
+                                                 recover);
+}
+
+// ---------------------------------------------------------------------------------------
+// exit rule (Section 3.3, Appendix A.1): EWMA over the accepted slots, AND of the enabled
+// thresholds at the first accepted step-split token
+// ---------------------------------------------------------------------------------------
+struct SxExitParams {
+  float alpha;
+  float thr[SX_MAX_SIGNALS];
+  int dir[SX_MAX_SIGNALS];
+  uint32_t enable;
+  int ema_positions;
+  const uint32_t *bitmap;
+  int stop_tok;
+};
+
+__global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float *x_state, int32_t *n_updates,
+                               int32_t *thinking, const float *slot_signal, const int32_t *cand,
+                               const int32_t *path, int path_stride, const int32_t *accept_len,
+                               const int32_t *recover, int32_t *exit_flag, int32_t *accept_out,
+                               int32_t *recover_out, float *smoothed, int32_t *status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int L = accept_len[b];
+  int flag = 0, Lo = L, ro = recover[b];
+  float x[SX_MAX_SIGNALS];
+  for (int i = 0; i < S; ++i) x[i] = x_state[(size_t)b * S + i];
+  int nu = n_updates[b];
+  if (thinking[b] != 0) {
+    for (int idx = 0; idx <= L && idx < path_stride; ++idx) {
+      const int slot = path[(size_t)b * path_stride + idx];
+      if (slot < 0 || slot >= P) { sx_set_status(status, SX_ERR_INVALID_ARG); break; }
+      const float *sg = slot_signal + ((size_t)b * P + slot) * S;
+      if (p.ema_positions == SX_EMA_VERIFIED_CONTEXT || idx == 0) {
+        bool none = false;
+        for (int i = 0; i < S; ++i) none |= isnan(sg[i]);
+        if (none) break;
+        for (int i = 0; i < S; ++i)
+          x[i] = (nu == 0) ? sg[i]
+                           : (float)((double)p.alpha * (double)sg[i] + (1.0 - (double)p.alpha) * (double)x[i]);
+        ++nu;
+      }
+      const int tok = cand[(size_t)b * P + slot];
+      bool split = true;
+      if (p.bitmap) split = (tok >= 0 && tok < V) ? ((p.bitmap[tok >> 5] >> (tok & 31)) & 1u) : false;
+      bool pass = true;
+      for (int i = 0; i < S; ++i) {
+        if (!((p.enable >> i) & 1u)) continue;
+        pass = pass && ((p.dir[i] == SX_DIR_GT) ? (x[i] > p.thr[i]) : (x[i] < p.thr[i]));
+      }
+      if (split && pass) {
+        flag = 1; Lo = idx; ro = p.stop_tok;
+        thinking[b] = 0;
+        break;
+      }
+    }
+    for (int i = 0; i < S; ++i) x_state[(size_t)b * S + i] = x[i];
+    n_updates[b] = nu;
+  }
+  exit_flag[b] = flag;
+  accept_out[b] = Lo;
+  recover_out[b] = ro;
+  for (int i = 0; i < S; ++i) smoothed[(size_t)b * S + i] = x[i];
+}
+
+void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
+                    const float *slot_signal, const int32_t *cand, const int32_t *path, int path_stride,
+                    const int32_t *accept_len, const int32_t *recover, int32_t *exit_flag,
+                    int32_t *accept_out, int32_t *recover_out, float *smoothed, int V, int32_t *status,
+                    cudaStream_t st) {
+  SxExitParams p;
+  p.alpha = cfg.alpha;
+  for (int i = 0; i < SX_MAX_SIGNALS; ++i) { p.thr[i] = cfg.thr[i]; p.dir[i] = cfg.dir[i]; }
+  p.enable = cfg.enable_mask;
+  p.ema_positions = cfg.ema_positions;
+  p.bitmap = cfg.split_bitmap_d;
+  p.stop_tok = cfg.stop_think_token;
+  sx_exit_kernel<<<(B + 31) / 32, 32, 0, st>>>(B, P, S, V, p, state.x_d, state.n_updates_d, state.thinking_d,
+                                               slot_signal, cand, path, path_stride, accept_len, recover,
+                                               exit_flag, accept_out, recover_out, smoothed, status);
+}
+
+// ---------------------------------------------------------------------------------------
+// draft tree bookkeeping.  Candidate ids follow generation order: depth 1 = [0, T); depth
+// r >= 2 = T + (r-2) T^2 + j T + t for the t-th child of the j-th expanded row.  Score =
+// fp32 sum of log-probabilities; better = higher score, then lower candidate id.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ bool sx_better(float sa, int ia, float sb, int ib) {
+  return sa > sb || (sa == sb && ia < ib);
+}
+
+__global__ void sx_tree_expand_kernel(SxTree t, int round, const int32_t *tok_rt, const float *logp_rt) {
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int T = t.T;
+  int32_t *ctok = t.cand_tok + (size_t)b * t.NC, *cpar = t.cand_parent + (size_t)b * t.NC;
+  int32_t *csrc = t.cand_src_row + (size_t)b * t.NC, *crow = t.cand_row + (size_t)b * t.NC;
+  float *csc = t.cand_score + (size_t)b * t.NC;
+  uint64_t *rmask = t.row_mask + (size_t)b * t.rows;
+  const int cnt = (round == 1) ? T : T * T;
+  const int base = (round == 1) ? 0 : T + (round - 2) * T * T;
+  if (round == 1 && tid == 0) rmask[0] = 1ull;
+  for (int i = tid; i < cnt; i += blockDim.x) {
+    const int j = i / T, tt = i % T;
+    const int rrow = (round == 1) ? b : b * T + j;            // row of this round's launch
+    float ps = 0.f;
+    int pc = -1, src = 0;
+    if (round > 1) {
+      pc = t.sel_cid[b * T + j];
+      ps = csc[pc];
+      src = 1 + (round - 2) * T + j;
+    }
+    ctok[base + i] = tok_rt[(size_t)rrow * T + tt];
+    csc[base + i] = ps + logp_rt[(size_t)rrow * T + tt];
+    cpar[base + i] = pc;
+    csrc[base + i] = src;
+    crow[base + i] = -1;
+  }
+  __syncthreads();
+  if (round >= t.D) return;
+  // choose the T best of this depth for the next round (rank by counting)
+  for (int i = tid; i < cnt; i += blockDim.x) {
+    const float s = csc[base + i];
+    int rank = 0;
+    for (int k = 0; k < cnt; ++k) rank += sx_better(csc[base + k], k, s, i) ? 1 : 0;
+    if (rank < T) {
+      const int cid = base + i;
+      const int rid = 1 + (round - 1) * T + rank;           // drafted row of the next round
+      const int nr = b * T + rank;
+      t.sel_cid[nr] = cid;
+      t.sel_tok[nr] = ctok[cid];
+      t.feat_idx[nr] = b * t.rows + csrc[cid];
+      t.hid_idx[nr] = b * t.rows + rid;
+      const uint64_t mk = rmask[csrc[cid]] | (1ull << rid);
+      t.next_mask[nr] = mk;
+      rmask[rid] = mk;
+      crow[cid] = rid;
+    }
+  }
+}
+
+void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
+                           cudaStream_t st) {
+  sx_tree_expand_kernel<<<B, 64, 0, st>>>(t, round, tok_rt, logp_rt);
+}
+
+__global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_iter_out o) {
+  extern __shared__ int sx_tl[];           // kept[NC], slot_of[NC]
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int NC = t.NC, P = 1 + t.max_nodes, T = t.T;
+  int *kept = sx_tl, *slot_of = sx_tl + NC;
+  const int32_t *ctok = t.cand_tok + (size_t)b * NC, *cpar = t.cand_parent + (size_t)b * NC;
+  const int32_t *csrc = t.cand_src_row + (size_t)b * NC, *crow = t.cand_row + (size_t)b * NC;
+  const float *csc = t.cand_score + (size_t)b * NC;
+  for (int i = tid; i < NC; i += blockDim.x) {
+    const float s = csc[i];
+    int rank = 0;
+    for (int k = 0; k < NC; ++k) rank += sx_better(csc[k], k, s, i) ? 1 : 0;
+    kept[i] = rank < t.max_nodes;
+  }
+  __syncthreads();
+  for (int i = tid; i < NC; i += blockDim.x) {
+    int s = 1;
+    for (int k = 0; k < i; ++k) s += kept[k];
+    slot_of[i] = kept[i] ? s : -1;
+  }
+  __syncthreads();
+  const float qnan = __int_as_float(0x7fc00000);
+  if (tid == 0) {
+    const size_t at = (size_t)b * P;
+    o.cand_tok_d[at] = tok0[b];
+    if (o.parent_d) o.parent_d[at] = -1;
+    if (o.depth_d) o.depth_d[at] = 0;
+    if (o.slot_row_d) o.slot_row_d[at] = 0;
+    if (o.slot_src_row_d) o.slot_src_row_d[at] = -1;
+    for (int s = 0; s < S; ++s) o.slot_signal_d[at * S + s] = t.row_sig[((size_t)b * t.rows) * S + s];
+  }
+  for (int i = tid; i < NC; i += blockDim.x) {
+    if (!kept[i]) continue;
+    const size_t at = (size_t)b * P + slot_of[i];
+    const int depth = (i < T) ? 1 : 2 + (i - T) / (T * T);
+    o.cand_tok_d[at] = ctok[i];
+    if (o.parent_d) o.parent_d[at] = (cpar[i] < 0) ? 0 : slot_of[cpar[i]];
+    if (o.depth_d) o.depth_d[at] = depth;
+    if (o.slot_row_d) o.slot_row_d[at] = crow[i];
+    if (o.slot_src_row_d) o.slot_src_row_d[at] = csrc[i];
+    for (int s = 0; s < S; ++s)
+      o.slot_signal_d[at * S + s] = (crow[i] >= 0) ? t.row_sig[((size_t)b * t.rows + crow[i]) * S + s] : qnan;
+  }
+}
+
+void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
+                           cudaStream_t st) {
+  sx_tree_layout_kernel<<<B, 256, (size_t)2 * t.NC * sizeof(int), st>>>(t, S, tok0, o);
+}

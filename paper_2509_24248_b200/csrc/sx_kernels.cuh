@@ -1,0 +1,81 @@
+// Launch wrappers of the non-GEMM kernels (defined in sx_kernels.cu) and of the GEMMs
+// (sx_gemm.cu).  Host-side only.
+#pragma once
+#include "sx_common.cuh"
+
+// affine-or-indirect row addressing: index(r) = idx ? idx[r] : r * mul + add
+struct SxIndex {
+  const int32_t *idx;
+  int mul, add;
+};
+
+struct SxShape {
+  int H, nq, nkv, d, F, V, S, page;
+  float eps, theta;
+  int act[SX_MAX_SIGNALS];
+};
+
+void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
+                            SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status, cudaStream_t st);
+
+// v = sum_s part[s][r][:] (+ residual); out_v = bf16(v); out_n = bf16(rmsnorm(out_v) * gamma);
+// out_user (optional) receives out_n at row index ui(r).
+void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+                           const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
+                           bf16 *out_user, SxIndex ui, cudaStream_t st);
+
+void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
+                               size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
+                               cudaStream_t st);
+
+void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits,
+                             size_t split_stride, bf16 *m_out, cudaStream_t st);
+
+int sx_attn_splits(const SxShape &sh, int R, int n_cap, int sm_count);
+size_t sx_attn_ws_bytes(const SxShape &sh, int R, int max_splits);
+void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, const bf16 *q, const sx_kv &kv,
+                         int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
+
+void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
+                             int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
+                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st);
+
+void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st);
+
+void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
+                      int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st);
+
+void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
+                    const float *slot_signal, const int32_t *cand, const int32_t *path, int path_stride,
+                    const int32_t *accept_len, const int32_t *recover, int32_t *exit_flag,
+                    int32_t *accept_out, int32_t *recover_out, float *smoothed, int V, int32_t *status,
+                    cudaStream_t st);
+
+// tree bookkeeping state (device, in the workspace), per sequence
+struct SxTree {
+  int T, D, rows, NC, max_nodes;
+  int32_t *cand_tok, *cand_parent, *cand_src_row, *cand_row;   // [B, NC]
+  float *cand_score;                                           // [B, NC]
+  uint64_t *row_mask;                                          // [B, rows]
+  int32_t *sel_cid;                                            // [B, T]
+  int32_t *sel_tok;                                            // [B*T] next round's input tokens
+  int32_t *feat_idx, *hid_idx;                                 // [B*T] next round's row addressing
+  uint64_t *next_mask;                                         // [B*T]
+  float *row_sig;                                              // [B, rows, S]
+};
+void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
+                           cudaStream_t st);
+void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
+                           cudaStream_t st);
+
+// ---- GEMMs (sx_gemm.cu) -------------------------------------------------------------------
+// part[s][r][n] = sum over the s-th K range of X[r][k] * W[n][k]   (fp32)
+struct SxGemmPlan { int splits; };
+int sx_gemm_pick_splits(int N, int K, int sm_count);
+sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part,
+                                 int splits, size_t split_stride, int32_t *status, cudaStream_t st);
+// head: per-CTA partial results out[cta][row]; returns the number of CTAs used in *G
+sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
+                         SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
+                         int32_t *status, cudaStream_t st);
+int sx_head_max_rows(int T);

@@ -1,0 +1,304 @@
+"""GPU-vs-oracle comparison of one speculative-exit iteration.
+
+Rules: draft tokens, tree layout, target tokens, accepted lengths, paths, recover tokens and
+exit flags must match exactly; signals within 1e-2 absolute; hidden states within 2e-2
+relative L2 per row.  The only exemption: a decision whose deciding margin in the oracle is
+below 1e-3 * |largest value| (top-2 logit gap for an argmax, k-th vs (k+1)-th for a top-k,
+score margin for a tree selection).  There the oracle adopts the GPU's choice - after checking
+that it is a valid choice within that margin - so that everything downstream is still compared
+exactly.  Exempt decisions are counted and reported.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List
+
+import torch
+
+from oracle import specexit_oracle as orc
+from paper_2509_24248_b200 import binding, synth
+from tests import harness
+
+REL_GAP = 1e-3
+SIGNAL_ATOL = 1e-2
+HIDDEN_REL_L2 = 2e-2
+
+
+class ParityError(AssertionError):
+    pass
+
+
+@dataclass
+class Report:
+    exempt: List[str] = field(default_factory=list)
+    max_signal_err: float = 0.0
+    max_hidden_rel: float = 0.0
+    accept_len: List[int] = field(default_factory=list)
+    exit_flag: List[int] = field(default_factory=list)
+
+
+def _rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
+    return float((a - b).norm() / b.norm().clamp_min(1e-30))
+
+
+class GpuChooser:
+    """Decision hook for the oracle: keeps the oracle's choice when the GPU agrees, adopts the
+    GPU's when it differs only within the near-tie margin, raises otherwise."""
+
+    def __init__(self, rep: Report, cand_tok=None, tree=None, T=1):
+        self.rep, self.cand_tok, self.tree, self.T = rep, cand_tok, tree, T
+
+    def _children_base(self, row: int) -> int:
+        T = self.T
+        if row == 0:
+            return 0
+        r, j = 2 + (row - 1) // T, (row - 1) % T
+        return T + (r - 2) * T * T + j * T
+
+    def __call__(self, kind, key, values, k, default):
+        if kind == "tok":
+            b, kk = key
+            g = int(self.cand_tok[b, kk])
+            if g == int(default[0]):
+                return default
+            top = float(values.max())
+            if 0 <= g < values.numel() and top - float(values[g]) <= REL_GAP * abs(top):
+                self.rep.exempt.append(f"draft token b={b} k={kk}")
+                return [g]
+            raise ParityError(f"draft token b={b} k={kk}: gpu {g} vs oracle {int(default[0])} "
+                              f"(gap {orc.top_gap(values):.3e})")
+        if kind == "topk":
+            b, row = key
+            base = self._children_base(row)
+            gids = [int(t) for t in self.tree["tok"][b, base:base + k]]
+            if gids == [int(i) for i in default]:
+                return default
+            top = float(values.max())
+            delta = REL_GAP * abs(top)
+            kth = float(values[default[-1]])
+            vals = [float(values[i]) for i in gids]
+            rest = values.clone()
+            rest[gids] = -float("inf")
+            ok = (len(set(gids)) == k and min(vals) >= kth - delta and float(rest.max()) <= min(vals) + delta
+                  and all(vals[i] >= vals[i + 1] - delta for i in range(k - 1)))
+            if ok:
+                self.rep.exempt.append(f"top-{k} b={b} row={row}")
+                return gids
+            raise ParityError(f"top-{k} b={b} row={row}: gpu {gids} vs oracle {list(default)}")
+        if kind in ("expand", "keep"):
+            score = dict(values)
+            if kind == "expand":
+                b, depth = key
+                rows = self.tree["row"][b]
+                gsel = sorted((int(rows[cid]), cid) for cid, _ in values if int(rows[cid]) >= 0)
+                gids = [cid for _, cid in gsel]
+            else:
+                (b,) = key
+                gids = sorted(self.tree["kept"][b])
+            if list(gids) == list(default):
+                return default
+            best = max(abs(s) for s in score.values())
+            delta = REL_GAP * best
+            dset, gset = set(default), set(gids)
+            worst_in = min(score[c] for c in gids)
+            best_out = max([score[c] for c in score if c not in gset], default=-float("inf"))
+            ok = len(gset) == len(dset) and best_out <= worst_in + delta
+            if kind == "expand":
+                sv = [score[c] for c in gids]
+                ok = ok and all(sv[i] >= sv[i + 1] - delta for i in range(len(sv) - 1))
+            if ok:
+                self.rep.exempt.append(f"tree {kind} {key}")
+                return gids
+            raise ParityError(f"tree {kind} {key}: gpu {gids} vs oracle {list(default)}")
+        raise ValueError(kind)
+
+
+def make_gpu(case: harness.Case, act=(0, 0, 0)) -> binding.SpecExit:
+    wl = case.wl
+    sx = binding.SpecExit(wl.shape, case.weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
+                          wl.max_nodes, act=act)
+    sx.set_kv(case.kv)
+    return sx
+
+
+def to_params(sx: binding.SpecExit, cfg: orc.ExitCfg) -> binding.ExitParams:
+    bm = None if cfg.split_bitmap is None else cfg.split_bitmap.to(sx.dev)
+    return binding.ExitParams(alpha=cfg.alpha, thr=tuple(cfg.thr), dir=tuple(cfg.dir),
+                              enable_mask=cfg.enable_mask, ema_positions=cfg.ema_positions,
+                              split_bitmap=bm, stop_think_token=cfg.stop_think_token)
+
+
+def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, parent, slot_signal,
+                  out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int):
+    """verify + exit comparison, shared by chain and tree."""
+    B, P = cand_tok.shape
+    tt, gap = orc.target_argmax(model, th)
+    g_tt = out["target_tok_d"].cpu().to(torch.int64)
+    forced = {}
+    for b in range(B):
+        for j in range(P):
+            if int(g_tt[b, j]) != int(tt[b, j]):
+                if float(gap[b, j]) < REL_GAP:
+                    forced[(b, j)] = int(g_tt[b, j])
+                    rep.exempt.append(f"target token b={b} slot={j}")
+                else:
+                    raise ParityError(f"target token b={b} slot={j}: gpu {int(g_tt[b, j])} vs {int(tt[b, j])} "
+                                      f"gap {float(gap[b, j]):.3e}")
+    v = orc.verify(model, th, cand_tok, parent, forced_target=forced)
+    g_L = out["accept_len_d"].cpu().to(torch.int64)
+    g_path = out["path_d"].cpu().to(torch.int64)
+    g_rec = out["recover_tok_d"].cpu().to(torch.int64)
+    for b in range(B):
+        L = int(v.accept_len[b])
+        if int(g_L[b]) != L:
+            raise ParityError(f"accept_len b={b}: gpu {int(g_L[b])} vs {L}")
+        want = v.path[b] + [-1] * (K + 1 - len(v.path[b]))
+        if g_path[b].tolist() != want:
+            raise ParityError(f"path b={b}: gpu {g_path[b].tolist()} vs {want}")
+        if int(g_rec[b]) != int(v.recover_tok[b]):
+            raise ParityError(f"recover token b={b}")
+        if not 0 <= L <= K:
+            raise ParityError("accept_len out of range")
+    st = state0.clone()
+    e = orc.exit_update(cfg, st, slot_signal, cand_tok, v.path, v.accept_len, v.recover_tok)
+    g_flag = out["exit_flag_d"].cpu().to(torch.int64)
+    g_Lo = out["accept_len_out_d"].cpu().to(torch.int64)
+    g_ro = out["recover_tok_out_d"].cpu().to(torch.int64)
+    g_sm = out["smoothed_d"].cpu().to(torch.float64)
+    for b in range(B):
+        if int(g_flag[b]) != int(e.exit_flag[b]):
+            # a smoothed value within the signal tolerance of its threshold may fall either way
+            near = any(((cfg.enable_mask >> i) & 1) and abs(float(e.smoothed[b, i]) - cfg.thr[i]) < 1e-3
+                       for i in range(slot_signal.shape[2]))
+            if not near:
+                raise ParityError(f"exit flag b={b}: gpu {int(g_flag[b])} vs {int(e.exit_flag[b])}")
+            rep.exempt.append(f"exit flag b={b} (smoothed value at threshold)")
+            continue
+        if int(g_Lo[b]) != int(e.accept_len[b]) or int(g_ro[b]) != int(e.recover_tok[b]):
+            raise ParityError(f"exit outputs b={b}")
+        err = float((g_sm[b] - e.smoothed[b]).abs().max())
+        rep.max_signal_err = max(rep.max_signal_err, err)
+        if err > SIGNAL_ATOL:
+            raise ParityError(f"smoothed signals b={b}: {err}")
+        if int(gstate["thinking"][b]) != int(st.thinking[b]) or int(gstate["n_updates"][b]) != int(st.n_updates[b]):
+            raise ParityError(f"exit state b={b}")
+    rep.accept_len = [int(x) for x in g_Lo]
+    rep.exit_flag = [int(x) for x in g_flag]
+    return v, e
+
+
+def _compare_rows(rep: Report, what: str, g_hid: torch.Tensor, o_hid: torch.Tensor):
+    for i in range(o_hid.shape[0]):
+        rel = _rel_l2(g_hid[i].to(torch.float64), o_hid[i])
+        rep.max_hidden_rel = max(rep.max_hidden_rel, rel)
+        if not rel <= HIDDEN_REL_L2:
+            raise ParityError(f"hidden {what} row {i}: rel L2 {rel}")
+
+
+def _compare_signals(rep: Report, g: torch.Tensor, o: torch.Tensor):
+    gn, on = torch.isnan(g), torch.isnan(o)
+    if not torch.equal(gn, on):
+        raise ParityError("signal NaN pattern (slots never drafted from) differs")
+    err = float((g[~gn].to(torch.float64) - o[~on]).abs().max()) if (~gn).any() else 0.0
+    rep.max_signal_err = max(rep.max_signal_err, err)
+    if err > SIGNAL_ATOL:
+        raise ParityError(f"signals differ by {err}")
+
+
+def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0: orc.ExitState = None,
+              sx: binding.SpecExit = None) -> Report:
+    wl = case.wl
+    rep = Report()
+    cfg = cfg or harness.default_exit_cfg(wl)
+    model = harness.oracle_model(case, act=act)
+    d0 = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    th = harness.chain_target_hidden(case, d0)             # inputs of the verify step, fixed from here
+    own = sx is None
+    sx = sx or make_gpu(case, act)
+    out = sx.new_outputs(wl.B)
+    gst = sx.new_state(wl.B)
+    state0 = state0 or orc.ExitState.fresh(wl.B, wl.shape.S)
+    gst["x"].copy_(state0.x.to(torch.float32))
+    gst["n_updates"].copy_(state0.n_updates.to(torch.int32))
+    gst["thinking"].copy_(state0.thinking.to(torch.int32))
+    sx.sx_spec_exit_iter(to_params(sx, cfg), gst, case.f0.to(sx.dev), case.t0.to(sx.dev), th.to(sx.dev), out)
+    torch.cuda.synchronize()
+    sx.check_status("sx_spec_exit_iter")
+    g_tok = out["cand_tok_d"].cpu().to(torch.int64)
+    chooser = GpuChooser(rep, cand_tok=g_tok)
+    d = d0
+    if not torch.equal(g_tok, d0.cand_tok):
+        d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, chooser=chooser)
+        if not torch.equal(g_tok, d.cand_tok):
+            raise ParityError("draft tokens differ after adopting near-ties")
+    g_hid = out["hidden_d"].cpu()
+    for b in range(wl.B):
+        _compare_rows(rep, f"b={b}", g_hid[b], d.hidden[b])
+    _compare_signals(rep, out["slot_signal_d"].cpu(), d.slot_signal)
+    P = wl.K + 1
+    want_par = torch.arange(-1, wl.K).repeat(wl.B, 1)
+    if not torch.equal(out["parent_d"].cpu().to(torch.int64), want_par):
+        raise ParityError("chain parents")
+    _compare_tail(rep, model, cfg, state0, th, d.cand_tok, None, d.slot_signal, out,
+                  {k: v.cpu() for k, v in gst.items()}, wl.K)
+    if own:
+        sx.close()
+    return rep
+
+
+def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: binding.SpecExit = None) -> Report:
+    wl = case.wl
+    rep = Report()
+    cfg = cfg or harness.default_exit_cfg(wl)
+    model = harness.oracle_model(case, act=act)
+    T, D = wl.topk, wl.K
+    d0 = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes)
+    th = harness.tree_target_hidden(case, d0)
+    own = sx is None
+    sx = sx or make_gpu(case, act)
+    out = sx.new_outputs(wl.B)
+    gst = sx.new_state(wl.B)
+    state0 = orc.ExitState.fresh(wl.B, wl.shape.S)
+    sx.sx_spec_exit_iter(to_params(sx, cfg), gst, case.f0.to(sx.dev), case.t0.to(sx.dev), th.to(sx.dev), out)
+    torch.cuda.synchronize()
+    sx.check_status("sx_spec_exit_iter")
+    o = {k: v.cpu() for k, v in out.items()}
+    # the GPU's kept set as candidate ids: a candidate is identified by (source row, token)
+    NC = T + (D - 1) * T * T
+
+    def src_row(cid):
+        if cid < T:
+            return 0
+        r, j = 2 + (cid - T) // (T * T), ((cid - T) % (T * T)) // T
+        return 1 + (r - 2) * T + j
+
+    kept = []
+    for b in range(wl.B):
+        lut = {(src_row(c), int(o["tree_cand_tok_d"][b, c])): c for c in range(NC)}
+        ks = []
+        for s in range(1, wl.P):
+            key = (int(o["slot_src_row_d"][b, s]), int(o["cand_tok_d"][b, s]))
+            if key not in lut:
+                raise ParityError(f"tree slot b={b} s={s} does not name a generated candidate")
+            ks.append(lut[key])
+        kept.append(ks)
+    chooser = GpuChooser(rep, tree={"tok": o["tree_cand_tok_d"], "row": o["tree_cand_row_d"], "kept": kept}, T=T)
+    d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes, chooser=chooser)
+    for b in range(wl.B):
+        for c in d.cands[b]:
+            if int(o["tree_cand_tok_d"][b, c.cid]) != c.tok or int(o["tree_cand_row_d"][b, c.cid]) != c.row:
+                raise ParityError(f"tree candidate b={b} cid={c.cid}")
+            if abs(float(o["tree_cand_score_d"][b, c.cid]) - c.score) > 1e-3 * max(1.0, abs(c.score)):
+                raise ParityError(f"tree score b={b} cid={c.cid}: {float(o['tree_cand_score_d'][b, c.cid])} vs {c.score}")
+    for name, want in (("cand_tok_d", d.cand_tok), ("parent_d", d.parent), ("depth_d", d.depth),
+                       ("slot_row_d", d.slot_row), ("slot_src_row_d", d.slot_src_row)):
+        if not torch.equal(o[name].to(torch.int64), want):
+            raise ParityError(f"tree layout {name}")
+    for b in range(wl.B):
+        _compare_rows(rep, f"b={b}", o["hidden_d"][b], d.hidden[b])
+    _compare_signals(rep, o["slot_signal_d"], d.slot_signal)
+    _compare_tail(rep, model, cfg, state0, th, d.cand_tok, d.parent, d.slot_signal, out,
+                  {k: v.cpu() for k, v in gst.items()}, wl.K)
+    if own:
+        sx.close()
+    return rep
