@@ -160,8 +160,8 @@ class PagedKV:
             n = self.len[b]
             npg = (n + self.page - 1) // self.page
             pages = self.table[b, :npg].to(torch.int64)
-            kk = self.k[pages].permute(1, 0, 2, 3).reshape(self.k.shape[1], npg * self.page, -1)
-            vv = self.v[pages].permute(1, 0, 2, 3).reshape(self.v.shape[1], npg * self.page, -1)
+            kk = self.k[pages].permute(1, 0, 2, 3).reshape(self.k.shape[1], npg * self.page, self.k.shape[3])
+            vv = self.v[pages].permute(1, 0, 2, 3).reshape(self.v.shape[1], npg * self.page, self.v.shape[3])
             self._prefix[b] = (kk[:, :n].to(F64), vv[:, :n].to(F64))
         return self._prefix[b]
 

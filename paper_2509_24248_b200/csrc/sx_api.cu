@@ -238,7 +238,7 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
   c->launches += 8;   // embed, 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
-  SX_TRY(head(c, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, T > 1 ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
+  SX_TRY(head(c, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
               status, st));
   return SX_OK;
 }
