@@ -1,0 +1,345 @@
+"""Benchmark of the speculative-exit step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C1] [--impl reference]
+
+One step = one whole speculative-exit iteration (all draft rounds, verification, acceptance,
+exit decision) over one batch of synthetic input.  Prints ONE JSON line (rank 0).
+
+value      iterations/s with every input resident in HBM, timed with CUDA events over K steps
+e2e        the same through the host-buffer entry point: pinned host inputs are copied in and
+           the step's results copied out inside the timed region
+roofline   the dominant kernel (extended LM head of a draft round): algorithmic bytes of one
+           launch / its mean duration, against the measured HBM copy bandwidth
+cpu_baseline  the CPU oracle on the same workload (a bounded sample), host cores of this machine
+
+Multi-GPU (torchrun): the path shards by sequence with no exchange step, so every rank runs an
+independent replica of the workload ("weak" scaling); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_24248_b200 import synth  # noqa: E402
+
+METRIC = "spec-exit iterations/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
+    """Bytes one iteration has to move: every weight matrix once per dependent draft round,
+    every live KV byte once per round, the verify head once."""
+    s = wl.shape
+    layer = 2 * s.H * s.H + s.H * s.qkv_rows + s.n_q * s.d * s.H + 3 * s.H * s.F
+    head = (s.V + s.S) * s.H
+    rounds = wl.K
+    w_round = 2 * (layer + head)
+    kv_round = int(sum(int(n) for n in lens)) * s.n_kv * s.d * 2 * 2
+    total = rounds * (w_round + kv_round) + 2 * s.V * s.H
+    return {"total": total, "head_launch": 2 * head, "w_round": w_round, "kv_round": kv_round}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def build_inputs(wl: synth.Workload):
+    lens = synth.cache_lengths(wl)
+    kv = synth.make_kv(wl.shape, lens, wl.draft_rows, wl.seed)
+    weights = synth.make_weights(wl.shape, wl.seed)
+    f0, t0 = synth.make_f0_t0(wl)
+    return lens, kv, weights, f0, t0
+
+
+def run_reference(args, wl):
+    """The CPU oracle as it stands, on this machine's host cores; each step is a bounded sample."""
+    from oracle import specexit_oracle as orc
+    from tests import harness
+    case = harness.build_case(wl, poison_tail=False)
+    model = harness.oracle_model(case)
+    cfg = harness.default_exit_cfg(wl)
+
+    def one():
+        kv = harness.oracle_kv(case)
+        if wl.mode == synth.CHAIN:
+            d = orc.draft_chain(model, kv, case.f0, case.t0, wl.K)
+            th = harness.chain_target_hidden(case, d)
+            v = orc.verify(model, th, d.cand_tok)
+        else:
+            d = orc.draft_tree(model, kv, case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
+            th = harness.tree_target_hidden(case, d)
+            v = orc.verify(model, th, d.cand_tok, d.parent)
+        e = orc.exit_update(cfg, orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path, v.accept_len,
+                            v.recover_tok)
+        return int((e.accept_len + 1).sum())
+
+    for _ in range(args.warmup):
+        one()
+    t0 = time.perf_counter()
+    toks = 0
+    for _ in range(args.steps):
+        toks += one()
+    dt = time.perf_counter() - t0
+    ms = dt / args.steps * 1e3
+    val = 1e3 / ms
+    cores = torch.get_num_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "iterations/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "verified_tokens_per_s": toks / dt,
+            "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree"},
+            "cpu_baseline": {"value": val, "unit": "iterations/s", "cores": cores, "kind": "oracle",
+                             "sample": f"{args.steps} whole iteration(s) of {wl.name} (draft rounds + verify + exit)"},
+            "e2e": {"value": val, "unit": "iterations/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="C1")
+    ap.add_argument("--impl", default="b200")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = synth.workload(args.workload)
+
+    if args.impl == "reference":
+        if rank == 0:
+            if args.steps > 3:
+                args.steps = 3
+            args.warmup = min(args.warmup, 1)
+            run_reference(args, wl)
+        return
+
+    from paper_2509_24248_b200 import binding
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+
+    lens, kv, weights, f0, t0 = build_inputs(wl)
+    sx = binding.SpecExit(wl.shape, weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
+                          wl.max_nodes, device=str(dev))
+    sx.set_kv(kv)
+    del weights
+    P, H, S = wl.P, wl.shape.H, wl.shape.S
+    params = binding.ExitParams(alpha=wl.alpha, thr=(wl.thr, 0.8, 100.0), enable_mask=0b001,
+                                stop_think_token=min(7, wl.shape.V - 1))
+    out = sx.new_outputs(wl.B)
+    state = sx.new_state(wl.B)
+    state0 = {k: v.clone() for k, v in state.items()}
+    f0_d, t0_d = f0.to(dev), t0.to(dev)
+
+    # target hiddens: the draft hiddens of a set-up pass plus the workload's noise (outside the timed region)
+    th_d = torch.zeros(wl.B, P, H, dtype=torch.bfloat16, device=dev)
+    sx.sx_spec_exit_iter(params, state, f0_d, t0_d, th_d, out)
+    torch.cuda.synchronize()
+    sx.check_status("set-up pass")
+    hid = out["hidden_d"].float().cpu()
+    base = torch.empty(wl.B, P, H)
+    if wl.mode == synth.CHAIN:
+        base[:, :wl.K] = hid
+        base[:, wl.K] = hid[:, wl.K - 1]
+    else:
+        row = out["slot_row_d"].cpu().long()
+        src = out["slot_src_row_d"].cpu().long().clamp_min(0)
+        pick = torch.where(row >= 0, row, src)
+        base = torch.gather(hid, 1, pick.unsqueeze(-1).expand(-1, -1, H))
+    th = synth.noisy_hidden(base.to(torch.bfloat16), synth.unit_noise(wl, P), synth.noise_sigmas(wl).view(-1, 1, 1))
+    th_d.copy_(th)
+
+    def reset_state():
+        for k in state:
+            state[k].copy_(state0[k])
+
+    def step():
+        reset_state()
+        sx.sx_spec_exit_iter(params, state, f0_d, t0_d, th_d, out)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    sx.check_status("warm-up")
+
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    launches0 = sx.launch_count()
+    sx.profile_begin()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    verified = torch.zeros((), dtype=torch.int64, device=dev)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+        verified += (out["accept_len_out_d"] + 1).sum()
+    ev1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    prof = sx.profile_end()
+    launches = sx.launch_count() - launches0
+    sx.check_status("timed region")
+    ms_total = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms = ms_total / args.steps
+    value = world * 1e3 / ms
+    vtok = world * float(verified.item()) / (ms_total / 1e3)
+
+    # end to end: host buffers in, results out, through the host entry point
+    stage = {"feat0": torch.empty_like(f0_d), "tok0": torch.empty_like(t0_d), "target_hidden": torch.empty_like(th_d)}
+    f0_h, t0_h, th_h = f0.pin_memory(), t0.pin_memory(), th.pin_memory()
+    res_h = {"accept_len": torch.zeros(wl.B, dtype=torch.int32).pin_memory(),
+             "recover_tok": torch.zeros(wl.B, dtype=torch.int32).pin_memory(),
+             "exit_flag": torch.zeros(wl.B, dtype=torch.int32).pin_memory(),
+             "smoothed": torch.zeros(wl.B, S, dtype=torch.float32).pin_memory()}
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        reset_state()
+        sx.sx_spec_exit_iter_host(params, state, f0_h, t0_h, th_h, stage, out, res_h)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t_start = time.perf_counter()
+    for _ in range(e2e_steps):
+        reset_state()
+        sx.sx_spec_exit_iter_host(params, state, f0_h, t0_h, th_h, stage, out, res_h)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t_start) * 1e3 / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = wl.B * H * 2 + wl.B * 4 + wl.B * P * H * 2
+    d2h = wl.B * (3 * 4 + S * 4)
+
+    if rank != 0:
+        return
+    ab = algorithmic_bytes(wl, lens)
+    peak, peak_kind = measured_peaks()
+    head = prof.get("head_draft", {"ms": None, "n": 0})
+    head_ms = head["ms"] / head["n"] if head["n"] else None
+    achieved = ab["head_launch"] / (head_ms * 1e-3) / 1e9 if head_ms else None
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.txt")
+    if os.path.exists(tp):
+        for line in open(tp):
+            if line.startswith(f"{wl.name}.head_draft.dram_bytes_per_launch="):
+                traffic = float(line.split("=")[1])
+    line = {
+        "metric": METRIC, "value": value, "unit": "iterations/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "verified_tokens_per_s": vtok, "sequence_iterations_per_s": value * wl.B,
+        "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree",
+                   "cached_tokens": int(sum(int(n) for n in lens)),
+                   "l2": "no flush: each iteration streams %.2f GB of weights and KV, far beyond the 126 MB L2"
+                         % (ab["total"] / 1e9)},
+        "step_roofline": {"bytes_per_iteration": ab["total"], "hbm_bound_ms": ab["total"] / (peak * 1e9) * 1e3,
+                          "frac": (ab["total"] / (peak * 1e9) * 1e3) / ms, "peak_gbs": peak, "peak_kind": peak_kind},
+        "roofline": {"kernel": "extended LM head of one draft round", "bound": "hbm", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak if achieved else None,
+                     "traffic": traffic, "launch_ms": head_ms, "peak_kind": peak_kind},
+        "kernel_ms_per_step": {k: (v["ms"] / args.steps) for k, v in prof.items()},
+        "clocks": clocks,
+        "e2e": {"value": world * 1e3 / e2e_ms, "unit": "iterations/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        t1 = time.perf_counter()
+        from oracle import specexit_oracle as orc
+        from tests import harness
+        case = harness.build_case(wl, poison_tail=False)
+        model = harness.oracle_model(case)
+        t2 = time.perf_counter()
+        if wl.mode == synth.CHAIN:
+            d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+            v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok)
+        else:
+            d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
+            v = orc.verify(model, harness.tree_target_hidden(case, d), d.cand_tok, d.parent)
+        orc.exit_update(harness.default_exit_cfg(wl), orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path,
+                        v.accept_len, v.recover_tok)
+        dt = time.perf_counter() - t2
+        line["cpu_baseline"] = {"value": 1.0 / dt, "unit": "iterations/s", "cores": torch.get_num_threads(),
+                                "kind": "oracle", "sample": f"1 whole iteration of {wl.name} ({dt:.1f} s)"}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -229,6 +229,18 @@ sx_status sx_spec_exit_iter_host(sx_ctx *ctx, const sx_kv *kv, const sx_exit_cfg
                                  int32_t *exit_flag_h, float *smoothed_h, void *ws_d,
                                  size_t ws_bytes, int32_t *status_d, void *stream);
 
+/* Per-kernel-class device timing for the benchmark (the paper has no counterpart).  Between
+ * begin and end every launch of the classes below is bracketed by CUDA events on its stream;
+ * sx_profile_end - to be called after the caller has synchronised the stream - returns the
+ * summed milliseconds and the number of launches per class and stops recording. */
+enum {
+  SX_PROF_HEAD_DRAFT = 0, SX_PROF_HEAD_VERIFY = 1, SX_PROF_GEMM_FC = 2, SX_PROF_GEMM_QKV = 3,
+  SX_PROF_GEMM_O = 4, SX_PROF_GEMM_GATE_UP = 5, SX_PROF_GEMM_DOWN = 6, SX_PROF_ATTENTION = 7,
+  SX_PROF_CLASSES = 8
+};
+sx_status sx_profile_begin(sx_ctx *ctx);
+sx_status sx_profile_end(sx_ctx *ctx, float *ms_out, int32_t *count_out);
+
 #ifdef __cplusplus
 }
 #endif

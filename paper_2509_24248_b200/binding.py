@@ -26,7 +26,9 @@ EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
-           "sx_spec_exit_iter_host"]
+           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end"]
+PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
+                "attention"]
 
 
 class SxError(RuntimeError):
@@ -113,6 +115,10 @@ def load_library() -> C.CDLL:
     lib.sx_spec_exit_iter_host.restype = i32
     lib.sx_spec_exit_iter_host.argtypes = [vp, C.POINTER(KV), C.POINTER(ExitCfg), C.POINTER(ExitState), vp, vp,
                                            vp, vp, vp, vp, C.POINTER(IterOut), vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.sx_profile_begin.restype = i32
+    lib.sx_profile_begin.argtypes = [vp]
+    lib.sx_profile_end.restype = i32
+    lib.sx_profile_end.argtypes = [vp, vp, vp]
     _lib = lib
     return lib
 
@@ -248,6 +254,16 @@ class SpecExit:
 
     def launch_count(self) -> int:
         return int(self.lib.sx_launch_count(self.h))
+
+    def profile_begin(self) -> None:
+        _check(self.lib.sx_profile_begin(self.h), "sx_profile_begin")
+
+    def profile_end(self) -> Dict[str, Dict[str, float]]:
+        """Call after synchronising.  Returns {class: {"ms": summed ms, "n": launches}}."""
+        ms = (C.c_float * len(PROF_CLASSES))()
+        n = (C.c_int32 * len(PROF_CLASSES))()
+        _check(self.lib.sx_profile_end(self.h, ms, n), "sx_profile_end")
+        return {name: {"ms": float(ms[i]), "n": int(n[i])} for i, name in enumerate(PROF_CLASSES) if n[i]}
 
     # ---- entry points (same names as the C ABI) ------------------------------------------------
     def sx_draft_step(self, round_: int, feat: torch.Tensor, tok: torch.Tensor,

@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument checks, workspace carve-up and the launch sequence of one
 // speculative-exit iteration.  Nothing here synchronises or allocates device memory.
 #include <new>
+#include <vector>
 #include <stdio.h>
 #include <string.h>
 
@@ -21,7 +22,54 @@ struct sx_ctx {
       off_tok_rt, off_logp_rt, off_tree, total;
   // tree sub-offsets relative to off_tree
   size_t t_tok, t_par, t_src, t_row, t_score, t_rmask, t_selcid, t_seltok, t_fidx, t_hidx, t_nmask, t_rsig;
+  // optional per-class event timing
+  bool prof_on;
+  std::vector<cudaEvent_t> *prof_ev;     // pairs: start, stop
+  std::vector<int> *prof_cls;
+  size_t prof_used;
 };
+
+static void prof_mark(sx_ctx *c, int cls, bool start, cudaStream_t st) {
+  if (!c->prof_on) return;
+  if (start) {
+    if (c->prof_used + 2 > c->prof_ev->size()) {
+      if (c->prof_ev->size() >= 400000) { c->prof_on = false; return; }
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { c->prof_on = false; return; }
+      c->prof_ev->push_back(a);
+      c->prof_ev->push_back(b);
+      c->prof_cls->push_back(cls);
+    } else {
+      (*c->prof_cls)[c->prof_used / 2] = cls;
+    }
+    cudaEventRecord((*c->prof_ev)[c->prof_used], st);
+  } else {
+    cudaEventRecord((*c->prof_ev)[c->prof_used + 1], st);
+    c->prof_used += 2;
+  }
+}
+
+extern "C" sx_status sx_profile_begin(sx_ctx *c) {
+  if (!c) return SX_ERR_INVALID_ARG;
+  c->prof_used = 0;
+  c->prof_on = true;
+  return SX_OK;
+}
+
+extern "C" sx_status sx_profile_end(sx_ctx *c, float *ms_out, int32_t *count_out) {
+  if (!c || !ms_out || !count_out) return SX_ERR_INVALID_ARG;
+  c->prof_on = false;
+  for (int i = 0; i < SX_PROF_CLASSES; ++i) { ms_out[i] = 0.f; count_out[i] = 0; }
+  for (size_t i = 0; i + 1 < c->prof_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, (*c->prof_ev)[i], (*c->prof_ev)[i + 1]) != cudaSuccess) return SX_ERR_CUDA;
+    const int cls = (*c->prof_cls)[i / 2];
+    ms_out[cls] += ms;
+    count_out[cls] += 1;
+  }
+  c->prof_used = 0;
+  return SX_OK;
+}
 
 static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
@@ -61,6 +109,8 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
+  c->prof_ev = new std::vector<cudaEvent_t>();
+  c->prof_cls = new std::vector<int>();
   c->sh.H = m->H; c->sh.nq = m->n_q_heads; c->sh.nkv = m->n_kv_heads; c->sh.d = m->head_dim;
   c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.S = m->n_signals; c->sh.page = m->page_size;
   c->sh.eps = m->rms_eps; c->sh.theta = m->rope_theta;
@@ -146,7 +196,15 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   return SX_OK;
 }
 
-extern "C" void sx_destroy(sx_ctx *c) { delete c; }
+extern "C" void sx_destroy(sx_ctx *c) {
+  if (!c) return;
+  if (c->prof_ev) {
+    for (cudaEvent_t e : *c->prof_ev) cudaEventDestroy(e);
+    delete c->prof_ev;
+    delete c->prof_cls;
+  }
+  delete c;
+}
 extern "C" size_t sx_workspace_bytes(const sx_ctx *c) { return c ? c->total : 0; }
 extern "C" int64_t sx_launch_count(const sx_ctx *c) { return c ? c->launches : 0; }
 
@@ -178,18 +236,21 @@ static SxTree tree_view(const sx_ctx *c, char *ws) {
 #define SX_TRY(e) do { sx_status _s = (e); if (_s != SX_OK) return _s; } while (0)
 
 // GEMM + its split-K buffer; returns the split count used
-static sx_status gemm(sx_ctx *c, const void *W, int N, int K, const bf16 *X, int R, char *ws, int *splits,
+static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf16 *X, int R, char *ws, int *splits,
                       size_t *stride, int32_t *status, cudaStream_t st) {
   int sp = sx_gemm_pick_splits(N, K, c->sm_count);
   if (sp > c->max_splits) sp = c->max_splits;
   *splits = sp;
   *stride = (size_t)R * N;
   c->launches += 1;
-  return sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, status, st);
+  prof_mark(c, cls, true, st);
+  sx_status rc = sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, status, st);
+  prof_mark(c, cls, false, st);
+  return rc;
 }
 
 // head over R rows in chunks the kernel can hold; merges into tok/logp/signals
-static sx_status head(sx_ctx *c, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
+static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
                       int32_t *status, cudaStream_t st) {
   const int cap = sx_head_max_rows(T);
@@ -198,8 +259,10 @@ static sx_status head(sx_ctx *c, const void *W, int Ntot, int V, int S, const bf
   for (int r0 = 0; r0 < R; r0 += cap) {
     const int rc = (R - r0 < cap) ? R - r0 : cap;
     int G = 0;
+    prof_mark(c, cls, true, st);
     SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
                           c->head_rows, &G, z, S, c->sm_count, status, st));
+    prof_mark(c, cls, false, st);
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
     if (s2.idx) s2.idx += r0; else s2.add += r0 * s2.mul;
@@ -224,21 +287,23 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   rm.cache_len = kv->cache_len_d; rm.row_mask = row_mask;
   int sp; size_t stride;
   sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
-  SX_TRY(gemm(c, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
+  SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
-  SX_TRY(gemm(c, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
+  SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
   sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st);
   const int nsplit = sx_attn_splits(s, R, kv->max_pages * s.page, c->sm_count);
+  prof_mark(c, SX_PROF_ATTENTION, true, st);
   sx_launch_attention(s, rm, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st);
-  SX_TRY(gemm(c, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
+  prof_mark(c, SX_PROF_ATTENTION, false, st);
+  SX_TRY(gemm(c, SX_PROF_GEMM_O, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st);
-  SX_TRY(gemm(c, c->w.wgate_up_d, 2 * s.F, s.H, n, R, ws, &sp, &stride, status, st));
+  SX_TRY(gemm(c, SX_PROF_GEMM_GATE_UP, c->w.wgate_up_d, 2 * s.F, s.H, n, R, ws, &sp, &stride, status, st));
   sx_launch_finish_swiglu(s, R, part, sp, stride, m, st);
-  SX_TRY(gemm(c, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
+  SX_TRY(gemm(c, SX_PROF_GEMM_DOWN, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
   c->launches += 8;   // embed, 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
-  SX_TRY(head(c, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
+  SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
               status, st));
   return SX_OK;
 }
@@ -274,7 +339,7 @@ extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *
   if (parent_d && P > SX_MAX_VERIFY_SLOTS) return SX_ERR_UNSUPPORTED;
   SX_TRY(check_ws(c, ws_d, ws_bytes));
   cudaStream_t st = (cudaStream_t)stream;
-  SX_TRY(head(c, c->w.target_head_d, c->sh.V, c->sh.V, 0, (const bf16 *)target_hidden_d, batch * P, 1, 0, (char *)ws_d,
+  SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, c->sh.V, c->sh.V, 0, (const bf16 *)target_hidden_d, batch * P, 1, 0, (char *)ws_d,
               target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st));
   sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st);
   c->launches += 1;
