@@ -224,9 +224,11 @@ class DraftModel:
             out[h] = p @ Vall[kvh]
         return out
 
-    def round(self, kv: PagedKV, rows: List[Row]) -> Tuple[torch.Tensor, HeadOut]:
+    def round(self, kv: PagedKV, rows: List[Row], head_input=None) -> Tuple[torch.Tensor, HeadOut]:
         """One draft pass over ``rows``; appends their K/V to the cache.  Returns the
-        final-normed hidden ``g [R, H]`` (bf16 values) and the head outputs."""
+        final-normed hidden ``g [R, H]`` (bf16 values) and the head outputs.
+        ``head_input(rows, g)`` (replay hook) may name the hidden the head is evaluated on, so
+        that a test can check the head's decisions on another implementation's hidden."""
         sh, w = self.sh, self.w
         R = len(rows)
         toks = torch.tensor([r.tok for r in rows], dtype=torch.int64)
@@ -251,7 +253,7 @@ class DraftModel:
         m = bf16r(silu(gu[:, :sh.F]) * gu[:, sh.F:])
         y = bf16r(a + linear(m, w["wdown"]))
         g = bf16r(rmsnorm(y, w["normf"], sh.eps))
-        return g, self.head(g)
+        return g, self.head(g if head_input is None else head_input(rows, g))
 
 
 # --------------------------------------------------------------------------------------
@@ -268,7 +270,8 @@ class ChainDraft:
 
 
 def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, K: int,
-                forced: Optional[Dict[Tuple[int, int], int]] = None, chooser=None) -> ChainDraft:
+                forced: Optional[Dict[Tuple[int, int], int]] = None, chooser=None,
+                before_round=None, head_input=None) -> ChainDraft:
     """K autoregressive draft rounds per sequence.  ``forced[(b, k)]`` (k = 1..K) replaces
     the k-th draft token of sequence b (used to replay a near-tie the other way);
     ``chooser("tok", (b, k), logits, 1, [tok]) -> [tok]`` may do the same on the fly."""
@@ -281,10 +284,15 @@ def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tens
     gap = torch.empty(B, K, dtype=F64)
     feat = f0.to(F64)
     for k in range(1, K + 1):
+        if before_round is not None and k > 1:
+            # replay hook: lets a test restart round k from another implementation's state
+            # (its previous hidden and the K/V it appended), so that each round is compared
+            # on identical inputs; returns the feature to use
+            feat = before_round(k, kv, feat)
         rows = [Row(b=b, feat=feat[b], tok=int(cand[b, k - 1]), pos=kv.len[b] + k - 1,
                     slot=kv.len[b] + k - 1,
                     visible=[kv.len[b] + j for j in range(k)]) for b in range(B)]
-        g, ho = model.round(kv, rows)
+        g, ho = model.round(kv, rows, head_input)
         for b in range(B):
             tok = argmax_low(ho.logits[b])
             gap[b, k - 1] = top_gap(ho.logits[b])
@@ -331,7 +339,7 @@ class TreeDraft:
 
 def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, depth: int,
                topk: int, max_nodes: int, override: Optional[Dict[Tuple, List[int]]] = None,
-               chooser=None) -> TreeDraft:
+               chooser=None, before_round=None, head_input=None) -> TreeDraft:
     """Tree drafting.  Round 1 drafts the root; round r >= 2 expands the `topk` best
     candidates of depth r-1 (score = sum of log-probabilities; ties: lower candidate id).
     After the last round the `max_nodes` best candidates overall are kept and laid out in
@@ -370,13 +378,16 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
                 visible=[kv.len[b]]) for b in range(B)]
     for b in range(B):
         row_vis[b][0] = [kv.len[b]]
-    g, ho = model.round(kv, rows)
+    g, ho = model.round(kv, rows, head_input)
     for b in range(B):
         hidden[b, 0] = g[b]
         row_sig[b, 0] = ho.s[b]
         emit(b, 0, -1, 0.0, 1, ho.logits[b])
 
     for r in range(2, depth + 1):
+        feat_src = hidden
+        if before_round is not None:
+            feat_src = before_round(r, kv, hidden)   # replay hook, see draft_chain
         rows, owner = [], []
         for b in range(B):
             level = [c for c in cands[b] if c.depth == r - 1]
@@ -399,10 +410,10 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
                 c.row = rid
                 vis = list(row_vis[b][c.src_row]) + [kv.len[b] + rid]
                 row_vis[b][rid] = vis
-                rows.append(Row(b=b, feat=hidden[b, c.src_row], tok=c.tok,
+                rows.append(Row(b=b, feat=feat_src[b, c.src_row], tok=c.tok,
                                 pos=kv.len[b] + r - 1, slot=kv.len[b] + rid, visible=vis))
                 owner.append((b, rid, c))
-        g, ho = model.round(kv, rows)
+        g, ho = model.round(kv, rows, head_input)
         for i, (b, rid, c) in enumerate(owner):
             hidden[b, rid] = g[i]
             row_sig[b, rid] = ho.s[i]

@@ -41,9 +41,8 @@ __global__ void sx_gemm_partial_ref_kernel(const bf16 *W, int N, int K, const bf
   }
 }
 
-int sx_gemm_pick_splits(int N, int K, int sm_count) { return 1; }
 
-sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
+sx_status sx_ref_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
                                  size_t split_stride, int32_t *status, cudaStream_t st) {
   if (splits != 1 || (K % 8) != 0) return SX_ERR_UNSUPPORTED;
   sx_gemm_partial_ref_kernel<<<(N + 3) / 4, 128, 0, st>>>(W, N, K, X, R, part);
@@ -87,13 +86,13 @@ __global__ void sx_head_ref_kernel(const bf16 *W, int Ntot, int V, int K, const 
   sx_head_flush(hs, R, tid, parts + (size_t)blockIdx.x * part_stride);
 }
 
-int sx_head_max_rows(int T) { return SX_REF_RC; }
+int sx_ref_head_max_rows(int T) { return SX_REF_RC; }
 
-void sx_gemm_init(int device) {
+void sx_ref_init(int device) {
   cudaFuncSetAttribute(sx_head_ref_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
 }
 
-sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
+sx_status sx_ref_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
                          int32_t *status, cudaStream_t st) {
   if ((K % 8) != 0 || R > SX_REF_RC) return SX_ERR_UNSUPPORTED;

@@ -1,0 +1,445 @@
+// Skinny GEMMs on the 5th-generation tensor cores (sm_100a): weights stream through a TMA-fed
+// shared-memory ring, tcgen05.mma accumulates into TMEM, the epilogue reads TMEM back.
+//
+//   out[r][n] = sum_k X[r][k] * W[n][k]        W: [n_rows, K] bf16 row-major (K-major)
+//                                              X: [R, K]      bf16 row-major (K-major)
+//
+// The product is formed "swapped": a tile of 128 weight rows is the M side of the MMA, the R
+// token rows (padded to a multiple of 16, at most 256) are the N side, so that a handful of
+// token rows still fills the 128 TMEM lanes.  Every shape this path sees is bound by the weight
+// stream from HBM; the design goal is bytes in flight (deep ring, one persistent CTA per SM),
+// not MMA rate.
+//
+// Warp roles (192 threads): warp 0 = TMA producer (one lane), warp 1 = MMA issuer (one lane,
+// owns the TMEM allocation), warps 2-5 = epilogue (one TMEM lane quarter each).  Two TMEM
+// accumulators let the epilogue of one tile overlap the main loop of the next.
+//
+// Every wait on an mbarrier is bounded; when one runs out the CTA raises SX_ERR_TIMEOUT in the
+// status word, stops issuing work, lets in-flight copies land, frees its TMEM and returns.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <mutex>
+#include <unordered_map>
+
+#include "sx_head_epilogue.cuh"
+#include "sx_kernels.cuh"
+
+#define SX_BK 64                 // K elements per stage (128 bytes: one swizzle row)
+#define SX_A_BYTES (SX_TILE_M * SX_BK * 2)
+#define SX_WAIT_LIMIT (1u << 24)
+#define SX_SMEM_MAX 232448
+
+struct SxTcParams {
+  int n_rows, num_kb, R, nmma, num_tiles, splits, kb_per_split, stages, acc_cols, tmem_cols;
+  float *part;
+  size_t split_stride;
+  int V, S, T, lse, part_stride;
+  SxHeadPartial *parts;
+  float *z;
+  int32_t *status;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// bounded wait; false = gave up (or another role already did)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  for (uint32_t i = 0; i < SX_WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+      : "memory");
+}
+
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_alloc(uint32_t slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 x bf16 -> fp32, M = 128, K = 16
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float *v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart,
+// 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  uint64_t d = (uint64_t)((addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major), 16 B units
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+  d |= (uint64_t)1 << 46;                 // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// barrier over the 128 epilogue threads that also ANDs a flag, so that they all take the same branch
+__device__ __forceinline__ bool epi_all(bool ok) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred pi, po;\n\t"
+      "setp.ne.u32 pi, %1, 0;\n\t"
+      "bar.red.and.pred po, 1, 128, pi;\n\t"
+      "selp.u32 %0, 1, 0, po;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return out != 0;
+}
+
+template <bool HEAD>
+__global__ void __launch_bounds__(192, 1)
+sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, SxTcParams p) {
+  extern __shared__ uint8_t sx_tc_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)sx_tc_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t stage_bytes = SX_A_BYTES + (uint32_t)p.nmma * 128u;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * stage_bytes);
+  uint64_t *full = bars, *empty = bars + p.stages, *tfull = bars + 2 * p.stages, *tempty = tfull + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty + 2);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  uint8_t *epi_smem = reinterpret_cast<uint8_t *>(tmem_slot + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.stages; ++i) {
+      mbar_init(smem_u32(&full[i]), 1);
+      mbar_init(smem_u32(&empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&tfull[i]), 1);
+      mbar_init(smem_u32(&tempty[i]), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tc_alloc(smem_u32(tmem_slot), (uint32_t)p.tmem_cols);
+    tc_relinquish();
+  }
+  SxHeadSmem hs;
+  if (HEAD) {
+    hs = sx_head_carve(epi_smem, p.R, p.T, p.lse);
+    if (warp >= 2) sx_head_init(hs, p.R, threadIdx.x - 64);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int items = HEAD ? p.num_tiles : p.num_tiles * p.splits;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+        const int tile = HEAD ? item : item / p.splits;
+        const int sp = HEAD ? 0 : item % p.splits;
+        const int kb0 = sp * p.kb_per_split;
+        const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = smem_u32(&full[stage]);
+          const uint32_t dst = smem_u32(smem + (size_t)stage * stage_bytes);
+          mbar_expect_tx(fb, stage_bytes);
+          tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
+          tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = nmma, M = 128
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.nmma >> 3) << 17) |
+                             ((uint32_t)(SX_TILE_M >> 4) << 24);
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+        const int sp = HEAD ? 0 : item % p.splits;
+        const int kb0 = sp * p.kb_per_split;
+        const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+        if (!mbar_wait(smem_u32(&tempty[acc]), acc_phase ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.acc_cols);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(smem_u32(&full[stage]), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a = smem_u32(smem + (size_t)stage * stage_bytes);
+          const uint32_t b = a + SX_A_BYTES;
+#pragma unroll
+          for (int k = 0; k < SX_BK / 16; ++k)
+            tc_mma(d_tmem, smem_desc(a + k * 32), smem_desc(b + k * 32), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          tc_commit(smem_u32(&empty[stage]));          // frees the stage once these MMAs have read it
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&tfull[acc]));              // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    const int q = warp & 3;                            // TMEM lane quarter this warp may read
+    const int et = q * 32 + lane;                      // row of the tile owned by this thread
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+      const int tile = HEAD ? item : item / p.splits;
+      const int sp = HEAD ? 0 : item % p.splits;
+      if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
+      const int n = tile * SX_TILE_M + et;
+      for (int c0 = 0; c0 < p.nmma && c0 < p.R; c0 += 16) {
+        float v[16];
+        tc_ld16(taddr + c0, v);
+        if (!HEAD) {
+          if (n < p.n_rows) {
+            float *dst = p.part + (size_t)sp * p.split_stride + n;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (c0 + j < p.R) dst[(size_t)(c0 + j) * p.n_rows] = v[j];
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int r = c0 + j;
+            if (r < p.R) {
+              sx_head_column(hs, r, v[j], (uint32_t)n, n < p.V, q, lane);
+              if (n >= p.V && n < p.V + p.S) p.z[(size_t)r * p.S + (n - p.V)] = v[j];
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tempty[acc]));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      if (HEAD && p.T > 1) {
+        epi_bar();
+        sx_head_merge_pending(hs, p.R, et);
+        epi_bar();
+      }
+    }
+    if (HEAD) {
+      epi_bar();
+      sx_head_flush(hs, p.R, et, p.parts + (size_t)blockIdx.x * p.part_stride);
+    }
+  }
+  if (*abort_flag) {
+    // a wait ran out: report, give copies already in flight time to land, then tear down
+    if (threadIdx.x == 0) sx_set_status(p.status, SX_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+static PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+static std::mutex g_mu;
+struct MapKey {
+  const void *ptr; int rows, cols, box_rows;
+  bool operator==(const MapKey &o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey &k) const {
+    return std::hash<const void *>()(k.ptr) ^ ((size_t)k.rows * 1000003u) ^ ((size_t)k.cols * 7919u) ^ ((size_t)k.box_rows << 48);
+  }
+};
+static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_maps;
+
+static bool get_map(const void *ptr, int rows, int cols, int box_rows, CUtensorMap *out) {
+  std::lock_guard<std::mutex> lk(g_mu);
+  if (!g_encode) {
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) return false;
+    g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  MapKey key{ptr, rows, cols, box_rows};
+  auto it = g_maps.find(key);
+  if (it != g_maps.end()) { *out = it->second; return true; }
+  CUtensorMap m;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {SX_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult rc = g_encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (rc != CUDA_SUCCESS) return false;
+  if (g_maps.size() > 4096) g_maps.clear();
+  g_maps.emplace(key, m);
+  *out = m;
+  return true;
+}
+
+static int pow2_at_least(int v) { int p = 32; while (p < v) p <<= 1; return p; }
+
+static bool fill_common(SxTcParams &p, int n_rows, int K, int R, size_t epi_bytes) {
+  p.n_rows = n_rows;
+  p.num_kb = (K + SX_BK - 1) / SX_BK;
+  p.R = R;
+  p.nmma = ((R + 15) / 16) * 16;
+  if (p.nmma > 256) return false;
+  p.num_tiles = (n_rows + SX_TILE_M - 1) / SX_TILE_M;
+  p.acc_cols = p.nmma;
+  p.tmem_cols = pow2_at_least(2 * p.nmma);
+  const size_t stage_bytes = SX_A_BYTES + (size_t)p.nmma * 128;
+  const size_t fixed = 1024 + 256 + 64 + epi_bytes + 64;
+  int stages = (int)((SX_SMEM_MAX - fixed) / stage_bytes);
+  if (stages > 10) stages = 10;
+  if (stages < 2) return false;
+  p.stages = stages;
+  return true;
+}
+
+static size_t smem_bytes(const SxTcParams &p, size_t epi_bytes) {
+  return 1024 + (size_t)p.stages * (SX_A_BYTES + (size_t)p.nmma * 128) + (size_t)(2 * p.stages + 4) * 8 + 16 + epi_bytes + 64;
+}
+
+void sx_tc_init(int device) {
+  cudaFuncSetAttribute(sx_tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
+  cudaFuncSetAttribute(sx_tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
+}
+
+// Choose the K split: fill the SMs in whole waves, keep at least 4 k-blocks per item.
+int sx_tc_pick_splits(int N, int K, int sm_count) {
+  const int tiles = (N + SX_TILE_M - 1) / SX_TILE_M;
+  const int num_kb = (K + SX_BK - 1) / SX_BK;
+  int best = 1;
+  double best_eff = 0.0;
+  for (int s = 1; s <= 16; ++s) {
+    const int per = (num_kb + s - 1) / s;
+    if (per < 4 && s > 1) break;
+    const int real = (num_kb + per - 1) / per;
+    if (real != s) continue;
+    const int items = tiles * s;
+    const int waves = (items + sm_count - 1) / sm_count;
+    const double eff = (double)items / ((double)waves * sm_count);
+    if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+  }
+  return best;
+}
+
+sx_status sx_tc_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
+                             size_t split_stride, int sm_count, int32_t *status, cudaStream_t st) {
+  if ((K % 8) != 0 || R < 1) return SX_ERR_UNSUPPORTED;
+  for (int r0 = 0; r0 < R; r0 += 256) {
+    const int rc = (R - r0 < 256) ? R - r0 : 256;
+    SxTcParams p;
+    memset(&p, 0, sizeof(p));
+    if (!fill_common(p, N, K, rc, 0)) return SX_ERR_UNSUPPORTED;
+    p.kb_per_split = (p.num_kb + splits - 1) / splits;
+    p.splits = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;
+    if (p.splits != splits) return SX_ERR_INVALID_ARG;
+    p.part = part + (size_t)r0 * N;
+    p.split_stride = split_stride;
+    p.status = status;
+    CUtensorMap mw, mx;
+    if (!get_map(W, N, K, SX_TILE_M, &mw) || !get_map(X + (size_t)r0 * K, rc, K, p.nmma, &mx)) return SX_ERR_CUDA;
+    const int items = p.num_tiles * p.splits;
+    const int grid = items < sm_count ? items : sm_count;
+    sx_tc_gemm_kernel<false><<<grid, 192, smem_bytes(p, 0), st>>>(mw, mx, p);
+  }
+  return SX_OK;
+}
+
+int sx_tc_head_max_rows(int T) { return T > 1 ? 64 : 256; }
+
+sx_status sx_tc_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
+                     SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
+                     cudaStream_t st) {
+  if ((K % 8) != 0 || R < 1 || R > sx_tc_head_max_rows(T)) return SX_ERR_UNSUPPORTED;
+  SxTcParams p;
+  memset(&p, 0, sizeof(p));
+  const size_t epi = sx_head_smem_bytes(R, T, lse);
+  if (!fill_common(p, Ntot, K, R, epi)) return SX_ERR_UNSUPPORTED;
+  p.splits = 1;
+  p.kb_per_split = p.num_kb;
+  p.V = V; p.S = S; p.T = T; p.lse = lse; p.parts = parts; p.part_stride = part_stride; p.z = z; p.status = status;
+  CUtensorMap mw, mx;
+  if (!get_map(W, Ntot, K, SX_TILE_M, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
+  const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
+  sx_tc_gemm_kernel<true><<<grid, 192, smem_bytes(p, epi), st>>>(mw, mx, p);
+  *G = grid;
+  return SX_OK;
+}

@@ -7,6 +7,14 @@ below 1e-3 * |largest value| (top-2 logit gap for an argmax, k-th vs (k+1)-th fo
 score margin for a tree selection).  There the oracle adopts the GPU's choice - after checking
 that it is a valid choice within that margin - so that everything downstream is still compared
 exactly.  Exempt decisions are counted and reported.
+
+How the two runs are lined up.  Each draft round is compared on identical inputs: before round
+k the oracle is handed the GPU's state (its previous hiddens as features, the K/V rows it
+appended), computes its own hidden for the round - compared against the tolerance - and then
+evaluates the head on the GPU's hidden of that row, so that the integer decisions (argmax,
+top-k, everything the tree builds from them) are taken by both sides from the same input in the
+same precision.  A free-running oracle pass is made as well (its hiddens define the target
+hiddens fed to verification, and its drift from the GPU is reported).
 """
 from __future__ import annotations
 
@@ -35,6 +43,8 @@ class Report:
     max_hidden_rel: float = 0.0
     accept_len: List[int] = field(default_factory=list)
     exit_flag: List[int] = field(default_factory=list)
+    free_running_tokens_equal: bool = True
+    free_running_hidden_rel: float = 0.0
 
 
 def _rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
@@ -111,6 +121,21 @@ class GpuChooser:
                 return gids
             raise ParityError(f"tree {kind} {key}: gpu {gids} vs oracle {list(default)}")
         raise ValueError(kind)
+
+
+def _kv_replay(sx: binding.SpecExit, case: harness.Case):
+    """Returns f(kv, rows): copies the K/V the GPU appended for the given drafted rows of every
+    sequence into the oracle's cache."""
+    gk, gv = sx.kv["k_pages"].cpu(), sx.kv["v_pages"].cpu()
+    table, lens, page = case.kv["page_table"], case.kv["cache_len"], case.wl.shape.page
+
+    def f(kv, rows):
+        for b in range(case.wl.B):
+            for i in rows:
+                slot = int(lens[b]) + i
+                pp = int(table[b, slot // page])
+                kv.write(b, slot, gk[pp, :, slot % page], gv[pp, :, slot % page])
+    return f
 
 
 def make_gpu(case: harness.Case, act=(0, 0, 0)) -> binding.SpecExit:
@@ -225,13 +250,32 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     torch.cuda.synchronize()
     sx.check_status("sx_spec_exit_iter")
     g_tok = out["cand_tok_d"].cpu().to(torch.int64)
-    chooser = GpuChooser(rep, cand_tok=g_tok)
-    d = d0
-    if not torch.equal(g_tok, d0.cand_tok):
-        d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, chooser=chooser)
-        if not torch.equal(g_tok, d.cand_tok):
-            raise ParityError("draft tokens differ after adopting near-ties")
     g_hid = out["hidden_d"].cpu()
+    rep.free_running_tokens_equal = bool(torch.equal(g_tok, d0.cand_tok))
+    # Replay: every round of the oracle restarts from the GPU's state (its previous hidden and the
+    # K/V rows it appended), so each round is compared on identical inputs.  Without this the two
+    # runs drift apart round by round: bf16 re-rounding turns summation-order noise into ulp-level
+    # differences within one round, and the feedback through the next round's feature compounds it.
+    chooser = GpuChooser(rep, cand_tok=g_tok)
+    replay = _kv_replay(sx, case)
+
+    def before_round(k, kv, feat):
+        replay(kv, range(0, k - 1))
+        return g_hid[:, k - 2].to(torch.float64)
+
+    lens = [int(n) for n in case.kv["cache_len"]]
+
+    def head_input(rows, g):
+        # decisions of the head are checked on the GPU's own hidden of that row (same precision,
+        # same input); the oracle's hidden is compared separately against the tolerance
+        return torch.stack([g_hid[r.b, r.slot - lens[r.b]].to(torch.float64) for r in rows])
+
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, chooser=chooser,
+                        before_round=before_round, head_input=head_input)
+    if not torch.equal(g_tok, d.cand_tok):
+        raise ParityError("draft tokens differ after adopting near-ties")
+    rep.free_running_hidden_rel = max(_rel_l2(g_hid[b, wl.K - 1].to(torch.float64), d0.hidden[b, wl.K - 1])
+                                      for b in range(wl.B))
     for b in range(wl.B):
         _compare_rows(rep, f"b={b}", g_hid[b], d.hidden[b])
     _compare_signals(rep, out["slot_signal_d"].cpu(), d.slot_signal)
@@ -283,7 +327,23 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
             ks.append(lut[key])
         kept.append(ks)
     chooser = GpuChooser(rep, tree={"tok": o["tree_cand_tok_d"], "row": o["tree_cand_row_d"], "kept": kept}, T=T)
-    d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes, chooser=chooser)
+    replay = _kv_replay(sx, case)
+    g_hid = o["hidden_d"]
+
+    def before_round(r, kv, hidden):
+        done = 1 + (r - 2) * T                    # rows drafted before round r
+        replay(kv, range(0, done))
+        src = hidden.clone()
+        src[:, :done] = g_hid[:, :done].to(torch.float64)
+        return src
+
+    lens = [int(n) for n in case.kv["cache_len"]]
+
+    def head_input(rows, g):
+        return torch.stack([g_hid[r.b, r.slot - lens[r.b]].to(torch.float64) for r in rows])
+
+    d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes, chooser=chooser,
+                       before_round=before_round, head_input=head_input)
     for b in range(wl.B):
         for c in d.cands[b]:
             if int(o["tree_cand_tok_d"][b, c.cid]) != c.tok or int(o["tree_cand_row_d"][b, c.cid]) != c.row:

@@ -1,0 +1,24 @@
+"""Full-size benchmark configurations: CUDA path vs the CPU oracle on the same seeded inputs,
+in the launch configuration bench.py times."""
+import pytest
+
+from paper_2509_24248_b200 import synth
+from tests import harness, parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_chain_config(name):
+    wl = synth.workload(name)
+    rep = parity.run_chain(harness.build_case(wl, poison_tail=True))
+    print(f"{name}: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
+          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
+    assert len(rep.exempt) <= max(2, wl.B * (wl.K + 1) // 10)
+
+
+def test_tree_config4():
+    wl = synth.workload("C4")
+    rep = parity.run_tree(harness.build_case(wl, poison_tail=True))
+    print(f"C4: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
+          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
