@@ -46,7 +46,8 @@ enum {
   SX_ERR_CAPACITY = -3,    /* page table too short / token id out of range (device) */
   SX_ERR_WORKSPACE = -4,
   SX_ERR_CUDA = -5,
-  SX_ERR_TIMEOUT = -6      /* a bounded device-side wait expired */
+  SX_ERR_TIMEOUT = -6,     /* a bounded device-side wait expired */
+  SX_ERR_STATIC_LIMIT = -7 /* request larger than a fixed built-in buffer (sx_verify_noalloc) */
 };
 
 enum { SX_MODE_CHAIN = 0, SX_MODE_TREE = 1 };
@@ -240,6 +241,34 @@ enum {
 };
 sx_status sx_profile_begin(sx_ctx *ctx);
 sx_status sx_profile_end(sx_ctx *ctx, float *ms_out, int32_t *count_out);
+
+/* Verification for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience).  Some hosts of this library hold no allocator at the point
+ * where a draft is verified: an inference server whose memory pool owns the whole device and
+ * hands out fixed buffers only, a plugin called inside a latency-critical section where
+ * cudaMalloc (which may synchronise the device) is off limits, or a process that runs under a
+ * hard memory quota fixed at start-up.  Such a caller has nowhere to put the workspace that
+ * sx_verify wants.  sx_verify_noalloc computes exactly what sx_verify computes - target LM head
+ * with fused argmax over batch * P hidden states, then greedy acceptance - but needs neither a
+ * context nor a workspace: the head kernel's per-CTA partial results live in a fixed array inside
+ * the library image (SX_NOALLOC_SCRATCH_BYTES, about 0.7 MB, held by every GPU that loads the
+ * library until the process exits).  The call allocates and frees no device memory.
+ *   - Limit: batch * P <= SX_NOALLOC_MAX_ROWS; beyond it the call returns SX_ERR_STATIC_LIMIT and
+ *     launches nothing.  Tree mode (parent_d != NULL) also needs P <= SX_MAX_VERIFY_SLOTS.
+ *   - target_head_d is the [vocab, H] bf16 head; the other arguments are those of sx_verify.
+ *   - The first call on a device resolves the array's device address and sets kernel attributes
+ *     for that device (which must be current); make that first call outside any stream capture.
+ *   - All calls on a device share the array and it keeps the previous call's contents.  Nothing
+ *     in it needs clearing (every slice that is read was written by the same call), but two
+ *     calls that overlap on one GPU - different streams or threads - race on it: keep them on
+ *     one stream or order them yourself. */
+#define SX_NOALLOC_MAX_ROWS 64
+#define SX_NOALLOC_SCRATCH_BYTES (160 * SX_NOALLOC_MAX_ROWS * (8 * SX_MAX_TOPK + 8))
+sx_status sx_verify_noalloc(const void *target_head_d, int32_t vocab, int32_t H, int32_t batch,
+                            int32_t P, const void *target_hidden_d, const int32_t *cand_tok_d,
+                            const int32_t *parent_d, int32_t *target_tok_d, int32_t *accept_len_d,
+                            int32_t *path_d, int32_t path_stride, int32_t *recover_tok_d,
+                            int32_t *status_d, void *stream);
 
 #ifdef __cplusplus
 }

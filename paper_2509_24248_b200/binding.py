@@ -26,7 +26,7 @@ EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
-           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end"]
+           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -119,6 +119,8 @@ def load_library() -> C.CDLL:
     lib.sx_profile_begin.argtypes = [vp]
     lib.sx_profile_end.restype = i32
     lib.sx_profile_end.argtypes = [vp, vp, vp]
+    lib.sx_verify_noalloc.restype = i32
+    lib.sx_verify_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -154,6 +156,26 @@ class ExitParams:
         c.split_bitmap_d = _p(self.split_bitmap)
         c.stop_think_token = self.stop_think_token
         return c
+
+
+NOALLOC_MAX_ROWS = 64
+
+
+def sx_verify_noalloc(target_head: torch.Tensor, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
+                      parent: Optional[torch.Tensor], out: Dict[str, torch.Tensor], status: torch.Tensor) -> None:
+    """Verification without a context or a workspace, for callers that may not allocate device
+    memory: every buffer, results included, is handed in by the caller (``out`` holds
+    ``target_tok [B,P]``, ``accept_len [B]``, ``path [B,stride]`` and ``recover_tok [B]``, all
+    int32 on the device) and the library's scratch is a fixed array inside its own image.  At most
+    ``NOALLOC_MAX_ROWS`` hidden states (B * P) per call; calls on one device share the scratch,
+    so keep them on one stream."""
+    lib = load_library()
+    B, P = cand_tok.shape
+    V, H = target_head.shape
+    _check(lib.sx_verify_noalloc(target_head.data_ptr(), V, H, B, P, target_hidden.data_ptr(), cand_tok.data_ptr(),
+                                 _p(parent), out["target_tok"].data_ptr(), out["accept_len"].data_ptr(),
+                                 out["path"].data_ptr(), int(out["path"].shape[1]), out["recover_tok"].data_ptr(),
+                                 status.data_ptr(), torch.cuda.current_stream().cuda_stream), "sx_verify_noalloc")
 
 
 class SpecExit:

@@ -82,6 +82,7 @@ extern "C" const char *sx_strerror(sx_status s) {
     case SX_ERR_WORKSPACE: return "workspace too small or misaligned";
     case SX_ERR_CUDA: return "CUDA runtime error";
     case SX_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case SX_ERR_STATIC_LIMIT: return "request exceeds the fixed built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -21,9 +21,9 @@
 
 void sx_gemm_init(int device);
 
-#define SX_NOALLOC_MAX_ROWS 64      // batch * P accepted by sx_verify_noalloc
 #define SX_NOALLOC_MAX_CTAS 160     // CTAs of the head kernel that may leave a partial result
-#define SX_NOALLOC_SCRATCH_BYTES (SX_NOALLOC_MAX_CTAS * SX_NOALLOC_MAX_ROWS * sizeof(SxHeadPartial))
+static_assert(SX_NOALLOC_SCRATCH_BYTES == SX_NOALLOC_MAX_CTAS * SX_NOALLOC_MAX_ROWS * sizeof(SxHeadPartial),
+              "the header's SX_NOALLOC_SCRATCH_BYTES must match the partial-result record");
 
 // In host code this name is only a handle for the runtime, never a device address: the address
 // comes from cudaGetSymbolAddress, once per device.
