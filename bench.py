@@ -65,11 +65,25 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        self.t0 = self.t1 = None
+
+    def wait_ready(self, timeout: float = 10.0):
+        """nvidia-smi takes a second or two to start and perturbs launches while it does; the timed
+        region begins only after its first sample has arrived."""
+        t = time.time()
+        while self.proc is not None and not self.rows and time.time() - t < timeout:
+            time.sleep(0.05)
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -78,7 +92,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -90,7 +104,10 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], None, set()
-        for r in self.rows:
+        inside = [r for (t, r) in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t) + 0.1]
+        if not inside:                      # region shorter than the sampling period: nearest samples
+            inside = [r for (_, r) in self.rows[-2:]]
+        for r in inside:
             try:
                 sm.append(float(r[0]))
                 mx = float(r[1])
@@ -157,12 +174,11 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="C1")
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -225,16 +241,18 @@ def main():
         reset_state()
         sx.sx_spec_exit_iter(params, state, f0_d, t0_d, th_d, out)
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(max(3, args.warmup)):
         step()
     torch.cuda.synchronize()
     sx.check_status("warm-up")
+    sampler.wait_ready()
 
-    sampler = ClockSampler(local)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    sampler.mark_begin()
     launches0 = sx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     verified = torch.zeros((), dtype=torch.int64, device=dev)
@@ -244,6 +262,7 @@ def main():
         verified += (out["accept_len_out_d"] + 1).sum()
     ev1.record()
     torch.cuda.synchronize()
+    sampler.mark_end()
     if dist is not None:
         dist.barrier()
     launches = sx.launch_count() - launches0
@@ -273,7 +292,7 @@ def main():
              "recover_tok": torch.zeros(wl.B, dtype=torch.int32).pin_memory(),
              "exit_flag": torch.zeros(wl.B, dtype=torch.int32).pin_memory(),
              "smoothed": torch.zeros(wl.B, S, dtype=torch.float32).pin_memory()}
-    e2e_steps = max(3, min(args.steps, 50))
+    e2e_steps = max(3, min(args.steps, 200))
     for _ in range(3):
         reset_state()
         sx.sx_spec_exit_iter_host(params, state, f0_h, t0_h, th_h, stage, out, res_h)

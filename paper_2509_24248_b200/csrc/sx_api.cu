@@ -7,8 +7,6 @@
 
 #include "sx_kernels.cuh"
 
-void sx_gemm_init(int device);
-
 struct sx_ctx {
   SxShape sh;
   sx_weights w;
@@ -16,7 +14,7 @@ struct sx_ctx {
   int max_batch, Rmax, VR, sm_count, device;
   int rows_per_seq, P, NC;
   int64_t launches;
-  int max_splits, part_N, attn_max_splits, head_G, head_rows;
+  int max_splits, part_N, head_G, head_rows;
   // workspace offsets (bytes)
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
       off_tok_rt, off_logp_rt, off_tree, total;
@@ -106,6 +104,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (m->n_signals < 0 || m->n_signals > SX_MAX_SIGNALS || m->vocab < 1 || m->page_size < 1)
     return SX_ERR_UNSUPPORTED;
   if (m->H > 16384) return SX_ERR_UNSUPPORTED;
+  if (!(m->head_dim == 16 || m->head_dim == 32 || m->head_dim == 64 || m->head_dim == 128)) return SX_ERR_UNSUPPORTED;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
@@ -156,7 +155,6 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->part_N = s.H;
   if ((s.nq + 2 * s.nkv) * s.d > c->part_N) c->part_N = (s.nq + 2 * s.nkv) * s.d;
   if (2 * s.F > c->part_N) c->part_N = 2 * s.F;
-  c->attn_max_splits = 64;
   c->head_G = 2 * c->sm_count;
   c->head_rows = R > 256 ? R : 256;
   size_t o = 0;
@@ -170,7 +168,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->off_m = take((size_t)R * s.F * 2);
   c->off_g = take((size_t)R * s.H * 2);
   c->off_part = take((size_t)c->max_splits * R * c->part_N * 4);
-  c->off_attn = take(sx_attn_ws_bytes(s, R, c->attn_max_splits));
+  c->off_attn = take(sx_attn_ws_bytes(s, max_batch, T, c->sm_count));
   c->off_hparts = take((size_t)c->head_G * c->head_rows * sizeof(SxHeadPartial));
   c->off_z = take((size_t)R * SX_MAX_SIGNALS * 4);
   c->off_tok_rt = take((size_t)R * SX_MAX_TOPK * 4);
@@ -245,7 +243,7 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
   *stride = (size_t)R * N;
   c->launches += 1;
   prof_mark(c, cls, true, st);
-  sx_status rc = sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, status, st);
+  sx_status rc = sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, c->sm_count, status, st);
   prof_mark(c, cls, false, st);
   return rc;
 }
@@ -292,9 +290,11 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
   sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st);
-  const int nsplit = sx_attn_splits(s, R, kv->max_pages * s.page, c->sm_count);
+  const int B = kv->batch, nr = R / B;
+  const int E = (c->dc.mode == SX_MODE_CHAIN) ? round : (round == 1 ? 1 : 1 + (round - 1) * c->dc.topk);
+  const int nsplit = sx_attn_splits(s, B, nr, kv->max_pages * s.page, c->sm_count);
   prof_mark(c, SX_PROF_ATTENTION, true, st);
-  sx_launch_attention(s, rm, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st);
+  sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st);
   prof_mark(c, SX_PROF_ATTENTION, false, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_O, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st);

@@ -50,6 +50,19 @@ __device__ __forceinline__ SxRowInfo sx_row_info(const SxRowMap &m, int r) {
   return i;
 }
 
+// placement only (sequence, cached length, position, drafted-row index): touches nothing a kernel
+// of the same iteration writes, so it may run before the wait on the preceding kernel
+__device__ __forceinline__ SxRowInfo sx_row_place(const SxRowMap &m, int r) {
+  SxRowInfo i;
+  if (m.mode == SX_MODE_CHAIN) { i.b = r; i.rel = m.round - 1; }
+  else if (m.round == 1) { i.b = r; i.rel = 0; }
+  else { i.b = r / m.topk; i.rel = 1 + (m.round - 2) * m.topk + (r % m.topk); }
+  i.mask = 0ull;
+  i.n = m.cache_len[i.b];
+  i.pos = i.n + m.round - 1;
+  return i;
+}
+
 __device__ __forceinline__ void sx_set_status(int32_t *status, int32_t code) {
   if (status) atomicMin(status, code);
 }

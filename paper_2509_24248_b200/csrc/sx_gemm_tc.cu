@@ -24,6 +24,7 @@
 
 #include "sx_head_epilogue.cuh"
 #include "sx_kernels.cuh"
+#include "sx_launch.cuh"
 
 #define SX_BK 64                 // K elements per stage (128 bytes: one swizzle row)
 #define SX_A_BYTES (SX_TILE_M * SX_BK * 2)
@@ -171,6 +172,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   uint8_t *epi_smem = reinterpret_cast<uint8_t *>(tmem_slot + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  sx_pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int i = 0; i < p.stages; ++i) {
       mbar_init(smem_u32(&full[i]), 1);
@@ -201,22 +203,38 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   if (warp == 0) {
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      int stage = 0;
-      uint32_t phase = 0;
+      // The weight tiles depend on nothing: the first ring of them is requested before the wait on
+      // the preceding kernel, the activation tiles of those stages right after it.
+      //   pass 0: weights of the first `stages` k-blocks     pass 1: their activations
+      //   pass 2: every later k-block, weights and activations together
       bool ok = true;
-      for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
-        const int tile = HEAD ? item : item / p.splits;
-        const int sp = HEAD ? 0 : item % p.splits;
-        const int kb0 = sp * p.kb_per_split;
-        const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t fb = smem_u32(&full[stage]);
-          const uint32_t dst = smem_u32(smem + (size_t)stage * stage_bytes);
-          mbar_expect_tx(fb, stage_bytes);
-          tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
-          tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
-          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      for (int pass = 0; pass < 3 && ok; ++pass) {
+        if (pass == 1) sx_pdl_wait();
+        int stage = 0, cnt = 0;
+        uint32_t phase = 0;
+        for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+          const int tile = HEAD ? item : item / p.splits;
+          const int sp = HEAD ? 0 : item % p.splits;
+          const int kb0 = sp * p.kb_per_split;
+          const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+          for (int kb = kb0; kb < kb1; ++kb, ++cnt) {
+            if (pass < 2 && cnt >= p.stages) break;
+            const uint32_t fb = smem_u32(&full[stage]);
+            const uint32_t dst = smem_u32(smem + (size_t)stage * stage_bytes);
+            if (pass == 0) {
+              mbar_expect_tx(fb, stage_bytes);
+              tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
+            } else if (pass == 1) {
+              tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
+            } else if (cnt >= p.stages) {
+              if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+              mbar_expect_tx(fb, stage_bytes);
+              tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
+              tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
+            }
+            if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          }
+          if (pass < 2 && cnt >= p.stages) break;
         }
       }
     }
@@ -256,6 +274,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     const int et = q * 32 + lane;                      // row of the tile owned by this thread
     int acc = 0;
     uint32_t acc_phase = 0;
+    sx_pdl_wait();
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
       const int tile = HEAD ? item : item / p.splits;
       const int sp = HEAD ? 0 : item % p.splits;
@@ -376,13 +395,13 @@ static size_t smem_bytes(const SxTcParams &p, size_t epi_bytes) {
   return 1024 + (size_t)p.stages * (SX_A_BYTES + (size_t)p.nmma * 128) + (size_t)(2 * p.stages + 4) * 8 + 16 + epi_bytes + 64;
 }
 
-void sx_tc_init(int device) {
+void sx_gemm_init(int device) {
   cudaFuncSetAttribute(sx_tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
   cudaFuncSetAttribute(sx_tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
 }
 
 // Choose the K split: fill the SMs in whole waves, keep at least 4 k-blocks per item.
-int sx_tc_pick_splits(int N, int K, int sm_count) {
+int sx_gemm_pick_splits(int N, int K, int sm_count) {
   const int tiles = (N + SX_TILE_M - 1) / SX_TILE_M;
   const int num_kb = (K + SX_BK - 1) / SX_BK;
   int best = 1;
@@ -400,8 +419,8 @@ int sx_tc_pick_splits(int N, int K, int sm_count) {
   return best;
 }
 
-sx_status sx_tc_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
-                             size_t split_stride, int sm_count, int32_t *status, cudaStream_t st) {
+sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
+                                 size_t split_stride, int sm_count, int32_t *status, cudaStream_t st) {
   if ((K % 8) != 0 || R < 1) return SX_ERR_UNSUPPORTED;
   for (int r0 = 0; r0 < R; r0 += 256) {
     const int rc = (R - r0 < 256) ? R - r0 : 256;
@@ -418,17 +437,18 @@ sx_status sx_tc_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, 
     if (!get_map(W, N, K, SX_TILE_M, &mw) || !get_map(X + (size_t)r0 * K, rc, K, p.nmma, &mx)) return SX_ERR_CUDA;
     const int items = p.num_tiles * p.splits;
     const int grid = items < sm_count ? items : sm_count;
-    sx_tc_gemm_kernel<false><<<grid, 192, smem_bytes(p, 0), st>>>(mw, mx, p);
+    if (sx_launch(sx_tc_gemm_kernel<false>, dim3(grid), dim3(192), smem_bytes(p, 0), st, mw, mx, p) != cudaSuccess)
+      return SX_ERR_CUDA;
   }
   return SX_OK;
 }
 
-int sx_tc_head_max_rows(int T) { return T > 1 ? 64 : 256; }
+int sx_head_max_rows(int T) { return T > 1 ? 64 : 256; }
 
-sx_status sx_tc_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
-                     SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
-                     cudaStream_t st) {
-  if ((K % 8) != 0 || R < 1 || R > sx_tc_head_max_rows(T)) return SX_ERR_UNSUPPORTED;
+sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
+                         SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
+                         cudaStream_t st) {
+  if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T)) return SX_ERR_UNSUPPORTED;
   SxTcParams p;
   memset(&p, 0, sizeof(p));
   const size_t epi = sx_head_smem_bytes(R, T, lse);
@@ -439,7 +459,8 @@ sx_status sx_tc_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R
   CUtensorMap mw, mx;
   if (!get_map(W, Ntot, K, SX_TILE_M, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
   const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
-  sx_tc_gemm_kernel<true><<<grid, 192, smem_bytes(p, epi), st>>>(mw, mx, p);
+  if (sx_launch(sx_tc_gemm_kernel<true>, dim3(grid), dim3(192), smem_bytes(p, epi), st, mw, mx, p) != cudaSuccess)
+    return SX_ERR_CUDA;
   *G = grid;
   return SX_OK;
 }

@@ -4,6 +4,7 @@
 #include <math.h>
 
 #include "sx_kernels.cuh"
+#include "sx_launch.cuh"
 
 __device__ __forceinline__ int sx_index(const SxIndex &x, int r) { return x.idx ? x.idx[r] : r * x.mul + x.add; }
 
@@ -12,6 +13,8 @@ __device__ __forceinline__ int sx_index(const SxIndex &x, int r) { return x.idx 
 // ---------------------------------------------------------------------------------------
 __global__ void sx_embed_concat_kernel(int H, int V, const bf16 *feat, SxIndex fi, const int32_t *tok,
                                        SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int r = blockIdx.x;
   int t = tok[sx_index(ti, r)];
   if (t < 0 || t >= V) {
@@ -23,35 +26,66 @@ __global__ void sx_embed_concat_kernel(int H, int V, const bf16 *feat, SxIndex f
   uint4 *o = reinterpret_cast<uint4 *>(u + (size_t)r * 2 * H);
   const int n = H / 8;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    o[i] = f[i];
-    o[n + i] = e[i];
+    const uint4 a = f[i], b = e[i];
+    o[i] = a;
+    o[n + i] = b;
   }
 }
 
 void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
                             SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status, cudaStream_t st) {
-  sx_embed_concat_kernel<<<R, 128, 0, st>>>(sh.H, sh.V, feat, fi, tok, ti, embed, u, status);
+  int threads = ((sh.H / 8 + 31) / 32) * 32;
+  if (threads > 512) threads = 512;
+  sx_launch(sx_embed_concat_kernel, dim3(R), dim3(threads), 0, st, sh.H, sh.V, feat, fi, tok, ti, embed, u, status);
 }
 
 // ---------------------------------------------------------------------------------------
-// split-K finisher + RMSNorm
+// split-K finisher + RMSNorm.  One CTA per row; a thread owns 4 consecutive elements per pass
+// and issues the loads of all splits before it adds them (in split order).
 // ---------------------------------------------------------------------------------------
-__global__ void sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t split_stride,
-                                      const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
-                                      bf16 *out_user, SxIndex ui) {
+// sum over the splits, in split order, of 4 consecutive floats; loads go out four splits at a time
+__device__ __forceinline__ float4 sx_sum_splits4(const float *p, int splits, size_t split_stride) {
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < splits; s0 += 4) {
+    float4 v[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+      if (s0 + s < splits) v[s] = *reinterpret_cast<const float4 *>(p + (size_t)(s0 + s) * split_stride);
+#pragma unroll
+    for (int s = 0; s < 4; ++s)
+      if (s0 + s < splits) { a.x += v[s].x; a.y += v[s].y; a.z += v[s].z; a.w += v[s].w; }
+  }
+  return a;
+}
+
+__global__ void __launch_bounds__(512)
+sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t split_stride,
+                      const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
+                      bf16 *out_user, SxIndex ui) {
   extern __shared__ float sx_buf[];
   __shared__ float red[32];
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int r = blockIdx.x;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < H; i += blockDim.x) {
-    float v = 0.f;
-    for (int s = 0; s < splits; ++s) v += part[s * split_stride + (size_t)r * H + i];
-    if (residual) v += __bfloat162float(residual[(size_t)r * H + i]);
-    const bf16 vb = __float2bfloat16_rn(v);
-    if (out_v) out_v[(size_t)r * H + i] = vb;
-    const float vf = __bfloat162float(vb);
-    sx_buf[i] = vf;
-    ss += vf * vf;
+  for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+    float4 v = sx_sum_splits4(part + (size_t)r * H + i, splits, split_stride);
+    if (residual) {
+      const uint2 ru = *reinterpret_cast<const uint2 *>(residual + (size_t)r * H + i);
+      const float2 r0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ru.x));
+      const float2 r1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ru.y));
+      v.x += r0.x; v.y += r0.y; v.z += r1.x; v.w += r1.y;
+    }
+    __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+    if (out_v) {
+      uint2 w;
+      w.x = *reinterpret_cast<uint32_t *>(&b0);
+      w.y = *reinterpret_cast<uint32_t *>(&b1);
+      *reinterpret_cast<uint2 *>(out_v + (size_t)r * H + i) = w;
+    }
+    const float2 f0 = __bfloat1622float2(b0), f1 = __bfloat1622float2(b1);
+    *reinterpret_cast<float4 *>(sx_buf + i) = make_float4(f0.x, f0.y, f1.x, f1.y);
+    ss += (f0.x * f0.x + f0.y * f0.y) + (f1.x * f1.x + f1.y * f1.y);
   }
   ss = sx_warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -64,295 +98,122 @@ __global__ void sx_finish_norm_kernel(int H, float eps, const float *part, int s
   __syncthreads();
   const float scale = rsqrtf(red[0] / (float)H + eps);
   bf16 *user = out_user ? out_user + (size_t)sx_index(ui, r) * H : nullptr;
-  for (int i = threadIdx.x; i < H; i += blockDim.x) {
-    const bf16 nb = __float2bfloat16_rn(sx_buf[i] * scale * __bfloat162float(gamma[i]));
-    if (out_n) out_n[(size_t)r * H + i] = nb;
-    if (user) user[i] = nb;
+  for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4 *>(sx_buf + i);
+    const uint2 gu = *reinterpret_cast<const uint2 *>(gamma + i);
+    const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gu.x));
+    const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gu.y));
+    __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x * scale * g0.x, v.y * scale * g0.y);
+    __nv_bfloat162 b1 = __floats2bfloat162_rn(v.z * scale * g1.x, v.w * scale * g1.y);
+    uint2 w;
+    w.x = *reinterpret_cast<uint32_t *>(&b0);
+    w.y = *reinterpret_cast<uint32_t *>(&b1);
+    if (out_n) *reinterpret_cast<uint2 *>(out_n + (size_t)r * H + i) = w;
+    if (user) *reinterpret_cast<uint2 *>(user + i) = w;
   }
 }
 
 void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
                            bf16 *out_user, SxIndex ui, cudaStream_t st) {
-  sx_finish_norm_kernel<<<R, 256, sh.H * sizeof(float), st>>>(sh.H, sh.eps, part, splits, split_stride,
-                                                               residual, gamma, out_v, out_n, out_user, ui);
+  int threads = ((sh.H / 4 + 31) / 32) * 32;
+  if (threads > 512) threads = 512;
+  sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * sizeof(float), st, sh.H, sh.eps, part, splits,
+            split_stride, residual, gamma, out_v, out_n, out_user, ui);
 }
 
 // ---------------------------------------------------------------------------------------
-// split-K finisher of the QKV projection + rotary (rotate-half pairing) + KV append
+// split-K finisher of the QKV projection + rotary (rotate-half pairing) + KV append.
+// One CTA per (head, row); thread i owns the pair (i, i + d/2).
 // ---------------------------------------------------------------------------------------
 __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, SxRowMap rm, const float *part,
                                           int splits, size_t split_stride, bf16 *q_out, sx_kv kv, int page,
                                           int32_t *status) {
-  const int r = blockIdx.x;
-  const SxRowInfo ri = sx_row_info(rm, r);
-  const int N = (nq + 2 * nkv) * d;
+  sx_pdl_launch_dependents();
+  const int hh = blockIdx.x, r = blockIdx.y;
+  const int i = threadIdx.x;
   const int half = d / 2;
-  const int slot = ri.n + ri.rel;
-  const int lp = slot / page, off = slot % page;
-  int pp = -1;
-  if (lp < kv.max_pages) pp = kv.page_table_d[(size_t)ri.b * kv.max_pages + lp];
-  const bool can_write = (pp >= 0 && pp < kv.num_pages);
-  if (!can_write && threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY);
-  bf16 *kp = reinterpret_cast<bf16 *>(kv.k_pages_d);
-  bf16 *vp = reinterpret_cast<bf16 *>(kv.v_pages_d);
-  const float *row = part + (size_t)r * N;
-  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+  const bool rot = hh < nq + nkv;                 // q and k heads rotate, v heads do not
+  const SxRowInfo ri = sx_row_place(rm, r);       // reads cache_len only (an input of the iteration)
+  float c = 1.f, s = 0.f;
+  if (rot && i < half) {
     // the angle needs more than fp32 at positions in the tens of thousands
     const double inv = exp2(-(2.0 * (double)i / (double)d) * log2(theta));
     double sn, cs;
     sincos((double)ri.pos * inv, &sn, &cs);
-    const float c = (float)cs, s = (float)sn;
-    for (int h = 0; h < nq + nkv; ++h) {
-      float x1 = 0.f, x2 = 0.f;
-      for (int sp = 0; sp < splits; ++sp) {
-        x1 += row[sp * split_stride + h * d + i];
-        x2 += row[sp * split_stride + h * d + i + half];
-      }
-      const bf16 y1 = __float2bfloat16_rn(x1 * c - x2 * s);
-      const bf16 y2 = __float2bfloat16_rn(x2 * c + x1 * s);
-      if (h < nq) {
-        q_out[(size_t)r * nq * d + h * d + i] = y1;
-        q_out[(size_t)r * nq * d + h * d + i + half] = y2;
-      } else if (can_write) {
-        const size_t base = (((size_t)pp * nkv + (h - nq)) * page + off) * d;
-        kp[base + i] = y1;
-        kp[base + i + half] = y2;
-      }
-    }
-    if (can_write) {
-      for (int h = 0; h < nkv; ++h) {
-        float v1 = 0.f, v2 = 0.f;
-        for (int sp = 0; sp < splits; ++sp) {
-          v1 += row[sp * split_stride + (nq + nkv + h) * d + i];
-          v2 += row[sp * split_stride + (nq + nkv + h) * d + i + half];
-        }
-        const size_t base = (((size_t)pp * nkv + h) * page + off) * d;
-        vp[base + i] = __float2bfloat16_rn(v1);
-        vp[base + i + half] = __float2bfloat16_rn(v2);
-      }
-    }
+    c = (float)cs;
+    s = (float)sn;
   }
+  sx_pdl_wait();
+  if (i >= half) return;
+  const int N = (nq + 2 * nkv) * d;
+  const float *row = part + (size_t)r * N + hh * d;
+  float x1 = 0.f, x2 = 0.f;
+  for (int sp = 0; sp < splits; ++sp) {
+    x1 += row[sp * split_stride + i];
+    x2 += row[sp * split_stride + i + half];
+  }
+  bf16 y1, y2;
+  if (rot) {
+    y1 = __float2bfloat16_rn(x1 * c - x2 * s);
+    y2 = __float2bfloat16_rn(x2 * c + x1 * s);
+  } else {
+    y1 = __float2bfloat16_rn(x1);
+    y2 = __float2bfloat16_rn(x2);
+  }
+  if (hh < nq) {
+    q_out[((size_t)r * nq + hh) * d + i] = y1;
+    q_out[((size_t)r * nq + hh) * d + i + half] = y2;
+    return;
+  }
+  const int slot = ri.n + ri.rel;
+  const int lp = slot / page, off = slot % page;
+  int pp = -1;
+  if (lp < kv.max_pages) pp = kv.page_table_d[(size_t)ri.b * kv.max_pages + lp];
+  if (pp < 0 || pp >= kv.num_pages) {
+    if (i == 0) sx_set_status(status, SX_ERR_CAPACITY);
+    return;
+  }
+  const int kh = (hh < nq + nkv) ? hh - nq : hh - nq - nkv;
+  bf16 *dst = reinterpret_cast<bf16 *>(hh < nq + nkv ? kv.k_pages_d : kv.v_pages_d) +
+              (((size_t)pp * nkv + kh) * page + off) * d;
+  dst[i] = y1;
+  dst[i + half] = y2;
 }
 
 void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
                                cudaStream_t st) {
-  sx_finish_qkv_rope_kernel<<<rm.R, 128, 0, st>>>(sh.nq, sh.nkv, sh.d, (double)sh.theta, rm, part, splits,
-                                                   split_stride, q_out, kv, sh.page, status);
+  int threads = ((sh.d / 2 + 31) / 32) * 32;
+  sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv, sh.d,
+            (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, status);
 }
 
 // ---------------------------------------------------------------------------------------
 // split-K finisher of gate/up + SwiGLU
 // ---------------------------------------------------------------------------------------
 __global__ void sx_finish_swiglu_kernel(int F, const float *part, int splits, size_t split_stride, bf16 *m_out) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int r = blockIdx.y;
   const float *row = part + (size_t)r * 2 * F;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < F; i += gridDim.x * blockDim.x) {
-    float g = 0.f, u = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      g += row[s * split_stride + i];
-      u += row[s * split_stride + F + i];
-    }
-    const float si = g / (1.0f + expf(-g));
-    m_out[(size_t)r * F + i] = __float2bfloat16_rn(si * u);
-  }
+  const int i = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= F) return;
+  const float4 g = sx_sum_splits4(row + i, splits, split_stride);
+  const float4 u = sx_sum_splits4(row + F + i, splits, split_stride);
+  const float m0 = g.x / (1.0f + expf(-g.x)) * u.x, m1 = g.y / (1.0f + expf(-g.y)) * u.y;
+  const float m2 = g.z / (1.0f + expf(-g.z)) * u.z, m3 = g.w / (1.0f + expf(-g.w)) * u.w;
+  __nv_bfloat162 b0 = __floats2bfloat162_rn(m0, m1), b1 = __floats2bfloat162_rn(m2, m3);
+  uint2 w;
+  w.x = *reinterpret_cast<uint32_t *>(&b0);
+  w.y = *reinterpret_cast<uint32_t *>(&b1);
+  *reinterpret_cast<uint2 *>(m_out + (size_t)r * F + i) = w;
 }
 
 void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                              bf16 *m_out, cudaStream_t st) {
-  dim3 grid((sh.F + 1023) / 1024, R);
-  if (grid.x < 1) grid.x = 1;
-  sx_finish_swiglu_kernel<<<grid, 256, 0, st>>>(sh.F, part, splits, split_stride, m_out);
-}
-
-// ---------------------------------------------------------------------------------------
-// split-K decode attention over the paged cache.
-// Block = (split, kv head, row).  A key's head_dim spans d/8 lanes (16-byte loads); a warp
-// works on 32/(d/8) keys at once; the G query heads of the group share every K/V load.
-// The last split also takes the visible drafted rows (slots n + bit).
-// Partials: ws_ml[r][hq][split] = (m, l), ws_o[r][hq][split][d] (unnormalised).
-// ---------------------------------------------------------------------------------------
-template <int G>
-__global__ void sx_attn_split_kernel(int nq, int nkv, int d, int page, float scale, SxRowMap rm, const bf16 *q,
-                                     sx_kv kv, int nsplit, float2 *ws_ml, float *ws_o, int32_t *status) {
-  extern __shared__ float sx_sm[];
-  const int split = blockIdx.x, kvh = blockIdx.y, r = blockIdx.z;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int lpk = d >> 3;                 // lanes per key
-  const int kpw = 32 / lpk;               // keys per warp step
-  const int grp = lane / lpk, sub = lane % lpk;
-  const SxRowInfo ri = sx_row_info(rm, r);
-  const int n = ri.n;
-  const int chunk = (n + nsplit - 1) / nsplit;
-  const int k0 = split * chunk;
-  const int k1 = min(n, k0 + chunk);
-  const int n_extra = (split == nsplit - 1) ? __popcll(ri.mask) : 0;
-  const int total = max(0, k1 - k0) + n_extra;
-
-  float qf[G][8], acc[G][8], m[G], l[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    const uint4 qu = *reinterpret_cast<const uint4 *>(q + ((size_t)r * nq + kvh * G + g) * d + sub * 8);
-    sx_unpack8(qu, qf[g]);
-    m[g] = -INFINITY;
-    l[g] = 0.f;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[g][j] = 0.f;
-  }
-  const bf16 *kp = reinterpret_cast<const bf16 *>(kv.k_pages_d);
-  const bf16 *vp = reinterpret_cast<const bf16 *>(kv.v_pages_d);
-  const int32_t *table = kv.page_table_d + (size_t)ri.b * kv.max_pages;
-  const int step = 4 * kpw;
-  for (int base = 0; base < total; base += step) {
-    const int t = base + warp * kpw + grp;
-    const bool live = t < total;
-    int slot = 0;
-    if (live) {
-      if (t < k1 - k0) {
-        slot = k0 + t;
-      } else {                                   // the (t - (k1-k0))-th set bit of the mask
-        int want = t - max(0, k1 - k0);
-        uint64_t mm = ri.mask;
-        for (int z = 0; z < want; ++z) mm &= mm - 1;
-        slot = n + (__ffsll((long long)mm) - 1);
-      }
-    }
-    bool ok = live;
-    size_t off = 0;
-    if (live) {
-      const int lp = slot / page;
-      int pp = (lp < kv.max_pages) ? table[lp] : -1;
-      if (pp < 0 || pp >= kv.num_pages) { ok = false; sx_set_status(status, SX_ERR_CAPACITY); }
-      else off = (((size_t)pp * nkv + kvh) * page + (slot % page)) * d + sub * 8;
-    }
-    float kf[8], vf[8];
-    if (ok) {
-      sx_unpack8(*reinterpret_cast<const uint4 *>(kp + off), kf);
-      sx_unpack8(*reinterpret_cast<const uint4 *>(vp + off), vf);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { kf[j] = 0.f; vf[j] = 0.f; }
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float s = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) s = fmaf(qf[g][j], kf[j], s);
-      for (int o = lpk >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      s *= scale;
-      if (ok) {
-        const float mn = fmaxf(m[g], s);
-        const float corr = __expf(m[g] - mn);
-        const float p = __expf(s - mn);
-        l[g] = l[g] * corr + p;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[g][j] = acc[g][j] * corr + p * vf[j];
-        m[g] = mn;
-      }
-    }
-  }
-  // merge the key groups of a warp, then the warps
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    for (int o = lpk; o < 32; o <<= 1) {
-      const float mo = __shfl_xor_sync(0xffffffffu, m[g], o);
-      const float lo = __shfl_xor_sync(0xffffffffu, l[g], o);
-      const float mn = fmaxf(m[g], mo);
-      const float c0 = (m[g] == -INFINITY) ? 0.f : __expf(m[g] - mn);
-      const float c1 = (mo == -INFINITY) ? 0.f : __expf(mo - mn);
-      l[g] = l[g] * c0 + lo * c1;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float ao = __shfl_xor_sync(0xffffffffu, acc[g][j], o);
-        acc[g][j] = acc[g][j] * c0 + ao * c1;
-      }
-      m[g] = mn;
-    }
-  }
-  // shared: [4 warps][G][2 + d]
-  float *sm = sx_sm;
-  const int per = 2 + d;
-  if (grp == 0) {
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float *dst = sm + ((size_t)warp * G + g) * per;
-      if (sub == 0) { dst[0] = m[g]; dst[1] = l[g]; }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) dst[2 + sub * 8 + j] = acc[g][j];
-    }
-  }
-  __syncthreads();
-  for (int e = tid; e < G * d; e += blockDim.x) {
-    const int g = e / d, j = e % d;
-    float mm = -INFINITY;
-    for (int w = 0; w < 4; ++w) mm = fmaxf(mm, sm[((size_t)w * G + g) * per]);
-    float ll = 0.f, a = 0.f;
-    for (int w = 0; w < 4; ++w) {
-      const float *src = sm + ((size_t)w * G + g) * per;
-      const float c = (src[0] == -INFINITY) ? 0.f : __expf(src[0] - mm);
-      ll += src[1] * c;
-      a += src[2 + j] * c;
-    }
-    const size_t hq = (size_t)r * nq + kvh * G + g;
-    ws_o[(hq * nsplit + split) * d + j] = a;
-    if (j == 0) ws_ml[hq * nsplit + split] = make_float2(mm, ll);
-  }
-}
-
-__global__ void sx_attn_combine_kernel(int nq, int d, int nsplit, const float2 *ws_ml, const float *ws_o,
-                                       bf16 *o_out) {
-  const size_t hq = (size_t)blockIdx.y * nq + blockIdx.x;
-  float mm = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) mm = fmaxf(mm, ws_ml[hq * nsplit + s].x);
-  float ll = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float2 t = ws_ml[hq * nsplit + s];
-    if (t.x != -INFINITY) ll += t.y * __expf(t.x - mm);
-  }
-  for (int j = threadIdx.x; j < d; j += blockDim.x) {
-    float a = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
-      const float2 t = ws_ml[hq * nsplit + s];
-      if (t.x != -INFINITY) a += ws_o[(hq * nsplit + s) * d + j] * __expf(t.x - mm);
-    }
-    o_out[hq * d + j] = __float2bfloat16_rn(a / ll);
-  }
-}
-
-int sx_attn_splits(const SxShape &sh, int R, int n_cap, int sm_count) {
-  int want = (4 * sm_count + R * sh.nkv - 1) / (R * sh.nkv);
-  int by_len = (n_cap + 255) / 256;
-  int s = want < by_len ? want : by_len;
-  if (s < 1) s = 1;
-  if (s > 64) s = 64;
-  return s;
-}
-
-size_t sx_attn_ws_bytes(const SxShape &sh, int R, int max_splits) {
-  return (size_t)R * sh.nq * max_splits * (sh.d + 2) * sizeof(float);
-}
-
-void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, const bf16 *q, const sx_kv &kv, int nsplit,
-                         float *ws, bf16 *o_out, int32_t *status, cudaStream_t st) {
-  const int R = rm.R;
-  float2 *ws_ml = reinterpret_cast<float2 *>(ws);
-  float *ws_o = ws + (size_t)R * sh.nq * nsplit * 2;
-  const int G = sh.nq / sh.nkv;
-  dim3 grid(nsplit, sh.nkv, R);
-  const size_t smem = (size_t)4 * G * (2 + sh.d) * sizeof(float);
-  const float scale = 1.0f / sqrtf((float)sh.d);
-#define SX_ATTN(GG)                                                                                          \
-  sx_attn_split_kernel<GG><<<grid, 128, smem, st>>>(sh.nq, sh.nkv, sh.d, sh.page, scale, rm, q, kv, nsplit, \
-                                                    ws_ml, ws_o, status)
-  switch (G) {
-    case 1: SX_ATTN(1); break;
-    case 2: SX_ATTN(2); break;
-    case 4: SX_ATTN(4); break;
-    default: SX_ATTN(8); break;
-  }
-#undef SX_ATTN
-  sx_attn_combine_kernel<<<dim3(sh.nq, R), 64, 0, st>>>(sh.nq, sh.d, nsplit, ws_ml, ws_o, o_out);
+  dim3 grid((sh.F / 4 + 127) / 128, R);
+  sx_launch(sx_finish_swiglu_kernel, grid, dim3(128), 0, st, sh.F, part, splits, split_stride, m_out);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -361,6 +222,8 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, const bf16 *q, c
 __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
                                         const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
                                         SxIndex toi, float *logp_out, float *sig_out, SxIndex si) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   extern __shared__ unsigned long long sx_cand[];      // [G * T]
   __shared__ unsigned long long wbest[4];
   __shared__ float s_lse;
@@ -402,15 +265,16 @@ __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int p
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
                              float *logp_out, float *sig_out, SxIndex si, cudaStream_t st) {
-  sx_head_finalize_kernel<<<R, 128, (size_t)G * T * 8, st>>>(parts, G, part_stride, T, lse, z, S, sh.act[0],
-                                                              sh.act[1], sh.act[2], tok_out, toi, logp_out,
-                                                              sig_out, si);
+  sx_launch(sx_head_finalize_kernel, dim3(R), dim3(128), (size_t)G * T * 8, st, parts, G, part_stride, T, lse, z, S,
+            sh.act[0], sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si);
 }
 
 // ---------------------------------------------------------------------------------------
 // chain layout: slot j holds the j-th draft token; the signal of slot j comes from round j+1
 // ---------------------------------------------------------------------------------------
 __global__ void sx_chain_layout_kernel(int B, int K, int S, const int32_t *tok0, sx_iter_out o) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int P = K + 1;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= B * P) return;
@@ -426,7 +290,7 @@ __global__ void sx_chain_layout_kernel(int B, int K, int S, const int32_t *tok0,
 
 void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st) {
   const int n = B * (K + 1);
-  sx_chain_layout_kernel<<<(n + 127) / 128, 128, 0, st>>>(B, K, S, tok0, o);
+  sx_launch(sx_chain_layout_kernel, dim3((n + 127) / 128), dim3(128), 0, st, B, K, S, tok0, o);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -434,6 +298,8 @@ void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_i
 // ---------------------------------------------------------------------------------------
 __global__ void sx_accept_kernel(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                                  int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int32_t *c = cand + (size_t)b * P, *t = target + (size_t)b * P;
@@ -462,8 +328,8 @@ __global__ void sx_accept_kernel(int B, int P, const int32_t *cand, const int32_
 
 void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                       int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st) {
-  sx_accept_kernel<<<(B + 31) / 32, 32, 0, st>>>(B, P, cand, parent, target, accept_len, path, path_stride,
-                                                 recover);
+  sx_launch(sx_accept_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, cand, parent, target, accept_len, path,
+            path_stride, recover);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -485,6 +351,8 @@ __global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float
                                const int32_t *path, int path_stride, const int32_t *accept_len,
                                const int32_t *recover, int32_t *exit_flag, int32_t *accept_out,
                                int32_t *recover_out, float *smoothed, int32_t *status) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= B) return;
   const int L = accept_len[b];
@@ -541,9 +409,9 @@ void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_s
   p.ema_positions = cfg.ema_positions;
   p.bitmap = cfg.split_bitmap_d;
   p.stop_tok = cfg.stop_think_token;
-  sx_exit_kernel<<<(B + 31) / 32, 32, 0, st>>>(B, P, S, V, p, state.x_d, state.n_updates_d, state.thinking_d,
-                                               slot_signal, cand, path, path_stride, accept_len, recover,
-                                               exit_flag, accept_out, recover_out, smoothed, status);
+  sx_launch(sx_exit_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, S, V, p, state.x_d, state.n_updates_d,
+            state.thinking_d, slot_signal, cand, path, path_stride, accept_len, recover, exit_flag, accept_out,
+            recover_out, smoothed, status);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -556,6 +424,8 @@ __device__ __forceinline__ bool sx_better(float sa, int ia, float sb, int ib) {
 }
 
 __global__ void sx_tree_expand_kernel(SxTree t, int round, const int32_t *tok_rt, const float *logp_rt) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int b = blockIdx.x, tid = threadIdx.x;
   const int T = t.T;
   int32_t *ctok = t.cand_tok + (size_t)b * t.NC, *cpar = t.cand_parent + (size_t)b * t.NC;
@@ -606,10 +476,12 @@ __global__ void sx_tree_expand_kernel(SxTree t, int round, const int32_t *tok_rt
 
 void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
                            cudaStream_t st) {
-  sx_tree_expand_kernel<<<B, 64, 0, st>>>(t, round, tok_rt, logp_rt);
+  sx_launch(sx_tree_expand_kernel, dim3(B), dim3(64), 0, st, t, round, tok_rt, logp_rt);
 }
 
 __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_iter_out o) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   extern __shared__ int sx_tl[];           // kept[NC], slot_of[NC]
   const int b = blockIdx.x, tid = threadIdx.x;
   const int NC = t.NC, P = 1 + t.max_nodes, T = t.T;
@@ -656,5 +528,5 @@ __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_i
 
 void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
                            cudaStream_t st) {
-  sx_tree_layout_kernel<<<B, 256, (size_t)2 * t.NC * sizeof(int), st>>>(t, S, tok0, o);
+  sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)2 * t.NC * sizeof(int), st, t, S, tok0, o);
 }

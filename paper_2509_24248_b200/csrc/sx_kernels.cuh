@@ -1,5 +1,5 @@
 // Launch wrappers of the non-GEMM kernels (defined in sx_kernels.cu) and of the GEMMs
-// (sx_gemm.cu).  Host-side only.
+// (sx_gemm_tc.cu) and of the attention (sx_attention.cu).  Host-side only.
 #pragma once
 #include "sx_common.cuh"
 
@@ -31,10 +31,13 @@ void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const floa
 void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits,
                              size_t split_stride, bf16 *m_out, cudaStream_t st);
 
-int sx_attn_splits(const SxShape &sh, int R, int n_cap, int sm_count);
-size_t sx_attn_ws_bytes(const SxShape &sh, int R, int max_splits);
-void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, const bf16 *q, const sx_kv &kv,
-                         int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
+// decode attention (sx_attention.cu).  B sequences with nr rows each this round, E drafted slots
+// behind the cached prefix (this round's rows included).
+bool sx_attn_supported(const SxShape &sh);
+int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count);
+size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_count);
+void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
+                         const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
 
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
@@ -68,12 +71,14 @@ void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok
 void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
                            cudaStream_t st);
 
-// ---- GEMMs (sx_gemm.cu) -------------------------------------------------------------------
+// ---- GEMMs (sx_gemm_tc.cu) ----------------------------------------------------------------
 // part[s][r][n] = sum over the s-th K range of X[r][k] * W[n][k]   (fp32)
 struct SxGemmPlan { int splits; };
 int sx_gemm_pick_splits(int N, int K, int sm_count);
 sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part,
-                                 int splits, size_t split_stride, int32_t *status, cudaStream_t st);
+                                 int splits, size_t split_stride, int sm_count, int32_t *status,
+                                 cudaStream_t st);
+void sx_gemm_init(int device);
 // head: per-CTA partial results out[cta][row]; returns the number of CTAs used in *G
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,

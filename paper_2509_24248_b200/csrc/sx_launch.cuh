@@ -1,0 +1,34 @@
+// Launch helper with programmatic dependent launch: a kernel launched through sx_launch may be
+// scheduled while its predecessor in the stream is still draining, so that its prologue (and,
+// for the GEMMs, the first ring of weight tiles, which depend on nothing) overlaps the
+// predecessor's tail.  Every kernel launched this way executes sx_pdl_wait() before it reads or
+// writes anything another kernel of the stream produces or consumes; completion is therefore
+// transitive along the stream exactly as with plain stream order.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <string.h>
+
+#include <utility>
+
+__device__ __forceinline__ void sx_pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void sx_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t sx_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             Args &&...args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}

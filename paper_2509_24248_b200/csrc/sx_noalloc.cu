@@ -19,8 +19,6 @@
 
 #include "sx_kernels.cuh"
 
-void sx_gemm_init(int device);
-
 #define SX_NOALLOC_MAX_CTAS 160     // CTAs of the head kernel that may leave a partial result
 static_assert(SX_NOALLOC_SCRATCH_BYTES == SX_NOALLOC_MAX_CTAS * SX_NOALLOC_MAX_ROWS * sizeof(SxHeadPartial),
               "the header's SX_NOALLOC_SCRATCH_BYTES must match the partial-result record");
