@@ -148,6 +148,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->device = dev;
   c->sm_count = prop.multiProcessorCount;
   sx_gemm_init(dev);
+  sx_attn_init(dev);
 
   const SxShape &s = c->sh;
   const int R = c->Rmax;

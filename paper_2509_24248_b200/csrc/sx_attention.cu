@@ -1,64 +1,115 @@
 // Decode attention over the paged bf16 KV cache, split over the keys ("split-K").
 //
-// One warp owns one work item: (sequence b, KV head h, tile of 16 queries, chunk of keys).  The
-// queries of an item are the G query heads of the KV head's group for every row the sequence
-// drafts this round (1 row in a chain, top-k sibling rows in a tree), so each K/V byte is read
-// once per sequence and round whatever the group size or the number of siblings.
+// One warp owns one work item: (sequence b, KV head h, tile of 8 queries, chunk of keys).  The
+// queries of a (b, h) pair are the G query heads of the KV head's group for every row the
+// sequence drafts this round (1 row in a chain, top-k sibling rows in a tree); when they need
+// more than one tile, the tiles go to sibling warps that share one staged copy of the keys and
+// values, so each K/V byte leaves HBM once per sequence and round whatever the group size or
+// the number of siblings.
 //
-// The products run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 out) with
-// every operand fetched straight from global memory into its fragment registers by 16-byte
-// loads: the contraction index of Q.K^T (head dimension) and the column index of P.V (head
-// dimension again) may be permuted freely, so each lane loads 8 consecutive elements of one key
-// and uses them as the fragment entries of two k-steps (Q.K^T) or of eight column tiles (P.V).
-// Every 32-byte sector that is fetched is fully used, nothing is staged in shared memory, and
-// the bytes in flight are the 16 loads per lane of a 16-key step, re-issued for the next step as soon
-// as the current one has consumed its registers.
+// Both products run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32 out)
+// in transposed form, keys (then head-dimension rows) on the 16-row side and the 8 queries on
+// the 8-column side:
+//     S^T[key][q]  = sum_d K[key][d] Q[q][d]          A = K rows,   B = Q^T
+//     O^T[d][q]   += sum_key V[key][d] P[key][q]      A = V^T,      B = P^T
+// The contraction index of the first product and the row index of the second (both the head
+// dimension) may be permuted freely, so every lane fetches 8 consecutive elements of one K or
+// V row with one 16-byte copy and uses them as fragment entries of two k-steps (K) or of four
+// row tiles (V): each 32-byte sector that is fetched is fully used.  P^T is obtained from the
+// accumulator layout of S^T with two movmatrix transposes.
+//
+// The copies are asynchronous (cp.async) into a small shared-memory ring addressed by lane, i.e.
+// the ring only extends the register file so that further 16-key steps are in flight while one
+// is being computed; a lane reads back what it, or the same lane of a sibling warp, requested,
+// so the ring needs no swizzle and, with one query tile, no barrier.
 //
 // Softmax is the usual running (max, sum) in fp32 with exponentials in base 2; P is rounded to
 // bf16 for the second product.  A warp leaves (m, l, unnormalised O) per query and chunk; the
-// combine kernel merges the chunks and writes bf16.
+// merge kernel combines the chunks and writes bf16.
 #include <math.h>
+#include <stdlib.h>
 
 #include "sx_kernels.cuh"
 #include "sx_launch.cuh"
 
-#define SX_ATTN_WARPS 4
+#define SX_ATTN_MAX_STAGES 8    // 16-key steps staged per warp group: one being consumed, the rest in flight
+#define SX_ATTN_SMEM_BUDGET (200 * 1024)
+#define SX_ATTN_MAX_TILES 8     // query tiles (of 8) per (sequence, KV head): group size * sibling rows <= 64
 
-__device__ __forceinline__ void sx_mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void sx_mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                            uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
       "{%0, %1, %2, %3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-
+// transpose of an 8x8 matrix of 16-bit elements held one row pair per lane
+__device__ __forceinline__ uint32_t sx_movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ float sx_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t sx_pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-
 __device__ __forceinline__ uint32_t sx_word(const uint4 &u, int i) {
   return i == 0 ? u.x : (i == 1 ? u.y : (i == 2 ? u.z : u.w));
 }
+// 16-byte asynchronous copy global -> shared; reads nothing and writes zeros when !valid
+__device__ __forceinline__ void sx_cp_async16(uint32_t smem_dst, const void *gsrc, bool valid) {
+  const uint32_t bytes = valid ? 16u : 0u;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void sx_cp_async16_full(uint32_t smem_dst, const void *gsrc) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void sx_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void sx_cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// waits until at most n (0..6) of this lane's copy groups are pending
+__device__ __forceinline__ void sx_cp_async_wait_n(int n) {
+  switch (n) {
+    case 0: sx_cp_async_wait<0>(); break;
+    case 1: sx_cp_async_wait<1>(); break;
+    case 2: sx_cp_async_wait<2>(); break;
+    case 3: sx_cp_async_wait<3>(); break;
+    case 4: sx_cp_async_wait<4>(); break;
+    case 5: sx_cp_async_wait<5>(); break;
+    default: sx_cp_async_wait<6>(); break;
+  }
+}
+// barrier over the `threads` threads of warp group `grp` (ids 1 and 2; a CTA holds at most two
+// groups of more than one warp)
+__device__ __forceinline__ void sx_group_bar(int grp, int threads) {
+  if (grp == 0) asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");
+  else asm volatile("bar.sync 2, %0;" ::"r"(threads) : "memory");
+}
 
-// storage position of head-dimension element d inside a partial-output row (the order in which
-// the accumulator fragments hold it): column tile (d / 64) * 8 + d % 8, column (d % 64) / 8
-__host__ __device__ __forceinline__ int sx_attn_perm(int d) { return (((d >> 6) << 3) + (d & 7)) * 8 + ((d & 63) >> 3); }
-
-template <int D>
-__global__ void __launch_bounds__(SX_ATTN_WARPS * 32, 2)
-sx_attn_mma_kernel(int nq, int nkv, int G, int page, float scale_log2, SxRowMap rm, int nr, int E, int MT,
-                   const bf16 *__restrict__ q, sx_kv kv, int nsplit, float2 *__restrict__ ws_ml,
+// NT = query tiles per (sequence, KV head) = warps per group (MULTI: NT > 1); gpc = groups per CTA.
+template <int D, bool MULTI>
+__global__ void __launch_bounds__(256, 1)
+sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale_log2, SxRowMap rm, int nr, int E,
+                   int NT, int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit, float2 *__restrict__ ws_ml,
                    float *__restrict__ ws_o, int32_t *status) {
-  constexpr int NC = (D + 31) / 32;       // 32-element chunks of the head dimension (Q.K^T)
-  constexpr int NH = (D + 63) / 64;       // 64-element halves of the head dimension (P.V)
-  constexpr int DS = NH * 64;             // partial-output row length
+  constexpr int NC = (D + 31) / 32;       // 32-element chunks of the head dimension (first product)
+  constexpr int NH = (D + 63) / 64;       // 64-element halves of the head dimension (second product)
+  constexpr int NL = 2 * NC + 4 * NH;     // 16-byte copies per lane and 16-key step
+  extern __shared__ uint4 sx_stage[];     // [groups][stages][NL][32 lanes]
   sx_pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const int wg = blockIdx.x * SX_ATTN_WARPS + warp;
-  const int split = wg / MT, mt = wg - split * MT;
-  if (split >= nsplit) return;
+  const int grp = MULTI ? warp / NT : warp, qt = MULTI ? warp - grp * NT : 0;
+  const int split = blockIdx.x * gpc + grp;
+  if (grp >= gpc || split >= nsplit) return;
   const int b = blockIdx.z, h = blockIdx.y;
+  const uint32_t stg = (uint32_t)__cvta_generic_to_shared(sx_stage) +
+                       (uint32_t)((grp * stages * NL * 32 + lane) * sizeof(uint4));
   sx_pdl_wait();
   const int n = rm.cache_len[b];
   const int total = n + E;
@@ -68,59 +119,60 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, float scale_log2, SxRowMap 
   const int k1 = min(total, k0 + chunk);
   const int NQ = nr * G;
 
-  // the two query rows of this lane
+  // B fragments of Q^T: lane (g, t) holds query g of the tile, elements t*8.. of every 32-chunk
+  uint32_t qb[NC][4];
+  {
+    const int m = qt * 8 + g;
+    const bool valid = m < NQ;
+    const int j = valid ? m / G : 0;
+    const int r = b * nr + j;
+    const bf16 *qp = q + ((size_t)r * nq + h * G + (valid ? m - j * G : 0)) * D;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      uint4 u = make_uint4(0, 0, 0, 0);
+      if (valid && c * 32 + t * 8 < D) u = *reinterpret_cast<const uint4 *>(qp + c * 32 + t * 8);
+      qb[c][0] = u.x; qb[c][1] = u.y; qb[c][2] = u.z; qb[c][3] = u.w;
+    }
+  }
+  // the two queries whose scores this lane holds (columns 2t and 2t + 1 of the tile)
   int hq[2];
   bool qv[2];
   uint64_t vis[2];
-  const bf16 *qp[2];
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
-    const int m = mt * 16 + g + i * 8;
+    const int m = qt * 8 + 2 * t + i;
     qv[i] = m < NQ;
-    const int j = qv[i] ? m / G : 0, gh = qv[i] ? m - (m / G) * G : 0;
+    const int j = qv[i] ? m / G : 0;
     const int r = b * nr + j;
-    hq[i] = r * nq + h * G + gh;
-    qp[i] = q + (size_t)hq[i] * D;
+    hq[i] = r * nq + h * G + (qv[i] ? m - j * G : 0);
     if (rm.mode == SX_MODE_TREE && rm.round > 1) vis[i] = rm.row_mask[r];
     else vis[i] = (E >= 64) ? ~0ull : ((1ull << E) - 1ull);
   }
-  uint32_t qa[NC][2][4];
-#pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    uint4 u0 = make_uint4(0, 0, 0, 0), u1 = u0;
-    if (c * 32 + t * 8 < D) {
-      if (qv[0]) u0 = *reinterpret_cast<const uint4 *>(qp[0] + c * 32 + t * 8);
-      if (qv[1]) u1 = *reinterpret_cast<const uint4 *>(qp[1] + c * 32 + t * 8);
-    }
-    qa[c][0][0] = u0.x; qa[c][0][1] = u1.x; qa[c][0][2] = u0.y; qa[c][0][3] = u1.y;
-    qa[c][1][0] = u0.z; qa[c][1][1] = u1.z; qa[c][1][2] = u0.w; qa[c][1][3] = u1.w;
-  }
 
-  float o[NH * 8][4];
+  float o[NH * 4][4];
 #pragma unroll
-  for (int j = 0; j < NH * 8; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
+  for (int j = 0; j < NH * 4; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
   float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
 
   const bf16 *kp = reinterpret_cast<const bf16 *>(kv.k_pages_d);
   const bf16 *vp = reinterpret_cast<const bf16 *>(kv.v_pages_d);
   const int32_t *table = kv.page_table_d + (size_t)b * kv.max_pages;
   // page-table entries of the chunk, one per lane, when they fit
-  const int lp_first = k0 / page;
-  const int lp_last = (k1 > k0) ? (k1 - 1) / page : lp_first;
+  const int lp_first = (page_shift >= 0) ? (k0 >> page_shift) : k0 / page;
+  const int lp_last = (k1 > k0) ? ((page_shift >= 0) ? ((k1 - 1) >> page_shift) : (k1 - 1) / page) : lp_first;
   const bool tbl_in_regs = (lp_last - lp_first) < 32;
   int tbl = -1;
   if (tbl_in_regs && lp_first + lane <= lp_last && lp_first + lane < kv.max_pages) tbl = table[lp_first + lane];
   bool bad = false;
   const bool one_page = (page & 15) == 0;        // chunks start on multiples of 16: a step never straddles pages
-
-  // The K registers are refilled for step i + 1 as soon as step i's Q.K^T has consumed them, the V
-  // registers as soon as its P.V has: about one step's worth of loads is in flight all the time.
-  uint4 kr[2][NC], vr[4][NH];
+  // element offsets of this lane inside a 16-key block that lies in one page
+  const int klane = g * D + t * 8;               // K: keys g and g + 8, elements t*8.. of every chunk
+  const int vlane = 2 * t * D + g * 8;           // V: keys 2t, 2t+1, 2t+8, 2t+9, elements g*8.. of every half
 
   // offset of the K/V row of `slot` (and whether it may be read); every lane takes part in the shuffle
   auto row_offset = [&](int slot, bool &ok) -> size_t {
     const bool live = slot < k1;
-    const int lp = live ? slot / page : lp_first;
+    const int lp = live ? ((page_shift >= 0) ? (slot >> page_shift) : slot / page) : lp_first;
     int pp;
     if (tbl_in_regs) pp = __shfl_sync(0xffffffffu, tbl, lp - lp_first);
     else pp = (lp < kv.max_pages) ? table[lp] : -1;
@@ -128,136 +180,157 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, float scale_log2, SxRowMap 
     if (live && !ok) bad = true;
     return ok ? (((size_t)pp * nkv + h) * page + (slot - lp * page)) * D : 0;
   };
-  auto issue_k = [&](uint4 (&dst)[2][NC], int s0) {
-    bool ok0, ok1;
-    size_t o0, o1;
-    if (one_page) {
-      const size_t base = row_offset(s0, ok0);
-      o0 = base + (size_t)g * D;
-      o1 = o0 + (size_t)8 * D;
-      ok1 = ok0 && (s0 + 8 + g < k1);
-      ok0 = ok0 && (s0 + g < k1);
-    } else {
-      o0 = row_offset(s0 + g, ok0);
-      o1 = row_offset(s0 + 8 + g, ok1);
+  // Requests the 16 keys from s0 into stage buffer `buf`: copy j < 2 NC is chunk j % NC of key
+  // g (j < NC) or g + 8, the others are half (j - 2 NC) % NH of the keys 2t, 2t+1, 2t+8, 2t+9.
+  // The NT warps of a group take every NT-th copy each (bit j of `mine`).
+  uint32_t mine = 0xffffffffu;
+  if (MULTI) {
+    mine = 0u;
+    for (int j = qt; j < NL; j += NT) mine |= 1u << j;
+  }
+  auto issue = [&](int buf, int s0) {
+    const uint32_t dst = stg + (uint32_t)(buf * NL * 32 * sizeof(uint4));
+    bool okb = false;
+    size_t base = 0;
+    if (one_page) base = row_offset(s0, okb);
+    if (one_page && okb && s0 + 16 <= k1) {
+      const bf16 *kb = kp + base + klane, *vb = vp + base + vlane;
+#pragma unroll
+      for (int j = 0; j < NL; ++j) {
+        if (MULTI && !((mine >> j) & 1u)) continue;
+        if (j < 2 * NC) {
+          const int nt = j / NC, c = j % NC;
+          if (D % 32 == 0) sx_cp_async16_full(dst + j * 512, kb + nt * 8 * D + c * 32);
+          else sx_cp_async16(dst + j * 512, kb + nt * 8 * D + c * 32, c * 32 + t * 8 < D);
+        } else {
+          const int kk = (j - 2 * NC) / NH, hf = (j - 2 * NC) % NH;
+          if (D % 64 == 0) sx_cp_async16_full(dst + j * 512, vb + ((kk >> 1) * 8 + (kk & 1)) * D + hf * 64);
+          else sx_cp_async16(dst + j * 512, vb + ((kk >> 1) * 8 + (kk & 1)) * D + hf * 64, hf * 64 + g * 8 < D);
+        }
+      }
+      return;
     }
+    bool ok[6];
+    size_t of[6];
+#pragma unroll
+    for (int i = 0; i < 6; ++i) {
+      const int key = (i < 2) ? i * 8 + g : ((i - 2) >> 1) * 8 + 2 * t + ((i - 2) & 1);
+      if (one_page) { of[i] = base + (size_t)key * D; ok[i] = okb && (s0 + key < k1); }
+      else of[i] = row_offset(s0 + key, ok[i]);
+    }
+#pragma unroll
+    for (int j = 0; j < NL; ++j) {
+      if (MULTI && !((mine >> j) & 1u)) continue;
+      if (j < 2 * NC) {
+        const int nt = j / NC, c = j % NC;
+        const bool v = ok[nt] && (c * 32 + t * 8 < D);
+        sx_cp_async16(dst + j * 512, kp + (v ? of[nt] + c * 32 + t * 8 : 0), v);
+      } else {
+        const int kk = (j - 2 * NC) / NH, hf = (j - 2 * NC) % NH;
+        const bool v = ok[2 + kk] && (hf * 64 + g * 8 < D);
+        sx_cp_async16(dst + j * 512, vp + (v ? of[2 + kk] + hf * 64 + g * 8 : 0), v);
+      }
+    }
+  };
+
+  const int nsteps = (k1 > k0) ? (k1 - k0 + 15) >> 4 : 0;
+  for (int i = 0; i < stages - 1; ++i) {
+    if (i < nsteps) issue(i, k0 + i * 16);
+    sx_cp_async_commit();
+  }
+  int buf = 0;
+  for (int it = 0; it < nsteps; ++it) {
+    const int s0 = k0 + it * 16;
+    sx_cp_async_wait_n(stages - 2);                         // this lane's copies of step `it` have landed
+    if (MULTI) sx_group_bar(grp, NT * 32);                   // ... and those of the other warps of the group
+    {
+      // the buffer consumed in the previous step is free now: request step it + STAGES - 1 into it
+      const int nb = (buf == 0) ? stages - 1 : buf - 1;
+      if (it + stages - 1 < nsteps) issue(nb, s0 + (stages - 1) * 16);
+      sx_cp_async_commit();
+    }
+    const uint4 *src = sx_stage + (size_t)(grp * stages + buf) * NL * 32 + lane;
+    // ---- S^T = K.Q^T for 16 keys x 8 queries: two accumulation chains --------------------------
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
-      dst[0][c] = make_uint4(0, 0, 0, 0);
-      dst[1][c] = make_uint4(0, 0, 0, 0);
-      if (c * 32 + t * 8 < D) {
-        if (ok0) dst[0][c] = *reinterpret_cast<const uint4 *>(kp + o0 + c * 32 + t * 8);
-        if (ok1) dst[1][c] = *reinterpret_cast<const uint4 *>(kp + o1 + c * 32 + t * 8);
-      }
+      const uint4 ka = src[c * 32], kb8 = src[(NC + c) * 32];      // keys g and g + 8
+      sx_mma_bf16(s, ka.x, kb8.x, ka.y, kb8.y, qb[c][0], qb[c][1]);
+      sx_mma_bf16(s2, ka.z, kb8.z, ka.w, kb8.w, qb[c][2], qb[c][3]);
     }
-  };
-  auto issue_v = [&](uint4 (&dst)[4][NH], int s0) {
-    bool ok[4];
-    size_t of[4];
-    if (one_page) {
-      bool okb;
-      const size_t base = row_offset(s0, okb);
+    // s[0], s[1]: key g, queries 2t, 2t+1;  s[2], s[3]: key g + 8
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk) {
-        const int key = (kk >> 1) * 8 + 2 * t + (kk & 1);
-        of[kk] = base + (size_t)key * D;
-        ok[kk] = okb && (s0 + key < k1);
-      }
-    } else {
-#pragma unroll
-      for (int kk = 0; kk < 4; ++kk) of[kk] = row_offset(s0 + (kk >> 1) * 8 + 2 * t + (kk & 1), ok[kk]);
-    }
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk)
-#pragma unroll
-      for (int hf = 0; hf < NH; ++hf) {
-        dst[kk][hf] = make_uint4(0, 0, 0, 0);
-        if (ok[kk] && hf * 64 + g * 8 < D) dst[kk][hf] = *reinterpret_cast<const uint4 *>(vp + of[kk] + hf * 64 + g * 8);
-      }
-  };
-  if (k0 < k1) {
-    issue_k(kr, k0);
-    issue_v(vr, k0);
-  }
-  for (int s0 = k0; s0 < k1; s0 += 16) {
-    const bool more = s0 + 16 < k1;
-    // ---- S = Q.K^T for 16 keys ----------------------------------------------------------
-    float s[2][4];
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt) {
-      s[nt][0] = 0.f; s[nt][1] = 0.f; s[nt][2] = 0.f; s[nt][3] = 0.f;
-#pragma unroll
-      for (int c = 0; c < NC; ++c) {
-        sx_mma_bf16(s[nt], qa[c][0], kr[nt][c].x, kr[nt][c].y);
-        sx_mma_bf16(s[nt], qa[c][1], kr[nt][c].z, kr[nt][c].w);
-      }
-    }
-    if (more) issue_k(kr, s0 + 16);
-    const bool edge = s0 + 16 > n;             // the step touches drafted rows or the end of the chunk
-#pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
+    for (int i = 0; i < 4; ++i) s[i] = (s[i] + s2[i]) * scale_log2;
+    if (s0 + 16 > n) {                       // the step touches drafted rows or the end of the chunk
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        float v = s[nt][i] * scale_log2;
-        if (edge) {
-          const int slot = s0 + nt * 8 + 2 * t + (i & 1);
-          const bool seen = slot < n || (slot < k1 && ((vis[i >> 1] >> (slot - n)) & 1ull));
-          if (!seen) v = -INFINITY;
-        }
-        s[nt][i] = v;
-      }
-    // ---- running softmax ---------------------------------------------------------------------
-    uint32_t pa[4];
-#pragma unroll
-    for (int rw = 0; rw < 2; ++rw) {
-      float mx = fmaxf(fmaxf(s[0][2 * rw], s[0][2 * rw + 1]), fmaxf(s[1][2 * rw], s[1][2 * rw + 1]));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      const float mnew = fmaxf(mrun[rw], mx);
-      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
-      const float corr = exp2f(mrun[rw] - msafe);
-      const float p00 = exp2f(s[0][2 * rw] - msafe), p01 = exp2f(s[0][2 * rw + 1] - msafe);
-      const float p10 = exp2f(s[1][2 * rw] - msafe), p11 = exp2f(s[1][2 * rw + 1] - msafe);
-      lrun[rw] = lrun[rw] * corr + ((p00 + p01) + (p10 + p11));
-      mrun[rw] = mnew;
-      pa[rw] = sx_pack_bf16x2(p00, p01);
-      pa[2 + rw] = sx_pack_bf16x2(p10, p11);
-      if (__any_sync(0xffffffffu, corr != 1.0f)) {
-#pragma unroll
-        for (int j = 0; j < NH * 8; ++j) { o[j][2 * rw] *= corr; o[j][2 * rw + 1] *= corr; }
+        const int slot = s0 + g + (i >> 1) * 8;
+        const bool seen = slot < n || (slot < k1 && ((vis[i & 1] >> (slot - n)) & 1ull));
+        if (!seen) s[i] = -INFINITY;
       }
     }
-    // ---- O += P.V ---------------------------------------------------------------------------------
+    // ---- running softmax over the keys (rows): lanes with equal t hold the same two queries ------
+    float corr[2];
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      float mx = fmaxf(s[i], s[2 + i]);
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+      const float mnew = fmaxf(mrun[i], mx);
+      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
+      corr[i] = sx_ex2(mrun[i] - msafe);
+      s[i] = sx_ex2(s[i] - msafe);
+      s[2 + i] = sx_ex2(s[2 + i] - msafe);
+      lrun[i] = lrun[i] * corr[i] + (s[i] + s[2 + i]);
+      mrun[i] = mnew;
+    }
+    if (__any_sync(0xffffffffu, corr[0] != 1.0f || corr[1] != 1.0f)) {
+#pragma unroll
+      for (int j = 0; j < NH * 4; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[1]; o[j][2] *= corr[0]; o[j][3] *= corr[1]; }
+    }
+    // P^T fragments: (P[key 2t][q g], P[key 2t+1][q g]) and the same for keys 8..15
+    const uint32_t pb0 = sx_movmatrix_trans(sx_pack_bf16x2(s[0], s[1]));
+    const uint32_t pb1 = sx_movmatrix_trans(sx_pack_bf16x2(s[2], s[3]));
+    // ---- O^T += V^T.P^T: row tile (hf, ep) holds d = hf*64 + g*8 + 2ep (row g) and + 1 (row g + 8) ---
+#pragma unroll
+    for (int hf = 0; hf < NH; ++hf) {
+      const uint4 v0 = src[(2 * NC + 0 * NH + hf) * 32], v1 = src[(2 * NC + 1 * NH + hf) * 32];
+      const uint4 v2 = src[(2 * NC + 2 * NH + hf) * 32], v3 = src[(2 * NC + 3 * NH + hf) * 32];
+#pragma unroll
+      for (int ep = 0; ep < 4; ++ep) {
+        const uint32_t w0 = sx_word(v0, ep), w1 = sx_word(v1, ep), w2 = sx_word(v2, ep), w3 = sx_word(v3, ep);
+        sx_mma_bf16(o[hf * 4 + ep], __byte_perm(w0, w1, 0x5410u), __byte_perm(w0, w1, 0x7632u),
+                    __byte_perm(w2, w3, 0x5410u), __byte_perm(w2, w3, 0x7632u), pb0, pb1);
+      }
+    }
+    buf = (buf + 1 == stages) ? 0 : buf + 1;
+  }
+  sx_cp_async_wait<0>();
+  if (__any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(status, SX_ERR_CAPACITY);
+  // ---- leave the partial result: O[q][d] natural order, d = hf*64 + g*8 + 2ep + {0, 1} -------------------
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    float l = lrun[i];
+    l += __shfl_xor_sync(0xffffffffu, l, 4);
+    l += __shfl_xor_sync(0xffffffffu, l, 8);
+    l += __shfl_xor_sync(0xffffffffu, l, 16);
+    if (!qv[i]) continue;
+    const size_t at = (size_t)hq[i] * nsplit + split;
+    if (g == 0) ws_ml[at] = make_float2(mrun[i], l);
+    float *dst = ws_o + at * D;
 #pragma unroll
     for (int hf = 0; hf < NH; ++hf)
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
-        const uint32_t b0 = __byte_perm(sx_word(vr[0][hf], e >> 1), sx_word(vr[1][hf], e >> 1), sel);
-        const uint32_t b1 = __byte_perm(sx_word(vr[2][hf], e >> 1), sx_word(vr[3][hf], e >> 1), sel);
-        sx_mma_bf16(o[hf * 8 + e], pa, b0, b1);
+      for (int ep = 0; ep < 4; ++ep) {
+        const int d = hf * 64 + g * 8 + 2 * ep;
+        if (d < D) *reinterpret_cast<float2 *>(dst + d) = make_float2(o[hf * 4 + ep][i], o[hf * 4 + ep][2 + i]);
       }
-    if (more) issue_v(vr, s0 + 16);
-  }
-  if (__any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(status, SX_ERR_CAPACITY);
-  // ---- leave the partial result ------------------------------------------------------------------
-#pragma unroll
-  for (int rw = 0; rw < 2; ++rw) {
-    float l = lrun[rw];
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (!qv[rw]) continue;
-    const size_t at = (size_t)hq[rw] * nsplit + split;
-    if (t == 0) ws_ml[at] = make_float2(mrun[rw], l);
-    float *dst = ws_o + at * DS;
-#pragma unroll
-    for (int j = 0; j < NH * 8; ++j)
-      *reinterpret_cast<float2 *>(dst + j * 8 + 2 * t) = make_float2(o[j][2 * rw], o[j][2 * rw + 1]);
   }
 }
 
 // o[hq][d] = sum_s O_s[d] 2^(m_s - M) / sum_s l_s 2^(m_s - M)
-__global__ void sx_attn_merge_kernel(int nq, int d, int ds, int nsplit, const float2 *__restrict__ ws_ml,
+__global__ void sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__restrict__ ws_ml,
                                      const float *__restrict__ ws_o, bf16 *__restrict__ o_out) {
   extern __shared__ float sx_w[];          // [nsplit] weights 2^(m_s - M)
   __shared__ float s_red[2];
@@ -282,30 +355,45 @@ __global__ void sx_attn_merge_kernel(int nq, int d, int ds, int nsplit, const fl
   __syncthreads();
   const float inv = 1.0f / s_red[0];
   for (int j = tid; j < d; j += blockDim.x) {
-    const int at = sx_attn_perm(j);
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
     int s = 0;
     for (; s + 4 <= nsplit; s += 4) {
-      a0 += ws_o[(hq * nsplit + s) * ds + at] * sx_w[s];
-      a1 += ws_o[(hq * nsplit + s + 1) * ds + at] * sx_w[s + 1];
-      a2 += ws_o[(hq * nsplit + s + 2) * ds + at] * sx_w[s + 2];
-      a3 += ws_o[(hq * nsplit + s + 3) * ds + at] * sx_w[s + 3];
+      a0 += ws_o[(hq * nsplit + s) * d + j] * sx_w[s];
+      a1 += ws_o[(hq * nsplit + s + 1) * d + j] * sx_w[s + 1];
+      a2 += ws_o[(hq * nsplit + s + 2) * d + j] * sx_w[s + 2];
+      a3 += ws_o[(hq * nsplit + s + 3) * d + j] * sx_w[s + 3];
     }
-    for (; s < nsplit; ++s) a0 += ws_o[(hq * nsplit + s) * ds + at] * sx_w[s];
+    for (; s < nsplit; ++s) a0 += ws_o[(hq * nsplit + s) * d + j] * sx_w[s];
     o_out[hq * d + j] = __float2bfloat16_rn(((a0 + a1) + (a2 + a3)) * inv);
   }
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static int attn_ds(int d) { return ((d + 63) / 64) * 64; }
+static int attn_loads(int d) { return 2 * ((d + 31) / 32) + 4 * ((d + 63) / 64); }
+static int attn_tiles(const SxShape &sh, int nr) { return (nr * (sh.nq / sh.nkv) + 7) / 8; }
+static int attn_groups_per_cta(int NT) { return NT >= 4 ? 1 : 4 / NT; }
 
-// Key chunks per (sequence, KV head, query tile): enough warps to fill the machine a few times
-// over, at least 64 keys each.
+void sx_attn_init(int device) {
+  const int smem = SX_ATTN_SMEM_BUDGET;
+  cudaFuncSetAttribute(sx_attn_mma_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+}
+
+// Key chunks per (sequence, KV head): enough warp groups to fill the machine a few times over,
+// at least 64 keys each.
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count) {
-  const int G = sh.nq / sh.nkv;
-  const int MT = (nr * G + 15) / 16;
-  const int groups = B * sh.nkv * MT;
-  int want = (sm_count * 8 * 3 + groups - 1) / groups;
+  const int NT = attn_tiles(sh, nr);
+  const int groups = B * sh.nkv;
+  static int waves = -1;
+  if (waves < 0) { const char *e = getenv("SX_ATTN_WAVES_DBG"); waves = e ? atoi(e) : 3; }
+  const int warps_wanted = sm_count * 12 * waves;
+  int want = (warps_wanted / NT + groups - 1) / groups;
   int by_len = (n_cap + 63) / 64;
   int s = want < by_len ? want : by_len;
   if (s < 1) s = 1;
@@ -320,25 +408,49 @@ size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_cou
       const size_t rows = (size_t)B * nr * sh.nq * sx_attn_splits(sh, B, nr, 1 << 30, sm_count);
       if (rows > worst) worst = rows;
     }
-  return worst * (attn_ds(sh.d) + 2) * sizeof(float);
+  return worst * (sh.d + 2) * sizeof(float);
 }
 
-bool sx_attn_supported(const SxShape &sh) { return sh.d == 16 || sh.d == 32 || sh.d == 64 || sh.d == 128; }
+bool sx_attn_supported(const SxShape &sh) {
+  return (sh.d == 16 || sh.d == 32 || sh.d == 64 || sh.d == 128) &&
+         attn_tiles(sh, SX_MAX_TOPK) <= SX_ATTN_MAX_TILES;
+}
 
 void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q, const sx_kv &kv,
                          int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st) {
   const int R = B * nr;
   const int G = sh.nq / sh.nkv;
-  const int MT = (nr * G + 15) / 16;
-  const int ds = attn_ds(sh.d);
+  const int NT = attn_tiles(sh, nr);
+  const int gpc = attn_groups_per_cta(NT);
   float2 *ws_ml = reinterpret_cast<float2 *>(ws);
   float *ws_o = ws + (size_t)R * sh.nq * nsplit * 2;
   const float scale_log2 = (float)(1.4426950408889634 / sqrt((double)sh.d));
-  dim3 grid((nsplit * MT + SX_ATTN_WARPS - 1) / SX_ATTN_WARPS, sh.nkv, B);
-  dim3 block(SX_ATTN_WARPS * 32);
-#define SX_ATTN(DD)                                                                                              \
-  sx_launch(sx_attn_mma_kernel<DD>, grid, block, 0, st, sh.nq, sh.nkv, G, sh.page, scale_log2, rm, nr, E, MT, q, kv, \
-            nsplit, ws_ml, ws_o, status)
+  int page_shift = -1;
+  if ((sh.page & (sh.page - 1)) == 0)
+    for (page_shift = 0; (1 << page_shift) < sh.page; ++page_shift) {}
+  dim3 grid((nsplit + gpc - 1) / gpc, sh.nkv, B);
+  dim3 block(32 * NT * gpc);
+  // Stages per group: a group of NT warps shares one ring, so it gets NT times the depth of a
+  // single warp's (two steps), within the shared-memory budget.
+  int stages = 2 * NT;
+  {
+    static int dbg = -1;
+    if (dbg < 0) { const char *e = getenv("SX_ATTN_STAGES_DBG"); dbg = e ? atoi(e) : 0; }
+    if (dbg > 0) stages = dbg * NT;
+  }
+  if (stages > SX_ATTN_MAX_STAGES) stages = SX_ATTN_MAX_STAGES;
+  const size_t stage_bytes = (size_t)attn_loads(sh.d) * 32 * sizeof(uint4);
+  while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
+  const size_t smem = (size_t)gpc * stages * stage_bytes;
+#define SX_ATTN(DD)                                                                                                    \
+  do {                                                                                                                 \
+    if (NT > 1)                                                                                                        \
+      sx_launch(sx_attn_mma_kernel<DD, true>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, \
+                rm, nr, E, NT, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status);                                       \
+    else                                                                                                               \
+      sx_launch(sx_attn_mma_kernel<DD, false>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift,            \
+                scale_log2, rm, nr, E, NT, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status);                           \
+  } while (0)
   switch (sh.d) {
     case 16: SX_ATTN(16); break;
     case 32: SX_ATTN(32); break;
@@ -346,6 +458,6 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
     default: SX_ATTN(128); break;
   }
 #undef SX_ATTN
-  sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3(128), (size_t)nsplit * sizeof(float), st, sh.nq, sh.d, ds, nsplit,
+  sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3(128), (size_t)nsplit * sizeof(float), st, sh.nq, sh.d, nsplit,
             (const float2 *)ws_ml, (const float *)ws_o, o_out);
 }

@@ -34,6 +34,7 @@ void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int sp
 // decode attention (sx_attention.cu).  B sequences with nr rows each this round, E drafted slots
 // behind the cached prefix (this round's rows included).
 bool sx_attn_supported(const SxShape &sh);
+void sx_attn_init(int device);
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count);
 size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_count);
 void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
