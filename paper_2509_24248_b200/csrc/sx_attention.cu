@@ -12,16 +12,13 @@
 // the 8-column side:
 //     S^T[key][q]  = sum_d K[key][d] Q[q][d]          A = K rows,   B = Q^T
 //     O^T[d][q]   += sum_key V[key][d] P[key][q]      A = V^T,      B = P^T
-// The contraction index of the first product and the row index of the second (both the head
-// dimension) may be permuted freely, so every lane fetches 8 consecutive elements of one K or
-// V row with one 16-byte copy and uses them as fragment entries of two k-steps (K) or of four
-// row tiles (V): each 32-byte sector that is fetched is fully used.  P^T is obtained from the
-// accumulator layout of S^T with two movmatrix transposes.
+// P^T is obtained from the accumulator layout of S^T with two movmatrix transposes.
 //
-// The copies are asynchronous (cp.async) into a small shared-memory ring addressed by lane, i.e.
-// the ring only extends the register file so that further 16-key steps are in flight while one
-// is being computed; a lane reads back what it, or the same lane of a sibling warp, requested,
-// so the ring needs no swizzle and, with one query tile, no barrier.
+// K and V rows are staged in a shared-memory ring by asynchronous 16-byte copies (cp.async) that
+// are fully coalesced - a step's 16 rows of one page are one contiguous block and every copy
+// instruction moves 512 consecutive bytes of it - and land at XOR-swizzled chunk positions, from
+// which ldmatrix (plain for K, transposing for V) delivers the A fragments without bank
+// conflicts or register shuffling.  Several 16-key steps are in flight while one is computed.
 //
 // Softmax is the usual running (max, sum) in fp32 with exponentials in base 2; P is rounded to
 // bf16 for the second product.  A warp leaves (m, l, unnormalised O) per query and chunk; the
@@ -59,9 +56,6 @@ __device__ __forceinline__ uint32_t sx_pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t *>(&v);
 }
-__device__ __forceinline__ uint32_t sx_word(const uint4 &u, int i) {
-  return i == 0 ? u.x : (i == 1 ? u.y : (i == 2 ? u.z : u.w));
-}
 // 16-byte asynchronous copy global -> shared; reads nothing and writes zeros when !valid
 __device__ __forceinline__ void sx_cp_async16(uint32_t smem_dst, const void *gsrc, bool valid) {
   const uint32_t bytes = valid ? 16u : 0u;
@@ -92,24 +86,44 @@ __device__ __forceinline__ void sx_group_bar(int grp, int threads) {
   else asm volatile("bar.sync 2, %0;" ::"r"(threads) : "memory");
 }
 
+// four 8x8 matrices of 16-bit elements from shared memory into MMA fragment registers; lane l
+// gives the address of row l % 8 of matrix l / 8
+__device__ __forceinline__ void sx_ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void sx_ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2,
+                                                     uint32_t &r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+// XOR applied to the 16-byte chunk index of a staged K/V row so that the eight rows of an
+// ldmatrix phase fall into different bank groups (rows are D * 2 bytes apart)
+template <int D>
+__device__ __forceinline__ int sx_attn_swz(int key) {
+  return D >= 64 ? (key & 7) : (D == 32 ? ((key >> 1) & 3) : ((key >> 2) & 1));
+}
+
 // NT = query tiles per (sequence, KV head) = warps per group (MULTI: NT > 1); gpc = groups per CTA.
 template <int D, bool MULTI>
 __global__ void __launch_bounds__(256, 1)
 sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale_log2, SxRowMap rm, int nr, int E,
-                   int NT, int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit, float2 *__restrict__ ws_ml,
-                   float *__restrict__ ws_o, int32_t *status) {
-  constexpr int NC = (D + 31) / 32;       // 32-element chunks of the head dimension (first product)
-  constexpr int NH = (D + 63) / 64;       // 64-element halves of the head dimension (second product)
-  constexpr int NL = 2 * NC + 4 * NH;     // 16-byte copies per lane and 16-key step
-  extern __shared__ uint4 sx_stage[];     // [groups][stages][NL][32 lanes]
+                   int NT, int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit,
+                   float2 *__restrict__ ws_ml, float *__restrict__ ws_o, int32_t *status) {
+  constexpr int CPR = D / 8;              // 16-byte chunks per K/V row
+  constexpr int NLK = D / 16;             // copies per lane for the 16 K rows of a step (as many for V)
+  constexpr int NKS = D / 16;             // k-steps of the first product = 16-row tiles of the second
+  constexpr int BLK = 16 * D * 2;         // bytes of the K (or V) block of a step
+  extern __shared__ uint4 sx_stage[];     // [groups][stages][K block | V block]
   sx_pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int grp = MULTI ? warp / NT : warp, qt = MULTI ? warp - grp * NT : 0;
   const int split = blockIdx.x * gpc + grp;
   if (grp >= gpc || split >= nsplit) return;
   const int b = blockIdx.z, h = blockIdx.y;
-  const uint32_t stg = (uint32_t)__cvta_generic_to_shared(sx_stage) +
-                       (uint32_t)((grp * stages * NL * 32 + lane) * sizeof(uint4));
+  const uint32_t stg = (uint32_t)__cvta_generic_to_shared(sx_stage) + (uint32_t)(grp * stages * 2 * BLK);
   sx_pdl_wait();
   const int n = rm.cache_len[b];
   const int total = n + E;
@@ -119,8 +133,8 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   const int k1 = min(total, k0 + chunk);
   const int NQ = nr * G;
 
-  // B fragments of Q^T: lane (g, t) holds query g of the tile, elements t*8.. of every 32-chunk
-  uint32_t qb[NC][4];
+  // B fragments of Q^T: lane (g, t) holds query g of the tile: elements 16ks + 2t, +1 and 16ks + 8 + 2t, +1
+  uint32_t qb[NKS][2];
   {
     const int m = qt * 8 + g;
     const bool valid = m < NQ;
@@ -128,10 +142,9 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     const int r = b * nr + j;
     const bf16 *qp = q + ((size_t)r * nq + h * G + (valid ? m - j * G : 0)) * D;
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      uint4 u = make_uint4(0, 0, 0, 0);
-      if (valid && c * 32 + t * 8 < D) u = *reinterpret_cast<const uint4 *>(qp + c * 32 + t * 8);
-      qb[c][0] = u.x; qb[c][1] = u.y; qb[c][2] = u.z; qb[c][3] = u.w;
+    for (int ks = 0; ks < NKS; ++ks) {
+      qb[ks][0] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 2 * t) : 0u;
+      qb[ks][1] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 8 + 2 * t) : 0u;
     }
   }
   // the two queries whose scores this lane holds (columns 2t and 2t + 1 of the tile)
@@ -149,9 +162,9 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     else vis[i] = (E >= 64) ? ~0ull : ((1ull << E) - 1ull);
   }
 
-  float o[NH * 4][4];
+  float o[NKS][4];
 #pragma unroll
-  for (int j = 0; j < NH * 4; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
+  for (int j = 0; j < NKS; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
   float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
 
   const bf16 *kp = reinterpret_cast<const bf16 *>(kv.k_pages_d);
@@ -165,10 +178,27 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   if (tbl_in_regs && lp_first + lane <= lp_last && lp_first + lane < kv.max_pages) tbl = table[lp_first + lane];
   bool bad = false;
   const bool one_page = (page & 15) == 0;        // chunks start on multiples of 16: a step never straddles pages
-  // element offsets of this lane inside a 16-key block that lies in one page
-  const int klane = g * D + t * 8;               // K: keys g and g + 8, elements t*8.. of every chunk
-  const int vlane = 2 * t * D + g * 8;           // V: keys 2t, 2t+1, 2t+8, 2t+9, elements g*8.. of every half
-
+  // ---- staging plan ---------------------------------------------------------------------------
+  // A step's 16 K rows (then its 16 V rows) are one contiguous block when they share a page; lane
+  // l of copy i moves the 16-byte chunk i * 32 + l of the block, i.e. every copy instruction reads
+  // 512 contiguous bytes.  In shared memory chunk j of row `key` sits at key * CPR + (j ^ swz(key)).
+  uint32_t cdst[NLK];
+#pragma unroll
+  for (int i = 0; i < NLK; ++i) {
+    const int ch = i * 32 + lane, key = ch / CPR, j = ch % CPR;
+    cdst[i] = (uint32_t)((key * CPR + (j ^ sx_attn_swz<D>(key))) * 16);
+  }
+  // ldmatrix row addresses (relative to the stage buffer) for every k-step / row tile
+  uint32_t ka[NKS], va[NKS];
+  {
+    const int keyA = (lane & 7) + ((lane >> 3) & 1) * 8, hiA = lane >> 4;
+    const int keyV = (lane & 7) + (lane >> 4) * 8, hiV = (lane >> 3) & 1;
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) {
+      ka[ks] = (uint32_t)(keyA * 2 * D + (((2 * ks + hiA) ^ sx_attn_swz<D>(keyA)) << 4));
+      va[ks] = (uint32_t)(BLK + keyV * 2 * D + (((2 * ks + hiV) ^ sx_attn_swz<D>(keyV)) << 4));
+    }
+  }
   // offset of the K/V row of `slot` (and whether it may be read); every lane takes part in the shuffle
   auto row_offset = [&](int slot, bool &ok) -> size_t {
     const bool live = slot < k1;
@@ -180,56 +210,35 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     if (live && !ok) bad = true;
     return ok ? (((size_t)pp * nkv + h) * page + (slot - lp * page)) * D : 0;
   };
-  // Requests the 16 keys from s0 into stage buffer `buf`: copy j < 2 NC is chunk j % NC of key
-  // g (j < NC) or g + 8, the others are half (j - 2 NC) % NH of the keys 2t, 2t+1, 2t+8, 2t+9.
-  // The NT warps of a group take every NT-th copy each (bit j of `mine`).
+  // The NT warps of a group take every NT-th copy each (bit c of `mine`; K copies first, then V).
   uint32_t mine = 0xffffffffu;
   if (MULTI) {
     mine = 0u;
-    for (int j = qt; j < NL; j += NT) mine |= 1u << j;
+    for (int c = qt; c < 2 * NLK; c += NT) mine |= 1u << c;
   }
   auto issue = [&](int buf, int s0) {
-    const uint32_t dst = stg + (uint32_t)(buf * NL * 32 * sizeof(uint4));
+    const uint32_t dst = stg + (uint32_t)(buf * 2 * BLK);
     bool okb = false;
     size_t base = 0;
     if (one_page) base = row_offset(s0, okb);
     if (one_page && okb && s0 + 16 <= k1) {
-      const bf16 *kb = kp + base + klane, *vb = vp + base + vlane;
+      const bf16 *kb = kp + base + lane * 8, *vb = vp + base + lane * 8;
 #pragma unroll
-      for (int j = 0; j < NL; ++j) {
-        if (MULTI && !((mine >> j) & 1u)) continue;
-        if (j < 2 * NC) {
-          const int nt = j / NC, c = j % NC;
-          if (D % 32 == 0) sx_cp_async16_full(dst + j * 512, kb + nt * 8 * D + c * 32);
-          else sx_cp_async16(dst + j * 512, kb + nt * 8 * D + c * 32, c * 32 + t * 8 < D);
-        } else {
-          const int kk = (j - 2 * NC) / NH, hf = (j - 2 * NC) % NH;
-          if (D % 64 == 0) sx_cp_async16_full(dst + j * 512, vb + ((kk >> 1) * 8 + (kk & 1)) * D + hf * 64);
-          else sx_cp_async16(dst + j * 512, vb + ((kk >> 1) * 8 + (kk & 1)) * D + hf * 64, hf * 64 + g * 8 < D);
-        }
+      for (int i = 0; i < NLK; ++i) {
+        if (!MULTI || ((mine >> i) & 1u)) sx_cp_async16_full(dst + cdst[i], kb + i * 256);
+        if (!MULTI || ((mine >> (NLK + i)) & 1u)) sx_cp_async16_full(dst + BLK + cdst[i], vb + i * 256);
       }
       return;
     }
-    bool ok[6];
-    size_t of[6];
 #pragma unroll
-    for (int i = 0; i < 6; ++i) {
-      const int key = (i < 2) ? i * 8 + g : ((i - 2) >> 1) * 8 + 2 * t + ((i - 2) & 1);
-      if (one_page) { of[i] = base + (size_t)key * D; ok[i] = okb && (s0 + key < k1); }
-      else of[i] = row_offset(s0 + key, ok[i]);
-    }
-#pragma unroll
-    for (int j = 0; j < NL; ++j) {
-      if (MULTI && !((mine >> j) & 1u)) continue;
-      if (j < 2 * NC) {
-        const int nt = j / NC, c = j % NC;
-        const bool v = ok[nt] && (c * 32 + t * 8 < D);
-        sx_cp_async16(dst + j * 512, kp + (v ? of[nt] + c * 32 + t * 8 : 0), v);
-      } else {
-        const int kk = (j - 2 * NC) / NH, hf = (j - 2 * NC) % NH;
-        const bool v = ok[2 + kk] && (hf * 64 + g * 8 < D);
-        sx_cp_async16(dst + j * 512, vp + (v ? of[2 + kk] + hf * 64 + g * 8 : 0), v);
-      }
+    for (int i = 0; i < NLK; ++i) {
+      const int ch = i * 32 + lane, key = ch / CPR, j = ch % CPR;
+      bool ok;
+      size_t of;
+      if (one_page) { of = base + (size_t)key * D; ok = okb && (s0 + key < k1); }
+      else of = row_offset(s0 + key, ok);
+      if (!MULTI || ((mine >> i) & 1u)) sx_cp_async16(dst + cdst[i], kp + (ok ? of + j * 8 : 0), ok);
+      if (!MULTI || ((mine >> (NLK + i)) & 1u)) sx_cp_async16(dst + BLK + cdst[i], vp + (ok ? of + j * 8 : 0), ok);
     }
   };
 
@@ -242,21 +251,23 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   for (int it = 0; it < nsteps; ++it) {
     const int s0 = k0 + it * 16;
     sx_cp_async_wait_n(stages - 2);                         // this lane's copies of step `it` have landed
-    if (MULTI) sx_group_bar(grp, NT * 32);                   // ... and those of the other warps of the group
+    if (MULTI) sx_group_bar(grp, NT * 32);                  // ... and those of every other lane of the group
+    else __syncwarp();
     {
-      // the buffer consumed in the previous step is free now: request step it + STAGES - 1 into it
+      // the buffer consumed in the previous step is free now: request step it + stages - 1 into it
       const int nb = (buf == 0) ? stages - 1 : buf - 1;
       if (it + stages - 1 < nsteps) issue(nb, s0 + (stages - 1) * 16);
       sx_cp_async_commit();
     }
-    const uint4 *src = sx_stage + (size_t)(grp * stages + buf) * NL * 32 + lane;
+    const uint32_t sb = stg + (uint32_t)(buf * 2 * BLK);
     // ---- S^T = K.Q^T for 16 keys x 8 queries: two accumulation chains --------------------------
     float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const uint4 ka = src[c * 32], kb8 = src[(NC + c) * 32];      // keys g and g + 8
-      sx_mma_bf16(s, ka.x, kb8.x, ka.y, kb8.y, qb[c][0], qb[c][1]);
-      sx_mma_bf16(s2, ka.z, kb8.z, ka.w, kb8.w, qb[c][2], qb[c][3]);
+    for (int ks = 0; ks < NKS; ++ks) {
+      uint32_t a0, a1, a2, a3;
+      sx_ldmatrix_x4(sb + ka[ks], a0, a1, a2, a3);
+      if (ks & 1) sx_mma_bf16(s2, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+      else sx_mma_bf16(s, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
     }
     // s[0], s[1]: key g, queries 2t, 2t+1;  s[2], s[3]: key g + 8
 #pragma unroll
@@ -287,28 +298,23 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     }
     if (__any_sync(0xffffffffu, corr[0] != 1.0f || corr[1] != 1.0f)) {
 #pragma unroll
-      for (int j = 0; j < NH * 4; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[1]; o[j][2] *= corr[0]; o[j][3] *= corr[1]; }
+      for (int j = 0; j < NKS; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[1]; o[j][2] *= corr[0]; o[j][3] *= corr[1]; }
     }
     // P^T fragments: (P[key 2t][q g], P[key 2t+1][q g]) and the same for keys 8..15
     const uint32_t pb0 = sx_movmatrix_trans(sx_pack_bf16x2(s[0], s[1]));
     const uint32_t pb1 = sx_movmatrix_trans(sx_pack_bf16x2(s[2], s[3]));
-    // ---- O^T += V^T.P^T: row tile (hf, ep) holds d = hf*64 + g*8 + 2ep (row g) and + 1 (row g + 8) ---
+    // ---- O^T += V^T.P^T: tile dt holds d = 16 dt + g (rows g) and 16 dt + 8 + g (rows g + 8) ------------
 #pragma unroll
-    for (int hf = 0; hf < NH; ++hf) {
-      const uint4 v0 = src[(2 * NC + 0 * NH + hf) * 32], v1 = src[(2 * NC + 1 * NH + hf) * 32];
-      const uint4 v2 = src[(2 * NC + 2 * NH + hf) * 32], v3 = src[(2 * NC + 3 * NH + hf) * 32];
-#pragma unroll
-      for (int ep = 0; ep < 4; ++ep) {
-        const uint32_t w0 = sx_word(v0, ep), w1 = sx_word(v1, ep), w2 = sx_word(v2, ep), w3 = sx_word(v3, ep);
-        sx_mma_bf16(o[hf * 4 + ep], __byte_perm(w0, w1, 0x5410u), __byte_perm(w0, w1, 0x7632u),
-                    __byte_perm(w2, w3, 0x5410u), __byte_perm(w2, w3, 0x7632u), pb0, pb1);
-      }
+    for (int dt = 0; dt < NKS; ++dt) {
+      uint32_t a0, a1, a2, a3;
+      sx_ldmatrix_x4_trans(sb + va[dt], a0, a1, a2, a3);
+      sx_mma_bf16(o[dt], a0, a1, a2, a3, pb0, pb1);
     }
     buf = (buf + 1 == stages) ? 0 : buf + 1;
   }
   sx_cp_async_wait<0>();
   if (__any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(status, SX_ERR_CAPACITY);
-  // ---- leave the partial result: O[q][d] natural order, d = hf*64 + g*8 + 2ep + {0, 1} -------------------
+  // ---- leave the partial result: O[q][d] ----------------------------------------------------------------
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     float l = lrun[i];
@@ -320,12 +326,10 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     if (g == 0) ws_ml[at] = make_float2(mrun[i], l);
     float *dst = ws_o + at * D;
 #pragma unroll
-    for (int hf = 0; hf < NH; ++hf)
-#pragma unroll
-      for (int ep = 0; ep < 4; ++ep) {
-        const int d = hf * 64 + g * 8 + 2 * ep;
-        if (d < D) *reinterpret_cast<float2 *>(dst + d) = make_float2(o[hf * 4 + ep][i], o[hf * 4 + ep][2 + i]);
-      }
+    for (int dt = 0; dt < NKS; ++dt) {
+      dst[dt * 16 + g] = o[dt][i];
+      dst[dt * 16 + 8 + g] = o[dt][2 + i];
+    }
   }
 }
 
@@ -369,7 +373,6 @@ __global__ void sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static int attn_loads(int d) { return 2 * ((d + 31) / 32) + 4 * ((d + 63) / 64); }
 static int attn_tiles(const SxShape &sh, int nr) { return (nr * (sh.nq / sh.nkv) + 7) / 8; }
 static int attn_groups_per_cta(int NT) { return NT >= 4 ? 1 : 4 / NT; }
 
@@ -439,7 +442,7 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
     if (dbg > 0) stages = dbg * NT;
   }
   if (stages > SX_ATTN_MAX_STAGES) stages = SX_ATTN_MAX_STAGES;
-  const size_t stage_bytes = (size_t)attn_loads(sh.d) * 32 * sizeof(uint4);
+  const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
   const size_t smem = (size_t)gpc * stages * stage_bytes;
 #define SX_ATTN(DD)                                                                                                    \
