@@ -30,6 +30,8 @@
 #define SX_A_BYTES (SX_TILE_M * SX_BK * 2)
 #define SX_WAIT_LIMIT (1u << 24)
 #define SX_SMEM_MAX 232448
+#define SX_ARGMAX_CHUNKS 8        // 32-row chunks of token rows in the plain-argmax epilogue (<= 256 rows)
+#define SX_ARGMAX_SMEM (128 * 33 * 4)
 
 struct SxTcParams {
   int n_rows, num_kb, R, nmma, num_tiles, splits, kb_per_split, stages, acc_cols, tmem_cols;
@@ -275,6 +277,88 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     int acc = 0;
     uint32_t acc_phase = 0;
     sx_pdl_wait();
+    if (HEAD && p.T == 1 && !p.lse) {
+      // Plain argmax (chain drafting, verification).  The logits of a tile go through a small
+      // shared-memory buffer, 32 token rows at a time, so that afterwards a thread owns one token
+      // row (column of the tile) and a quarter of the vocabulary rows: it scans them in index
+      // order with a strict compare and keeps its running best in registers for the whole
+      // kernel - no reductions across lanes and no atomics in the loop.
+      float *tb = reinterpret_cast<float *>(epi_smem);          // [128 rows][33]
+      const int tid = threadIdx.x - 64, col = tid & 31, part = tid >> 5;
+      float bestv[SX_ARGMAX_CHUNKS];
+      int besti[SX_ARGMAX_CHUNKS];
+#pragma unroll
+      for (int ch = 0; ch < SX_ARGMAX_CHUNKS; ++ch) { bestv[ch] = -INFINITY; besti[ch] = -1; }
+      for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
+        const int n = item * SX_TILE_M + et;
+        const bool in_vocab = n < p.V;
+        const bool is_signal = n >= p.V && n < p.V + p.S;
+#pragma unroll
+        for (int ch = 0; ch < SX_ARGMAX_CHUNKS; ++ch) {
+          if (ch * 32 < p.R) {
+            float v[32];
+            tc_ld16(taddr + ch * 32, v);
+            if (ch * 32 + 16 < p.nmma) tc_ld16(taddr + ch * 32 + 16, v + 16);
+            else {
+#pragma unroll
+              for (int j = 16; j < 32; ++j) v[j] = 0.f;
+            }
+            if ((ch + 1) * 32 >= p.R) {                           // last chunk: the accumulator is free again
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&tempty[acc]));
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) tb[et * 33 + j] = in_vocab ? v[j] : -INFINITY;
+            if (is_signal) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (ch * 32 + j < p.R) p.z[(size_t)(ch * 32 + j) * p.S + (n - p.V)] = v[j];
+            }
+            epi_bar();
+            if (ch * 32 + col < p.R) {
+              float bv = bestv[ch];
+              int bi = besti[ch];
+              const float *src = tb + (part * 32) * 33 + col;
+              const int base = item * SX_TILE_M + part * 32;
+#pragma unroll
+              for (int rr = 0; rr < 32; ++rr) {
+                const float x = src[rr * 33];
+                if (x > bv) { bv = x; bi = base + rr; }
+              }
+              bestv[ch] = bv;
+              besti[ch] = bi;
+            }
+            epi_bar();
+          }
+        }
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      // merge the four row quarters per token row (quarter order = index order) and leave the result
+      epi_bar();
+      int *ci = reinterpret_cast<int *>(tb + 4 * 256);
+#pragma unroll
+      for (int ch = 0; ch < SX_ARGMAX_CHUNKS; ++ch)
+        if (ch * 32 + col < p.R) { tb[part * 256 + ch * 32 + col] = bestv[ch]; ci[part * 256 + ch * 32 + col] = besti[ch]; }
+      epi_bar();
+      SxHeadPartial *out = p.parts + (size_t)blockIdx.x * p.part_stride;
+      for (int r = tid; r < p.R; r += 128) {
+        float bv = tb[r];
+        int bi = ci[r];
+        for (int w = 1; w < 4; ++w)
+          if (tb[w * 256 + r] > bv) { bv = tb[w * 256 + r]; bi = ci[w * 256 + r]; }
+        SxHeadPartial hp;
+        hp.top[0] = (bi >= 0) ? sx_pack(bv, (uint32_t)bi) : 0ull;
+#pragma unroll
+        for (int tt = 1; tt < SX_MAX_TOPK; ++tt) hp.top[tt] = 0ull;
+        hp.m = -INFINITY;
+        hp.l = 0.f;
+        out[r] = hp;
+      }
+    } else {
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
       const int tile = HEAD ? item : item / p.splits;
       const int sp = HEAD ? 0 : item % p.splits;
@@ -316,6 +400,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
     if (HEAD) {
       epi_bar();
       sx_head_flush(hs, p.R, et, p.parts + (size_t)blockIdx.x * p.part_stride);
+    }
     }
   }
   if (*abort_flag) {
@@ -451,7 +536,8 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
   if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T)) return SX_ERR_UNSUPPORTED;
   SxTcParams p;
   memset(&p, 0, sizeof(p));
-  const size_t epi = sx_head_smem_bytes(R, T, lse);
+  size_t epi = sx_head_smem_bytes(R, T, lse);
+  if (T == 1 && !lse && epi < SX_ARGMAX_SMEM) epi = SX_ARGMAX_SMEM;
   if (!fill_common(p, Ntot, K, R, epi)) return SX_ERR_UNSUPPORTED;
   p.splits = 1;
   p.kb_per_split = p.num_kb;
