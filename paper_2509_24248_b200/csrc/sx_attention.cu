@@ -106,16 +106,19 @@ __device__ __forceinline__ int sx_attn_swz(int key) {
   return D >= 64 ? (key & 7) : (D == 32 ? ((key >> 1) & 3) : ((key >> 2) & 1));
 }
 
-// NT = query tiles per (sequence, KV head) = warps per group (MULTI: NT > 1); gpc = groups per CTA.
-template <int D, bool MULTI>
+// NT = warps per group = query tiles per (sequence, KV head), rounded up to a power of two (a
+// warp without queries still does its share of the copies); gpc = groups per CTA.
+template <int D, int NT>
 __global__ void __launch_bounds__(256, 1)
 sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale_log2, SxRowMap rm, int nr, int E,
-                   int NT, int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit,
+                   int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit,
                    float2 *__restrict__ ws_ml, float *__restrict__ ws_o, int32_t *status) {
   constexpr int CPR = D / 8;              // 16-byte chunks per K/V row
   constexpr int NLK = D / 16;             // copies per lane for the 16 K rows of a step (as many for V)
   constexpr int NKS = D / 16;             // k-steps of the first product = 16-row tiles of the second
   constexpr int BLK = 16 * D * 2;         // bytes of the K (or V) block of a step
+  constexpr bool MULTI = NT > 1;
+  constexpr int CNT = (NLK + NT - 1) / NT;  // K copies (and V copies) this warp requests per step
   extern __shared__ uint4 sx_stage[];     // [groups][stages][K block | V block]
   sx_pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -182,11 +185,12 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   // A step's 16 K rows (then its 16 V rows) are one contiguous block when they share a page; lane
   // l of copy i moves the 16-byte chunk i * 32 + l of the block, i.e. every copy instruction reads
   // 512 contiguous bytes.  In shared memory chunk j of row `key` sits at key * CPR + (j ^ swz(key)).
-  uint32_t cdst[NLK];
+  // The NT warps of a group take every NT-th copy each: this warp's k-th copy is copy qt + k * NT.
+  uint32_t cdst[CNT];
 #pragma unroll
-  for (int i = 0; i < NLK; ++i) {
-    const int ch = i * 32 + lane, key = ch / CPR, j = ch % CPR;
-    cdst[i] = (uint32_t)((key * CPR + (j ^ sx_attn_swz<D>(key))) * 16);
+  for (int k = 0; k < CNT; ++k) {
+    const int ch = (qt + k * NT) * 32 + lane, key = ch / CPR, j = ch % CPR;
+    cdst[k] = (uint32_t)((key * CPR + (j ^ sx_attn_swz<D>(key))) * 16);
   }
   // ldmatrix row addresses (relative to the stage buffer) for every k-step / row tile
   uint32_t ka[NKS], va[NKS];
@@ -210,35 +214,33 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     if (live && !ok) bad = true;
     return ok ? (((size_t)pp * nkv + h) * page + (slot - lp * page)) * D : 0;
   };
-  // The NT warps of a group take every NT-th copy each (bit c of `mine`; K copies first, then V).
-  uint32_t mine = 0xffffffffu;
-  if (MULTI) {
-    mine = 0u;
-    for (int c = qt; c < 2 * NLK; c += NT) mine |= 1u << c;
-  }
   auto issue = [&](int buf, int s0) {
     const uint32_t dst = stg + (uint32_t)(buf * 2 * BLK);
     bool okb = false;
     size_t base = 0;
     if (one_page) base = row_offset(s0, okb);
     if (one_page && okb && s0 + 16 <= k1) {
-      const bf16 *kb = kp + base + lane * 8, *vb = vp + base + lane * 8;
+      const bf16 *kb = kp + base + (qt * 32 + lane) * 8, *vb = vp + base + (qt * 32 + lane) * 8;
 #pragma unroll
-      for (int i = 0; i < NLK; ++i) {
-        if (!MULTI || ((mine >> i) & 1u)) sx_cp_async16_full(dst + cdst[i], kb + i * 256);
-        if (!MULTI || ((mine >> (NLK + i)) & 1u)) sx_cp_async16_full(dst + BLK + cdst[i], vb + i * 256);
+      for (int k = 0; k < CNT; ++k) {
+        if (NLK % NT == 0 || qt + k * NT < NLK) {
+          sx_cp_async16_full(dst + cdst[k], kb + k * NT * 256);
+          sx_cp_async16_full(dst + BLK + cdst[k], vb + k * NT * 256);
+        }
       }
       return;
     }
 #pragma unroll
-    for (int i = 0; i < NLK; ++i) {
-      const int ch = i * 32 + lane, key = ch / CPR, j = ch % CPR;
+    for (int k = 0; k < CNT; ++k) {
+      const int ch = (qt + k * NT) * 32 + lane, key = ch / CPR, j = ch % CPR;
       bool ok;
       size_t of;
       if (one_page) { of = base + (size_t)key * D; ok = okb && (s0 + key < k1); }
-      else of = row_offset(s0 + key, ok);
-      if (!MULTI || ((mine >> i) & 1u)) sx_cp_async16(dst + cdst[i], kp + (ok ? of + j * 8 : 0), ok);
-      if (!MULTI || ((mine >> (NLK + i)) & 1u)) sx_cp_async16(dst + BLK + cdst[i], vp + (ok ? of + j * 8 : 0), ok);
+      else of = row_offset(s0 + (key < 16 ? key : 0), ok);
+      if (NLK % NT == 0 || qt + k * NT < NLK) {
+        sx_cp_async16(dst + cdst[k], kp + (ok ? of + j * 8 : 0), ok);
+        sx_cp_async16(dst + BLK + cdst[k], vp + (ok ? of + j * 8 : 0), ok);
+      }
     }
   };
 
@@ -373,19 +375,25 @@ __global__ void sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static int attn_tiles(const SxShape &sh, int nr) { return (nr * (sh.nq / sh.nkv) + 7) / 8; }
+static int attn_tiles(const SxShape &sh, int nr) {
+  const int t = (nr * (sh.nq / sh.nkv) + 7) / 8;
+  return t <= 1 ? 1 : (t <= 2 ? 2 : (t <= 4 ? 4 : 8));
+}
 static int attn_groups_per_cta(int NT) { return NT >= 4 ? 1 : 4 / NT; }
 
-void sx_attn_init(int device) {
+template <int D>
+static void attn_init_d() {
   const int smem = SX_ATTN_SMEM_BUDGET;
-  cudaFuncSetAttribute(sx_attn_mma_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+}
+void sx_attn_init(int device) {
+  attn_init_d<16>();
+  attn_init_d<32>();
+  attn_init_d<64>();
+  attn_init_d<128>();
 }
 
 // Key chunks per (sequence, KV head): enough warp groups to fill the machine a few times over,
@@ -445,21 +453,23 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
   const size_t smem = (size_t)gpc * stages * stage_bytes;
-#define SX_ATTN(DD)                                                                                                    \
-  do {                                                                                                                 \
-    if (NT > 1)                                                                                                        \
-      sx_launch(sx_attn_mma_kernel<DD, true>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, \
-                rm, nr, E, NT, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status);                                       \
-    else                                                                                                               \
-      sx_launch(sx_attn_mma_kernel<DD, false>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift,            \
-                scale_log2, rm, nr, E, NT, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status);                           \
-  } while (0)
+#define SX_ATTN_NT(DD, NN)                                                                                        \
+  sx_launch(sx_attn_mma_kernel<DD, NN>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, rm, \
+            nr, E, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status)
+#define SX_ATTN(DD)                                  \
+  switch (NT) {                                      \
+    case 1: SX_ATTN_NT(DD, 1); break;                \
+    case 2: SX_ATTN_NT(DD, 2); break;                \
+    case 4: SX_ATTN_NT(DD, 4); break;                \
+    default: SX_ATTN_NT(DD, 8); break;               \
+  }
   switch (sh.d) {
     case 16: SX_ATTN(16); break;
     case 32: SX_ATTN(32); break;
     case 64: SX_ATTN(64); break;
     default: SX_ATTN(128); break;
   }
+#undef SX_ATTN_NT
 #undef SX_ATTN
   sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3(128), (size_t)nsplit * sizeof(float), st, sh.nq, sh.d, nsplit,
             (const float2 *)ws_ml, (const float *)ws_o, o_out);
