@@ -106,9 +106,10 @@ __device__ __forceinline__ int sx_attn_swz(int key) {
   return D >= 64 ? (key & 7) : (D == 32 ? ((key >> 1) & 3) : ((key >> 2) & 1));
 }
 
-// NT = warps per group = query tiles per (sequence, KV head), rounded up to a power of two (a
-// warp without queries still does its share of the copies); gpc = groups per CTA.
-template <int D, int NT>
+// A warp handles NQT tiles of 8 queries (the A fragments of K and V are fetched once per step and
+// used for all of them); NT warps form a group that shares one staged copy of the keys and values
+// (a warp without queries still does its share of the copies); gpc = groups per CTA.
+template <int D, int NT, int NQT>
 __global__ void __launch_bounds__(256, 1)
 sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale_log2, SxRowMap rm, int nr, int E,
                    int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit,
@@ -137,38 +138,44 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   const int NQ = nr * G;
 
   // B fragments of Q^T: lane (g, t) holds query g of the tile: elements 16ks + 2t, +1 and 16ks + 8 + 2t, +1
-  uint32_t qb[NKS][2];
-  {
-    const int m = qt * 8 + g;
+  uint32_t qb[NQT][NKS][2];
+#pragma unroll
+  for (int u = 0; u < NQT; ++u) {
+    const int m = (qt * NQT + u) * 8 + g;
     const bool valid = m < NQ;
     const int j = valid ? m / G : 0;
     const int r = b * nr + j;
     const bf16 *qp = q + ((size_t)r * nq + h * G + (valid ? m - j * G : 0)) * D;
 #pragma unroll
     for (int ks = 0; ks < NKS; ++ks) {
-      qb[ks][0] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 2 * t) : 0u;
-      qb[ks][1] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 8 + 2 * t) : 0u;
+      qb[u][ks][0] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 2 * t) : 0u;
+      qb[u][ks][1] = valid ? *reinterpret_cast<const uint32_t *>(qp + ks * 16 + 8 + 2 * t) : 0u;
     }
   }
   // the two queries whose scores this lane holds (columns 2t and 2t + 1 of the tile)
-  int hq[2];
-  bool qv[2];
-  uint64_t vis[2];
+  int hq[NQT][2];
+  bool qv[NQT][2];
+  uint64_t vis[NQT][2];
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    const int m = qt * 8 + 2 * t + i;
-    qv[i] = m < NQ;
-    const int j = qv[i] ? m / G : 0;
-    const int r = b * nr + j;
-    hq[i] = r * nq + h * G + (qv[i] ? m - j * G : 0);
-    if (rm.mode == SX_MODE_TREE && rm.round > 1) vis[i] = rm.row_mask[r];
-    else vis[i] = (E >= 64) ? ~0ull : ((1ull << E) - 1ull);
-  }
+  for (int u = 0; u < NQT; ++u)
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int m = (qt * NQT + u) * 8 + 2 * t + i;
+      qv[u][i] = m < NQ;
+      const int j = qv[u][i] ? m / G : 0;
+      const int r = b * nr + j;
+      hq[u][i] = r * nq + h * G + (qv[u][i] ? m - j * G : 0);
+      if (rm.mode == SX_MODE_TREE && rm.round > 1) vis[u][i] = rm.row_mask[r];
+      else vis[u][i] = (E >= 64) ? ~0ull : ((1ull << E) - 1ull);
+    }
 
-  float o[NKS][4];
+  float o[NQT][NKS][4], mrun[NQT][2], lrun[NQT][2];
 #pragma unroll
-  for (int j = 0; j < NKS; ++j) { o[j][0] = 0.f; o[j][1] = 0.f; o[j][2] = 0.f; o[j][3] = 0.f; }
-  float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
+  for (int u = 0; u < NQT; ++u) {
+#pragma unroll
+    for (int j = 0; j < NKS; ++j) { o[u][j][0] = 0.f; o[u][j][1] = 0.f; o[u][j][2] = 0.f; o[u][j][3] = 0.f; }
+    mrun[u][0] = -INFINITY; mrun[u][1] = -INFINITY; lrun[u][0] = 0.f; lrun[u][1] = 0.f;
+  }
 
   const bf16 *kp = reinterpret_cast<const bf16 *>(kv.k_pages_d);
   const bf16 *vp = reinterpret_cast<const bf16 *>(kv.v_pages_d);
@@ -262,55 +269,70 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
       sx_cp_async_commit();
     }
     const uint32_t sb = stg + (uint32_t)(buf * 2 * BLK);
-    // ---- S^T = K.Q^T for 16 keys x 8 queries: two accumulation chains --------------------------
-    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- S^T = K.Q^T for 16 keys x 8 NQT queries: two accumulation chains per query tile -------
+    float s[NQT][4], s2[NQT][4];
+#pragma unroll
+    for (int u = 0; u < NQT; ++u)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { s[u][i] = 0.f; s2[u][i] = 0.f; }
 #pragma unroll
     for (int ks = 0; ks < NKS; ++ks) {
       uint32_t a0, a1, a2, a3;
       sx_ldmatrix_x4(sb + ka[ks], a0, a1, a2, a3);
-      if (ks & 1) sx_mma_bf16(s2, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-      else sx_mma_bf16(s, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-    }
-    // s[0], s[1]: key g, queries 2t, 2t+1;  s[2], s[3]: key g + 8
 #pragma unroll
-    for (int i = 0; i < 4; ++i) s[i] = (s[i] + s2[i]) * scale_log2;
-    if (s0 + 16 > n) {                       // the step touches drafted rows or the end of the chunk
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int slot = s0 + g + (i >> 1) * 8;
-        const bool seen = slot < n || (slot < k1 && ((vis[i & 1] >> (slot - n)) & 1ull));
-        if (!seen) s[i] = -INFINITY;
+      for (int u = 0; u < NQT; ++u) {
+        if (ks & 1) sx_mma_bf16(s2[u], a0, a1, a2, a3, qb[u][ks][0], qb[u][ks][1]);
+        else sx_mma_bf16(s[u], a0, a1, a2, a3, qb[u][ks][0], qb[u][ks][1]);
       }
     }
-    // ---- running softmax over the keys (rows): lanes with equal t hold the same two queries ------
-    float corr[2];
+    // s[u][0], s[u][1]: key g, queries 2t, 2t+1 of tile u;  s[u][2], s[u][3]: key g + 8
+    const bool edge = s0 + 16 > n;             // the step touches drafted rows or the end of the chunk
+    uint32_t pb0[NQT], pb1[NQT];
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      float mx = fmaxf(s[i], s[2 + i]);
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-      const float mnew = fmaxf(mrun[i], mx);
-      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
-      corr[i] = sx_ex2(mrun[i] - msafe);
-      s[i] = sx_ex2(s[i] - msafe);
-      s[2 + i] = sx_ex2(s[2 + i] - msafe);
-      lrun[i] = lrun[i] * corr[i] + (s[i] + s[2 + i]);
-      mrun[i] = mnew;
-    }
-    if (__any_sync(0xffffffffu, corr[0] != 1.0f || corr[1] != 1.0f)) {
+    for (int u = 0; u < NQT; ++u) {
 #pragma unroll
-      for (int j = 0; j < NKS; ++j) { o[j][0] *= corr[0]; o[j][1] *= corr[1]; o[j][2] *= corr[0]; o[j][3] *= corr[1]; }
+      for (int i = 0; i < 4; ++i) s[u][i] = (s[u][i] + s2[u][i]) * scale_log2;
+      if (edge) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int slot = s0 + g + (i >> 1) * 8;
+          const bool seen = slot < n || (slot < k1 && ((vis[u][i & 1] >> (slot - n)) & 1ull));
+          if (!seen) s[u][i] = -INFINITY;
+        }
+      }
+      // running softmax over the keys (rows): lanes with equal t hold the same two queries
+      float corr[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        float mx = fmaxf(s[u][i], s[u][2 + i]);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+        const float mnew = fmaxf(mrun[u][i], mx);
+        const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
+        corr[i] = sx_ex2(mrun[u][i] - msafe);
+        s[u][i] = sx_ex2(s[u][i] - msafe);
+        s[u][2 + i] = sx_ex2(s[u][2 + i] - msafe);
+        lrun[u][i] = lrun[u][i] * corr[i] + (s[u][i] + s[u][2 + i]);
+        mrun[u][i] = mnew;
+      }
+      if (__any_sync(0xffffffffu, corr[0] != 1.0f || corr[1] != 1.0f)) {
+#pragma unroll
+        for (int j = 0; j < NKS; ++j) {
+          o[u][j][0] *= corr[0]; o[u][j][1] *= corr[1]; o[u][j][2] *= corr[0]; o[u][j][3] *= corr[1];
+        }
+      }
+      // P^T fragments: (P[key 2t][q g], P[key 2t+1][q g]) and the same for keys 8..15
+      pb0[u] = sx_movmatrix_trans(sx_pack_bf16x2(s[u][0], s[u][1]));
+      pb1[u] = sx_movmatrix_trans(sx_pack_bf16x2(s[u][2], s[u][3]));
     }
-    // P^T fragments: (P[key 2t][q g], P[key 2t+1][q g]) and the same for keys 8..15
-    const uint32_t pb0 = sx_movmatrix_trans(sx_pack_bf16x2(s[0], s[1]));
-    const uint32_t pb1 = sx_movmatrix_trans(sx_pack_bf16x2(s[2], s[3]));
     // ---- O^T += V^T.P^T: tile dt holds d = 16 dt + g (rows g) and 16 dt + 8 + g (rows g + 8) ------------
 #pragma unroll
     for (int dt = 0; dt < NKS; ++dt) {
       uint32_t a0, a1, a2, a3;
       sx_ldmatrix_x4_trans(sb + va[dt], a0, a1, a2, a3);
-      sx_mma_bf16(o[dt], a0, a1, a2, a3, pb0, pb1);
+#pragma unroll
+      for (int u = 0; u < NQT; ++u) sx_mma_bf16(o[u][dt], a0, a1, a2, a3, pb0[u], pb1[u]);
     }
     buf = (buf + 1 == stages) ? 0 : buf + 1;
   }
@@ -318,21 +340,23 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
   if (__any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(status, SX_ERR_CAPACITY);
   // ---- leave the partial result: O[q][d] ----------------------------------------------------------------
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    float l = lrun[i];
-    l += __shfl_xor_sync(0xffffffffu, l, 4);
-    l += __shfl_xor_sync(0xffffffffu, l, 8);
-    l += __shfl_xor_sync(0xffffffffu, l, 16);
-    if (!qv[i]) continue;
-    const size_t at = (size_t)hq[i] * nsplit + split;
-    if (g == 0) ws_ml[at] = make_float2(mrun[i], l);
-    float *dst = ws_o + at * D;
+  for (int u = 0; u < NQT; ++u)
 #pragma unroll
-    for (int dt = 0; dt < NKS; ++dt) {
-      dst[dt * 16 + g] = o[dt][i];
-      dst[dt * 16 + 8 + g] = o[dt][2 + i];
+    for (int i = 0; i < 2; ++i) {
+      float l = lrun[u][i];
+      l += __shfl_xor_sync(0xffffffffu, l, 4);
+      l += __shfl_xor_sync(0xffffffffu, l, 8);
+      l += __shfl_xor_sync(0xffffffffu, l, 16);
+      if (!qv[u][i]) continue;
+      const size_t at = (size_t)hq[u][i] * nsplit + split;
+      if (g == 0) ws_ml[at] = make_float2(mrun[u][i], l);
+      float *dst = ws_o + at * D;
+#pragma unroll
+      for (int dt = 0; dt < NKS; ++dt) {
+        dst[dt * 16 + g] = o[u][dt][i];
+        dst[dt * 16 + 8 + g] = o[u][dt][2 + i];
+      }
     }
-  }
 }
 
 // o[hq][d] = sum_s O_s[d] 2^(m_s - M) / sum_s l_s 2^(m_s - M)
@@ -375,19 +399,25 @@ __global__ void sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-static int attn_tiles(const SxShape &sh, int nr) {
+// 8-query tiles per (sequence, KV head), rounded up to a power of two; a warp takes two of them
+// when there are at least two
+static int attn_qtiles(const SxShape &sh, int nr) {
   const int t = (nr * (sh.nq / sh.nkv) + 7) / 8;
   return t <= 1 ? 1 : (t <= 2 ? 2 : (t <= 4 ? 4 : 8));
+}
+static int attn_tiles(const SxShape &sh, int nr) {          // warps per group
+  const int t = attn_qtiles(sh, nr);
+  return t >= 2 ? t / 2 : 1;
 }
 static int attn_groups_per_cta(int NT) { return NT >= 4 ? 1 : 4 / NT; }
 
 template <int D>
 static void attn_init_d() {
   const int smem = SX_ATTN_SMEM_BUDGET;
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 void sx_attn_init(int device) {
   attn_init_d<16>();
@@ -424,7 +454,7 @@ size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_cou
 
 bool sx_attn_supported(const SxShape &sh) {
   return (sh.d == 16 || sh.d == 32 || sh.d == 64 || sh.d == 128) &&
-         attn_tiles(sh, SX_MAX_TOPK) <= SX_ATTN_MAX_TILES;
+         attn_qtiles(sh, SX_MAX_TOPK) <= SX_ATTN_MAX_TILES;
 }
 
 void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q, const sx_kv &kv,
@@ -453,15 +483,15 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
   const size_t smem = (size_t)gpc * stages * stage_bytes;
-#define SX_ATTN_NT(DD, NN)                                                                                        \
-  sx_launch(sx_attn_mma_kernel<DD, NN>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, rm, \
+#define SX_ATTN_NT(DD, NN, QQ)                                                                                    \
+  sx_launch(sx_attn_mma_kernel<DD, NN, QQ>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, rm, \
             nr, E, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status)
 #define SX_ATTN(DD)                                  \
-  switch (NT) {                                      \
-    case 1: SX_ATTN_NT(DD, 1); break;                \
-    case 2: SX_ATTN_NT(DD, 2); break;                \
-    case 4: SX_ATTN_NT(DD, 4); break;                \
-    default: SX_ATTN_NT(DD, 8); break;               \
+  switch (attn_qtiles(sh, nr)) {                     \
+    case 1: SX_ATTN_NT(DD, 1, 1); break;             \
+    case 2: SX_ATTN_NT(DD, 1, 2); break;             \
+    case 4: SX_ATTN_NT(DD, 2, 2); break;             \
+    default: SX_ATTN_NT(DD, 4, 2); break;            \
   }
   switch (sh.d) {
     case 16: SX_ATTN(16); break;
