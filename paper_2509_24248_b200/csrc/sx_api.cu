@@ -253,7 +253,7 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
 static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
                       int32_t *status, cudaStream_t st) {
-  const int cap = sx_head_max_rows(T);
+  const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
   for (int r0 = 0; r0 < R; r0 += cap) {

@@ -10,7 +10,6 @@ typedef __nv_bfloat16 bf16;
 
 #define SX_WARP 32
 #define SX_TILE_M 128          // weight rows per GEMM tile
-#define SX_HEAD_PEND 128       // pending top-k entries per row and tile (= SX_TILE_M)
 
 // How the rows of one draft round map to sequences, positions and cache slots.
 struct SxRowMap {
@@ -117,8 +116,8 @@ __device__ __forceinline__ float sx_activate(float z, int act) {
 }
 
 // ----------------------------------------------------------------------------------------
-// Head epilogue state: per-row running top-T (value, index) and log-sum-exp over the
-// vocabulary rows a CTA has seen.  Lives in shared memory; see sx_head_epilogue.cuh.
+// What a CTA of the head kernel leaves per token row for the merge kernel: its top-T (value,
+// index) pairs and the log-sum-exp state over the vocabulary rows it has seen.
 // ----------------------------------------------------------------------------------------
 struct SxHeadPartial {       // what a CTA leaves behind for the merge, per row
   unsigned long long top[SX_MAX_TOPK];   // packed (value, index), best first; 0 = empty

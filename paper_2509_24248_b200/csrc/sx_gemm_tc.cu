@@ -22,7 +22,6 @@
 #include <mutex>
 #include <unordered_map>
 
-#include "sx_head_epilogue.cuh"
 #include "sx_kernels.cuh"
 #include "sx_launch.cuh"
 
@@ -32,6 +31,7 @@
 #define SX_SMEM_MAX 232448
 #define SX_ARGMAX_CHUNKS 8        // 32-row chunks of token rows in the plain-argmax epilogue (<= 256 rows)
 #define SX_ARGMAX_SMEM (128 * 33 * 4)
+#define SX_TOPK_SMEM (4 * 64 * 18 * 4)  // merge buffer of the top-8 epilogue: 4 quarters x 64 rows x 18 words
 
 struct SxTcParams {
   int n_rows, num_kb, R, nmma, num_tiles, splits, kb_per_split, stages, acc_cols, tmem_cols;
@@ -190,11 +190,6 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
   if (warp == 1) {
     tc_alloc(smem_u32(tmem_slot), (uint32_t)p.tmem_cols);
     tc_relinquish();
-  }
-  SxHeadSmem hs;
-  if (HEAD) {
-    hs = sx_head_carve(epi_smem, p.R, p.T, p.lse);
-    if (warp >= 2) sx_head_init(hs, p.R, threadIdx.x - 64);
   }
   tc_fence_before();
   __syncthreads();
@@ -358,49 +353,174 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         hp.l = 0.f;
         out[r] = hp;
       }
+    } else if (HEAD) {
+      // Top-8 (value, index) and log-sum-exp per token row (tree drafting; at most 64 token rows).
+      // Same data flow as above: a thread owns one token row and a quarter of the vocabulary rows
+      // of each tile, and keeps a sorted list of its 8 best and a running (max, sum) in registers.
+      float *tb = reinterpret_cast<float *>(epi_smem);          // [128 rows][33]
+      const int tid = threadIdx.x - 64, col = tid & 31, part = tid >> 5;
+      const float LOG2E = 1.4426950408889634f;
+      float tv[2][8], m2[2], ll[2];
+      int ti[2][8];
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch) {
+        m2[ch] = -INFINITY;
+        ll[ch] = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { tv[ch][k] = -INFINITY; ti[ch][k] = -1; }
+      }
+      for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
+        const int n = item * SX_TILE_M + et;
+        const bool in_vocab = n < p.V;
+        const bool is_signal = n >= p.V && n < p.V + p.S;
+#pragma unroll
+        for (int ch = 0; ch < 2; ++ch) {
+          if (ch * 32 < p.R) {
+            {
+              float v[32];
+              tc_ld16(taddr + ch * 32, v);
+              if (ch * 32 + 16 < p.nmma) tc_ld16(taddr + ch * 32 + 16, v + 16);
+              else {
+#pragma unroll
+                for (int j = 16; j < 32; ++j) v[j] = 0.f;
+              }
+              if ((ch + 1) * 32 >= p.R) {                         // last chunk: the accumulator is free again
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tempty[acc]));
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) tb[et * 33 + j] = in_vocab ? v[j] : -INFINITY;
+              if (is_signal) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (ch * 32 + j < p.R) p.z[(size_t)(ch * 32 + j) * p.S + (n - p.V)] = v[j];
+              }
+            }
+            epi_bar();
+            if (ch * 32 + col < p.R) {
+              const float *src = tb + (part * 32) * 33 + col;
+              const int base = item * SX_TILE_M + part * 32;
+              float x[32];
+#pragma unroll
+              for (int rr = 0; rr < 32; ++rr) x[rr] = src[rr * 33];
+              if (p.lse) {
+                float mx = x[0];
+#pragma unroll
+                for (int rr = 1; rr < 32; ++rr) mx = fmaxf(mx, x[rr]);
+                const float mnew = fmaxf(m2[ch], mx * LOG2E);
+                if (mnew > -INFINITY) {
+                  float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                  for (int rr = 0; rr < 32; rr += 2) {
+                    a0 += exp2f(fmaf(x[rr], LOG2E, -mnew));
+                    a1 += exp2f(fmaf(x[rr + 1], LOG2E, -mnew));
+                  }
+                  ll[ch] = ll[ch] * exp2f(m2[ch] - mnew) + (a0 + a1);
+                  m2[ch] = mnew;
+                }
+              }
+#pragma unroll
+              for (int rr = 0; rr < 32; ++rr) {
+                const float xv = x[rr];
+                if (xv > tv[ch][7]) {
+                  // entries >= xv stay in front of it (they have lower indices), the rest move down
+                  bool ge[8];
+#pragma unroll
+                  for (int k = 0; k < 8; ++k) ge[k] = tv[ch][k] >= xv;
+#pragma unroll
+                  for (int k = 7; k >= 1; --k) {
+                    tv[ch][k] = ge[k] ? tv[ch][k] : (ge[k - 1] ? xv : tv[ch][k - 1]);
+                    ti[ch][k] = ge[k] ? ti[ch][k] : (ge[k - 1] ? base + rr : ti[ch][k - 1]);
+                  }
+                  if (!ge[0]) { tv[ch][0] = xv; ti[ch][0] = base + rr; }
+                }
+              }
+            }
+            epi_bar();
+          }
+        }
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      // merge the four row quarters per token row, in quarter (= index) order
+      epi_bar();
+      int *tbi = reinterpret_cast<int *>(tb);
+#pragma unroll
+      for (int ch = 0; ch < 2; ++ch)
+        if (ch * 32 + col < p.R) {
+          const int at = (part * 64 + ch * 32 + col) * 18;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) { tb[at + k] = tv[ch][k]; tbi[at + 8 + k] = ti[ch][k]; }
+          tb[at + 16] = m2[ch];
+          tb[at + 17] = ll[ch];
+        }
+      epi_bar();
+      SxHeadPartial *out = p.parts + (size_t)blockIdx.x * p.part_stride;
+      if (tid < p.R) {
+        const int r = tid;
+        float bv[8], M = tb[r * 18 + 16];
+        int bi[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { bv[k] = tb[r * 18 + k]; bi[k] = tbi[r * 18 + 8 + k]; }
+        for (int w = 1; w < 4; ++w) {
+          const int at = (w * 64 + r) * 18;
+          M = fmaxf(M, tb[at + 16]);
+          for (int e = 0; e < 8; ++e) {
+            const float xv = tb[at + e];
+            const int xi = tbi[at + 8 + e];
+            if (xv > bv[7]) {
+              bool ge[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) ge[k] = bv[k] >= xv;
+#pragma unroll
+              for (int k = 7; k >= 1; --k) {
+                bv[k] = ge[k] ? bv[k] : (ge[k - 1] ? xv : bv[k - 1]);
+                bi[k] = ge[k] ? bi[k] : (ge[k - 1] ? xi : bi[k - 1]);
+              }
+              if (!ge[0]) { bv[0] = xv; bi[0] = xi; }
+            }
+          }
+        }
+        float L = 0.f;
+        for (int w = 0; w < 4; ++w) {
+          const int at = (w * 64 + r) * 18;
+          if (tb[at + 17] > 0.f) L += tb[at + 17] * exp2f(tb[at + 16] - M);
+        }
+        SxHeadPartial hp;
+#pragma unroll
+        for (int k = 0; k < SX_MAX_TOPK; ++k)
+          hp.top[k] = (k < p.T && bi[k] >= 0) ? sx_pack(bv[k], (uint32_t)bi[k]) : 0ull;
+        hp.m = (L > 0.f) ? M * 0.6931471805599453f : -INFINITY;
+        hp.l = L;
+        out[r] = hp;
+      }
     } else {
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
-      const int tile = HEAD ? item : item / p.splits;
-      const int sp = HEAD ? 0 : item % p.splits;
-      if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
-      tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
-      const int n = tile * SX_TILE_M + et;
-      for (int c0 = 0; c0 < p.nmma && c0 < p.R; c0 += 16) {
-        float v[16];
-        tc_ld16(taddr + c0, v);
-        if (!HEAD) {
+      // plain GEMM: this split's partial sums to global memory
+      for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int tile = item / p.splits;
+        const int sp = item % p.splits;
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
+        const int n = tile * SX_TILE_M + et;
+        for (int c0 = 0; c0 < p.nmma && c0 < p.R; c0 += 16) {
+          float v[16];
+          tc_ld16(taddr + c0, v);
           if (n < p.n_rows) {
             float *dst = p.part + (size_t)sp * p.split_stride + n;
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               if (c0 + j < p.R) dst[(size_t)(c0 + j) * p.n_rows] = v[j];
           }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int r = c0 + j;
-            if (r < p.R) {
-              sx_head_column(hs, r, v[j], (uint32_t)n, n < p.V, q, lane);
-              if (n >= p.V && n < p.V + p.S) p.z[(size_t)r * p.S + (n - p.V)] = v[j];
-            }
-          }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tempty[acc]));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tempty[acc]));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-      if (HEAD && p.T > 1) {
-        epi_bar();
-        sx_head_merge_pending(hs, p.R, et);
-        epi_bar();
-      }
-    }
-    if (HEAD) {
-      epi_bar();
-      sx_head_flush(hs, p.R, et, p.parts + (size_t)blockIdx.x * p.part_stride);
-    }
     }
   }
   if (*abort_flag) {
@@ -528,16 +648,15 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
   return SX_OK;
 }
 
-int sx_head_max_rows(int T) { return T > 1 ? 64 : 256; }
+int sx_head_max_rows(int T, int lse) { return (T == 1 && !lse) ? 256 : 64; }
 
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
                          cudaStream_t st) {
-  if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T)) return SX_ERR_UNSUPPORTED;
+  if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T, lse)) return SX_ERR_UNSUPPORTED;
   SxTcParams p;
   memset(&p, 0, sizeof(p));
-  size_t epi = sx_head_smem_bytes(R, T, lse);
-  if (T == 1 && !lse && epi < SX_ARGMAX_SMEM) epi = SX_ARGMAX_SMEM;
+  const size_t epi = (T == 1 && !lse) ? SX_ARGMAX_SMEM : SX_TOPK_SMEM;
   if (!fill_common(p, Ntot, K, R, epi)) return SX_ERR_UNSUPPORTED;
   p.splits = 1;
   p.kb_per_split = p.num_kb;

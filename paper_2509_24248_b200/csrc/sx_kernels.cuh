@@ -84,4 +84,4 @@ void sx_gemm_init(int device);
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
                          int32_t *status, cudaStream_t st);
-int sx_head_max_rows(int T);
+int sx_head_max_rows(int T, int lse);
