@@ -24,7 +24,6 @@
 // bf16 for the second product.  A warp leaves (m, l, unnormalised O) per query and chunk; the
 // merge kernel combines the chunks and writes bf16.
 #include <math.h>
-#include <stdlib.h>
 
 #include "sx_kernels.cuh"
 #include "sx_launch.cuh"
@@ -431,9 +430,7 @@ void sx_attn_init(int device) {
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count) {
   const int NT = attn_tiles(sh, nr);
   const int groups = B * sh.nkv;
-  static int waves = -1;
-  if (waves < 0) { const char *e = getenv("SX_ATTN_WAVES_DBG"); waves = e ? atoi(e) : 3; }
-  const int warps_wanted = sm_count * 12 * waves;
+  const int warps_wanted = sm_count * 12 * 3;
   int want = (warps_wanted / NT + groups - 1) / groups;
   int by_len = (n_cap + 63) / 64;
   int s = want < by_len ? want : by_len;
@@ -474,11 +471,6 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   // Stages per group: a group of NT warps shares one ring, so it gets NT times the depth of a
   // single warp's (two steps), within the shared-memory budget.
   int stages = 2 * NT;
-  {
-    static int dbg = -1;
-    if (dbg < 0) { const char *e = getenv("SX_ATTN_STAGES_DBG"); dbg = e ? atoi(e) : 0; }
-    if (dbg > 0) stages = dbg * NT;
-  }
   if (stages > SX_ATTN_MAX_STAGES) stages = SX_ATTN_MAX_STAGES;
   const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
