@@ -57,6 +57,28 @@ def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
     return {"total": total, "head_launch": 2 * head, "w_round": w_round, "kv_round": kv_round}
 
 
+def max_over_ranks(ms_local: float, dist, device) -> float:
+    """Replicas share nothing on the data path; the job's time is the slowest rank's."""
+    if dist is None:
+        return float(ms_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, dist, device) -> float:
+    if dist is None:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def whole_job_rate(units_all_ranks: float, ms_total: float) -> float:
+    """Units processed by all ranks per second of the slowest rank's time."""
+    return units_all_ranks / (ms_total / 1e3)
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -276,14 +298,10 @@ def main():
     torch.cuda.synchronize()
     prof = sx.profile_end()
     clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms = ms_total / args.steps
-    value = world * 1e3 / ms
-    vtok = world * float(verified.item()) / (ms_total / 1e3)
+    value = whole_job_rate(world * args.steps, ms_total)
+    vtok = whole_job_rate(sum_over_ranks(float(verified.item()), dist, dev), ms_total)
 
     # end to end: host buffers in, results out, through the host entry point
     stage = {"feat0": torch.empty_like(f0_d), "tok0": torch.empty_like(t0_d), "target_hidden": torch.empty_like(th_d)}
@@ -305,10 +323,7 @@ def main():
         sx.sx_spec_exit_iter_host(params, state, f0_h, t0_h, th_h, stage, out, res_h)
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t_start) * 1e3 / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = wl.B * H * 2 + wl.B * 4 + wl.B * P * H * 2
     d2h = wl.B * (3 * 4 + S * 4)
 
