@@ -252,7 +252,7 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
 // head over R rows in chunks the kernel can hold; merges into tok/logp/signals
 static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
-                      int32_t *status, cudaStream_t st) {
+                      int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0}) {
   const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
@@ -267,7 +267,8 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
     if (s2.idx) s2.idx += r0; else s2.add += r0 * s2.mul;
     sx_launch_head_finalize(c->sh, rc, parts, G, c->head_rows, T, lse, z, S, tok_out, t2,
-                            logp_out ? logp_out + (size_t)r0 * T : nullptr, sig_out, s2, st);
+                            logp_out ? logp_out + (size_t)r0 * T : nullptr, sig_out, s2, st,
+                            (R <= cap) ? nx : SxNextInput{nullptr, nullptr, nullptr, 0, 0});
     c->launches += 2;
   }
   return SX_OK;
@@ -276,7 +277,7 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
 static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const bf16 *feat, SxIndex fi,
                              const int32_t *tok, SxIndex ti, const uint64_t *row_mask, bf16 *hid_user, SxIndex ui,
                              int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si, char *ws,
-                             int32_t *status, cudaStream_t st) {
+                             int32_t *status, cudaStream_t st, bool input_ready = false, bool prepare_next = false) {
   const SxShape &s = c->sh;
   bf16 *u = (bf16 *)(ws + c->off_u), *x = (bf16 *)(ws + c->off_x), *n = (bf16 *)(ws + c->off_n);
   bf16 *q = (bf16 *)(ws + c->off_q), *o = (bf16 *)(ws + c->off_o), *a = (bf16 *)(ws + c->off_a);
@@ -286,7 +287,11 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   rm.mode = c->dc.mode; rm.round = round; rm.topk = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1; rm.R = R;
   rm.cache_len = kv->cache_len_d; rm.row_mask = row_mask;
   int sp; size_t stride;
-  sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
+  // input_ready: the previous round's merge kernel has already written u (chain drafting)
+  if (!input_ready) {
+    sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
+    c->launches += 1;
+  }
   SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
@@ -303,10 +308,12 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   sx_launch_finish_swiglu(s, R, part, sp, stride, m, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_DOWN, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
   sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
-  c->launches += 8;   // embed, 3 norms, rope, attention x2, swiglu
+  c->launches += 7;   // 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
   SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
-              status, st));
+              status, st,
+              prepare_next ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
+                           : SxNextInput{nullptr, nullptr, nullptr, 0, 0}));
   return SX_OK;
 }
 
@@ -385,12 +392,13 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
   if (c->dc.mode == SX_MODE_CHAIN) {
     sx_launch_chain_layout(B, K, S, tok0_d, *o, st);
     c->launches += 1;
+    const bool fuse = B <= sx_head_max_rows(1, 0);     // one head launch per round: its merge can write the next input
     for (int k = 1; k <= K; ++k) {
       const bf16 *feat = (k == 1) ? (const bf16 *)feat0_d : hid;
       SxIndex fi = (k == 1) ? SxIndex{nullptr, 1, 0} : SxIndex{nullptr, K, k - 2};
       SX_TRY(draft_round(c, kv, k, B, feat, fi, o->cand_tok_d, SxIndex{nullptr, P, k - 1}, nullptr, hid,
                          SxIndex{nullptr, K, k - 1}, o->cand_tok_d, SxIndex{nullptr, P, k}, nullptr,
-                         o->slot_signal_d, SxIndex{nullptr, P, k - 1}, ws, status_d, st));
+                         o->slot_signal_d, SxIndex{nullptr, P, k - 1}, ws, status_d, st, k > 1 && fuse, k < K && fuse));
     }
     SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
                      K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));

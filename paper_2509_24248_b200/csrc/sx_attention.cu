@@ -436,13 +436,13 @@ void sx_attn_init(int device) {
 }
 
 // Key chunks per (sequence, KV head): enough warp groups to fill the machine a few times over,
-// at least 64 keys each.
+// at least 32 keys each.
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count) {
   const int NT = attn_tiles(sh, nr);
   const int groups = B * sh.nkv;
   const int warps_wanted = sm_count * 12 * 3;
   int want = (warps_wanted / NT + groups - 1) / groups;
-  int by_len = (n_cap + 63) / 64;
+  int by_len = (n_cap + 31) / 32;
   int s = want < by_len ? want : by_len;
   if (s < 1) s = 1;
   if (s > 256) s = 256;

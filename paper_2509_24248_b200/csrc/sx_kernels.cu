@@ -58,13 +58,16 @@ __device__ __forceinline__ float4 sx_sum_splits4(const float *p, int splits, siz
   return a;
 }
 
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(1024)
 sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t split_stride,
                       const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
                       bf16 *out_user, SxIndex ui) {
-  extern __shared__ float sx_buf[];
+  extern __shared__ float sx_buf[];        // [H] values, then [H / 2] words of gain (bf16 pairs)
   __shared__ float red[32];
+  uint2 *gam = reinterpret_cast<uint2 *>(sx_buf + H);
   sx_pdl_launch_dependents();
+  // the gain is a weight: fetch it (from HBM) before waiting for the GEMM
+  for (int i = threadIdx.x; i < H / 4; i += blockDim.x) gam[i] = reinterpret_cast<const uint2 *>(gamma)[i];
   sx_pdl_wait();
   const int r = blockIdx.x;
   float ss = 0.f;
@@ -90,17 +93,16 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
   ss = sx_warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float t = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
-    t = sx_warp_sum(t);
-    if (threadIdx.x == 0) red[0] = t;
+  float tot = 0.f;
+  {
+    const int nw = blockDim.x >> 5;
+    for (int w = 0; w < nw; ++w) tot += red[w];           // same order in every thread
   }
-  __syncthreads();
-  const float scale = rsqrtf(red[0] / (float)H + eps);
+  const float scale = rsqrtf(tot / (float)H + eps);
   bf16 *user = out_user ? out_user + (size_t)sx_index(ui, r) * H : nullptr;
   for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4 *>(sx_buf + i);
-    const uint2 gu = *reinterpret_cast<const uint2 *>(gamma + i);
+    const uint2 gu = gam[i >> 2];
     const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gu.x));
     const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gu.y));
     __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x * scale * g0.x, v.y * scale * g0.y);
@@ -117,9 +119,11 @@ void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int spli
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
                            bf16 *out_user, SxIndex ui, cudaStream_t st) {
   int threads = ((sh.H / 4 + 31) / 32) * 32;
-  if (threads > 512) threads = 512;
-  sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * sizeof(float), st, sh.H, sh.eps, part, splits,
-            split_stride, residual, gamma, out_v, out_n, out_user, ui);
+  if (threads > 1024) threads = 1024;
+  if (sh.H * 6 > 48 * 1024)
+    cudaFuncSetAttribute(sx_finish_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.H * 6);
+  sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * (sizeof(float) + sizeof(bf16)), st, sh.H, sh.eps, part,
+            splits, split_stride, residual, gamma, out_v, out_n, out_user, ui);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -221,12 +225,13 @@ void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int sp
 // ---------------------------------------------------------------------------------------
 __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
                                         const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
-                                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si) {
-  sx_pdl_launch_dependents();
-  sx_pdl_wait();
+                                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si, SxNextInput nx) {
   extern __shared__ unsigned long long sx_cand[];      // [G * T]
   __shared__ unsigned long long wbest[4];
   __shared__ float s_lse;
+  __shared__ int s_tok;
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
   const int r = blockIdx.x, tid = threadIdx.x;
   for (int i = tid; i < G * T; i += blockDim.x) sx_cand[i] = parts[(size_t)(i / T) * part_stride + r].top[i % T];
   if (tid == 0 && lse) {
@@ -250,6 +255,7 @@ __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int p
     best = max(max(wbest[0], wbest[1]), max(wbest[2], wbest[3]));
     if (tid == 0) {
       tok_out[tbase + t] = (int32_t)sx_pack_index(best);
+      if (t == 0) s_tok = (int32_t)sx_pack_index(best);
       if (logp_out) logp_out[(size_t)r * T + t] = lse ? sx_pack_value(best) - s_lse : sx_pack_value(best);
     }
     for (int i = tid; i < G * T; i += blockDim.x)
@@ -260,13 +266,28 @@ __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int p
     const int a = tid == 0 ? act0 : (tid == 1 ? act1 : act2);
     sig_out[(size_t)sx_index(si, r) * S + tid] = sx_activate(z[(size_t)r * S + tid], a);
   }
+  if (nx.u) {
+    // chain drafting: the next round's input row [hidden of this round ; embedding of the chosen token]
+    __syncthreads();
+    int t = s_tok;
+    if (t < 0 || t >= nx.V) t = 0;
+    const uint4 *f = reinterpret_cast<const uint4 *>(nx.feat + (size_t)r * nx.H);
+    const uint4 *e = reinterpret_cast<const uint4 *>(nx.embed + (size_t)t * nx.H);
+    uint4 *o = reinterpret_cast<uint4 *>(nx.u + (size_t)r * 2 * nx.H);
+    const int n = nx.H / 8;
+    for (int i = tid; i < n; i += blockDim.x) {
+      const uint4 a = f[i], b = e[i];
+      o[i] = a;
+      o[n + i] = b;
+    }
+  }
 }
 
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
-                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st) {
+                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st, SxNextInput nx) {
   sx_launch(sx_head_finalize_kernel, dim3(R), dim3(128), (size_t)G * T * 8, st, parts, G, part_stride, T, lse, z, S,
-            sh.act[0], sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si);
+            sh.act[0], sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx);
 }
 
 // ---------------------------------------------------------------------------------------

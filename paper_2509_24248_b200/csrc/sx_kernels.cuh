@@ -40,9 +40,17 @@ size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_cou
 void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
                          const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
 
+// Optional fusion for chain drafting: the merge kernel also writes the next round's input row
+// u[r] = [feat[r] ; embed[token chosen for row r]] (u == nullptr: off).
+struct SxNextInput {
+  const bf16 *feat, *embed;
+  bf16 *u;
+  int H, V;
+};
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
-                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st);
+                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st,
+                             SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0});
 
 void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st);
 
