@@ -109,7 +109,7 @@ __device__ __forceinline__ int sx_attn_swz(int key) {
 // used for all of them); NT warps form a group that shares one staged copy of the keys and values
 // (a warp without queries still does its share of the copies); gpc = groups per CTA.
 template <int D, int NT, int NQT>
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(128, 3)
 sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale_log2, SxRowMap rm, int nr, int E,
                    int gpc, int stages, const bf16 *__restrict__ q, sx_kv kv, int nsplit,
                    float2 *__restrict__ ws_ml, float *__restrict__ ws_o, int32_t *status) {
