@@ -224,6 +224,27 @@ class DraftModel:
             out[h] = p @ Vall[kvh]
         return out
 
+    def layer_input(self, rows: List[Row]) -> Tuple[torch.Tensor, torch.Tensor]:
+        """u = [feature ; embedding], x = fc u, n1 = RMSNorm(x), and the fused q/k/v projection of
+        n1.  Returns ``x [R, H]`` (bf16 values) and ``qkv [R, (n_q + 2 n_kv) d]`` (unrounded)."""
+        sh, w = self.sh, self.w
+        toks = torch.tensor([r.tok for r in rows], dtype=torch.int64)
+        u = torch.cat([torch.stack([r.feat for r in rows]), w["embed"][toks].to(F64)], dim=1)
+        x = bf16r(linear(u, w["fc"]))
+        n1 = bf16r(rmsnorm(x, w["norm1"], sh.eps))
+        return x, linear(n1, w["wqkv"])
+
+    def append_kv(self, kv: PagedKV, rows: List[Row]) -> None:
+        """Writes the rows' K (rotated at their positions) and V into their cache slots.  With one
+        decoder layer the K/V of a position depend on that position's input only."""
+        sh = self.sh
+        nq, nk, d = sh.n_q, sh.n_kv, sh.d
+        _, qkv = self.layer_input(rows)
+        for i, r in enumerate(rows):
+            k = qkv[i, nq * d:(nq + nk) * d].view(nk, d)
+            v = qkv[i, (nq + nk) * d:].view(nk, d)
+            kv.write(r.b, r.slot, bf16r(rope(k, r.pos, sh.theta)), bf16r(v))
+
     def round(self, kv: PagedKV, rows: List[Row], head_input=None) -> Tuple[torch.Tensor, HeadOut]:
         """One draft pass over ``rows``; appends their K/V to the cache.  Returns the
         final-normed hidden ``g [R, H]`` (bf16 values) and the head outputs.
@@ -231,11 +252,7 @@ class DraftModel:
         that a test can check the head's decisions on another implementation's hidden."""
         sh, w = self.sh, self.w
         R = len(rows)
-        toks = torch.tensor([r.tok for r in rows], dtype=torch.int64)
-        u = torch.cat([torch.stack([r.feat for r in rows]), w["embed"][toks].to(F64)], dim=1)
-        x = bf16r(linear(u, w["fc"]))
-        n1 = bf16r(rmsnorm(x, w["norm1"], sh.eps))
-        qkv = linear(n1, w["wqkv"])
+        x, qkv = self.layer_input(rows)
         nq, nk, d = sh.n_q, sh.n_kv, sh.d
         o = torch.empty(R, nq * d, dtype=F64)
         qs = []
@@ -520,6 +537,49 @@ def verify(model: DraftModel, target_hidden: torch.Tensor, cand_tok: torch.Tenso
         L[b], rec[b] = l, r
         paths.append(p)
     return VerifyOut(tt, L, paths, rec, gap)
+
+
+# --------------------------------------------------------------------------------------
+# end of an iteration: Algorithm 1, "Update KV-cache and hidden states accordingly"
+# --------------------------------------------------------------------------------------
+@dataclass
+class CommitOut:
+    cache_len: List[int]      # cached length per sequence after the commit
+    feat0: torch.Tensor       # [B, H] feature of the next iteration's first draft row
+    tok0: torch.Tensor        # [B] its token (the recover token)
+
+
+def commit(model: DraftModel, kv: PagedKV, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
+           path: torch.Tensor, accept_len_out: torch.Tensor, recover_tok_out: torch.Tensor) -> CommitOut:
+    """Makes the verified tokens of an iteration part of the draft model's cached context.
+
+    Before the iteration sequence b had n cached positions.  Slot n holds the K/V of the last
+    accepted token of the previous iteration, computed in draft round 1 from its true feature:
+    it is kept.  The L accepted draft tokens (path slots 1..L) were drafted from draft hidden
+    states, so their K/V are recomputed ("catch-up") from the target's hidden states: the token
+    of path slot j is paired with the target hidden of path slot j - 1, the hidden that
+    predicted it, at position n + j.  The cached length becomes n + L + 1, and the next
+    iteration starts from (target hidden of path slot L, recover token).  ``accept_len_out`` and
+    ``recover_tok_out`` are the values after the exit rule (a cut path commits fewer tokens)."""
+    B = cand_tok.shape[0]
+    feat0 = torch.empty(B, model.sh.H, dtype=F64)
+    tok0 = torch.empty(B, dtype=torch.int64)
+    rows: List[Row] = []
+    new_len = []
+    for b in range(B):
+        n, L = kv.len[b], int(accept_len_out[b])
+        pb = [int(s) for s in path[b]]              # accepted slots, slot 0 first (tensor row or list)
+        for j in range(1, L + 1):
+            rows.append(Row(b=b, feat=bf16r(target_hidden[b, pb[j - 1]].to(F64)),
+                            tok=int(cand_tok[b, pb[j]]), pos=n + j, slot=n + j, visible=[]))
+        feat0[b] = bf16r(target_hidden[b, pb[L]].to(F64))
+        tok0[b] = int(recover_tok_out[b])
+        new_len.append(n + L + 1)
+    if rows:
+        model.append_kv(kv, rows)
+    kv.len = list(new_len)
+    kv._prefix.clear()
+    return CommitOut(new_len, feat0, tok0)
 
 
 # --------------------------------------------------------------------------------------

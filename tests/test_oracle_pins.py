@@ -632,3 +632,88 @@ def test_chain_iteration_end_to_end_properties():
     assert torch.equal(d2.hidden[1, :2], d.hidden[1, :2]) and int(d2.cand_tok[1, 2]) == alt
     assert not torch.equal(d2.hidden[1, 2], d.hidden[1, 2])
     assert torch.equal(d2.hidden[0], d.hidden[0])
+
+
+# ---------------------------------------------------------------- commit (Algorithm 1, KV-cache update)
+def test_commit_bookkeeping_and_pairing_on_a_tree_path():
+    # x = feature (fc = [I | 0]), k = first d components of rmsnorm(x) rotated, v = next d components
+    sh, w = _mini_model(H=4, n_q=1, n_kv=1, d=2, F=2, V=6, S=1, page=4, theta=1e4)
+    w["wqkv"][2, 0] = 1.0   # k0 <- n1[0]
+    w["wqkv"][3, 1] = 1.0   # k1 <- n1[1]
+    w["wqkv"][4, 2] = 1.0   # v0 <- n1[2]
+    w["wqkv"][5, 3] = 1.0   # v1 <- n1[3]
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    n = 5
+    kv = _mini_kv(sh, n, extra=6)
+    before_k, before_v = kv.k.clone(), kv.v.clone()
+    P = 8
+    th = torch.zeros(1, P, 4, dtype=torch.bfloat16)
+    for s in range(P):
+        th[0, s] = torch.tensor([1.0 + s, 2.0, -1.0, 0.5 * s], dtype=torch.bfloat16)
+    cand = torch.tensor([[9, 1, 2, 3, 4, 5, 0, 1]])
+    path = torch.tensor([[0, 3, 6, -1]])            # accepted: slot 3 (child of the root), then slot 6
+    out = orc.commit(model, kv, th, cand, path, torch.tensor([2]), torch.tensor([4]))
+    assert out.cache_len == [n + 3] and kv.len == [n + 3]
+    assert torch.equal(out.feat0[0], th[0, 6].to(F64)) and int(out.tok0[0]) == 4
+    # slot n + 1 pairs the hidden of path slot 0 with the token of path slot 3; the embedding is zero, so
+    # only the hidden matters: k = rot(n1[0:2], pos = n + 1), v = n1[2:4]
+    for j, src in ((1, 0), (2, 3)):
+        x = th[0, src].to(F64)
+        n1 = x / torch.sqrt((x * x).mean() + sh.eps)
+        n1 = n1.to(torch.bfloat16).to(F64)
+        pos = n + j
+        ang = pos * sh.theta ** (-0.0)               # d = 2: a single frequency, exponent 0
+        want_k = torch.tensor([n1[0] * math.cos(ang) - n1[1] * math.sin(ang),
+                               n1[1] * math.cos(ang) + n1[0] * math.sin(ang)], dtype=F64)
+        got_k, got_v = kv.read(0, n + j)
+        assert (got_k[0] - want_k).abs().max() < 1e-2 * max(1.0, float(want_k.abs().max()))
+        assert (got_v[0] - n1[2:4]).abs().max() < 1e-2
+    # nothing but the two catch-up slots was written
+    kv2 = kv.k.clone()
+    for j in (1, 2):
+        pp, off = kv._loc(0, n + j)
+        kv2[pp, :, off] = before_k[pp, :, off]
+    same = (kv2 == before_k) | (torch.isnan(kv2) & torch.isnan(before_k))
+    assert bool(same.all())
+
+
+def test_commit_with_nothing_accepted_keeps_the_cache_and_moves_on_by_one():
+    sh, w = _mini_model(H=4, n_q=1, n_kv=1, d=2, F=2, V=6, S=1, page=4)
+    model = orc.DraftModel(sh, w, act=(orc.ACT_SIGMOID,))
+    kv = _mini_kv(sh, 3, extra=4)
+    k0 = kv.k.clone()
+    th = torch.randn(1, 3, 4, generator=torch.Generator().manual_seed(1)).to(torch.bfloat16)
+    out = orc.commit(model, kv, th, torch.tensor([[1, 2, 3]]), torch.tensor([[0, -1, -1]]), torch.tensor([0]),
+                     torch.tensor([5]))
+    assert out.cache_len == [4] and int(out.tok0[0]) == 5 and torch.equal(out.feat0[0], th[0, 0].to(F64))
+    assert bool(((kv.k == k0) | (torch.isnan(kv.k) & torch.isnan(k0))).all())
+
+
+def test_commit_kv_against_float64_restatement_and_next_iteration_consistency():
+    # C0: after an iteration and its commit, every catch-up slot holds the K/V that the unrounded numpy
+    # restatement computes for (target hidden of the previous path slot, accepted token) at that position
+    wl = synth.workload("C0")
+    case = harness.build_case(wl, poison_tail=False)
+    model = harness.oracle_model(case)
+    kv = harness.oracle_kv(case)
+    d = orc.draft_chain(model, kv, case.f0, case.t0, wl.K)
+    th = harness.chain_target_hidden(case, d)
+    cand = d.cand_tok.clone()
+    cand[0, 1] = int(orc.target_argmax(model, th)[0][0, 0])        # make at least two tokens accepted
+    cand[0, 2] = int(orc.target_argmax(model, th)[0][0, 1])
+    v = orc.verify(model, th, cand)
+    L = int(v.accept_len[0])
+    assert L >= 2
+    n = int(case.kv["cache_len"][0])
+    out = orc.commit(model, kv, th, cand, v.path, v.accept_len, v.recover_tok)
+    assert out.cache_len[0] == n + L + 1
+    for j in range(1, L + 1):
+        f = th[0, j - 1].to(torch.float64).numpy()
+        pad = [np.zeros((1, wl.shape.n_kv, wl.shape.d))] * j          # position n + j
+        _, _, k_np, v_np = _np_forward(case, f, int(cand[0, j]), 0, pad, pad)
+        got_k, got_v = kv.read(0, n + j)
+        rel = lambda a, b: float(np.linalg.norm(a - b) / np.linalg.norm(b))
+        assert rel(got_k.numpy(), k_np[0]) < 1e-2 and rel(got_v.numpy(), v_np[0]) < 1e-2
+    # the next iteration drafts from the committed context without error and its first row sits at n + L + 1
+    d2 = orc.draft_chain(model, kv, out.feat0.to(torch.bfloat16), out.tok0, 2)
+    assert d2.cand_tok.shape == (1, 3) and kv.len[0] == n + L + 1
