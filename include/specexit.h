@@ -217,6 +217,27 @@ sx_status sx_spec_exit_iter(sx_ctx *ctx, const sx_kv *kv, const sx_exit_cfg *cfg
                             const void *target_hidden_d, const sx_iter_out *out, void *ws_d,
                             size_t ws_bytes, int32_t *status_d, void *stream);
 
+/* End of an iteration: Algorithm 1, "Update KV-cache and hidden states accordingly".  Makes the
+ * verified tokens part of the draft model's cached context and names the next iteration's
+ * first draft row.  For sequence b with n = cache_len[b] and L = accept_len_out_d[b] (the
+ * accepted length after the exit rule):
+ *   - slot n (the last accepted token of the previous iteration, keyed in draft round 1 from
+ *     its true feature) is kept;
+ *   - the token of path slot j (j = 1..L) is re-keyed from the TARGET's hidden state of path
+ *     slot j - 1, the state that predicted it: its K/V, at position n + j, overwrite the
+ *     drafted ones (the drafted K/V came from draft hidden states); drafted rows that were
+ *     not accepted are dropped;
+ *   - cache_len[b] becomes n + L + 1 (kv->cache_len_d is WRITTEN by this call);
+ *   - feat0_next_d[b] = target hidden of path slot L, tok0_next_d[b] = recover_tok_out_d[b].
+ * path_d [batch, path_stride] as produced by sx_verify, path_stride - 1 <= K of the plan.  The
+ * page table must cover cache_len + path_stride slots.  Work after this call sees the new
+ * lengths (the call ends with a kernel that later launches cannot overtake). */
+sx_status sx_commit(sx_ctx *ctx, const sx_kv *kv, int32_t P, const void *target_hidden_d,
+                    const int32_t *cand_tok_d, const int32_t *path_d, int32_t path_stride,
+                    const int32_t *accept_len_out_d, const int32_t *recover_tok_out_d,
+                    void *feat0_next_d, int32_t *tok0_next_d, void *ws_d, size_t ws_bytes,
+                    int32_t *status_d, void *stream);
+
 /* Same iteration with HOST buffers for the per-iteration inputs (feature, token, target
  * hiddens) and the per-iteration results (accepted length, recover token, exit flag, smoothed
  * signals): copies them in, runs sx_spec_exit_iter, copies the results out and synchronises

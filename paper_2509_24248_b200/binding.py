@@ -26,7 +26,7 @@ EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
-           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc"]
+           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -119,6 +119,8 @@ def load_library() -> C.CDLL:
     lib.sx_profile_begin.argtypes = [vp]
     lib.sx_profile_end.restype = i32
     lib.sx_profile_end.argtypes = [vp, vp, vp]
+    lib.sx_commit.restype = i32
+    lib.sx_commit.argtypes = [vp, C.POINTER(KV), i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
     lib.sx_verify_noalloc.restype = i32
     lib.sx_verify_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     _lib = lib
@@ -331,6 +333,19 @@ class SpecExit:
                                        Lo.data_ptr(), ro.data_ptr(), sm.data_ptr(), self.status.data_ptr(),
                                        self._stream()), "sx_exit_update")
         return ef, Lo, ro, sm
+
+    def sx_commit(self, target_hidden: torch.Tensor, cand_tok: torch.Tensor, path: torch.Tensor,
+                  accept_len_out: torch.Tensor, recover_tok_out: torch.Tensor):
+        """Commits the verified tokens (the context's ``cache_len`` tensor is advanced in place) and
+        returns the next iteration's first row ``(feat0 [B, H] bf16, tok0 [B] int32)``."""
+        B, P = cand_tok.shape
+        feat0 = torch.empty(B, self.shape.H, dtype=torch.bfloat16, device=self.dev)
+        tok0 = torch.empty(B, dtype=torch.int32, device=self.dev)
+        _check(self.lib.sx_commit(self.h, C.byref(self._kv_struct), P, target_hidden.data_ptr(), cand_tok.data_ptr(),
+                                  path.data_ptr(), int(path.shape[1]), accept_len_out.data_ptr(),
+                                  recover_tok_out.data_ptr(), feat0.data_ptr(), tok0.data_ptr(), self.ws_ptr,
+                                  self.ws_bytes, self.status.data_ptr(), self._stream()), "sx_commit")
+        return feat0, tok0
 
     def sx_spec_exit_iter(self, params: ExitParams, state: Dict[str, torch.Tensor], feat0: torch.Tensor,
                           tok0: torch.Tensor, target_hidden: torch.Tensor, out: Dict[str, torch.Tensor]) -> None:

@@ -17,7 +17,8 @@ struct sx_ctx {
   int max_splits, part_N, head_G, head_rows;
   // workspace offsets (bytes)
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
-      off_tok_rt, off_logp_rt, off_tree, total;
+      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, total;
+  int commit_rows, commit_N;
   // tree sub-offsets relative to off_tree
   size_t t_tok, t_par, t_src, t_row, t_score, t_rmask, t_selcid, t_seltok, t_fidx, t_hidx, t_nmask, t_rsig;
   // optional per-class event timing
@@ -68,6 +69,8 @@ extern "C" sx_status sx_profile_end(sx_ctx *c, float *ms_out, int32_t *count_out
   c->prof_used = 0;
   return SX_OK;
 }
+
+#define SX_COMMIT_MAX_SPLITS 4
 
 static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
@@ -174,6 +177,12 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->off_z = take((size_t)R * SX_MAX_SIGNALS * 4);
   c->off_tok_rt = take((size_t)R * SX_MAX_TOPK * 4);
   c->off_logp_rt = take((size_t)R * SX_MAX_TOPK * 4);
+  // commit: up to K catch-up rows per sequence through fc, norm and the K/V part of the projection
+  c->commit_rows = max_batch * dc->K;
+  c->commit_N = s.H > (s.nq + 2 * s.nkv) * s.d ? s.H : (s.nq + 2 * s.nkv) * s.d;
+  c->off_cu = take((size_t)c->commit_rows * 2 * s.H * 2);
+  c->off_cn = take((size_t)c->commit_rows * s.H * 2);
+  c->off_cpart = take((size_t)SX_COMMIT_MAX_SPLITS * c->commit_rows * c->commit_N * 4);
   c->off_tree = o;
   if (dc->mode == SX_MODE_TREE) {
     const size_t B = max_batch, NC = c->NC, rows = c->rows_per_seq;
@@ -286,6 +295,7 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   SxRowMap rm;
   rm.mode = c->dc.mode; rm.round = round; rm.topk = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1; rm.R = R;
   rm.cache_len = kv->cache_len_d; rm.row_mask = row_mask;
+  rm.valid_len = nullptr; rm.per_seq = 1;
   int sp; size_t stride;
   // input_ready: the previous round's merge kernel has already written u (chain drafting)
   if (!input_ready) {
@@ -431,6 +441,50 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
   return sx_exit_update(c, B, P, cfg, state, o->slot_signal_d, o->cand_tok_d, o->path_d, K + 1, o->accept_len_d,
                         o->recover_tok_d, o->exit_flag_d, o->accept_len_out_d, o->recover_tok_out_d, o->smoothed_d,
                         status_d, stream);
+}
+
+extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void *target_hidden_d,
+                               const int32_t *cand_tok_d, const int32_t *path_d, int32_t path_stride,
+                               const int32_t *accept_len_out_d, const int32_t *recover_tok_out_d, void *feat0_next_d,
+                               int32_t *tok0_next_d, void *ws_d, size_t ws_bytes, int32_t *status_d, void *stream) {
+  if (!c || !target_hidden_d || !cand_tok_d || !path_d || !accept_len_out_d || !recover_tok_out_d || !feat0_next_d ||
+      !tok0_next_d || !status_d)
+    return SX_ERR_INVALID_ARG;
+  SX_TRY(check_kv(c, kv));
+  SX_TRY(check_ws(c, ws_d, ws_bytes));
+  if (P < 1 || path_stride < 1 || path_stride - 1 > c->dc.K) return SX_ERR_INVALID_ARG;
+  if (((uintptr_t)target_hidden_d & 15) || ((uintptr_t)feat0_next_d & 15)) return SX_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  char *ws = (char *)ws_d;
+  const SxShape &s = c->sh;
+  const int B = kv->batch, M = path_stride - 1, R = B * M;
+  bf16 *u = (bf16 *)(ws + c->off_cu), *n = (bf16 *)(ws + c->off_cn);
+  float *part = (float *)(ws + c->off_cpart);
+  sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
+                          recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d, st);
+  c->launches += 1;
+  if (R > 0) {
+    int sp = sx_gemm_pick_splits(s.H, 2 * s.H, c->sm_count);
+    if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
+    SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 2 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
+                                  status_d, st));
+    sx_launch_finish_norm(s, R, part, sp, (size_t)R * s.H, nullptr, (const bf16 *)c->w.norm1_d, nullptr, n, nullptr,
+                          SxIndex{nullptr, 1, 0}, st);
+    const int N = (s.nq + 2 * s.nkv) * s.d;
+    sp = sx_gemm_pick_splits(N, s.H, c->sm_count);
+    if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
+    SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, s.H, n, R, part, sp, (size_t)R * N, c->sm_count, status_d,
+                                  st));
+    SxRowMap rm;
+    memset(&rm, 0, sizeof(rm));
+    rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
+    rm.valid_len = accept_len_out_d; rm.per_seq = M;
+    sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st);
+    c->launches += 4;
+  }
+  sx_launch_commit_advance(B, accept_len_out_d, const_cast<int32_t *>(kv->cache_len_d), st);
+  c->launches += 1;
+  return SX_OK;
 }
 
 extern "C" sx_status sx_spec_exit_iter_host(sx_ctx *c, const sx_kv *kv, const sx_exit_cfg *cfg,

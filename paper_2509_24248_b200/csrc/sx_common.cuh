@@ -19,7 +19,12 @@ struct SxRowMap {
   int R;                       // rows this round
   const int32_t *cache_len;    // [B]
   const uint64_t *row_mask;    // [R] tree rounds >= 2, else nullptr
+  // commit (mode SX_MODE_COMMIT): per_seq rows per sequence, row j of sequence b sits at slot and
+  // position n + 1 + j and exists only if j < valid_len[b]
+  const int32_t *valid_len;
+  int per_seq;
 };
+#define SX_MODE_COMMIT 2
 
 struct SxRowInfo {
   int b;          // sequence
@@ -53,6 +58,14 @@ __device__ __forceinline__ SxRowInfo sx_row_info(const SxRowMap &m, int r) {
 // of the same iteration writes, so it may run before the wait on the preceding kernel
 __device__ __forceinline__ SxRowInfo sx_row_place(const SxRowMap &m, int r) {
   SxRowInfo i;
+  if (m.mode == SX_MODE_COMMIT) {
+    i.b = r / m.per_seq;
+    i.rel = 1 + (r - i.b * m.per_seq);
+    i.mask = 0ull;
+    i.n = m.cache_len[i.b];
+    i.pos = i.n + i.rel;
+    return i;
+  }
   if (m.mode == SX_MODE_CHAIN) { i.b = r; i.rel = m.round - 1; }
   else if (m.round == 1) { i.b = r; i.rel = 0; }
   else { i.b = r / m.topk; i.rel = 1 + (m.round - 2) * m.topk + (r % m.topk); }

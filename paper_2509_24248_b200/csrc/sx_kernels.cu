@@ -132,9 +132,9 @@ void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int spli
 // ---------------------------------------------------------------------------------------
 __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, SxRowMap rm, const float *part,
                                           int splits, size_t split_stride, bf16 *q_out, sx_kv kv, int page,
-                                          int32_t *status) {
+                                          int head_begin, int32_t *status) {
   sx_pdl_launch_dependents();
-  const int hh = blockIdx.x, r = blockIdx.y;
+  const int hh = head_begin + blockIdx.x, r = blockIdx.y;
   const int i = threadIdx.x;
   const int half = d / 2;
   const bool rot = hh < nq + nkv;                 // q and k heads rotate, v heads do not
@@ -150,6 +150,7 @@ __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, 
   }
   sx_pdl_wait();
   if (i >= half) return;
+  if (rm.mode == SX_MODE_COMMIT && (ri.rel - 1) >= rm.valid_len[ri.b]) return;   // row does not exist
   const int N = (nq + 2 * nkv) * d;
   const float *row = part + (size_t)r * N + hh * d;
   float x1 = 0.f, x2 = 0.f;
@@ -189,8 +190,79 @@ void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const floa
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
                                cudaStream_t st) {
   int threads = ((sh.d / 2 + 31) / 32) * 32;
-  sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv, sh.d,
-            (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, status);
+  // q_out == nullptr: only the K and V heads (commit)
+  const int head_begin = q_out ? 0 : sh.nq;
+  sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv - head_begin, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv,
+            sh.d, (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, head_begin, status);
+}
+
+// ---------------------------------------------------------------------------------------
+// commit (Algorithm 1, "Update KV-cache and hidden states accordingly")
+// ---------------------------------------------------------------------------------------
+// Blocks [0, B * M): catch-up input row (b, j) = [target hidden of path slot j ; embedding of the
+// token of path slot j + 1] when j < L_b, zeros otherwise.  Blocks [B * M, B * M + B): the next
+// iteration's first row: feature = target hidden of path slot L_b, token = recover token.
+__global__ void sx_commit_gather_kernel(int B, int M, int P, int H, int V, const bf16 *th, const int32_t *cand,
+                                        const int32_t *path, int path_stride, const int32_t *accept_len,
+                                        const int32_t *recover, const bf16 *embed, bf16 *u, bf16 *feat0,
+                                        int32_t *tok0, int32_t *status) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int n8 = H / 8;
+  if ((int)blockIdx.x >= B * M) {
+    const int b = blockIdx.x - B * M;
+    int L = accept_len[b];
+    if (L < 0 || L >= path_stride) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_INVALID_ARG); L = 0; }
+    int slot = path[(size_t)b * path_stride + L];
+    if (slot < 0 || slot >= P) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_INVALID_ARG); slot = 0; }
+    const uint4 *src = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + slot) * H);
+    uint4 *dst = reinterpret_cast<uint4 *>(feat0 + (size_t)b * H);
+    for (int i = threadIdx.x; i < n8; i += blockDim.x) dst[i] = src[i];
+    if (threadIdx.x == 0) tok0[b] = recover[b];
+    return;
+  }
+  const int b = blockIdx.x / M, j = blockIdx.x - b * M;
+  uint4 *o = reinterpret_cast<uint4 *>(u + (size_t)blockIdx.x * 2 * H);
+  const int L = accept_len[b];
+  bool live = j < L && j + 1 < path_stride;
+  int s0 = 0, s1 = 0, t = 0;
+  if (live) {
+    s0 = path[(size_t)b * path_stride + j];
+    s1 = path[(size_t)b * path_stride + j + 1];
+    if (s0 < 0 || s0 >= P || s1 < 0 || s1 >= P) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_INVALID_ARG); live = false; }
+  }
+  if (live) {
+    t = cand[(size_t)b * P + s1];
+    if (t < 0 || t >= V) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY); t = 0; }
+  }
+  const uint4 *f = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + s0) * H);
+  const uint4 *e = reinterpret_cast<const uint4 *>(embed + (size_t)t * H);
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < n8; i += blockDim.x) {
+    o[i] = live ? f[i] : zero;
+    o[n8 + i] = live ? e[i] : zero;
+  }
+}
+
+// The last kernel of a commit.  It does not release its dependents early: whatever is launched
+// after it, however eagerly, starts once the new lengths are in memory.
+__global__ void sx_commit_advance_kernel(int B, const int32_t *accept_len, int32_t *cache_len) {
+  sx_pdl_wait();
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) cache_len[b] += accept_len[b] + 1;
+}
+
+void sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
+                             const int32_t *path, int path_stride, const int32_t *accept_len, const int32_t *recover,
+                             const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0, int32_t *status, cudaStream_t st) {
+  int threads = ((sh.H / 8 + 31) / 32) * 32;
+  if (threads > 512) threads = 512;
+  sx_launch(sx_commit_gather_kernel, dim3(B * M + B), dim3(threads), 0, st, B, M, P, sh.H, sh.V, th, cand, path,
+            path_stride, accept_len, recover, embed, u, feat0, tok0, status);
+}
+
+void sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st) {
+  sx_launch(sx_commit_advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, B, accept_len, cache_len);
 }
 
 // ---------------------------------------------------------------------------------------
