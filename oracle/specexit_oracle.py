@@ -585,6 +585,10 @@ def commit(model: DraftModel, kv: PagedKV, target_hidden: torch.Tensor, cand_tok
 # --------------------------------------------------------------------------------------
 # exit decision (Section 3.3; Appendix A.1: EWMA x_t = alpha s_t + (1 - alpha) x_{t-1})
 # --------------------------------------------------------------------------------------
+SMOOTH_EWMA, SMOOTH_NONE, SMOOTH_WINDOW, SMOOTH_MOMENTUM, SMOOTH_PARAGRAPH = 0, 1, 2, 3, 4
+HIST = 16        # samples of history kept per sequence (window and momentum rules, N <= 15)
+
+
 @dataclass
 class ExitCfg:
     alpha: float = 0.3
@@ -594,6 +598,8 @@ class ExitCfg:
     ema_positions: int = EMA_VERIFIED_CONTEXT
     split_bitmap: Optional[torch.Tensor] = None   # int32 words, bit t%32 of word t//32; None = all
     stop_think_token: int = 0
+    smoothing: int = SMOOTH_EWMA       # Appendix A.1, "Signal Smoothing"
+    window: int = 10                   # N of the sliding-window and momentum rules
 
 
 @dataclass
@@ -601,14 +607,20 @@ class ExitState:
     x: torch.Tensor          # [B, S] smoothed signals (fp32 values)
     n_updates: torch.Tensor  # [B]
     thinking: torch.Tensor   # [B] 1 while inside the reasoning phase
+    hist: Optional[torch.Tensor] = None      # [B, HIST, S] ring of the latest samples; sample i at i % HIST
+    par_sum: Optional[torch.Tensor] = None   # [B, S] sum of the samples of the current paragraph (fp32 values)
+    par_n: Optional[torch.Tensor] = None     # [B] their number
 
     @staticmethod
     def fresh(B: int, S: int = 3) -> "ExitState":
         return ExitState(torch.zeros(B, S, dtype=F64), torch.zeros(B, dtype=torch.int64),
-                         torch.ones(B, dtype=torch.int64))
+                         torch.ones(B, dtype=torch.int64), torch.zeros(B, HIST, S, dtype=F64),
+                         torch.zeros(B, S, dtype=F64), torch.zeros(B, dtype=torch.int64))
 
     def clone(self) -> "ExitState":
-        return ExitState(self.x.clone(), self.n_updates.clone(), self.thinking.clone())
+        c = lambda t: None if t is None else t.clone()
+        return ExitState(self.x.clone(), self.n_updates.clone(), self.thinking.clone(), c(self.hist),
+                         c(self.par_sum), c(self.par_n))
 
 
 def is_split(cfg: ExitCfg, tok: int) -> bool:
@@ -637,6 +649,41 @@ def ewma(cfg: ExitCfg, x: torch.Tensor, n_updates: int, s: torch.Tensor) -> torc
         return f32r(s)
     a = float(torch.tensor(cfg.alpha, dtype=torch.float32))   # alpha as the fp32 the kernel holds
     return f32r(a * s + (1.0 - a) * x)
+
+
+def smooth(cfg: ExitCfg, state: ExitState, b: int, s: torch.Tensor) -> torch.Tensor:
+    """Folds sample ``s`` (the n-th of sequence b, n = n_updates) into the state and returns the
+    smoothed score x_t of Appendix A.1.  Sums run oldest to newest in f64; x is stored as fp32.
+    Where fewer samples exist than a rule asks for, it uses those that exist (the paper does not
+    say): the window averages what it has; the momentum rule, which as printed predicts step t
+    from the samples before it, returns the sample itself while there is no earlier one."""
+    n = int(state.n_updates[b])
+    if cfg.smoothing == SMOOTH_EWMA:
+        return ewma(cfg, state.x[b], n, s)
+    if cfg.smoothing == SMOOTH_NONE:
+        return f32r(s)
+    if cfg.smoothing == SMOOTH_PARAGRAPH:
+        state.par_sum[b] = f32r(state.par_sum[b] + s)
+        state.par_n[b] += 1
+        return f32r(state.par_sum[b] / float(state.par_n[b]))
+    N = int(cfg.window)
+    assert 2 <= N < HIST
+    state.hist[b, n % HIST] = f32r(s)
+    at = lambda i: state.hist[b, i % HIST]          # sample i, i in (n - HIST, n]
+    if cfg.smoothing == SMOOTH_WINDOW:
+        m = min(n + 1, N)
+        acc = torch.zeros_like(s)
+        for i in range(n - m + 1, n + 1):
+            acc = acc + at(i)
+        return f32r(acc / float(m))
+    # momentum: x_t = s_{t-1} + (1 / (N - 1)) sum_{i = t-N+1}^{t-1} (s_i - s_{i-1}); the sum telescopes
+    if n == 0:
+        return f32r(s)
+    k = min(N - 1, n - 1)                            # differences available behind s_{t-1}
+    prev = at(n - 1)
+    if k == 0:
+        return f32r(prev)
+    return f32r(prev + (prev - at(n - 1 - k)) / float(k))
 
 
 @dataclass
@@ -668,10 +715,14 @@ def exit_update(cfg: ExitCfg, state: ExitState, slot_signal: torch.Tensor, cand_
             if cfg.ema_positions == EMA_VERIFIED_CONTEXT or idx == 0:
                 if bool(torch.isnan(sig).any()):
                     break                     # never drafted from this slot: nothing new to smooth
-                state.x[b] = ewma(cfg, state.x[b], int(state.n_updates[b]), sig)
+                state.x[b] = smooth(cfg, state, b, sig)
                 state.n_updates[b] += 1
-            if is_split(cfg, int(cand_tok[b, slot])) and thresholds_pass(cfg, state.x[b]):
+            split = is_split(cfg, int(cand_tok[b, slot]))
+            if split and thresholds_pass(cfg, state.x[b]):
                 ef[b], Lo[b], ro[b] = 1, idx, cfg.stop_think_token
                 state.thinking[b] = 0
                 break
+            if split and cfg.smoothing == SMOOTH_PARAGRAPH:
+                state.par_sum[b] = 0.0            # a paragraph delimiter went by: a new paragraph starts
+                state.par_n[b] = 0
     return ExitOut(ef, Lo, ro, state.x.clone())

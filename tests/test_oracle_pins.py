@@ -717,3 +717,56 @@ def test_commit_kv_against_float64_restatement_and_next_iteration_consistency():
     # the next iteration drafts from the committed context without error and its first row sits at n + L + 1
     d2 = orc.draft_chain(model, kv, out.feat0.to(torch.bfloat16), out.tok0, 2)
     assert d2.cand_tok.shape == (1, 3) and kv.len[0] == n + L + 1
+
+
+# ---------------------------------------------------------------- smoothing rules (Appendix A.1)
+def _run_rule(rule, samples, window=3, split_at=()):
+    """Feeds one sample per iteration (slot 0 only) and returns the smoothed values."""
+    V = 64
+    bm = torch.zeros(V // 32, dtype=torch.int32)
+    bm[0] = 1 << 5                                         # token 5 is the only step-split token
+    cfg = orc.ExitCfg(alpha=0.5, thr=(1e9, 0, 0), enable_mask=1, split_bitmap=bm, stop_think_token=1,
+                      smoothing=rule, window=window)
+    st = orc.ExitState.fresh(1, S=1)
+    xs = []
+    for i, s in enumerate(samples):
+        sig = torch.tensor([[[s], [float("nan")]]], dtype=F64)
+        tok = 5 if i in split_at else 7
+        out = orc.exit_update(cfg, st, sig, torch.tensor([[tok, 0]]), [[0]], torch.tensor([0]), torch.tensor([3]))
+        assert int(out.exit_flag[0]) == 0
+        xs.append(float(out.smoothed[0, 0]))
+    return xs
+
+
+def test_sliding_window_hand_values():
+    assert _run_rule(orc.SMOOTH_WINDOW, [1, 2, 3, 4, 5], window=3) == [1.0, 1.5, 2.0, 3.0, 4.0]
+
+
+def test_momentum_hand_values_and_linear_sequences_are_predicted_exactly():
+    # x_t = s_{t-1} + (s_{t-1} - s_{t-N}) / (N - 1) once N + 1 samples exist; fewer differences before
+    assert _run_rule(orc.SMOOTH_MOMENTUM, [1, 2, 4, 7, 11], window=3) == [1.0, 1.0, 3.0, 5.5, 9.5]
+    # literal form of the printed sum for t = 3, N = 3: s_2 + ((s_1 - s_0) + (s_2 - s_1)) / 2
+    assert 4 + ((2 - 1) + (4 - 2)) / 2 == 5.5
+    lin = [0.25 + 0.125 * i for i in range(14)]
+    xs = _run_rule(orc.SMOOTH_MOMENTUM, lin, window=10)
+    assert xs[2:] == lin[2:]
+
+
+def test_paragraph_mean_resets_at_a_split_token_and_none_passes_through():
+    assert _run_rule(orc.SMOOTH_PARAGRAPH, [2, 4, 6, 10], split_at=(1,)) == [2.0, 3.0, 6.0, 8.0]
+    assert _run_rule(orc.SMOOTH_NONE, [0.5, 0.25, 0.75]) == [0.5, 0.25, 0.75]
+
+
+@pytest.mark.parametrize("rule", [orc.SMOOTH_EWMA, orc.SMOOTH_NONE, orc.SMOOTH_WINDOW, orc.SMOOTH_MOMENTUM,
+                                  orc.SMOOTH_PARAGRAPH])
+def test_every_rule_is_the_identity_on_a_constant_signal(rule):
+    assert _run_rule(rule, [0.625] * 14, window=10) == [0.625] * 14
+
+
+def test_window_longer_than_the_ring_history_wraps_correctly():
+    s = [float(i % 7) for i in range(40)]
+    xs = _run_rule(orc.SMOOTH_WINDOW, s, window=10)
+    for t in range(40):
+        lo = max(0, t - 9)
+        want = float(torch.tensor(sum(s[lo:t + 1]) / (t + 1 - lo), dtype=torch.float32))
+        assert abs(xs[t] - want) < 1e-6
