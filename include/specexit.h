@@ -54,6 +54,12 @@ enum { SX_MODE_CHAIN = 0, SX_MODE_TREE = 1 };
 enum { SX_ACT_SIGMOID = 0, SX_ACT_EXPM1 = 1, SX_ACT_IDENTITY = 2 };   /* Eq. 3-5 */
 enum { SX_DIR_GT = 0, SX_DIR_LT = 1 };                                 /* Appendix A.1 thresholds */
 enum { SX_EMA_VERIFIED_CONTEXT = 0, SX_EMA_FIRST_ONLY = 1 };
+/* Appendix A.1 smoothing rules.  EWMA: x <- alpha s + (1 - alpha) x.  NONE: x = s.  WINDOW: mean of
+ * the last N samples (of those that exist).  MOMENTUM: x_t = s_{t-1} + (s_{t-1} - s_{t-N}) / (N - 1),
+ * the printed sum of differences telescoped, with as many differences as exist.  PARAGRAPH: mean
+ * of the samples since the last step-split token. */
+enum { SX_SMOOTH_EWMA = 0, SX_SMOOTH_NONE = 1, SX_SMOOTH_WINDOW = 2, SX_SMOOTH_MOMENTUM = 3, SX_SMOOTH_PARAGRAPH = 4 };
+#define SX_HIST 16
 
 #define SX_MAX_SIGNALS 3
 #define SX_MAX_TOPK 8
@@ -115,6 +121,8 @@ typedef struct {
   int32_t ema_positions;             /* which accepted slots feed the EWMA */
   const uint32_t *split_bitmap_d;    /* vocab bits, bit (t % 32) of word t / 32; NULL: every token splits */
   int32_t stop_think_token;
+  int32_t smoothing;                 /* SX_SMOOTH_*: Appendix A.1, "Signal Smoothing" */
+  int32_t window;                    /* N of the sliding-window and momentum rules, 2 <= N < SX_HIST */
 } sx_exit_cfg;
 
 /* Per-sequence state carried across iterations (device, caller-owned). */
@@ -122,6 +130,10 @@ typedef struct {
   float *x_d;            /* [batch, n_signals] smoothed signals */
   int32_t *n_updates_d;  /* [batch] samples folded in so far; 0 -> the next sample initialises x */
   int32_t *thinking_d;   /* [batch] 1 while inside the reasoning phase */
+  float *hist_d;         /* [batch, SX_HIST, n_signals] ring of the latest samples (sample i at i % SX_HIST);
+                            needed by SX_SMOOTH_WINDOW and SX_SMOOTH_MOMENTUM, else may be NULL */
+  float *par_sum_d;      /* [batch, n_signals] sum over the current paragraph; SX_SMOOTH_PARAGRAPH, else NULL */
+  int32_t *par_n_d;      /* [batch] samples in the current paragraph; SX_SMOOTH_PARAGRAPH, else NULL */
 } sx_exit_state;
 
 /* Outputs of one iteration; P = K + 1 (chain) or 1 + max_nodes (tree); rows = K (chain) or

@@ -23,6 +23,8 @@ MODE_CHAIN, MODE_TREE = 0, 1
 ACT_SIGMOID, ACT_EXPM1, ACT_IDENTITY = 0, 1, 2
 DIR_GT, DIR_LT = 0, 1
 EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
+SMOOTH_EWMA, SMOOTH_NONE, SMOOTH_WINDOW, SMOOTH_MOMENTUM, SMOOTH_PARAGRAPH = 0, 1, 2, 3, 4
+HIST = 16
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
@@ -61,11 +63,12 @@ class ExitCfg(C.Structure):
     _fields_ = [("alpha", C.c_float), ("thr", C.c_float * SX_MAX_SIGNALS),
                 ("dir", C.c_int32 * SX_MAX_SIGNALS), ("enable_mask", C.c_uint32),
                 ("ema_positions", C.c_int32), ("split_bitmap_d", C.c_void_p),
-                ("stop_think_token", C.c_int32)]
+                ("stop_think_token", C.c_int32), ("smoothing", C.c_int32), ("window", C.c_int32)]
 
 
 class ExitState(C.Structure):
-    _fields_ = [("x_d", C.c_void_p), ("n_updates_d", C.c_void_p), ("thinking_d", C.c_void_p)]
+    _fields_ = [("x_d", C.c_void_p), ("n_updates_d", C.c_void_p), ("thinking_d", C.c_void_p),
+                ("hist_d", C.c_void_p), ("par_sum_d", C.c_void_p), ("par_n_d", C.c_void_p)]
 
 
 _ITER_FIELDS = ("cand_tok_d", "parent_d", "depth_d", "slot_row_d", "slot_src_row_d", "hidden_d",
@@ -146,6 +149,8 @@ class ExitParams:
     ema_positions: int = EMA_VERIFIED_CONTEXT
     split_bitmap: Optional[torch.Tensor] = None     # int32 words on the device, or None
     stop_think_token: int = 0
+    smoothing: int = SMOOTH_EWMA
+    window: int = 10
 
     def struct(self) -> ExitCfg:
         c = ExitCfg()
@@ -157,6 +162,8 @@ class ExitParams:
         c.ema_positions = self.ema_positions
         c.split_bitmap_d = _p(self.split_bitmap)
         c.stop_think_token = self.stop_think_token
+        c.smoothing = self.smoothing
+        c.window = self.window
         return c
 
 
@@ -242,7 +249,10 @@ class SpecExit:
     def new_state(self, B: int) -> Dict[str, torch.Tensor]:
         return {"x": torch.zeros(B, self.shape.S, dtype=torch.float32, device=self.dev),
                 "n_updates": torch.zeros(B, dtype=torch.int32, device=self.dev),
-                "thinking": torch.ones(B, dtype=torch.int32, device=self.dev)}
+                "thinking": torch.ones(B, dtype=torch.int32, device=self.dev),
+                "hist": torch.zeros(B, HIST, self.shape.S, dtype=torch.float32, device=self.dev),
+                "par_sum": torch.zeros(B, self.shape.S, dtype=torch.float32, device=self.dev),
+                "par_n": torch.zeros(B, dtype=torch.int32, device=self.dev)}
 
     def new_outputs(self, B: int) -> Dict[str, torch.Tensor]:
         d, P, S = self.dev, self.P, self.shape.S
@@ -265,7 +275,8 @@ class SpecExit:
 
     @staticmethod
     def _state_struct(st: Dict[str, torch.Tensor]) -> ExitState:
-        return ExitState(st["x"].data_ptr(), st["n_updates"].data_ptr(), st["thinking"].data_ptr())
+        return ExitState(st["x"].data_ptr(), st["n_updates"].data_ptr(), st["thinking"].data_ptr(),
+                         _p(st.get("hist")), _p(st.get("par_sum")), _p(st.get("par_n")))
 
     def _stream(self) -> int:
         return torch.cuda.current_stream(self.dev).cuda_stream

@@ -376,6 +376,11 @@ extern "C" sx_status sx_exit_update(sx_ctx *c, int32_t batch, int32_t P, const s
   if (!state->x_d || !state->n_updates_d || !state->thinking_d || batch < 1 || P < 1 || path_stride < 1)
     return SX_ERR_INVALID_ARG;
   if (!(cfg->alpha >= 0.f && cfg->alpha <= 1.f)) return SX_ERR_INVALID_ARG;
+  if (cfg->smoothing < SX_SMOOTH_EWMA || cfg->smoothing > SX_SMOOTH_PARAGRAPH) return SX_ERR_INVALID_ARG;
+  if ((cfg->smoothing == SX_SMOOTH_WINDOW || cfg->smoothing == SX_SMOOTH_MOMENTUM) &&
+      (!state->hist_d || cfg->window < 2 || cfg->window >= SX_HIST))
+    return SX_ERR_INVALID_ARG;
+  if (cfg->smoothing == SX_SMOOTH_PARAGRAPH && (!state->par_sum_d || !state->par_n_d)) return SX_ERR_INVALID_ARG;
   sx_launch_exit(batch, P, c->sh.S, *cfg, *state, slot_signal_d, cand_tok_d, path_d, path_stride, accept_len_d,
                  recover_tok_d, exit_flag_d, accept_len_out_d, recover_tok_out_d, smoothed_out_d, c->sh.V, status_d,
                  (cudaStream_t)stream);

@@ -437,6 +437,9 @@ struct SxExitParams {
   int ema_positions;
   const uint32_t *bitmap;
   int stop_tok;
+  int smoothing, window;
+  float *hist, *par_sum;
+  int32_t *par_n;
 };
 
 __global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float *x_state, int32_t *n_updates,
@@ -462,9 +465,34 @@ __global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float
         bool none = false;
         for (int i = 0; i < S; ++i) none |= isnan(sg[i]);
         if (none) break;
-        for (int i = 0; i < S; ++i)
-          x[i] = (nu == 0) ? sg[i]
-                           : (float)((double)p.alpha * (double)sg[i] + (1.0 - (double)p.alpha) * (double)x[i]);
+        for (int i = 0; i < S; ++i) {
+          const float s = sg[i];
+          if (p.smoothing == SX_SMOOTH_EWMA) {
+            x[i] = (nu == 0) ? s : (float)((double)p.alpha * (double)s + (1.0 - (double)p.alpha) * (double)x[i]);
+          } else if (p.smoothing == SX_SMOOTH_NONE) {
+            x[i] = s;
+          } else if (p.smoothing == SX_SMOOTH_PARAGRAPH) {
+            float *ps = p.par_sum + (size_t)b * S + i;
+            *ps = (float)((double)*ps + (double)s);
+            x[i] = (float)((double)*ps / (double)(p.par_n[b] + 1));
+          } else {
+            float *h = p.hist + (size_t)b * SX_HIST * S + i;       // sample j of this signal at h[(j % SX_HIST) * S]
+            h[(nu % SX_HIST) * S] = s;
+            if (p.smoothing == SX_SMOOTH_WINDOW) {
+              const int m = min(nu + 1, p.window);
+              double acc = 0.0;
+              for (int j = nu - m + 1; j <= nu; ++j) acc += (double)h[(j % SX_HIST) * S];
+              x[i] = (float)(acc / (double)m);
+            } else if (nu == 0) {
+              x[i] = s;
+            } else {
+              const int k = min(p.window - 1, nu - 1);
+              const double prev = (double)h[((nu - 1) % SX_HIST) * S];
+              x[i] = (k == 0) ? (float)prev : (float)(prev + (prev - (double)h[((nu - 1 - k) % SX_HIST) * S]) / (double)k);
+            }
+          }
+        }
+        if (p.smoothing == SX_SMOOTH_PARAGRAPH) p.par_n[b] += 1;
         ++nu;
       }
       const int tok = cand[(size_t)b * P + slot];
@@ -479,6 +507,10 @@ __global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float
         flag = 1; Lo = idx; ro = p.stop_tok;
         thinking[b] = 0;
         break;
+      }
+      if (split && p.smoothing == SX_SMOOTH_PARAGRAPH) {       // a paragraph delimiter went by
+        for (int i = 0; i < S; ++i) p.par_sum[(size_t)b * S + i] = 0.f;
+        p.par_n[b] = 0;
       }
     }
     for (int i = 0; i < S; ++i) x_state[(size_t)b * S + i] = x[i];
@@ -502,6 +534,8 @@ void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_s
   p.ema_positions = cfg.ema_positions;
   p.bitmap = cfg.split_bitmap_d;
   p.stop_tok = cfg.stop_think_token;
+  p.smoothing = cfg.smoothing; p.window = cfg.window;
+  p.hist = state.hist_d; p.par_sum = state.par_sum_d; p.par_n = state.par_n_d;
   sx_launch(sx_exit_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, S, V, p, state.x_d, state.n_updates_d,
             state.thinking_d, slot_signal, cand, path, path_stride, accept_len, recover, exit_flag, accept_out,
             recover_out, smoothed, status);

@@ -150,7 +150,8 @@ def to_params(sx: binding.SpecExit, cfg: orc.ExitCfg) -> binding.ExitParams:
     bm = None if cfg.split_bitmap is None else cfg.split_bitmap.to(sx.dev)
     return binding.ExitParams(alpha=cfg.alpha, thr=tuple(cfg.thr), dir=tuple(cfg.dir),
                               enable_mask=cfg.enable_mask, ema_positions=cfg.ema_positions,
-                              split_bitmap=bm, stop_think_token=cfg.stop_think_token)
+                              split_bitmap=bm, stop_think_token=cfg.stop_think_token, smoothing=cfg.smoothing,
+                              window=cfg.window)
 
 
 def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, parent, slot_signal,
