@@ -306,15 +306,25 @@ __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int p
   sx_pdl_wait();
   const int r = blockIdx.x, tid = threadIdx.x;
   for (int i = tid; i < G * T; i += blockDim.x) sx_cand[i] = parts[(size_t)(i / T) * part_stride + r].top[i % T];
-  if (tid == 0 && lse) {
-    float mm = -INFINITY;
-    for (int g = 0; g < G; ++g) mm = fmaxf(mm, parts[(size_t)g * part_stride + r].m);
-    float ll = 0.f;
-    for (int g = 0; g < G; ++g) {
+  if (lse) {
+    // log-sum-exp over the CTAs' (max, sum) pairs: every thread takes a few of them
+    __shared__ float s_red[4];
+    float mloc = -INFINITY;
+    for (int g = tid; g < G; g += blockDim.x) mloc = fmaxf(mloc, parts[(size_t)g * part_stride + r].m);
+    mloc = sx_warp_max(mloc);
+    if ((tid & 31) == 0) s_red[tid >> 5] = mloc;
+    __syncthreads();
+    const float mm = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
+    __syncthreads();
+    float lloc = 0.f;
+    for (int g = tid; g < G; g += blockDim.x) {
       const SxHeadPartial &p = parts[(size_t)g * part_stride + r];
-      if (p.l > 0.f) ll += p.l * expf(p.m - mm);
+      if (p.l > 0.f) lloc += p.l * expf(p.m - mm);
     }
-    s_lse = mm + logf(ll);
+    lloc = sx_warp_sum(lloc);
+    if ((tid & 31) == 0) s_red[tid >> 5] = lloc;
+    __syncthreads();
+    if (tid == 0) s_lse = mm + logf((s_red[0] + s_red[1]) + (s_red[2] + s_red[3]));
   }
   __syncthreads();
   const int tbase = sx_index(toi, r);
