@@ -605,13 +605,15 @@ void sx_gemm_init(int device) {
   cudaFuncSetAttribute(sx_tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
 }
 
-// Choose the K split: fill the SMs in whole waves, keep at least 4 k-blocks per item.
+// Choose the K split: fill the SMs in whole waves, keep at least 4 k-blocks per item, and use at
+// most 4 splits: beyond that the extra partial sums (written, then read back by the finisher in
+// dependent batches) cost more than the better SM coverage gains (measured on C1 and C2).
 int sx_gemm_pick_splits(int N, int K, int sm_count) {
   const int tiles = (N + SX_TILE_M - 1) / SX_TILE_M;
   const int num_kb = (K + SX_BK - 1) / SX_BK;
   int best = 1;
   double best_eff = 0.0;
-  for (int s = 1; s <= 16; ++s) {
+  for (int s = 1; s <= 4; ++s) {
     const int per = (num_kb + s - 1) / s;
     if (per < 4 && s > 1) break;
     const int real = (num_kb + per - 1) / per;
