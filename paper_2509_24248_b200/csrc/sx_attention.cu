@@ -365,18 +365,18 @@ sx_attn_mma_kernel(int nq, int nkv, int G, int page, int page_shift, float scale
     }
 }
 
-// o[hq][d] = sum_s O_s[d] 2^(m_s - M) / sum_s l_s 2^(m_s - M).  One CTA of 256 threads per query row:
-// thread = (split group of 8, float4 of the head dimension), so that the loads of all splits are
-// in flight together; at most 256 splits.
-__global__ void __launch_bounds__(256)
+// o[hq][d] = sum_s O_s[d] 2^(m_s - M) / sum_s l_s 2^(m_s - M).  One CTA per query row: thread =
+// (split group, float4 of the head dimension), 8 or 32 groups, so that the loads of all splits
+// are in flight together; at most 256 splits.
+__global__ void __launch_bounds__(1024)
 sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__restrict__ ws_ml, const float *__restrict__ ws_o,
                      bf16 *__restrict__ o_out) {
   __shared__ float s_w[256];               // weights 2^(m_s - M)
-  __shared__ float s_red[8], s_sum[8];
-  __shared__ float4 s_acc[8][32];
+  __shared__ float s_red[32], s_sum[32];
+  __shared__ float4 s_acc[32][32];
   sx_pdl_launch_dependents();
   const size_t hq = (size_t)blockIdx.y * nq + blockIdx.x;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nw = blockDim.x >> 5;
   sx_pdl_wait();
   float2 ml = make_float2(-INFINITY, 0.f);
   if (tid < nsplit) ml = ws_ml[hq * nsplit + tid];
@@ -384,17 +384,16 @@ sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__restrict__ ws_ml
   if (lane == 0) s_red[warp] = mm;
   __syncthreads();
   mm = s_red[0];
-#pragma unroll
-  for (int w = 1; w < 8; ++w) mm = fmaxf(mm, s_red[w]);
+  for (int w = 1; w < nw && w < 8; ++w) mm = fmaxf(mm, s_red[w]);      // splits live in the first 256 threads
   const float wgt = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mm);
-  s_w[tid] = wgt;
+  if (tid < 256) s_w[tid] = wgt;
   const float ls = sx_warp_sum(ml.y * wgt);
   if (lane == 0) s_sum[warp] = ls;
   __syncthreads();
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   if (lane * 4 < d) {
     const float *src = ws_o + hq * nsplit * d + lane * 4;
-    for (int sp = warp; sp < nsplit; sp += 8) {
+    for (int sp = warp; sp < nsplit; sp += nw) {
       const float4 v = *reinterpret_cast<const float4 *>(src + (size_t)sp * d);
       const float w = s_w[sp];
       acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
@@ -404,12 +403,10 @@ sx_attn_merge_kernel(int nq, int d, int nsplit, const float2 *__restrict__ ws_ml
   __syncthreads();
   if (tid < d) {
     float ll = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) ll += s_sum[w];
+    for (int w = 0; w < nw && w < 8; ++w) ll += s_sum[w];
     const float *col = reinterpret_cast<const float *>(&s_acc[0][0]) + tid;
     float a = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) a += col[w * 128];
+    for (int w = 0; w < nw; ++w) a += col[w * 128];
     o_out[hq * d + tid] = __float2bfloat16_rn(a / ll);
   }
 }
@@ -510,6 +507,6 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   }
 #undef SX_ATTN_NT
 #undef SX_ATTN
-  sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3(256), 0, st, sh.nq, sh.d, nsplit, (const float2 *)ws_ml,
-            (const float *)ws_o, o_out);
+  sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3((nsplit > 64 && sh.nq * R <= 296) ? 1024 : 256), 0, st, sh.nq, sh.d, nsplit,
+            (const float2 *)ws_ml, (const float *)ws_o, o_out);
 }
