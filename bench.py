@@ -142,6 +142,43 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+def write_timeline(path: str, step, name: str) -> None:
+    """Three iterations under the CUPTI activity tracer; the middle one is written out.  A kernel's
+    'adds' is its completion time minus the latest completion before it: with programmatic dependent
+    launch kernels start early and wait, so durations overlap and only completions are meaningful."""
+    import collections
+    from torch.profiler import ProfilerActivity, profile
+    with profile(activities=[ProfilerActivity.CUDA]) as prof:
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+    ev = sorted((e for e in prof.events() if e.device_type.name == "CUDA" and e.name.startswith(("sx_", "void sx_"))),
+                key=lambda e: e.time_range.start)
+    n = len(ev) // 3
+    it = ev[n:2 * n]
+    t0 = it[0].time_range.start
+    prev_end = t0
+    agg = collections.OrderedDict()
+    lines = [f"workload {name}: one iteration, {len(it)} kernels; times in us", f"{'start':>9s} {'end':>9s} {'adds':>8s}  kernel"]
+    for e in it:
+        nm = e.name.split("(")[0].replace("void ", "")[:44]
+        end = e.time_range.end
+        adds = max(0.0, end - prev_end)
+        lines.append(f"{e.time_range.start - t0:9.2f} {end - t0:9.2f} {adds:8.2f}  {nm}")
+        a = agg.setdefault(nm, [0, 0.0])
+        a[0] += 1
+        a[1] += adds
+        prev_end = max(prev_end, end)
+    tot = sum(a[1] for a in agg.values())
+    lines.append("")
+    lines.append("sum of 'adds' per kernel (the first kernel absorbs the tail of the previous iteration):")
+    for k, a in sorted(agg.items(), key=lambda x: -x[1][1]):
+        lines.append(f"  {k:46s} n={a[0]:3d} {a[1]:9.1f} us {a[1] / tot * 100:5.1f} %  avg {a[1] / a[0]:7.2f}")
+    lines.append(f"  total {tot:.1f} us")
+    with open(path, "w") as f:
+        f.write("\n".join(lines) + "\n")
+
+
 def build_inputs(wl: synth.Workload):
     lens = synth.cache_lengths(wl)
     kv = synth.make_kv(wl.shape, lens, wl.draft_rows, wl.seed)
@@ -201,6 +238,10 @@ def main():
     ap.add_argument("--workload", default="C1")
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--timeline", default=None, metavar="FILE",
+                    help="also write a per-kernel timeline of one iteration (CUPTI through torch.profiler): when "
+                         "each kernel completed and how long after its predecessor, i.e. what it adds to the "
+                         "dependent chain once programmatic dependent launch has overlapped the rest")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -302,6 +343,9 @@ def main():
     ms = ms_total / args.steps
     value = whole_job_rate(world * args.steps, ms_total)
     vtok = whole_job_rate(sum_over_ranks(float(verified.item()), dist, dev), ms_total)
+
+    if args.timeline and rank == 0:
+        write_timeline(args.timeline, step, wl.name)
 
     # end to end: host buffers in, results out, through the host entry point
     stage = {"feat0": torch.empty_like(f0_d), "tok0": torch.empty_like(t0_d), "target_hidden": torch.empty_like(th_d)}
