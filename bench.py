@@ -319,10 +319,12 @@ def main():
     launches0 = sx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     verified = torch.zeros((), dtype=torch.int64, device=dev)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ev0.record()
-    for _ in range(args.steps):
+    for i in range(args.steps):
         step()
         verified += (out["accept_len_out_d"] + 1).sum()
+        marks[i].record()          # one event per iteration: per-iteration percentiles
     ev1.record()
     torch.cuda.synchronize()
     sampler.mark_end()
@@ -339,6 +341,8 @@ def main():
     torch.cuda.synchronize()
     prof = sx.profile_end()
     clocks = sampler.stop()
+    per_step = sorted(a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks))
+    pct = lambda q: per_step[min(len(per_step) - 1, int(q * len(per_step)))]
     ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms = ms_total / args.steps
     value = whole_job_rate(world * args.steps, ms_total)
@@ -389,6 +393,7 @@ def main():
         "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "verified_tokens_per_s": vtok, "sequence_iterations_per_s": value * wl.B,
+        "ms_per_step_percentiles": {"p10": pct(0.10), "p50": pct(0.50), "p90": pct(0.90)},
         "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree",
                    "cached_tokens": int(sum(int(n) for n in lens)),
                    "l2": "no flush: each iteration streams %.2f GB of weights and KV, far beyond the 126 MB L2"
