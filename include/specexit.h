@@ -165,9 +165,9 @@ typedef struct {
 typedef struct sx_ctx sx_ctx;
 
 /* Build a host-side plan for the given shapes.  Weight pointers are recorded, not copied.
- * Fails with SX_ERR_UNSUPPORTED for shapes the kernels do not cover (H, head_dim, ffn not
- * multiples of 8; head_dim > 256 or not a power of two; group size > 8; topk, rows or slots
- * beyond the SX_MAX_* limits). */
+ * Fails with SX_ERR_UNSUPPORTED for shapes the kernels do not cover: H, ffn not multiples of 8;
+ * head_dim other than 16, 32, 64 or 128; a group size (n_q_heads / n_kv_heads) other than 1, 2,
+ * 4 or 8; group size * topk > 64; topk, rows or slots beyond the SX_MAX_* limits. */
 sx_status sx_create(const sx_model_cfg *model, const sx_weights *weights, int32_t max_batch,
                     const sx_draft_cfg *draft, int32_t max_verify_rows, sx_ctx **out);
 void sx_destroy(sx_ctx *ctx);

@@ -70,7 +70,7 @@ extern "C" sx_status sx_profile_end(sx_ctx *c, float *ms_out, int32_t *count_out
   return SX_OK;
 }
 
-#define SX_COMMIT_MAX_SPLITS 4
+#define SX_COMMIT_MAX_SPLITS SX_GEMM_MAX_SPLITS
 
 static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 
@@ -107,7 +107,6 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (m->n_signals < 0 || m->n_signals > SX_MAX_SIGNALS || m->vocab < 1 || m->page_size < 1)
     return SX_ERR_UNSUPPORTED;
   if (m->H > 16384) return SX_ERR_UNSUPPORTED;
-  if (!(m->head_dim == 16 || m->head_dim == 32 || m->head_dim == 64 || m->head_dim == 128)) return SX_ERR_UNSUPPORTED;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
@@ -148,6 +147,10 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
     delete c;
     return SX_ERR_CUDA;
   }
+  if (!sx_attn_supported(c->sh)) {            // head_dim 16 / 32 / 64 / 128, group size * topk <= 64
+    delete c;
+    return SX_ERR_UNSUPPORTED;
+  }
   c->device = dev;
   c->sm_count = prop.multiProcessorCount;
   sx_gemm_init(dev);
@@ -155,7 +158,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
 
   const SxShape &s = c->sh;
   const int R = c->Rmax;
-  c->max_splits = 16;
+  c->max_splits = SX_GEMM_MAX_SPLITS;
   c->part_N = s.H;
   if ((s.nq + 2 * s.nkv) * s.d > c->part_N) c->part_N = (s.nq + 2 * s.nkv) * s.d;
   if (2 * s.F > c->part_N) c->part_N = 2 * s.F;

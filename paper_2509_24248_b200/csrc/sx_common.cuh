@@ -31,28 +31,7 @@ struct SxRowInfo {
   int n;          // cached prefix length
   int pos;        // rotary position
   int rel;        // drafted-row index within the sequence (slot = n + rel)
-  uint64_t mask;  // visible drafted rows (own bit included)
 };
-
-__device__ __forceinline__ SxRowInfo sx_row_info(const SxRowMap &m, int r) {
-  SxRowInfo i;
-  if (m.mode == SX_MODE_CHAIN) {
-    i.b = r;
-    i.rel = m.round - 1;
-    i.mask = (i.rel >= 63) ? ~0ull : ((2ull << i.rel) - 1ull);
-  } else if (m.round == 1) {
-    i.b = r;
-    i.rel = 0;
-    i.mask = 1ull;
-  } else {
-    i.b = r / m.topk;
-    i.rel = 1 + (m.round - 2) * m.topk + (r % m.topk);
-    i.mask = m.row_mask[r];
-  }
-  i.n = m.cache_len[i.b];
-  i.pos = i.n + m.round - 1;
-  return i;
-}
 
 // placement only (sequence, cached length, position, drafted-row index): touches nothing a kernel
 // of the same iteration writes, so it may run before the wait on the preceding kernel
@@ -61,7 +40,6 @@ __device__ __forceinline__ SxRowInfo sx_row_place(const SxRowMap &m, int r) {
   if (m.mode == SX_MODE_COMMIT) {
     i.b = r / m.per_seq;
     i.rel = 1 + (r - i.b * m.per_seq);
-    i.mask = 0ull;
     i.n = m.cache_len[i.b];
     i.pos = i.n + i.rel;
     return i;
@@ -69,7 +47,6 @@ __device__ __forceinline__ SxRowInfo sx_row_place(const SxRowMap &m, int r) {
   if (m.mode == SX_MODE_CHAIN) { i.b = r; i.rel = m.round - 1; }
   else if (m.round == 1) { i.b = r; i.rel = 0; }
   else { i.b = r / m.topk; i.rel = 1 + (m.round - 2) * m.topk + (r % m.topk); }
-  i.mask = 0ull;
   i.n = m.cache_len[i.b];
   i.pos = i.n + m.round - 1;
   return i;
@@ -109,18 +86,6 @@ __device__ __forceinline__ float sx_warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
-
-__device__ __forceinline__ void sx_unpack8(const uint4 &u, float *f) {
-  const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&u);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float2 t = __bfloat1622float2(p[i]);
-    f[2 * i] = t.x;
-    f[2 * i + 1] = t.y;
-  }
-}
-
-__device__ __forceinline__ float sx_round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 __device__ __forceinline__ float sx_activate(float z, int act) {
   if (act == SX_ACT_SIGMOID) return 1.0f / (1.0f + expf(-z));

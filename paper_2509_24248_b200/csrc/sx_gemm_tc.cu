@@ -613,7 +613,7 @@ int sx_gemm_pick_splits(int N, int K, int sm_count) {
   const int num_kb = (K + SX_BK - 1) / SX_BK;
   int best = 1;
   double best_eff = 0.0;
-  for (int s = 1; s <= 4; ++s) {
+  for (int s = 1; s <= SX_GEMM_MAX_SPLITS; ++s) {
     const int per = (num_kb + s - 1) / s;
     if (per < 4 && s > 1) break;
     const int real = (num_kb + per - 1) / per;

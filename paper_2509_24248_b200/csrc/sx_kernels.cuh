@@ -88,7 +88,7 @@ void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, c
 
 // ---- GEMMs (sx_gemm_tc.cu) ----------------------------------------------------------------
 // part[s][r][n] = sum over the s-th K range of X[r][k] * W[n][k]   (fp32)
-struct SxGemmPlan { int splits; };
+#define SX_GEMM_MAX_SPLITS 4      // sx_gemm_pick_splits never returns more
 int sx_gemm_pick_splits(int N, int K, int sm_count);
 sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part,
                                  int splits, size_t split_stride, int sm_count, int32_t *status,
