@@ -247,12 +247,20 @@ class SpecExit:
                              self.kv["k_pages"].data_ptr(), self.kv["v_pages"].data_ptr())
 
     def new_state(self, B: int) -> Dict[str, torch.Tensor]:
-        return {"x": torch.zeros(B, self.shape.S, dtype=torch.float32, device=self.dev),
-                "n_updates": torch.zeros(B, dtype=torch.int32, device=self.dev),
-                "thinking": torch.ones(B, dtype=torch.int32, device=self.dev),
-                "hist": torch.zeros(B, HIST, self.shape.S, dtype=torch.float32, device=self.dev),
-                "par_sum": torch.zeros(B, self.shape.S, dtype=torch.float32, device=self.dev),
-                "par_n": torch.zeros(B, dtype=torch.int32, device=self.dev)}
+        """Exit state of B sequences.  All arrays are views of one 4-byte-word buffer (``"_all"``), so
+        that a caller can save or restore the whole state with a single copy."""
+        S = self.shape.S
+        sizes = [("x", B * S, torch.float32, (B, S)), ("n_updates", B, torch.int32, (B,)),
+                 ("thinking", B, torch.int32, (B,)), ("hist", B * HIST * S, torch.float32, (B, HIST, S)),
+                 ("par_sum", B * S, torch.float32, (B, S)), ("par_n", B, torch.int32, (B,))]
+        words = sum(((n + 3) // 4) * 4 for _, n, _, _ in sizes)
+        buf = torch.zeros(words, dtype=torch.int32, device=self.dev)
+        st, at = {"_all": buf}, 0
+        for name, n, dt, shape in sizes:
+            st[name] = buf[at:at + n].view(dt).view(*shape)
+            at += ((n + 3) // 4) * 4
+        st["thinking"].fill_(1)
+        return st
 
     def new_outputs(self, B: int) -> Dict[str, torch.Tensor]:
         d, P, S = self.dev, self.P, self.shape.S
