@@ -295,54 +295,64 @@ void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int sp
 // ---------------------------------------------------------------------------------------
 // merge of the per-CTA head results: top-T ids (+ log-probabilities), activated signals
 // ---------------------------------------------------------------------------------------
-__global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
-                                        const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
-                                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si, SxNextInput nx) {
-  extern __shared__ unsigned long long sx_cand[];      // [G * T]
-  __shared__ unsigned long long wbest[4];
+// One CTA per token row, one thread per CTA of the head kernel (blockDim >= G).  Every per-CTA list
+// is sorted, so the global top-T is a tournament over the list heads: T rounds of a block-wide
+// maximum, the winner advances in its list.  Everything stays in registers.
+__global__ void __launch_bounds__(1024)
+sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
+                        const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
+                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si, SxNextInput nx) {
+  __shared__ unsigned long long s_best[2][32];
+  __shared__ float s_red[32];
   __shared__ float s_lse;
   __shared__ int s_tok;
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int r = blockIdx.x, tid = threadIdx.x;
-  for (int i = tid; i < G * T; i += blockDim.x) sx_cand[i] = parts[(size_t)(i / T) * part_stride + r].top[i % T];
-  if (lse) {
-    // log-sum-exp over the CTAs' (max, sum) pairs: every thread takes a few of them
-    __shared__ float s_red[4];
-    float mloc = -INFINITY;
-    for (int g = tid; g < G; g += blockDim.x) mloc = fmaxf(mloc, parts[(size_t)g * part_stride + r].m);
-    mloc = sx_warp_max(mloc);
-    if ((tid & 31) == 0) s_red[tid >> 5] = mloc;
-    __syncthreads();
-    const float mm = fmaxf(fmaxf(s_red[0], s_red[1]), fmaxf(s_red[2], s_red[3]));
-    __syncthreads();
-    float lloc = 0.f;
-    for (int g = tid; g < G; g += blockDim.x) {
-      const SxHeadPartial &p = parts[(size_t)g * part_stride + r];
-      if (p.l > 0.f) lloc += p.l * expf(p.m - mm);
-    }
-    lloc = sx_warp_sum(lloc);
-    if ((tid & 31) == 0) s_red[tid >> 5] = lloc;
-    __syncthreads();
-    if (tid == 0) s_lse = mm + logf((s_red[0] + s_red[1]) + (s_red[2] + s_red[3]));
+  const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = blockDim.x >> 5;
+  unsigned long long v[SX_MAX_TOPK];
+  float pm = -INFINITY, pl = 0.f;
+#pragma unroll
+  for (int k = 0; k < SX_MAX_TOPK; ++k) v[k] = 0ull;
+  if (tid < G) {
+    const SxHeadPartial &p = parts[(size_t)tid * part_stride + r];
+#pragma unroll
+    for (int k = 0; k < SX_MAX_TOPK; ++k)
+      if (k < T) v[k] = p.top[k];
+    pm = p.m;
+    pl = p.l;
   }
-  __syncthreads();
+  if (lse) {
+    float mm = sx_warp_max(pm);
+    if (lane == 0) s_red[warp] = mm;
+    __syncthreads();
+    mm = sx_warp_max(lane < nw ? s_red[lane] : -INFINITY);
+    __syncthreads();
+    float ll = sx_warp_sum(pl > 0.f ? pl * expf(pm - mm) : 0.f);
+    if (lane == 0) s_red[warp] = ll;
+    __syncthreads();
+    ll = sx_warp_sum(lane < nw ? s_red[lane] : 0.f);
+    if (tid == 0) s_lse = mm + logf(ll);
+  }
   const int tbase = sx_index(toi, r);
   for (int t = 0; t < T; ++t) {
-    unsigned long long best = 0ull;
-    for (int i = tid; i < G * T; i += blockDim.x) best = max(best, sx_cand[i]);
+    unsigned long long best = v[0];
+#pragma unroll
     for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
-    if ((tid & 31) == 0) wbest[tid >> 5] = best;
+    if (lane == 0) s_best[t & 1][warp] = best;
     __syncthreads();
-    best = max(max(wbest[0], wbest[1]), max(wbest[2], wbest[3]));
+    best = lane < nw ? s_best[t & 1][lane] : 0ull;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
     if (tid == 0) {
       tok_out[tbase + t] = (int32_t)sx_pack_index(best);
       if (t == 0) s_tok = (int32_t)sx_pack_index(best);
       if (logp_out) logp_out[(size_t)r * T + t] = lse ? sx_pack_value(best) - s_lse : sx_pack_value(best);
     }
-    for (int i = tid; i < G * T; i += blockDim.x)
-      if (sx_cand[i] == best) sx_cand[i] = 0ull;       // packed values are unique (index inside)
-    __syncthreads();
+    if (best != 0ull && v[0] == best) {          // packed values are unique (index inside): one winner
+#pragma unroll
+      for (int k = 0; k + 1 < SX_MAX_TOPK; ++k) v[k] = v[k + 1];
+      v[SX_MAX_TOPK - 1] = 0ull;
+    }
   }
   if (sig_out && tid < S) {
     const int a = tid == 0 ? act0 : (tid == 1 ? act1 : act2);
@@ -368,8 +378,10 @@ __global__ void sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int p
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
                              float *logp_out, float *sig_out, SxIndex si, cudaStream_t st, SxNextInput nx) {
-  sx_launch(sx_head_finalize_kernel, dim3(R), dim3(128), (size_t)G * T * 8, st, parts, G, part_stride, T, lse, z, S,
-            sh.act[0], sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx);
+  int threads = ((G + 31) / 32) * 32;              // one thread per CTA of the head kernel (G <= SM count)
+  if (threads < 128) threads = 128;
+  sx_launch(sx_head_finalize_kernel, dim3(R), dim3(threads), 0, st, parts, G, part_stride, T, lse, z, S, sh.act[0],
+            sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx);
 }
 
 // ---------------------------------------------------------------------------------------
