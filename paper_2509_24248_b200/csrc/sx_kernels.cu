@@ -411,39 +411,56 @@ void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_i
 // ---------------------------------------------------------------------------------------
 // greedy acceptance (Algorithm 1): chain prefix match, or the walk down the tree
 // ---------------------------------------------------------------------------------------
+// One warp per sequence; in a tree the lanes look for the accepted child together.
 __global__ void sx_accept_kernel(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                                  int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover) {
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (b >= B) return;
   const int32_t *c = cand + (size_t)b * P, *t = target + (size_t)b * P;
   int32_t *pa = path + (size_t)b * path_stride;
   int L = 0, cur = 0;
-  pa[0] = 0;
+  if (lane == 0) pa[0] = 0;
   if (!parent) {
-    while (L < P - 1 && c[L + 1] == t[L]) { ++L; if (L < path_stride) pa[L] = L; }
+    // longest prefix with cand[j + 1] == target[j]: first mismatch among the lanes' positions
+    for (int j0 = 0; j0 < P - 1; j0 += 32) {
+      const int j = j0 + lane;
+      const bool ok = j < P - 1 && c[j + 1] == t[j];
+      const unsigned miss = ~__ballot_sync(0xffffffffu, ok);
+      const int run = miss ? __ffs(miss) - 1 : 32;
+      if (lane < run && j0 + lane + 1 < path_stride) pa[j0 + lane + 1] = j0 + lane + 1;
+      L += run;
+      if (run < 32) break;
+    }
     cur = L;
   } else {
     const int32_t *par = parent + (size_t)b * P;
     for (;;) {
+      const int want = t[cur];
       int nxt = -1;
-      for (int s = 1; s < P; ++s)
-        if (par[s] == cur && c[s] == t[cur]) { nxt = s; break; }
+      for (int s0 = 1; s0 < P && nxt < 0; s0 += 32) {
+        const int sl = s0 + lane;
+        const bool hit = sl < P && par[sl] == cur && c[sl] == want;
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m) nxt = s0 + __ffs(m) - 1;            // lowest slot wins, as in a serial scan
+      }
       if (nxt < 0) break;
       cur = nxt;
       ++L;
-      if (L < path_stride) pa[L] = cur;
+      if (lane == 0 && L < path_stride) pa[L] = cur;
     }
   }
-  for (int j = L + 1; j < path_stride; ++j) pa[j] = -1;
-  accept_len[b] = L;
-  recover[b] = t[cur];
+  for (int j = L + 1 + lane; j < path_stride; j += 32) pa[j] = -1;
+  if (lane == 0) {
+    accept_len[b] = L;
+    recover[b] = t[cur];
+  }
 }
 
 void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                       int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st) {
-  sx_launch(sx_accept_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, cand, parent, target, accept_len, path,
+  sx_launch(sx_accept_kernel, dim3((B + 3) / 4), dim3(128), 0, st, B, P, cand, parent, target, accept_len, path,
             path_stride, recover);
 }
 
