@@ -193,12 +193,27 @@ class DraftModel:
         self.sh = shape
         self.w = weights
         self.act = tuple(act)
-        # the target's LM head; by default the draft's vocabulary rows
-        self.target_head = target_head if target_head is not None else weights["head"][:shape.V]
+        # The draft head may cover a reduced vocabulary: its first Vd rows score the draft ids
+        # 0..Vd-1, `draft_to_token` maps a draft id to the token id it stands for (identity when
+        # absent); the signal rows of Eq. 1 follow the Vd vocabulary rows.
+        self.Vd = int(weights["head"].shape[0]) - shape.S
+        m = weights.get("draft_to_token")
+        self.map = None if m is None else [int(t) for t in m]
+        assert self.map is None or len(self.map) == self.Vd
+        # the target's LM head; by default the draft's vocabulary rows (full vocabulary only)
+        if target_head is None:
+            target_head = weights.get("target_head")
+        if target_head is None:
+            assert self.Vd == shape.V, "a reduced draft vocabulary needs the target's own head"
+            target_head = weights["head"][:shape.V]
+        self.target_head = target_head
+
+    def to_token(self, draft_id: int) -> int:
+        return int(draft_id) if self.map is None else self.map[int(draft_id)]
 
     # Eq. 1: one matrix, vocabulary rows first, signal rows last, same hidden state
     def head(self, g: torch.Tensor) -> HeadOut:
-        V, S = self.sh.V, self.sh.S
+        V, S = self.Vd, self.sh.S
         full = f32r(linear(g, self.w["head"]))
         z = full[:, V:V + S]
         return HeadOut(logits=full[:, :V], z=z, s=f32r(activate(z, self.act)))
@@ -317,7 +332,7 @@ def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tens
                 tok = int(forced[(b, k)])
             if chooser is not None:
                 tok = int(chooser("tok", (b, k), ho.logits[b], 1, [tok])[0])
-            cand[b, k] = tok
+            cand[b, k] = model.to_token(tok)      # decisions are taken on draft ids, tokens are stored
         hidden[:, k - 1] = g
         sig[:, k - 1] = ho.s
         zz[:, k - 1] = ho.z
@@ -387,7 +402,7 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
         for t in ids:
             lp = f32r(logits[t] - lse)
             sc = f32r(torch.tensor(par_score, dtype=F64) + lp)
-            cands[b].append(Cand(cid=len(cands[b]), depth=dep, parent=par_cid, tok=int(t),
+            cands[b].append(Cand(cid=len(cands[b]), depth=dep, parent=par_cid, tok=model.to_token(t),
                                  logp=float(lp), score=float(sc), src_row=row))
 
     # round 1: the root row

@@ -30,7 +30,7 @@ TREE = 1
 # item ids for the per-item generators
 _IT = {"embed": 1, "fc": 2, "norm1": 3, "norm2": 4, "normf": 5, "wqkv": 6, "wo": 7,
        "wgate_up": 8, "wdown": 9, "head": 10, "k": 11, "v": 12, "f0": 13, "t0": 14,
-       "noise": 15, "sigma": 16, "lens": 17, "perm": 18, "noise2": 19}
+       "noise": 15, "sigma": 16, "lens": 17, "perm": 18, "noise2": 19, "d2t": 20, "target_head": 21}
 
 
 @dataclass(frozen=True)
@@ -45,6 +45,7 @@ class ModelShape:
     eps: float = 1e-6
     theta: float = 1e6
     page: int = 64
+    Vd: int = 0          # rows of a reduced draft vocabulary (0: the draft head covers all V ids)
 
     @property
     def qkv_rows(self) -> int:
@@ -139,8 +140,12 @@ def make_weights(shape: ModelShape, seed: int, std: float = 0.02) -> Dict[str, t
         "wo": _randn_bf16(s.H, s.n_q * s.d, std, 0.0, _gen(seed, "wo")),
         "wgate_up": _randn_bf16(2 * s.F, s.H, std, 0.0, _gen(seed, "wgate_up")),
         "wdown": _randn_bf16(s.H, s.F, std, 0.0, _gen(seed, "wdown")),
-        "head": _randn_bf16(s.V + s.S, s.H, std, 0.0, _gen(seed, "head")),
+        "head": _randn_bf16((s.Vd or s.V) + s.S, s.H, std, 0.0, _gen(seed, "head")),
     }
+    if s.Vd:
+        # reduced draft vocabulary: Vd distinct token ids in increasing order, and a target head of its own
+        w["draft_to_token"] = torch.sort(torch.randperm(s.V, generator=_gen(seed, "d2t"))[:s.Vd]).values.to(torch.int32)
+        w["target_head"] = _randn_bf16(s.V, s.H, std, 0.0, _gen(seed, "target_head"))
     return w
 
 

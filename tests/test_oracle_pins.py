@@ -770,3 +770,49 @@ def test_window_longer_than_the_ring_history_wraps_correctly():
         lo = max(0, t - 9)
         want = float(torch.tensor(sum(s[lo:t + 1]) / (t + 1 - lo), dtype=torch.float32))
         assert abs(xs[t] - want) < 1e-6
+
+
+# ---------------------------------------------------------------- reduced draft vocabulary (id map)
+def test_permuted_full_size_id_map_leaves_the_drafted_tokens_unchanged():
+    # head'[i] = head[pi[i]] with draft_to_token = pi scores the same tokens: chain and tree drafts agree
+    wl = harness.tiny_workload(B=2, K=3)
+    case = harness.build_case(wl, poison_tail=False)
+    sh = wl.shape
+    pi = torch.randperm(sh.V, generator=torch.Generator().manual_seed(8))
+    w2 = dict(case.weights)
+    w2["head"] = torch.cat([case.weights["head"][:sh.V][pi], case.weights["head"][sh.V:]], dim=0)
+    w2["draft_to_token"] = pi.to(torch.int32)
+    w2["target_head"] = case.weights["head"][:sh.V]
+    m1, m2 = orc.DraftModel(sh, case.weights), orc.DraftModel(sh, w2)
+    d1 = orc.draft_chain(m1, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    d2 = orc.draft_chain(m2, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    assert torch.equal(d1.cand_tok, d2.cand_tok)
+    assert (d1.hidden - d2.hidden).abs().max() == 0 and (d1.slot_signal[:, :-1] - d2.slot_signal[:, :-1]).abs().max() == 0
+    wt = harness.tiny_workload(B=2, K=3, mode=synth.TREE, topk=3, max_nodes=8)
+    ct = harness.build_case(wt, poison_tail=False, weights=case.weights)
+    t1 = orc.draft_tree(m1, harness.oracle_kv(ct), ct.f0, ct.t0, 3, 3, 8)
+    t2 = orc.draft_tree(m2, harness.oracle_kv(ct), ct.f0, ct.t0, 3, 3, 8)
+    assert torch.equal(t1.cand_tok, t2.cand_tok) and torch.equal(t1.parent, t2.parent)
+
+
+def test_reduced_draft_vocabulary_drafts_the_best_token_among_its_rows_only():
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=200, page=16, Vd=37)
+    wl = synth.Workload("rv", sh, B=3, mode=synth.CHAIN, K=2, len_lo=4, len_hi=20, seed=13)
+    case = harness.build_case(wl, poison_tail=False)
+    assert case.weights["head"].shape[0] == 37 + sh.S and case.weights["target_head"].shape[0] == 200
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    allowed = set(case.weights["draft_to_token"].tolist())
+    assert set(d.cand_tok[:, 1:].reshape(-1).tolist()) <= allowed
+    # brute force for round 1: numpy scan over the 37 rows on the oracle's own hidden
+    W = case.weights["head"][:37].to(torch.float64).numpy()
+    for b in range(wl.B):
+        logits = (W @ d.hidden[b, 0].numpy()).astype(np.float32)
+        assert int(case.weights["draft_to_token"][int(np.argmax(logits))]) == int(d.cand_tok[b, 1])
+    # the signal rows follow the 37 vocabulary rows
+    Wsig = case.weights["head"][37:].to(torch.float64).numpy()
+    z = (Wsig @ d.hidden[0, 0].numpy()).astype(np.float32)
+    assert np.allclose(z, d.z[0, 0].numpy(), atol=1e-6)
+    # verification uses the target's own full-vocabulary head
+    v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok)
+    assert int(v.target_tok.max()) < 200
