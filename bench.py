@@ -49,7 +49,7 @@ def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
     every live KV byte once per round, the verify head once."""
     s = wl.shape
     layer = 2 * s.H * s.H + s.H * s.qkv_rows + s.n_q * s.d * s.H + 3 * s.H * s.F
-    head = (s.V + s.S) * s.H
+    head = ((s.Vd or s.V) + s.S) * s.H
     rounds = wl.K
     w_round = 2 * (layer + head)
     kv_round = int(sum(int(n) for n in lens)) * s.n_kv * s.d * 2 * 2
@@ -237,6 +237,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="C1")
     ap.add_argument("--impl", default="b200")
+    ap.add_argument("--draft-vocab", type=int, default=0, metavar="VD",
+                    help="reduce the draft head to VD ids (id map + the target's own head); 0 = the workload as defined")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timeline", default=None, metavar="FILE",
                     help="also write a per-kernel timeline of one iteration (CUPTI through torch.profiler): when "
@@ -247,6 +249,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     wl = synth.workload(args.workload)
+    if args.draft_vocab:
+        import dataclasses
+        wl = dataclasses.replace(wl, name=f"{wl.name}+Vd{args.draft_vocab}",
+                                 shape=dataclasses.replace(wl.shape, Vd=args.draft_vocab))
 
     if args.impl == "reference":
         if rank == 0:

@@ -75,6 +75,9 @@ typedef struct {
   float rms_eps, rope_theta;
   int32_t page_size;                /* KV slots per page */
   int32_t act[SX_MAX_SIGNALS];      /* activation of each signal row */
+  int32_t draft_vocab;              /* rows of the draft head's vocabulary part; 0 = vocab.  A reduced
+                                       draft vocabulary (draft_vocab < vocab) scores draft ids
+                                       0..draft_vocab-1, see sx_weights.draft_to_token_d */
 } sx_model_cfg;
 
 typedef struct {
@@ -87,8 +90,13 @@ typedef struct {
   const void *wgate_up_d;     /* [2 * ffn, H]: gate rows, then up rows */
   const void *wdown_d;        /* [H, ffn] */
   const void *normf_d;        /* [H] final gain */
-  const void *head_d;         /* [vocab + n_signals, H]: Eq. 1, vocabulary rows first, signal rows last */
-  const void *target_head_d;  /* [vocab, H] target LM head; may alias head_d */
+  const void *head_d;         /* [draft_vocab + n_signals, H]: Eq. 1, vocabulary rows first, signal rows last */
+  const void *target_head_d;  /* [vocab, H] target LM head; may alias head_d when draft_vocab == vocab */
+  const int32_t *draft_to_token_d; /* [draft_vocab] token id of each draft id, distinct, each in
+                                      [0, vocab); NULL = identity (needs draft_vocab == vocab).
+                                      Every drafted token that leaves the library (draft_tok,
+                                      candidate ids) or feeds the embedding of the next round is
+                                      the mapped id; ties break toward the lower draft id. */
 } sx_weights;
 
 /* Paged KV cache of the draft layer.  Slot s of sequence b lives in physical page

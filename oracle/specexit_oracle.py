@@ -508,6 +508,92 @@ def target_argmax(model: DraftModel, target_hidden: torch.Tensor) -> Tuple[torch
     return tok.view(B, P), gap.view(B, P)
 
 
+# --------------------------------------------------------------------------------------
+# stochastic verification: speculative sampling with deterministic drafts
+# --------------------------------------------------------------------------------------
+# Speculative sampling (the acceptance rule the paper's background section cites) keeps a draft
+# token x with probability min(1, p(x) / q(x)) and otherwise draws from the normalised
+# max(0, p - q); p is the target's distribution at temperature tau, q the draft's.  The drafts
+# here are deterministic (the draft's argmax, or its top-k children in a tree), so q is a point
+# mass: x is kept with probability p(x), and a rejection draws from p with x removed.  Drawing
+# one token t ~ p and keeping x exactly when t == x has that joint law (P(t = x) = p(x); given
+# t != x, t follows p without x), and for the children c_1..c_m of a tree node tried one after
+# the other against the shrinking residual, P(c_i kept) = p(c_i) again, so "keep the child that
+# equals t, else recover t" is the same law.  The verification below is therefore the greedy
+# walk with the target's argmax replaced by a sample t ~ softmax(logits / tau).
+#
+# The sample is a Gumbel-max draw so that it depends on the random numbers element by element
+# and not on a summation order:  t = argmax_i (logit_i + tau * g_i),  g_i = -ln(-ln(u_i)),
+# with u_i a uniform on (0, 1) taken from the counter-based generator Philox4x32-10 (Salmon et
+# al., "Parallel random numbers: as easy as 1, 2, 3", 2011): the draw for sequence b, verify
+# slot j and token id i is word (i mod 4) of the block with counter (i div 4, j, b, offset) and
+# key (seed mod 2^32, seed div 2^32).  tau = 0 is greedy verification.
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter, key):
+    """Philox4x32 with 10 rounds on numpy arrays of uint64 holding 32-bit words.
+    ``counter``: four arrays (or ints), ``key``: two.  Returns the four output words."""
+    import numpy as np
+    m32 = np.uint64(0xFFFFFFFF)
+    c = [np.asarray(x, dtype=np.uint64) & m32 for x in counter]
+    c = list(np.broadcast_arrays(*c))
+    k0, k1 = np.uint64(int(key[0]) & 0xFFFFFFFF), np.uint64(int(key[1]) & 0xFFFFFFFF)
+    for rnd in range(10):
+        if rnd:
+            k0 = (k0 + np.uint64(PHILOX_W0)) & m32
+            k1 = (k1 + np.uint64(PHILOX_W1)) & m32
+        p0 = np.uint64(PHILOX_M0) * c[0]            # 32 x 32 -> 64 bit products
+        p1 = np.uint64(PHILOX_M1) * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & m32
+        hi1, lo1 = p1 >> np.uint64(32), p1 & m32
+        c = [hi1 ^ c[1] ^ k0, lo1, hi0 ^ c[3] ^ k1, lo0]
+    return c
+
+
+def uniform_open(word):
+    """A 32-bit word to a uniform strictly inside (0, 1): the top 23 bits k give (k + 1/2) / 2^23,
+    a value that float32 holds exactly."""
+    import numpy as np
+    return ((np.asarray(word, dtype=np.uint64) >> np.uint64(9)).astype(np.float64) + 0.5) / float(1 << 23)
+
+
+@dataclass
+class SampleCfg:
+    temperature: float = 0.0
+    seed: int = 0
+    offset: int = 0          # e.g. the iteration number: a fresh set of draws per iteration
+
+
+def gumbel_noise(cfg: SampleCfg, b: int, j: int, V: int) -> torch.Tensor:
+    """g_i for i in [0, V) of sequence b, verify slot j (float64)."""
+    import numpy as np
+    nblk = (V + 3) // 4
+    w = philox4x32_10((np.arange(nblk, dtype=np.uint64), j, b, cfg.offset),
+                      (cfg.seed & 0xFFFFFFFF, (cfg.seed >> 32) & 0xFFFFFFFF))
+    u = uniform_open(np.stack(w, axis=1).reshape(-1)[:V])
+    return torch.from_numpy(-np.log(-np.log(u)))
+
+
+def target_sample(model: DraftModel, target_hidden: torch.Tensor, cfg: SampleCfg
+                  ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """t[b, j] ~ softmax(logits[b, j] / tau) by Gumbel-max, and the relative top-2 gap of the
+    perturbed scores.  The temperature enters as its float32 value."""
+    B, P, H = target_hidden.shape
+    logits = f32r(linear(target_hidden.reshape(B * P, H).to(F64), model.target_head))
+    tau = float(torch.tensor(cfg.temperature, dtype=torch.float32))
+    tok = torch.zeros(B * P, dtype=torch.int64)
+    gap = torch.zeros(B * P, dtype=F64)
+    for r in range(B * P):
+        s = logits[r]
+        if tau > 0.0:
+            s = s + tau * gumbel_noise(cfg, r // P, r % P, s.numel())
+        tok[r] = argmax_low(s)
+        gap[r] = top_gap(s)
+    return tok.view(B, P), gap.view(B, P)
+
+
 def accept_chain(cand_tok: Sequence[int], target_tok: Sequence[int]) -> Tuple[int, List[int], int]:
     """Longest prefix of draft tokens that equal the target's greedy choice one slot
     earlier; the recover token is the target's choice after the last accepted slot."""
@@ -535,8 +621,13 @@ def accept_tree(cand_tok: Sequence[int], parent: Sequence[int], target_tok: Sequ
 
 def verify(model: DraftModel, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
            parent: Optional[torch.Tensor] = None,
-           forced_target: Optional[Dict[Tuple[int, int], int]] = None) -> VerifyOut:
-    tt, gap = target_argmax(model, target_hidden)
+           forced_target: Optional[Dict[Tuple[int, int], int]] = None,
+           sample: Optional[SampleCfg] = None) -> VerifyOut:
+    """Greedy verification, or (``sample`` with a positive temperature) speculative sampling."""
+    if sample is not None and sample.temperature > 0.0:
+        tt, gap = target_sample(model, target_hidden, sample)
+    else:
+        tt, gap = target_argmax(model, target_hidden)
     if forced_target:
         for (b, j), t in forced_target.items():
             tt[b, j] = t

@@ -107,6 +107,9 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (m->n_signals < 0 || m->n_signals > SX_MAX_SIGNALS || m->vocab < 1 || m->page_size < 1)
     return SX_ERR_UNSUPPORTED;
   if (m->H > 16384) return SX_ERR_UNSUPPORTED;
+  const int Vd = m->draft_vocab ? m->draft_vocab : m->vocab;
+  if (Vd < 1 || Vd > m->vocab) return SX_ERR_INVALID_ARG;
+  if (Vd < m->vocab && !w->draft_to_token_d) return SX_ERR_INVALID_ARG;   // a reduced vocabulary needs its id map
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
@@ -114,7 +117,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->prof_ev = new std::vector<cudaEvent_t>();
   c->prof_cls = new std::vector<int>();
   c->sh.H = m->H; c->sh.nq = m->n_q_heads; c->sh.nkv = m->n_kv_heads; c->sh.d = m->head_dim;
-  c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.S = m->n_signals; c->sh.page = m->page_size;
+  c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.Vd = Vd; c->sh.S = m->n_signals; c->sh.page = m->page_size;
   c->sh.eps = m->rms_eps; c->sh.theta = m->rope_theta;
   for (int i = 0; i < SX_MAX_SIGNALS; ++i) c->sh.act[i] = m->act[i];
   c->w = *w;
@@ -126,7 +129,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
     c->rows_per_seq = 1 + T * (dc->K - 1);
     c->P = 1 + dc->max_nodes;
     c->NC = T + (dc->K - 1) * T * T;
-    if (T < 1 || T > SX_MAX_TOPK || T > m->vocab || c->rows_per_seq > SX_MAX_TREE_ROWS ||
+    if (T < 1 || T > SX_MAX_TOPK || T > Vd || c->rows_per_seq > SX_MAX_TREE_ROWS ||
         c->P > SX_MAX_VERIFY_SLOTS || dc->max_nodes < 1 || dc->max_nodes > c->NC) {
       delete c;
       return SX_ERR_UNSUPPORTED;
@@ -264,7 +267,8 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
 // head over R rows in chunks the kernel can hold; merges into tok/logp/signals
 static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
-                      int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0}) {
+                      int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
+                      const int32_t *map = nullptr) {
   const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
@@ -280,7 +284,7 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     if (s2.idx) s2.idx += r0; else s2.add += r0 * s2.mul;
     sx_launch_head_finalize(c->sh, rc, parts, G, c->head_rows, T, lse, z, S, tok_out, t2,
                             logp_out ? logp_out + (size_t)r0 * T : nullptr, sig_out, s2, st,
-                            (R <= cap) ? nx : SxNextInput{nullptr, nullptr, nullptr, 0, 0});
+                            (R <= cap) ? nx : SxNextInput{nullptr, nullptr, nullptr, 0, 0}, map, V);
     c->launches += 2;
   }
   return SX_OK;
@@ -323,10 +327,11 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
   c->launches += 7;   // 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
-  SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.V + s.S, s.V, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
+  SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.Vd + s.S, s.Vd, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
               status, st,
               prepare_next ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
-                           : SxNextInput{nullptr, nullptr, nullptr, 0, 0}));
+                           : SxNextInput{nullptr, nullptr, nullptr, 0, 0},
+              c->w.draft_to_token_d));
   return SX_OK;
 }
 

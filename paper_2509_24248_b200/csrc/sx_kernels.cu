@@ -301,7 +301,8 @@ void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int sp
 __global__ void __launch_bounds__(1024)
 sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int T, int lse,
                         const float *z, int S, int act0, int act1, int act2, int32_t *tok_out,
-                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si, SxNextInput nx) {
+                        SxIndex toi, float *logp_out, float *sig_out, SxIndex si, SxNextInput nx,
+                        const int32_t *map, int Vd) {
   __shared__ unsigned long long s_best[2][32];
   __shared__ float s_red[32];
   __shared__ float s_lse;
@@ -344,8 +345,10 @@ sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int 
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
     if (tid == 0) {
-      tok_out[tbase + t] = (int32_t)sx_pack_index(best);
-      if (t == 0) s_tok = (int32_t)sx_pack_index(best);
+      int32_t id = (int32_t)sx_pack_index(best);
+      if (map) id = (id >= 0 && id < Vd) ? map[id] : 0;      // draft id -> token id (reduced draft vocabulary)
+      tok_out[tbase + t] = id;
+      if (t == 0) s_tok = id;
       if (logp_out) logp_out[(size_t)r * T + t] = lse ? sx_pack_value(best) - s_lse : sx_pack_value(best);
     }
     if (best != 0ull && v[0] == best) {          // packed values are unique (index inside): one winner
@@ -377,11 +380,12 @@ sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int 
 
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
-                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st, SxNextInput nx) {
+                             float *logp_out, float *sig_out, SxIndex si, cudaStream_t st, SxNextInput nx,
+                             const int32_t *map, int Vd) {
   int threads = ((G + 31) / 32) * 32;              // one thread per CTA of the head kernel (G <= SM count)
   if (threads < 128) threads = 128;
   sx_launch(sx_head_finalize_kernel, dim3(R), dim3(threads), 0, st, parts, G, part_stride, T, lse, z, S, sh.act[0],
-            sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx);
+            sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx, map, Vd);
 }
 
 // ---------------------------------------------------------------------------------------

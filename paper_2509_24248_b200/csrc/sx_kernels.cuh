@@ -11,6 +11,7 @@ struct SxIndex {
 
 struct SxShape {
   int H, nq, nkv, d, F, V, S, page;
+  int Vd;                      // vocabulary rows of the draft head (== V without a reduced draft vocabulary)
   float eps, theta;
   int act[SX_MAX_SIGNALS];
 };
@@ -56,7 +57,8 @@ struct SxNextInput {
 void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
                              float *logp_out, float *sig_out, SxIndex si, cudaStream_t st,
-                             SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0});
+                             SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
+                             const int32_t *map = nullptr, int Vd = 0);   // map: draft id -> token id
 
 void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st);
 

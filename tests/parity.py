@@ -55,8 +55,13 @@ class GpuChooser:
     """Decision hook for the oracle: keeps the oracle's choice when the GPU agrees, adopts the
     GPU's when it differs only within the near-tie margin, raises otherwise."""
 
-    def __init__(self, rep: Report, cand_tok=None, tree=None, T=1):
+    def __init__(self, rep: Report, cand_tok=None, tree=None, T=1, id_map=None):
         self.rep, self.cand_tok, self.tree, self.T = rep, cand_tok, tree, T
+        # the GPU reports token ids, the oracle asks in draft ids: invert the id map
+        self.inv = None if id_map is None else {int(t): i for i, t in enumerate(id_map)}
+
+    def _draft_id(self, tok: int) -> int:
+        return int(tok) if self.inv is None else self.inv.get(int(tok), -1)
 
     def _children_base(self, row: int) -> int:
         T = self.T
@@ -68,7 +73,7 @@ class GpuChooser:
     def __call__(self, kind, key, values, k, default):
         if kind == "tok":
             b, kk = key
-            g = int(self.cand_tok[b, kk])
+            g = self._draft_id(self.cand_tok[b, kk])
             if g == int(default[0]):
                 return default
             top = float(values.max())
@@ -80,7 +85,9 @@ class GpuChooser:
         if kind == "topk":
             b, row = key
             base = self._children_base(row)
-            gids = [int(t) for t in self.tree["tok"][b, base:base + k]]
+            gids = [self._draft_id(t) for t in self.tree["tok"][b, base:base + k]]
+            if min(gids) < 0:
+                raise ParityError(f"top-{k} b={b} row={row}: a gpu token is outside the draft vocabulary")
             if gids == [int(i) for i in default]:
                 return default
             top = float(values.max())
@@ -257,7 +264,7 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     # K/V rows it appended), so each round is compared on identical inputs.  Without this the two
     # runs drift apart round by round: bf16 re-rounding turns summation-order noise into ulp-level
     # differences within one round, and the feedback through the next round's feature compounds it.
-    chooser = GpuChooser(rep, cand_tok=g_tok)
+    chooser = GpuChooser(rep, cand_tok=g_tok, id_map=model.map)
     replay = _kv_replay(sx, case)
 
     def before_round(k, kv, feat):
@@ -327,7 +334,7 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
                 raise ParityError(f"tree slot b={b} s={s} does not name a generated candidate")
             ks.append(lut[key])
         kept.append(ks)
-    chooser = GpuChooser(rep, tree={"tok": o["tree_cand_tok_d"], "row": o["tree_cand_row_d"], "kept": kept}, T=T)
+    chooser = GpuChooser(rep, tree={"tok": o["tree_cand_tok_d"], "row": o["tree_cand_row_d"], "kept": kept}, T=T, id_map=model.map)
     replay = _kv_replay(sx, case)
     g_hid = o["hidden_d"]
 

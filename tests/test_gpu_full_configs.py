@@ -22,3 +22,14 @@ def test_tree_config4():
     rep = parity.run_tree(harness.build_case(wl, poison_tail=True))
     print(f"C4: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
           f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
+
+
+def test_chain_config1_with_a_32k_draft_vocabulary():
+    """C1's shapes with the draft head reduced to 32768 ids (id map + the target's own head)."""
+    import dataclasses
+    wl = synth.workload("C1")
+    wl = dataclasses.replace(wl, shape=dataclasses.replace(wl.shape, Vd=32768))
+    rep = parity.run_chain(harness.build_case(wl, poison_tail=True))
+    print(f"C1/Vd=32768: accept_len {rep.accept_len} exempt {rep.exempt} "
+          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
+    assert len(rep.exempt) <= 2

@@ -816,3 +816,124 @@ def test_reduced_draft_vocabulary_drafts_the_best_token_among_its_rows_only():
     # verification uses the target's own full-vocabulary head
     v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok)
     assert int(v.target_tok.max()) < 200
+
+
+# ---------------------------------------------------------------------------------------
+# stochastic verification (speculative sampling with deterministic drafts)
+# ---------------------------------------------------------------------------------------
+def test_philox_known_answers():
+    for row in _rows("philox4x32_10_kat.txt"):
+        w = [int(x, 16) for x in row]
+        out = orc.philox4x32_10(w[0:4], w[4:6])
+        assert [int(x) for x in out] == w[6:10]
+
+
+def test_philox_is_vectorised_over_counters_consistently():
+    ctr = np.arange(7, dtype=np.uint64)
+    blk = orc.philox4x32_10((ctr, 3, 5, 9), (11, 13))
+    for i in range(7):
+        one = orc.philox4x32_10((i, 3, 5, 9), (11, 13))
+        assert [int(x) for x in one] == [int(blk[k][i]) for k in range(4)]
+
+
+def test_uniform_is_strictly_inside_the_unit_interval_and_exact_in_float32():
+    w = np.array([0, 1, 511, 512, 0x7FFFFFFF, 0x80000000, 0xFFFFFFFF], dtype=np.uint64)
+    u = orc.uniform_open(w)
+    assert u.min() > 0.0 and u.max() < 1.0
+    assert np.array_equal(u.astype(np.float32).astype(np.float64), u)
+    assert u[0] == 2.0 ** -24 and u[-1] == 1.0 - 2.0 ** -24 and u[3] == 1.5 * 2.0 ** -23
+
+
+class _IdentityHead:
+    """Stand-in model whose target logits are the hidden state itself."""
+    def __init__(self, V):
+        self.target_head = torch.eye(V, dtype=torch.bfloat16)
+
+
+def _draws(logits, tau, n, seed=77, offset=3):
+    V = len(logits)
+    hid = torch.tensor(logits, dtype=torch.bfloat16).view(1, 1, V).repeat(1, n, 1)
+    tok, _ = orc.target_sample(_IdentityHead(V), hid, orc.SampleCfg(tau, seed, offset))
+    return tok.view(-1).numpy()
+
+
+def test_sampled_target_token_follows_the_softmax_at_that_temperature():
+    logits = [1.0, -0.5, 2.0, 0.25, 1.5, -2.0]            # exact in bf16
+    for tau in (0.5, 1.0, 2.0):
+        n = 20000
+        t = _draws(logits, tau, n)
+        p = np.exp(np.array(logits) / tau)
+        p /= p.sum()
+        f = np.bincount(t, minlength=len(logits)) / n
+        sd = np.sqrt(p * (1 - p) / n)
+        assert np.all(np.abs(f - p) < 5 * sd), (tau, f, p)
+
+
+def test_acceptance_law_of_speculative_sampling_with_a_point_mass_draft():
+    # accept x with probability min(1, p(x) / q(x)); otherwise draw from norm(max(0, p - q))
+    logits = [0.5, 1.75, -1.0, 1.0, 0.0]
+    x, n = 1, 30000
+    p = np.exp(np.array(logits))
+    p /= p.sum()
+    q = np.zeros_like(p)
+    q[x] = 1.0
+    accept_prob = min(1.0, p[x] / q[x])
+    resid = np.maximum(0.0, p - q)
+    resid /= resid.sum()
+    t = _draws(logits, 1.0, n, seed=5, offset=0)
+    cand = [9, x]                                             # slot 0: last accepted token; slot 1: the draft
+    acc, rec = [], []
+    for i in range(n):
+        L, path, r = orc.accept_chain(cand, [int(t[i]), 0])
+        acc.append(L)
+        if L == 0:
+            rec.append(r)
+    fa = np.mean(acc)
+    assert abs(fa - accept_prob) < 5 * math.sqrt(accept_prob * (1 - accept_prob) / n)
+    fr = np.bincount(np.array(rec), minlength=len(p)) / len(rec)
+    assert fr[x] == 0.0
+    assert np.all(np.abs(fr - resid) < 5 * np.sqrt(resid * (1 - resid) / len(rec)) + 1e-12)
+
+
+def test_tree_children_tried_in_turn_against_the_residual_keep_child_i_with_probability_p_i():
+    # closed form of the sequential rule: child i is reached when all earlier ones were refused,
+    # and is then kept with probability p(c_i) / (1 - p(c_1) - ... - p(c_{i-1}))
+    logits = [0.5, 1.75, -1.0, 1.0, 0.0, 0.75]
+    p = np.exp(np.array(logits))
+    p /= p.sum()
+    children = [3, 1, 4]
+    reach, gone = 1.0, 0.0
+    for c in children:
+        keep = p[c] / (1.0 - gone)
+        assert abs(reach * keep - p[c]) < 1e-15
+        reach *= 1.0 - keep
+        gone += p[c]
+    # ... and the coupled draw reproduces it: one level of a tree, children in slots 1..3
+    n = 30000
+    t = _draws(logits, 1.0, n, seed=6, offset=1)
+    cand, parent = [9] + children, [-1, 0, 0, 0]
+    kept = np.zeros(len(children) + 1)
+    for i in range(n):
+        L, path, r = orc.accept_tree(cand, parent, [int(t[i]), 0, 0, 0])
+        kept[path[1] if L else 0] += 1
+    f = kept / n
+    want = np.array([1.0 - p[children].sum()] + [p[c] for c in children])
+    assert np.all(np.abs(f - want) < 5 * np.sqrt(want * (1 - want) / n))
+
+
+def test_zero_temperature_is_greedy_verification_and_draws_differ_by_slot_sequence_and_offset():
+    wl = harness.tiny_workload(B=2, K=3, len_lo=6, len_hi=20)
+    case = harness.build_case(wl, poison_tail=False)
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    th = harness.chain_target_hidden(case, d)
+    v0 = orc.verify(model, th, d.cand_tok)
+    v1 = orc.verify(model, th, d.cand_tok, sample=orc.SampleCfg(0.0, 1, 2))
+    assert torch.equal(v0.target_tok, v1.target_tok) and torch.equal(v0.accept_len, v1.accept_len)
+    g = [orc.gumbel_noise(orc.SampleCfg(1.0, s, o), b, j, 50) for (s, o, b, j) in
+         [(1, 0, 0, 0), (1, 0, 0, 1), (1, 0, 1, 0), (1, 1, 0, 0), (2, 0, 0, 0), (1 + (1 << 32), 0, 0, 0)]]
+    for a, b in itertools.combinations(range(len(g)), 2):
+        assert not torch.equal(g[a], g[b])
+    # a very high temperature makes the draw nearly uniform: it leaves the greedy choice often
+    hot = orc.verify(model, th, d.cand_tok, sample=orc.SampleCfg(50.0, 1, 0))
+    assert not torch.equal(hot.target_tok, v0.target_tok)
