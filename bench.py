@@ -200,11 +200,11 @@ def run_reference(args, wl):
         if wl.mode == synth.CHAIN:
             d = orc.draft_chain(model, kv, case.f0, case.t0, wl.K)
             th = harness.chain_target_hidden(case, d)
-            v = orc.verify(model, th, d.cand_tok)
+            v = orc.verify(model, th, d.cand_tok, sample=orc.SampleCfg(args.temperature, 1234, 1))
         else:
             d = orc.draft_tree(model, kv, case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
             th = harness.tree_target_hidden(case, d)
-            v = orc.verify(model, th, d.cand_tok, d.parent)
+            v = orc.verify(model, th, d.cand_tok, d.parent, sample=orc.SampleCfg(args.temperature, 1234, 1))
         e = orc.exit_update(cfg, orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path, v.accept_len,
                             v.recover_tok)
         return int((e.accept_len + 1).sum())
@@ -237,6 +237,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="C1")
     ap.add_argument("--impl", default="b200")
+    ap.add_argument("--temperature", type=float, default=0.0,
+                    help="verify with stochastic acceptance at this temperature (0 = greedy, the headline setting)")
     ap.add_argument("--draft-vocab", type=int, default=0, metavar="VD",
                     help="reduce the draft head to VD ids (id map + the target's own head); 0 = the workload as defined")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -253,6 +255,9 @@ def main():
         import dataclasses
         wl = dataclasses.replace(wl, name=f"{wl.name}+Vd{args.draft_vocab}",
                                  shape=dataclasses.replace(wl.shape, Vd=args.draft_vocab))
+    if args.temperature > 0.0:
+        import dataclasses
+        wl = dataclasses.replace(wl, name=f"{wl.name}+tau{args.temperature:g}")
 
     if args.impl == "reference":
         if rank == 0:
@@ -305,8 +310,13 @@ def main():
     def reset_state():
         state["_all"].copy_(state0)          # one copy: all state arrays are views of this buffer
 
+    draws = [0]
+
     def step():
         reset_state()
+        if args.temperature > 0.0:
+            draws[0] += 1
+            sx.sx_set_sampling(args.temperature, 1234, draws[0])     # fresh draws every iteration
         sx.sx_spec_exit_iter(params, state, f0_d, t0_d, th_d, out)
 
     sampler = ClockSampler(local)
@@ -423,10 +433,12 @@ def main():
         t2 = time.perf_counter()
         if wl.mode == synth.CHAIN:
             d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
-            v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok)
+            v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok,
+                           sample=orc.SampleCfg(args.temperature, 1234, 1))
         else:
             d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
-            v = orc.verify(model, harness.tree_target_hidden(case, d), d.cand_tok, d.parent)
+            v = orc.verify(model, harness.tree_target_hidden(case, d), d.cand_tok, d.parent,
+                           sample=orc.SampleCfg(args.temperature, 1234, 1))
         orc.exit_update(harness.default_exit_cfg(wl), orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path,
                         v.accept_len, v.recover_tok)
         dt = time.perf_counter() - t2

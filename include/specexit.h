@@ -217,6 +217,22 @@ sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hi
                     int32_t *recover_tok_d, void *ws_d, size_t ws_bytes, int32_t *status_d,
                     void *stream);
 
+/* Stochastic acceptance: speculative sampling, the acceptance rule of the speculative-decoding
+ * scheme the method builds on (Section 2, background on speculative decoding; Algorithm 1,
+ * "accept tokens").  A draft token x is kept with probability min(1, p(x) / q(x)), else a token is
+ * drawn from the normalised max(0, p - q); p is the target's softmax at `temperature`.  The drafts
+ * of this library are deterministic (q is a point mass), so the rule is realised exactly by
+ * drawing one token t ~ p per verify slot and keeping a draft token where it equals t: the
+ * sx_verify and sx_spec_exit_iter calls that follow return that draw in target_tok_d and walk it
+ * as they walk the greedy choice (chain and tree alike; the recover token is the draw at the
+ * last accepted slot).  The draw is t = argmax_i (logit_i + temperature * g_i) with g_i =
+ * -ln(-ln(u_i)), u_i = (k + 1/2) / 2^23 for k the top 23 bits of word (i mod 4) of the
+ * Philox4x32-10 block with counter (i div 4, slot, sequence, offset) and key (seed mod 2^32,
+ * seed div 2^32).  Give every iteration its own offset.  temperature = 0 (the state of a new
+ * context) is greedy verification.  Host-side state, read when a call is issued; returns
+ * SX_ERR_INVALID_ARG for a negative or non-finite temperature. */
+sx_status sx_set_sampling(sx_ctx *ctx, float temperature, uint64_t seed, uint32_t offset);
+
 /* Exit decision (Section 3.3; Appendix A.1).  Walks path slots 0..accept_len; each slot that
  * carries a signal updates the EWMA (all of them, or only the first, per ema_positions); the
  * first slot whose token is a step-split token while the smoothed signals pass ends the

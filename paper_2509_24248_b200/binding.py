@@ -28,7 +28,8 @@ HIST = 16
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
-           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit"]
+           "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit",
+           "sx_set_sampling"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -104,6 +105,8 @@ def load_library() -> C.CDLL:
     lib.sx_workspace_bytes.argtypes = [vp]
     lib.sx_strerror.restype = C.c_char_p
     lib.sx_strerror.argtypes = [i32]
+    lib.sx_set_sampling.restype = i32
+    lib.sx_set_sampling.argtypes = [vp, C.c_float, C.c_uint64, C.c_uint32]
     lib.sx_launch_count.restype = C.c_int64
     lib.sx_launch_count.argtypes = [vp]
     lib.sx_draft_step.restype = i32
@@ -327,6 +330,10 @@ class SpecExit:
                                       logp.data_ptr(), sig.data_ptr(), self.ws_ptr, self.ws_bytes,
                                       self.status.data_ptr(), self._stream()), "sx_draft_step")
         return hid, tok_out, logp, sig
+
+    def sx_set_sampling(self, temperature: float, seed: int = 0, offset: int = 0) -> None:
+        """Stochastic acceptance for the verify calls that follow (0 = greedy)."""
+        _check(self.lib.sx_set_sampling(self.h, float(temperature), int(seed), int(offset)), "sx_set_sampling")
 
     def sx_verify(self, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
                   parent: Optional[torch.Tensor] = None, path_stride: Optional[int] = None):

@@ -19,6 +19,7 @@ struct sx_ctx {
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
       off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, total;
   int commit_rows, commit_N;
+  SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
   // tree sub-offsets relative to off_tree
   size_t t_tok, t_par, t_src, t_row, t_score, t_rmask, t_selcid, t_seltok, t_fidx, t_hidx, t_nmask, t_rsig;
   // optional per-class event timing
@@ -268,7 +269,7 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
 static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
                       int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
-                      const int32_t *map = nullptr) {
+                      const int32_t *map = nullptr, const SxSample *smp = nullptr) {
   const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
@@ -276,8 +277,10 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     const int rc = (R - r0 < cap) ? R - r0 : cap;
     int G = 0;
     prof_mark(c, cls, true, st);
+    SxSample sm2;
+    if (smp) { sm2 = *smp; sm2.row0 = r0; }
     SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
-                          c->head_rows, &G, z, S, c->sm_count, status, st));
+                          c->head_rows, &G, z, S, c->sm_count, status, st, smp ? &sm2 : nullptr));
     prof_mark(c, cls, false, st);
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
@@ -356,6 +359,15 @@ extern "C" sx_status sx_draft_step(sx_ctx *c, const sx_kv *kv, int32_t round, in
                      (char *)ws_d, status_d, (cudaStream_t)stream);
 }
 
+extern "C" sx_status sx_set_sampling(sx_ctx *c, float temperature, uint64_t seed, uint32_t offset) {
+  if (!c || !(temperature >= 0.f) || !(temperature < INFINITY)) return SX_ERR_INVALID_ARG;
+  c->smp.temp = temperature;
+  c->smp.k0 = (uint32_t)(seed & 0xffffffffull);
+  c->smp.k1 = (uint32_t)(seed >> 32);
+  c->smp.offset = offset;
+  return SX_OK;
+}
+
 extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *target_hidden_d,
                                const int32_t *cand_tok_d, const int32_t *parent_d, int32_t *target_tok_d,
                                int32_t *accept_len_d, int32_t *path_d, int32_t path_stride, int32_t *recover_tok_d,
@@ -366,8 +378,11 @@ extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *
   if (parent_d && P > SX_MAX_VERIFY_SLOTS) return SX_ERR_UNSUPPORTED;
   SX_TRY(check_ws(c, ws_d, ws_bytes));
   cudaStream_t st = (cudaStream_t)stream;
+  SxSample smp = c->smp;
+  smp.P = P;
   SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, c->sh.V, c->sh.V, 0, (const bf16 *)target_hidden_d, batch * P, 1, 0, (char *)ws_d,
-              target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st));
+              target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
+              SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, smp.temp > 0.f ? &smp : nullptr));
   sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st);
   c->launches += 1;
   return SX_OK;

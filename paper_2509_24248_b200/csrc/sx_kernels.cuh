@@ -96,8 +96,17 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
                                  int splits, size_t split_stride, int sm_count, int32_t *status,
                                  cudaStream_t st);
 void sx_gemm_init(int device);
+// Sampled verification: with temp > 0 the plain-argmax head returns, per row, the arg max of
+// logit + temp * Gumbel noise, i.e. a draw from softmax(logits / temp).  Row r of the launch is
+// verify slot (row0 + r) % P of sequence (row0 + r) / P; the noise of (sequence, slot, token id)
+// comes from Philox4x32-10 with key (k0, k1) and `offset` as the last counter word.
+struct SxSample {
+  float temp;
+  uint32_t k0, k1, offset;
+  int P, row0;
+};
 // head: per-CTA partial results out[cta][row]; returns the number of CTAs used in *G
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
-                         int32_t *status, cudaStream_t st);
+                         int32_t *status, cudaStream_t st, const SxSample *smp = nullptr);
 int sx_head_max_rows(int T, int lse);

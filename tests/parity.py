@@ -161,11 +161,19 @@ def to_params(sx: binding.SpecExit, cfg: orc.ExitCfg) -> binding.ExitParams:
                               window=cfg.window)
 
 
+def _set_sampling(sx: binding.SpecExit, sample) -> None:
+    if sample is None:
+        sx.sx_set_sampling(0.0)
+    else:
+        sx.sx_set_sampling(sample.temperature, sample.seed, sample.offset)
+
+
 def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, parent, slot_signal,
-                  out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int):
+                  out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int, sample=None):
     """verify + exit comparison, shared by chain and tree."""
     B, P = cand_tok.shape
-    tt, gap = orc.target_argmax(model, th)
+    sampling = sample is not None and sample.temperature > 0.0
+    tt, gap = orc.target_sample(model, th, sample) if sampling else orc.target_argmax(model, th)
     g_tt = out["target_tok_d"].cpu().to(torch.int64)
     forced = {}
     for b in range(B):
@@ -177,7 +185,7 @@ def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, 
                 else:
                     raise ParityError(f"target token b={b} slot={j}: gpu {int(g_tt[b, j])} vs {int(tt[b, j])} "
                                       f"gap {float(gap[b, j]):.3e}")
-    v = orc.verify(model, th, cand_tok, parent, forced_target=forced)
+    v = orc.verify(model, th, cand_tok, parent, forced_target=forced, sample=sample)
     g_L = out["accept_len_d"].cpu().to(torch.int64)
     g_path = out["path_d"].cpu().to(torch.int64)
     g_rec = out["recover_tok_d"].cpu().to(torch.int64)
@@ -239,7 +247,7 @@ def _compare_signals(rep: Report, g: torch.Tensor, o: torch.Tensor):
 
 
 def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0: orc.ExitState = None,
-              sx: binding.SpecExit = None) -> Report:
+              sx: binding.SpecExit = None, sample=None) -> Report:
     wl = case.wl
     rep = Report()
     cfg = cfg or harness.default_exit_cfg(wl)
@@ -254,8 +262,10 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     gst["x"].copy_(state0.x.to(torch.float32))
     gst["n_updates"].copy_(state0.n_updates.to(torch.int32))
     gst["thinking"].copy_(state0.thinking.to(torch.int32))
+    _set_sampling(sx, sample)
     sx.sx_spec_exit_iter(to_params(sx, cfg), gst, case.f0.to(sx.dev), case.t0.to(sx.dev), th.to(sx.dev), out)
     torch.cuda.synchronize()
+    _set_sampling(sx, None)
     sx.check_status("sx_spec_exit_iter")
     g_tok = out["cand_tok_d"].cpu().to(torch.int64)
     g_hid = out["hidden_d"].cpu()
@@ -292,13 +302,14 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     if not torch.equal(out["parent_d"].cpu().to(torch.int64), want_par):
         raise ParityError("chain parents")
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, None, d.slot_signal, out,
-                  {k: v.cpu() for k, v in gst.items()}, wl.K)
+                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample)
     if own:
         sx.close()
     return rep
 
 
-def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: binding.SpecExit = None) -> Report:
+def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: binding.SpecExit = None,
+             sample=None) -> Report:
     wl = case.wl
     rep = Report()
     cfg = cfg or harness.default_exit_cfg(wl)
@@ -311,8 +322,10 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
     out = sx.new_outputs(wl.B)
     gst = sx.new_state(wl.B)
     state0 = orc.ExitState.fresh(wl.B, wl.shape.S)
+    _set_sampling(sx, sample)
     sx.sx_spec_exit_iter(to_params(sx, cfg), gst, case.f0.to(sx.dev), case.t0.to(sx.dev), th.to(sx.dev), out)
     torch.cuda.synchronize()
+    _set_sampling(sx, None)
     sx.check_status("sx_spec_exit_iter")
     o = {k: v.cpu() for k, v in out.items()}
     # the GPU's kept set as candidate ids: a candidate is identified by (source row, token)
@@ -366,7 +379,7 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
         _compare_rows(rep, f"b={b}", o["hidden_d"][b], d.hidden[b])
     _compare_signals(rep, o["slot_signal_d"], d.slot_signal)
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, d.parent, d.slot_signal, out,
-                  {k: v.cpu() for k, v in gst.items()}, wl.K)
+                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample)
     if own:
         sx.close()
     return rep
