@@ -41,6 +41,16 @@ EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
 
 EXEMPT_REL_GAP = 1e-3
 
+# Draft layer shapes.  ARCH_CONCAT (the layer the rest of this file describes): the previous
+# hidden state and the token embedding are concatenated and mixed by fc (2H -> H) in every round.
+# ARCH_FUSED3 (the EAGLE-3-shaped layer; the paper trains its draft with that recipe but does not
+# describe the layer, so this follows that publication): round 1 receives three target features
+# (low / middle / high layer, 3H) fused by fc (3H -> H); the attention input is the
+# concatenation [RMSNorm_e(embedding) ; RMSNorm_1(x)] (2H) while the residual stream starts
+# from x itself; later rounds take the layer's own output y (before the final norm) as x,
+# without fc.  The head still reads RMSNorm_f(y).
+ARCH_CONCAT, ARCH_FUSED3 = 0, 1
+
 
 def bf16r(x: torch.Tensor) -> torch.Tensor:
     """Round to bf16 the way a kernel holding an fp32 value would; result kept as f64."""
@@ -193,6 +203,7 @@ class DraftModel:
         self.sh = shape
         self.w = weights
         self.act = tuple(act)
+        self.arch = int(getattr(shape, "arch", ARCH_CONCAT))
         # The draft head may cover a reduced vocabulary: its first Vd rows score the draft ids
         # 0..Vd-1, `draft_to_token` maps a draft id to the token id it stands for (identity when
         # absent); the signal rows of Eq. 1 follow the Vd vocabulary rows.
@@ -244,6 +255,14 @@ class DraftModel:
         n1.  Returns ``x [R, H]`` (bf16 values) and ``qkv [R, (n_q + 2 n_kv) d]`` (unrounded)."""
         sh, w = self.sh, self.w
         toks = torch.tensor([r.tok for r in rows], dtype=torch.int64)
+        if self.arch == ARCH_FUSED3:
+            # a row that carries the three target features (3H) goes through fc; a row that
+            # carries a draft hidden state (H) is x as it stands
+            x = torch.stack([bf16r(linear(r.feat.view(1, -1), w["fc"]))[0] if r.feat.numel() == 3 * sh.H
+                             else bf16r(r.feat) for r in rows])
+            e = w["embed"][toks].to(F64)
+            u = torch.cat([bf16r(rmsnorm(e, w["norm_e"], sh.eps)), bf16r(rmsnorm(x, w["norm1"], sh.eps))], dim=1)
+            return x, linear(u, w["wqkv"])
         u = torch.cat([torch.stack([r.feat for r in rows]), w["embed"][toks].to(F64)], dim=1)
         x = bf16r(linear(u, w["fc"]))
         n1 = bf16r(rmsnorm(x, w["norm1"], sh.eps))
@@ -284,6 +303,10 @@ class DraftModel:
         gu = linear(n2, w["wgate_up"])
         m = bf16r(silu(gu[:, :sh.F]) * gu[:, sh.F:])
         y = bf16r(a + linear(m, w["wdown"]))
+        if self.arch == ARCH_FUSED3:
+            # the hidden handed on (and compared) is y; the head reads its final norm
+            yh = y if head_input is None else head_input(rows, y)
+            return y, self.head(bf16r(rmsnorm(yh, w["normf"], sh.eps)))
         g = bf16r(rmsnorm(y, w["normf"], sh.eps))
         return g, self.head(g if head_input is None else head_input(rows, g))
 
@@ -668,7 +691,7 @@ def commit(model: DraftModel, kv: PagedKV, target_hidden: torch.Tensor, cand_tok
     iteration starts from (target hidden of path slot L, recover token).  ``accept_len_out`` and
     ``recover_tok_out`` are the values after the exit rule (a cut path commits fewer tokens)."""
     B = cand_tok.shape[0]
-    feat0 = torch.empty(B, model.sh.H, dtype=F64)
+    feat0 = torch.empty(B, target_hidden.shape[-1], dtype=F64)
     tok0 = torch.empty(B, dtype=torch.int64)
     rows: List[Row] = []
     new_len = []

@@ -30,7 +30,8 @@ TREE = 1
 # item ids for the per-item generators
 _IT = {"embed": 1, "fc": 2, "norm1": 3, "norm2": 4, "normf": 5, "wqkv": 6, "wo": 7,
        "wgate_up": 8, "wdown": 9, "head": 10, "k": 11, "v": 12, "f0": 13, "t0": 14,
-       "noise": 15, "sigma": 16, "lens": 17, "perm": 18, "noise2": 19, "d2t": 20, "target_head": 21}
+       "noise": 15, "sigma": 16, "lens": 17, "perm": 18, "noise2": 19, "d2t": 20, "target_head": 21,
+       "norm_e": 22}
 
 
 @dataclass(frozen=True)
@@ -46,6 +47,8 @@ class ModelShape:
     theta: float = 1e6
     page: int = 64
     Vd: int = 0          # rows of a reduced draft vocabulary (0: the draft head covers all V ids)
+    arch: int = 0        # 0: fc over [hidden ; embedding] every round; 1: three-feature fusion in
+    #                      round 1 and [norm(embedding) ; norm(hidden)] as the attention input
 
     @property
     def qkv_rows(self) -> int:
@@ -132,16 +135,18 @@ def make_weights(shape: ModelShape, seed: int, std: float = 0.02) -> Dict[str, t
     s = shape
     w = {
         "embed": _randn_bf16(s.V, s.H, std, 0.0, _gen(seed, "embed")),
-        "fc": _randn_bf16(s.H, 2 * s.H, std, 0.0, _gen(seed, "fc")),
+        "fc": _randn_bf16(s.H, (3 if s.arch else 2) * s.H, std, 0.0, _gen(seed, "fc")),
         "norm1": _randn_bf16(1, s.H, std, 1.0, _gen(seed, "norm1")).reshape(s.H),
         "norm2": _randn_bf16(1, s.H, std, 1.0, _gen(seed, "norm2")).reshape(s.H),
         "normf": _randn_bf16(1, s.H, std, 1.0, _gen(seed, "normf")).reshape(s.H),
-        "wqkv": _randn_bf16(s.qkv_rows, s.H, std, 0.0, _gen(seed, "wqkv")),
+        "wqkv": _randn_bf16(s.qkv_rows, (2 if s.arch else 1) * s.H, std, 0.0, _gen(seed, "wqkv")),
         "wo": _randn_bf16(s.H, s.n_q * s.d, std, 0.0, _gen(seed, "wo")),
         "wgate_up": _randn_bf16(2 * s.F, s.H, std, 0.0, _gen(seed, "wgate_up")),
         "wdown": _randn_bf16(s.H, s.F, std, 0.0, _gen(seed, "wdown")),
         "head": _randn_bf16((s.Vd or s.V) + s.S, s.H, std, 0.0, _gen(seed, "head")),
     }
+    if s.arch:
+        w["norm_e"] = _randn_bf16(1, s.H, std, 1.0, _gen(seed, "norm_e")).reshape(s.H)
     if s.Vd:
         # reduced draft vocabulary: Vd distinct token ids in increasing order, and a target head of its own
         w["draft_to_token"] = torch.sort(torch.randperm(s.V, generator=_gen(seed, "d2t"))[:s.Vd]).values.to(torch.int32)
@@ -201,7 +206,7 @@ def make_kv(shape: ModelShape, lens: torch.Tensor, extra_slots: int, seed: int,
 
 def make_f0_t0(w: Workload) -> Tuple[torch.Tensor, torch.Tensor]:
     """Target feature of the last accepted token (N(0,1), bf16) and that token's id."""
-    f0 = _randn_bf16(w.B, w.shape.H, 1.0, 0.0, _gen(w.seed, "f0"))
+    f0 = _randn_bf16(w.B, (3 if w.shape.arch else 1) * w.shape.H, 1.0, 0.0, _gen(w.seed, "f0"))
     t0 = torch.randint(0, w.shape.V, (w.B,), generator=_gen(w.seed, "t0"), dtype=torch.int32)
     return f0, t0
 

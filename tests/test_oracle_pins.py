@@ -1,6 +1,7 @@
 """Pins for the CPU oracle: hand-worked values, closed forms, textbook special cases,
 invariants and brute force.  None of these re-types the oracle's own formula: each expected
 value is derived independently (by hand, by a closed form, by enumeration, or by numpy)."""
+import dataclasses
 import itertools
 import math
 import os
@@ -546,9 +547,11 @@ def test_tree_top1_degenerates_to_chain():
 
 
 # ---------------------------------------------------------------- whole forward vs an independent restatement
-def _np_forward(case, f, tok, b, n_extra_k, n_extra_v):
+def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False):
     """float64 numpy restatement of one draft position without any intermediate rounding,
-    written against the logical (un-paged) cache."""
+    written against the logical (un-paged) cache.  ``fused3``: the layer with three-feature
+    fusion (f of length 3H goes through fc, f of length H is the residual stream itself) and
+    [norm(embedding) ; norm(x)] as the attention input; then y is returned as well."""
     sh, w = case.wl.shape, {k: v.to(torch.float64).numpy() for k, v in case.weights.items()}
     page = sh.page
     n = int(case.kv["cache_len"][b])
@@ -561,11 +564,15 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v):
     K = np.concatenate([K] + n_extra_k, axis=0) if n_extra_k else K
     Vv = np.concatenate([Vv] + n_extra_v, axis=0) if n_extra_v else Vv
     pos = K.shape[0]
-    u = np.concatenate([f, w["embed"][tok]])
-    x = w["fc"] @ u
-
     def norm(v, g):
         return v / np.sqrt((v ** 2).mean() + sh.eps) * g
+
+    if fused3:
+        x = w["fc"] @ f if f.size == 3 * sh.H else f
+        att_in = np.concatenate([norm(w["embed"][tok], w["norm_e"]), norm(x, w["norm1"])])
+    else:
+        x = w["fc"] @ np.concatenate([f, w["embed"][tok]])
+        att_in = norm(x, w["norm1"])
 
     def rot(v):
         out = v.copy()
@@ -576,7 +583,7 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v):
             out[:, i + h] = v[:, i + h] * math.cos(ang) + v[:, i] * math.sin(ang)
         return out
 
-    qkv = w["wqkv"] @ norm(x, w["norm1"])
+    qkv = w["wqkv"] @ att_in
     q = rot(qkv[:sh.n_q * sh.d].reshape(sh.n_q, sh.d))
     k = rot(qkv[sh.n_q * sh.d:(sh.n_q + sh.n_kv) * sh.d].reshape(sh.n_kv, sh.d))
     v = qkv[(sh.n_q + sh.n_kv) * sh.d:].reshape(sh.n_kv, sh.d)
@@ -593,6 +600,8 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v):
     gate, up = gu[:sh.F], gu[sh.F:]
     y = a + w["wdown"] @ (gate / (1 + np.exp(-gate)) * up)
     g = norm(y, w["normf"])
+    if fused3:
+        return g, w["head"] @ g, k[None], v[None], y
     return g, w["head"] @ g, k[None], v[None]
 
 
@@ -937,3 +946,82 @@ def test_zero_temperature_is_greedy_verification_and_draws_differ_by_slot_sequen
     # a very high temperature makes the draw nearly uniform: it leaves the greedy choice often
     hot = orc.verify(model, th, d.cand_tok, sample=orc.SampleCfg(50.0, 1, 0))
     assert not torch.equal(hot.target_tok, v0.target_tok)
+
+
+# ---------------------------------------------------------------------------------------
+# the draft layer with three-feature fusion and a concatenated attention input
+# ---------------------------------------------------------------------------------------
+_SH_F3 = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=200, page=16, arch=1)
+
+
+def test_fused3_round_one_reduces_to_the_concat_layer_when_the_extra_inputs_are_switched_off():
+    # concat layer whose fc ignores the embedding  ==  fused layer fed [f ; 0 ; 0] whose q/k/v
+    # projection ignores the (normalised) embedding half: same x, same residual, same y
+    wl0 = harness.tiny_workload(B=2, K=1, len_lo=7, len_hi=21)
+    c0 = harness.build_case(wl0, poison_tail=False)
+    sh0, H = wl0.shape, wl0.shape.H
+    w0 = dict(c0.weights)
+    fc0 = w0["fc"].clone()
+    fc0[:, H:] = 0
+    w0["fc"] = fc0
+    wl1 = dataclasses.replace(wl0, shape=dataclasses.replace(sh0, arch=1))
+    w1 = synth.make_weights(wl1.shape, wl1.seed)
+    for k in ("embed", "norm1", "norm2", "normf", "wo", "wgate_up", "wdown", "head"):
+        w1[k] = w0[k]
+    fc1 = w1["fc"].clone()
+    fc1[:, :H] = fc0[:, :H]
+    w1["fc"] = fc1
+    wq = torch.zeros_like(w1["wqkv"])
+    wq[:, H:] = w0["wqkv"]
+    w1["wqkv"] = wq
+    f3 = torch.cat([c0.f0, torch.zeros(wl0.B, 2 * H, dtype=c0.f0.dtype)], dim=1)
+    m0, m1 = orc.DraftModel(sh0, w0), orc.DraftModel(wl1.shape, w1)
+    kv0, kv1 = harness.oracle_kv(c0), harness.oracle_kv(c0)
+    d0 = orc.draft_chain(m0, kv0, c0.f0, c0.t0, 1)
+    d1 = orc.draft_chain(m1, kv1, f3, c0.t0, 1)
+    assert torch.equal(d0.cand_tok, d1.cand_tok)
+    assert torch.equal(d0.slot_signal[:, 0], d1.slot_signal[:, 0])
+    g_from_y = orc.bf16r(orc.rmsnorm(d1.hidden[:, 0], w1["normf"], sh0.eps))
+    assert torch.equal(g_from_y, d0.hidden[:, 0])
+    for b in range(wl0.B):
+        ka, va = kv0.read(b, kv0.len[b])
+        kb, vb = kv1.read(b, kv1.len[b])
+        assert torch.equal(ka, kb) and torch.equal(va, vb)
+    # ... and switching the other half off instead changes the result: the halves are not symmetric
+    wq2 = torch.zeros_like(wq)
+    wq2[:, :H] = w0["wqkv"]
+    w2 = dict(w1)
+    w2["wqkv"] = wq2
+    d2 = orc.draft_chain(orc.DraftModel(wl1.shape, w2), harness.oracle_kv(c0), f3, c0.t0, 1)
+    assert not torch.equal(d2.hidden, d1.hidden)
+
+
+def test_fused3_two_rounds_against_float64_restatement():
+    wl = synth.Workload("f3", _SH_F3, B=2, mode=synth.CHAIN, K=2, len_lo=9, len_hi=30, seed=51)
+    case = harness.build_case(wl, poison_tail=False)
+    assert case.f0.shape == (2, 3 * 64) and case.weights["fc"].shape == (64, 192)
+    assert case.weights["wqkv"].shape == (_SH_F3.qkv_rows, 128)
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 2)
+    for b in range(wl.B):
+        f = case.f0[b].to(torch.float64).numpy()
+        g1, logits1, k1, v1, y1 = _np_forward(case, f, int(case.t0[b]), b, [], [], fused3=True)
+        assert np.linalg.norm(d.hidden[b, 0].numpy() - y1) / np.linalg.norm(y1) < 1e-2
+        s1 = 1 / (1 + np.exp(-logits1[wl.shape.V:]))
+        assert np.abs(s1 - d.slot_signal[b, 0].numpy()).max() < 5e-3
+        assert int(np.argmax(logits1[:wl.shape.V])) == int(d.cand_tok[b, 1]) or float(d.gap[b, 0]) < 5e-2
+        # round 2 continues from y (not from its final norm, and without fc)
+        g2, logits2, _, _, y2 = _np_forward(case, y1, int(d.cand_tok[b, 1]), b, [k1], [v1], fused3=True)
+        assert np.linalg.norm(d.hidden[b, 1].numpy() - y2) / np.linalg.norm(y2) < 2e-2
+        wrong = _np_forward(case, g1, int(d.cand_tok[b, 1]), b, [k1], [v1], fused3=True)[4]
+        assert np.linalg.norm(d.hidden[b, 1].numpy() - wrong) / np.linalg.norm(wrong) > 5e-2
+
+
+def test_fused3_tree_with_one_child_per_node_is_the_chain():
+    wl = synth.Workload("f3t", _SH_F3, B=2, mode=synth.TREE, K=3, topk=1, max_nodes=3, len_lo=9, len_hi=30, seed=52)
+    case = harness.build_case(wl, poison_tail=False)
+    model = harness.oracle_model(case)
+    t = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, 3, 1, 3)
+    c = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 3)
+    assert torch.equal(t.cand_tok, c.cand_tok)
+    assert torch.equal(t.hidden, c.hidden)
