@@ -78,7 +78,20 @@ typedef struct {
   int32_t draft_vocab;              /* rows of the draft head's vocabulary part; 0 = vocab.  A reduced
                                        draft vocabulary (draft_vocab < vocab) scores draft ids
                                        0..draft_vocab-1, see sx_weights.draft_to_token_d */
+  int32_t arch;                     /* SX_ARCH_CONCAT (0) or SX_ARCH_FUSED3, see below */
 } sx_model_cfg;
+
+/* Shape of the draft layer.
+ * SX_ARCH_CONCAT: every round mixes [previous hidden ; token embedding] (2H) through fc (2H -> H);
+ *   the hidden handed from round to round (and returned) is the final-normed output.
+ * SX_ARCH_FUSED3 (the EAGLE-3-shaped layer, the recipe the paper trains its draft with): round 1
+ *   takes three target features per row (low / middle / high layer, [R, 3H]) fused by fc
+ *   (3H -> H) into x; the attention input is [RMSNorm_e(embedding) ; RMSNorm_1(x)] (2H, so wqkv is
+ *   [.., 2H]) and the residual stream starts from x; later rounds take the layer's own output y
+ *   (before the final norm) as x, without fc.  The head reads RMSNorm_f(y).  Every hidden state
+ *   this library returns or takes between rounds (hidden_out_d, iteration output hidden_d) is y.
+ *   sx_commit is not available for this layer yet (SX_ERR_UNSUPPORTED). */
+enum { SX_ARCH_CONCAT = 0, SX_ARCH_FUSED3 = 1 };
 
 typedef struct {
   const void *embed_d;        /* [vocab, H] */
@@ -97,6 +110,8 @@ typedef struct {
                                       Every drafted token that leaves the library (draft_tok,
                                       candidate ids) or feeds the embedding of the next round is
                                       the mapped id; ties break toward the lower draft id. */
+  const void *norm_e_d;            /* [H] gain of the embedding's RMSNorm; SX_ARCH_FUSED3 only (with that
+                                      layer fc_d is [H, 3H] and wqkv_d is [.., 2H], embedding half first) */
 } sx_weights;
 
 /* Paged KV cache of the draft layer.  Slot s of sequence b lives in physical page

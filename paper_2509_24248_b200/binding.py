@@ -42,13 +42,14 @@ class ModelCfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
                 ("n_signals", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
-                ("page_size", C.c_int32), ("act", C.c_int32 * SX_MAX_SIGNALS), ("draft_vocab", C.c_int32)]
+                ("page_size", C.c_int32), ("act", C.c_int32 * SX_MAX_SIGNALS), ("draft_vocab", C.c_int32),
+                ("arch", C.c_int32)]
 
 
 class Weights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("embed_d", "fc_d", "norm1_d", "wqkv_d", "wo_d", "norm2_d",
                                           "wgate_up_d", "wdown_d", "normf_d", "head_d", "target_head_d",
-                                          "draft_to_token_d")]
+                                          "draft_to_token_d", "norm_e_d")]
 
 
 class KV(C.Structure):
@@ -211,13 +212,15 @@ class SpecExit:
         if "target_head" not in self.w:
             self.w["target_head"] = self.w["head"]      # rows [0, V) of the shared head
         mc = ModelCfg(shape.H, shape.n_q, shape.n_kv, shape.d, shape.F, shape.V, shape.S, shape.eps,
-                      shape.theta, shape.page, (C.c_int32 * 3)(*act), getattr(shape, "Vd", 0))
+                      shape.theta, shape.page, (C.c_int32 * 3)(*act), getattr(shape, "Vd", 0),
+                      getattr(shape, "arch", 0))
         d2t = self.w.get("draft_to_token")
         if d2t is not None and (d2t.dtype != torch.int32 or d2t.numel() != (shape.Vd or shape.V)):
             raise SxError("draft_to_token must be int32 with one entry per draft id")
         ws = Weights(*[self.w[n].data_ptr() for n in ("embed", "fc", "norm1", "wqkv", "wo", "norm2",
                                                        "wgate_up", "wdown", "normf", "head", "target_head")],
-                     d2t.data_ptr() if d2t is not None else None)
+                     d2t.data_ptr() if d2t is not None else None,
+                     self.w["norm_e"].data_ptr() if "norm_e" in self.w else None)
         dc = DraftCfg(mode, K, topk, max_nodes)
         h = C.c_void_p()
         _check(self.lib.sx_create(C.byref(mc), C.byref(ws), max_batch, C.byref(dc), max_verify_rows,

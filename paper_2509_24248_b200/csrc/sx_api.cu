@@ -111,6 +111,8 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   const int Vd = m->draft_vocab ? m->draft_vocab : m->vocab;
   if (Vd < 1 || Vd > m->vocab) return SX_ERR_INVALID_ARG;
   if (Vd < m->vocab && !w->draft_to_token_d) return SX_ERR_INVALID_ARG;   // a reduced vocabulary needs its id map
+  if (m->arch != SX_ARCH_CONCAT && m->arch != SX_ARCH_FUSED3) return SX_ERR_UNSUPPORTED;
+  if (m->arch == SX_ARCH_FUSED3 && (!w->norm_e_d || ((uintptr_t)w->norm_e_d & 15))) return SX_ERR_INVALID_ARG;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
@@ -118,7 +120,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->prof_ev = new std::vector<cudaEvent_t>();
   c->prof_cls = new std::vector<int>();
   c->sh.H = m->H; c->sh.nq = m->n_q_heads; c->sh.nkv = m->n_kv_heads; c->sh.d = m->head_dim;
-  c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.Vd = Vd; c->sh.S = m->n_signals; c->sh.page = m->page_size;
+  c->sh.F = m->ffn; c->sh.V = m->vocab; c->sh.Vd = Vd; c->sh.arch = m->arch; c->sh.S = m->n_signals; c->sh.page = m->page_size;
   c->sh.eps = m->rms_eps; c->sh.theta = m->rope_theta;
   for (int i = 0; i < SX_MAX_SIGNALS; ++i) c->sh.act[i] = m->act[i];
   c->w = *w;
@@ -307,14 +309,30 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   rm.cache_len = kv->cache_len_d; rm.row_mask = row_mask;
   rm.valid_len = nullptr; rm.per_seq = 1;
   int sp; size_t stride;
-  // input_ready: the previous round's merge kernel has already written u (chain drafting)
-  if (!input_ready) {
-    sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
-    c->launches += 1;
+  const bool fused3 = s.arch == SX_ARCH_FUSED3;
+  if (fused3) {
+    // round 1: x = fc . [three target features]; later rounds: x = the source row's hidden (y).
+    // u = [norm_e(E[token]) ; norm_1(x)] feeds the q/k/v projection, x is the residual stream.
+    if (round == 1) {
+      if (fi.idx || fi.mul != 1 || fi.add != 0) return SX_ERR_UNSUPPORTED;      // the GEMM reads the rows in place
+      SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 3 * s.H, feat, R, ws, &sp, &stride, status, st));
+      sx_launch_fused_input(s, R, part, sp, stride, nullptr, fi, tok, ti, (const bf16 *)c->w.embed_d,
+                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st);
+    } else {
+      sx_launch_fused_input(s, R, nullptr, 0, 0, feat, fi, tok, ti, (const bf16 *)c->w.embed_d,
+                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st);
+    }
+    SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, 2 * s.H, u, R, ws, &sp, &stride, status, st));
+  } else {
+    // input_ready: the previous round's merge kernel has already written u (chain drafting)
+    if (!input_ready) {
+      sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
+      c->launches += 1;
+    }
+    SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
+    sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
+    SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
   }
-  SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
-  sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
-  SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
   sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st);
   const int B = kv->batch, nr = R / B;
   const int E = (c->dc.mode == SX_MODE_CHAIN) ? round : (round == 1 ? 1 : 1 + (round - 1) * c->dc.topk);
@@ -327,12 +345,13 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   SX_TRY(gemm(c, SX_PROF_GEMM_GATE_UP, c->w.wgate_up_d, 2 * s.F, s.H, n, R, ws, &sp, &stride, status, st));
   sx_launch_finish_swiglu(s, R, part, sp, stride, m, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_DOWN, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
-  sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st);
+  // the hidden handed to the caller (and to the next round) is g, or y for the fused layer
+  sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st, fused3 ? 1 : 0);
   c->launches += 7;   // 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
   SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.Vd + s.S, s.Vd, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
               status, st,
-              prepare_next ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
+              (prepare_next && !fused3) ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
                            : SxNextInput{nullptr, nullptr, nullptr, 0, 0},
               c->w.draft_to_token_d));
   return SX_OK;
@@ -430,7 +449,8 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
   if (c->dc.mode == SX_MODE_CHAIN) {
     sx_launch_chain_layout(B, K, S, tok0_d, *o, st);
     c->launches += 1;
-    const bool fuse = B <= sx_head_max_rows(1, 0);     // one head launch per round: its merge can write the next input
+    // one head launch per round: its merge can write the next input (concat layer only)
+    const bool fuse = B <= sx_head_max_rows(1, 0) && c->sh.arch == SX_ARCH_CONCAT;
     for (int k = 1; k <= K; ++k) {
       const bf16 *feat = (k == 1) ? (const bf16 *)feat0_d : hid;
       SxIndex fi = (k == 1) ? SxIndex{nullptr, 1, 0} : SxIndex{nullptr, K, k - 2};
@@ -481,6 +501,7 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
   SX_TRY(check_kv(c, kv));
   SX_TRY(check_ws(c, ws_d, ws_bytes));
   if (P < 1 || path_stride < 1 || path_stride - 1 > c->dc.K) return SX_ERR_INVALID_ARG;
+  if (c->sh.arch != SX_ARCH_CONCAT) return SX_ERR_UNSUPPORTED;
   if (((uintptr_t)target_hidden_d & 15) || ((uintptr_t)feat0_next_d & 15)) return SX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)ws_d;
@@ -527,7 +548,7 @@ extern "C" sx_status sx_spec_exit_iter_host(sx_ctx *c, const sx_kv *kv, const sx
     return SX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t B = kv->batch, H = c->sh.H;
-  if (cudaMemcpyAsync(stage_feat0_d, feat0_h, B * H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return SX_ERR_CUDA;
+  if (cudaMemcpyAsync(stage_feat0_d, feat0_h, B * H * 2 * (c->sh.arch == SX_ARCH_FUSED3 ? 3 : 1), cudaMemcpyHostToDevice, st) != cudaSuccess) return SX_ERR_CUDA;
   if (cudaMemcpyAsync(stage_tok0_d, tok0_h, B * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return SX_ERR_CUDA;
   if (cudaMemcpyAsync(stage_target_hidden_d, target_hidden_h, B * c->P * H * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return SX_ERR_CUDA;

@@ -61,7 +61,7 @@ __device__ __forceinline__ float4 sx_sum_splits4(const float *p, int splits, siz
 __global__ void __launch_bounds__(1024)
 sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t split_stride,
                       const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
-                      bf16 *out_user, SxIndex ui) {
+                      bf16 *out_user, SxIndex ui, int user_gets_v) {
   extern __shared__ float sx_buf[];        // [H] values, then [H / 2] words of gain (bf16 pairs)
   __shared__ float red[32];
   uint2 *gam = reinterpret_cast<uint2 *>(sx_buf + H);
@@ -71,6 +71,7 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
   sx_pdl_wait();
   const int r = blockIdx.x;
   float ss = 0.f;
+  bf16 *user = out_user ? out_user + (size_t)sx_index(ui, r) * H : nullptr;
   for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
     float4 v = sx_sum_splits4(part + (size_t)r * H + i, splits, split_stride);
     if (residual) {
@@ -80,11 +81,12 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
       v.x += r0.x; v.y += r0.y; v.z += r1.x; v.w += r1.y;
     }
     __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
-    if (out_v) {
+    if (out_v || (user && user_gets_v)) {
       uint2 w;
       w.x = *reinterpret_cast<uint32_t *>(&b0);
       w.y = *reinterpret_cast<uint32_t *>(&b1);
-      *reinterpret_cast<uint2 *>(out_v + (size_t)r * H + i) = w;
+      if (out_v) *reinterpret_cast<uint2 *>(out_v + (size_t)r * H + i) = w;
+      if (user && user_gets_v) *reinterpret_cast<uint2 *>(user + i) = w;
     }
     const float2 f0 = __bfloat1622float2(b0), f1 = __bfloat1622float2(b1);
     *reinterpret_cast<float4 *>(sx_buf + i) = make_float4(f0.x, f0.y, f1.x, f1.y);
@@ -99,7 +101,7 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
     for (int w = 0; w < nw; ++w) tot += red[w];           // same order in every thread
   }
   const float scale = rsqrtf(tot / (float)H + eps);
-  bf16 *user = out_user ? out_user + (size_t)sx_index(ui, r) * H : nullptr;
+  if (user_gets_v) user = nullptr;
   for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4 *>(sx_buf + i);
     const uint2 gu = gam[i >> 2];
@@ -117,13 +119,102 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
 
 void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
-                           bf16 *out_user, SxIndex ui, cudaStream_t st) {
+                           bf16 *out_user, SxIndex ui, cudaStream_t st, int user_gets_v) {
   int threads = ((sh.H / 4 + 31) / 32) * 32;
   if (threads > 1024) threads = 1024;
   if (sh.H * 6 > 48 * 1024)
     cudaFuncSetAttribute(sx_finish_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.H * 6);
   sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * (sizeof(float) + sizeof(bf16)), st, sh.H, sh.eps, part,
-            splits, split_stride, residual, gamma, out_v, out_n, out_user, ui);
+            splits, split_stride, residual, gamma, out_v, out_n, out_user, ui, user_gets_v);
+}
+
+// ---------------------------------------------------------------------------------------
+// Input of the layer with three-feature fusion: x = the fused feature (split-K sum of the fc
+// GEMM, round 1) or the hidden state of the source row (later rounds); the attention input is
+// u[r] = [ RMSNorm_e(E[token]) ; RMSNorm_1(x) ], the residual stream starts from x.
+// One CTA per row; a thread owns 4 consecutive elements per pass.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+sx_fused_input_kernel(int H, int V, float eps, const float *part, int splits, size_t split_stride, const bf16 *feat,
+                      SxIndex fi, const int32_t *tok, SxIndex ti, const bf16 *embed, const bf16 *gamma_e,
+                      const bf16 *gamma_h, bf16 *x_out, bf16 *u, int32_t *status) {
+  extern __shared__ float sx_buf[];        // [H] x, [H] embedding
+  __shared__ float red[2][32];
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int r = blockIdx.x;
+  int t = tok[sx_index(ti, r)];
+  if (t < 0 || t >= V) {
+    if (threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY);
+    t = 0;
+  }
+  float *xs = sx_buf, *es = sx_buf + H;
+  const bf16 *src = part ? nullptr : feat + (size_t)sx_index(fi, r) * H;
+  const bf16 *erow = embed + (size_t)t * H;
+  float sx = 0.f, se = 0.f;
+  for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+    uint2 xw;
+    if (part) {
+      const float4 v = sx_sum_splits4(part + (size_t)r * H + i, splits, split_stride);
+      __nv_bfloat162 b0 = __floats2bfloat162_rn(v.x, v.y), b1 = __floats2bfloat162_rn(v.z, v.w);
+      xw.x = *reinterpret_cast<uint32_t *>(&b0);
+      xw.y = *reinterpret_cast<uint32_t *>(&b1);
+    } else {
+      xw = *reinterpret_cast<const uint2 *>(src + i);
+    }
+    *reinterpret_cast<uint2 *>(x_out + (size_t)r * H + i) = xw;
+    const uint2 ew = *reinterpret_cast<const uint2 *>(erow + i);
+    const float2 x0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xw.x));
+    const float2 x1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&xw.y));
+    const float2 e0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ew.x));
+    const float2 e1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ew.y));
+    *reinterpret_cast<float4 *>(xs + i) = make_float4(x0.x, x0.y, x1.x, x1.y);
+    *reinterpret_cast<float4 *>(es + i) = make_float4(e0.x, e0.y, e1.x, e1.y);
+    sx += (x0.x * x0.x + x0.y * x0.y) + (x1.x * x1.x + x1.y * x1.y);
+    se += (e0.x * e0.x + e0.y * e0.y) + (e1.x * e1.x + e1.y * e1.y);
+  }
+  sx = sx_warp_sum(sx);
+  se = sx_warp_sum(se);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sx; red[1][threadIdx.x >> 5] = se; }
+  __syncthreads();
+  float tx = 0.f, te = 0.f;
+  {
+    const int nw = blockDim.x >> 5;
+    for (int w = 0; w < nw; ++w) { tx += red[0][w]; te += red[1][w]; }    // same order in every thread
+  }
+  const float scx = rsqrtf(tx / (float)H + eps), sce = rsqrtf(te / (float)H + eps);
+  bf16 *urow = u + (size_t)r * 2 * H;
+  for (int i = threadIdx.x * 4; i < H; i += blockDim.x * 4) {
+    const float4 xv = *reinterpret_cast<const float4 *>(xs + i), ev = *reinterpret_cast<const float4 *>(es + i);
+    const uint2 ge = *reinterpret_cast<const uint2 *>(gamma_e + i), gh = *reinterpret_cast<const uint2 *>(gamma_h + i);
+    const float2 a0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ge.x));
+    const float2 a1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ge.y));
+    const float2 h0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gh.x));
+    const float2 h1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gh.y));
+    __nv_bfloat162 p0 = __floats2bfloat162_rn(ev.x * sce * a0.x, ev.y * sce * a0.y);
+    __nv_bfloat162 p1 = __floats2bfloat162_rn(ev.z * sce * a1.x, ev.w * sce * a1.y);
+    __nv_bfloat162 q0 = __floats2bfloat162_rn(xv.x * scx * h0.x, xv.y * scx * h0.y);
+    __nv_bfloat162 q1 = __floats2bfloat162_rn(xv.z * scx * h1.x, xv.w * scx * h1.y);
+    uint2 w;
+    w.x = *reinterpret_cast<uint32_t *>(&p0);
+    w.y = *reinterpret_cast<uint32_t *>(&p1);
+    *reinterpret_cast<uint2 *>(urow + i) = w;
+    w.x = *reinterpret_cast<uint32_t *>(&q0);
+    w.y = *reinterpret_cast<uint32_t *>(&q1);
+    *reinterpret_cast<uint2 *>(urow + H + i) = w;
+  }
+}
+
+void sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+                           const bf16 *feat, SxIndex fi, const int32_t *tok, SxIndex ti, const bf16 *embed,
+                           const bf16 *gamma_e, const bf16 *gamma_h, bf16 *x_out, bf16 *u, int32_t *status,
+                           cudaStream_t st) {
+  int threads = ((sh.H / 4 + 31) / 32) * 32;
+  if (threads > 1024) threads = 1024;
+  if (sh.H * 8 > 48 * 1024)
+    cudaFuncSetAttribute(sx_fused_input_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.H * 8);
+  sx_launch(sx_fused_input_kernel, dim3(R), dim3(threads), (size_t)sh.H * 8, st, sh.H, sh.V, sh.eps, part, splits,
+            split_stride, feat, fi, tok, ti, embed, gamma_e, gamma_h, x_out, u, status);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -11,6 +11,7 @@ struct SxIndex {
 
 struct SxShape {
   int H, nq, nkv, d, F, V, S, page;
+  int arch;                    // SX_ARCH_CONCAT | SX_ARCH_FUSED3
   int Vd;                      // vocabulary rows of the draft head (== V without a reduced draft vocabulary)
   float eps, theta;
   int act[SX_MAX_SIGNALS];
@@ -23,7 +24,14 @@ void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex 
 // out_user (optional) receives out_n at row index ui(r).
 void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
-                           bf16 *out_user, SxIndex ui, cudaStream_t st);
+                           bf16 *out_user, SxIndex ui, cudaStream_t st, int user_gets_v = 0);
+
+// Layer with three-feature fusion: x_out[r] = bf16(sum of the fc partials) (part != nullptr) or the
+// hidden of row fi(r) of `feat`; u[r] = [rmsnorm(E[token]) * gamma_e ; rmsnorm(x) * gamma_h].
+void sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+                           const bf16 *feat, SxIndex fi, const int32_t *tok, SxIndex ti, const bf16 *embed,
+                           const bf16 *gamma_e, const bf16 *gamma_h, bf16 *x_out, bf16 *u, int32_t *status,
+                           cudaStream_t st);
 
 void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
