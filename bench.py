@@ -48,12 +48,18 @@ def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
     """Bytes one iteration has to move: every weight matrix once per dependent draft round,
     every live KV byte once per round, the verify head once."""
     s = wl.shape
-    layer = 2 * s.H * s.H + s.H * s.qkv_rows + s.n_q * s.d * s.H + 3 * s.H * s.F
     head = ((s.Vd or s.V) + s.S) * s.H
     rounds = wl.K
-    w_round = 2 * (layer + head)
     kv_round = int(sum(int(n) for n in lens)) * s.n_kv * s.d * 2 * 2
-    total = rounds * (w_round + kv_round) + 2 * s.V * s.H
+    if s.arch:
+        # three-feature layer: fc (3H -> H) in round 1 only, q/k/v projection over 2H every round
+        layer = 2 * s.H * s.qkv_rows + s.n_q * s.d * s.H + 3 * s.H * s.F
+        w_round = 2 * (layer + head)
+        total = rounds * (w_round + kv_round) + 2 * 3 * s.H * s.H + 2 * s.V * s.H
+    else:
+        layer = 2 * s.H * s.H + s.H * s.qkv_rows + s.n_q * s.d * s.H + 3 * s.H * s.F
+        w_round = 2 * (layer + head)
+        total = rounds * (w_round + kv_round) + 2 * s.V * s.H
     return {"total": total, "head_launch": 2 * head, "w_round": w_round, "kv_round": kv_round}
 
 
@@ -239,6 +245,9 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="verify with stochastic acceptance at this temperature (0 = greedy, the headline setting)")
+    ap.add_argument("--layer", choices=["concat", "fused3"], default="concat",
+                    help="draft layer: fc over [hidden ; embedding] every round (the headline setting), or "
+                         "three-feature fusion in round 1 with [norm(embedding) ; norm(hidden)] as attention input")
     ap.add_argument("--draft-vocab", type=int, default=0, metavar="VD",
                     help="reduce the draft head to VD ids (id map + the target's own head); 0 = the workload as defined")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -258,6 +267,9 @@ def main():
     if args.temperature > 0.0:
         import dataclasses
         wl = dataclasses.replace(wl, name=f"{wl.name}+tau{args.temperature:g}")
+    if args.layer == "fused3":
+        import dataclasses
+        wl = dataclasses.replace(wl, name=f"{wl.name}+fused3", shape=dataclasses.replace(wl.shape, arch=1))
 
     if args.impl == "reference":
         if rank == 0:
@@ -387,7 +399,7 @@ def main():
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t_start) * 1e3 / e2e_steps
     e2e_ms = max_over_ranks(e2e_ms, dist, dev)
-    h2d = wl.B * H * 2 + wl.B * 4 + wl.B * P * H * 2
+    h2d = int(f0_h.numel()) * 2 + wl.B * 4 + wl.B * P * H * 2
     d2h = wl.B * (3 * 4 + S * 4)
 
     if rank != 0:

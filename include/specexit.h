@@ -90,7 +90,8 @@ typedef struct {
  *   [.., 2H]) and the residual stream starts from x; later rounds take the layer's own output y
  *   (before the final norm) as x, without fc.  The head reads RMSNorm_f(y).  Every hidden state
  *   this library returns or takes between rounds (hidden_out_d, iteration output hidden_d) is y.
- *   sx_commit is not available for this layer yet (SX_ERR_UNSUPPORTED). */
+ *   sx_commit takes the three target features of every verify slot ([batch, P, 3H]) as its
+ *   target_hidden_d and returns a [batch, 3H] feat0_next_d. */
 enum { SX_ARCH_CONCAT = 0, SX_ARCH_FUSED3 = 1 };
 
 typedef struct {

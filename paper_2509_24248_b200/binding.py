@@ -371,9 +371,11 @@ class SpecExit:
     def sx_commit(self, target_hidden: torch.Tensor, cand_tok: torch.Tensor, path: torch.Tensor,
                   accept_len_out: torch.Tensor, recover_tok_out: torch.Tensor):
         """Commits the verified tokens (the context's ``cache_len`` tensor is advanced in place) and
-        returns the next iteration's first row ``(feat0 [B, H] bf16, tok0 [B] int32)``."""
+        returns the next iteration's first row ``(feat0 [B, H] bf16, tok0 [B] int32)``.  With the
+        three-feature layer ``target_hidden`` is ``[B, P, 3H]`` (the target features of every verify
+        slot) and ``feat0`` is ``[B, 3H]``."""
         B, P = cand_tok.shape
-        feat0 = torch.empty(B, self.shape.H, dtype=torch.bfloat16, device=self.dev)
+        feat0 = torch.empty(B, int(target_hidden.shape[-1]), dtype=torch.bfloat16, device=self.dev)
         tok0 = torch.empty(B, dtype=torch.int32, device=self.dev)
         _check(self.lib.sx_commit(self.h, C.byref(self._kv_struct), P, target_hidden.data_ptr(), cand_tok.data_ptr(),
                                   path.data_ptr(), int(path.shape[1]), accept_len_out.data_ptr(),

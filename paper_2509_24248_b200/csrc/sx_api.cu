@@ -17,7 +17,7 @@ struct sx_ctx {
   int max_splits, part_N, head_G, head_rows;
   // workspace offsets (bytes)
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
-      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, total;
+      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, total;
   int commit_rows, commit_N;
   SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
   // tree sub-offsets relative to off_tree
@@ -189,9 +189,13 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   // commit: up to K catch-up rows per sequence through fc, norm and the K/V part of the projection
   c->commit_rows = max_batch * dc->K;
   c->commit_N = s.H > (s.nq + 2 * s.nkv) * s.d ? s.H : (s.nq + 2 * s.nkv) * s.d;
-  c->off_cu = take((size_t)c->commit_rows * 2 * s.H * 2);
+  c->off_cu = take((size_t)c->commit_rows * (s.arch == SX_ARCH_FUSED3 ? 3 : 2) * s.H * 2);
   c->off_cn = take((size_t)c->commit_rows * s.H * 2);
   c->off_cpart = take((size_t)SX_COMMIT_MAX_SPLITS * c->commit_rows * c->commit_N * 4);
+  if (s.arch == SX_ARCH_FUSED3) {
+    c->off_cu2 = take((size_t)c->commit_rows * 2 * s.H * 2);
+    c->off_ctok = take((size_t)c->commit_rows * 4);
+  }
   c->off_tree = o;
   if (dc->mode == SX_MODE_TREE) {
     const size_t B = max_batch, NC = c->NC, rows = c->rows_per_seq;
@@ -501,7 +505,6 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
   SX_TRY(check_kv(c, kv));
   SX_TRY(check_ws(c, ws_d, ws_bytes));
   if (P < 1 || path_stride < 1 || path_stride - 1 > c->dc.K) return SX_ERR_INVALID_ARG;
-  if (c->sh.arch != SX_ARCH_CONCAT) return SX_ERR_UNSUPPORTED;
   if (((uintptr_t)target_hidden_d & 15) || ((uintptr_t)feat0_next_d & 15)) return SX_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)ws_d;
@@ -509,6 +512,39 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
   const int B = kv->batch, M = path_stride - 1, R = B * M;
   bf16 *u = (bf16 *)(ws + c->off_cu), *n = (bf16 *)(ws + c->off_cn);
   float *part = (float *)(ws + c->off_cpart);
+  if (s.arch == SX_ARCH_FUSED3) {
+    // target_hidden_d holds the three target features of every verify slot ([batch, P, 3H]):
+    // catch-up rows go through fc (3H -> H), the two input norms and the K/V part of the projection
+    bf16 *u2 = (bf16 *)(ws + c->off_cu2);
+    int32_t *trow = (int32_t *)(ws + c->off_ctok);
+    sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
+                            recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d,
+                            st, trow);
+    c->launches += 1;
+    if (R > 0) {
+      int sp = sx_gemm_pick_splits(s.H, 3 * s.H, c->sm_count);
+      if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
+      SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 3 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
+                                    status_d, st));
+      sx_launch_fused_input(s, R, part, sp, (size_t)R * s.H, nullptr, SxIndex{nullptr, 1, 0}, trow, SxIndex{nullptr, 1, 0},
+                            (const bf16 *)c->w.embed_d, (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, n, u2,
+                            status_d, st);
+      const int N = (s.nq + 2 * s.nkv) * s.d;
+      sp = sx_gemm_pick_splits(N, 2 * s.H, c->sm_count);
+      if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
+      SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, 2 * s.H, u2, R, part, sp, (size_t)R * N, c->sm_count,
+                                    status_d, st));
+      SxRowMap rm;
+      memset(&rm, 0, sizeof(rm));
+      rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
+      rm.valid_len = accept_len_out_d; rm.per_seq = M;
+      sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st);
+      c->launches += 4;
+    }
+    sx_launch_commit_advance(B, accept_len_out_d, const_cast<int32_t *>(kv->cache_len_d), st);
+    c->launches += 1;
+    return SX_OK;
+  }
   sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
                           recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d, st);
   c->launches += 1;

@@ -293,27 +293,30 @@ void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const floa
 // Blocks [0, B * M): catch-up input row (b, j) = [target hidden of path slot j ; embedding of the
 // token of path slot j + 1] when j < L_b, zeros otherwise.  Blocks [B * M, B * M + B): the next
 // iteration's first row: feature = target hidden of path slot L_b, token = recover token.
-__global__ void sx_commit_gather_kernel(int B, int M, int P, int H, int V, const bf16 *th, const int32_t *cand,
+// FW is the width of a target feature row (H, or 3H for the layer with three-feature fusion).
+// With tok_rows == nullptr a catch-up row is [feature ; embedding] (FW == H); otherwise it is the
+// feature alone and the row's token goes to tok_rows.
+__global__ void sx_commit_gather_kernel(int B, int M, int P, int H, int FW, int V, const bf16 *th, const int32_t *cand,
                                         const int32_t *path, int path_stride, const int32_t *accept_len,
-                                        const int32_t *recover, const bf16 *embed, bf16 *u, bf16 *feat0,
-                                        int32_t *tok0, int32_t *status) {
+                                        const int32_t *recover, const bf16 *embed, bf16 *u, int32_t *tok_rows,
+                                        bf16 *feat0, int32_t *tok0, int32_t *status) {
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int n8 = H / 8;
+  const int n8 = H / 8, f8 = FW / 8;
   if ((int)blockIdx.x >= B * M) {
     const int b = blockIdx.x - B * M;
     int L = accept_len[b];
     if (L < 0 || L >= path_stride) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_INVALID_ARG); L = 0; }
     int slot = path[(size_t)b * path_stride + L];
     if (slot < 0 || slot >= P) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_INVALID_ARG); slot = 0; }
-    const uint4 *src = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + slot) * H);
-    uint4 *dst = reinterpret_cast<uint4 *>(feat0 + (size_t)b * H);
-    for (int i = threadIdx.x; i < n8; i += blockDim.x) dst[i] = src[i];
+    const uint4 *src = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + slot) * FW);
+    uint4 *dst = reinterpret_cast<uint4 *>(feat0 + (size_t)b * FW);
+    for (int i = threadIdx.x; i < f8; i += blockDim.x) dst[i] = src[i];
     if (threadIdx.x == 0) tok0[b] = recover[b];
     return;
   }
   const int b = blockIdx.x / M, j = blockIdx.x - b * M;
-  uint4 *o = reinterpret_cast<uint4 *>(u + (size_t)blockIdx.x * 2 * H);
+  uint4 *o = reinterpret_cast<uint4 *>(u + (size_t)blockIdx.x * (tok_rows ? FW : 2 * H));
   const int L = accept_len[b];
   bool live = j < L && j + 1 < path_stride;
   int s0 = 0, s1 = 0, t = 0;
@@ -326,9 +329,14 @@ __global__ void sx_commit_gather_kernel(int B, int M, int P, int H, int V, const
     t = cand[(size_t)b * P + s1];
     if (t < 0 || t >= V) { if (threadIdx.x == 0) sx_set_status(status, SX_ERR_CAPACITY); t = 0; }
   }
-  const uint4 *f = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + s0) * H);
+  const uint4 *f = reinterpret_cast<const uint4 *>(th + ((size_t)b * P + s0) * FW);
   const uint4 *e = reinterpret_cast<const uint4 *>(embed + (size_t)t * H);
   const uint4 zero = make_uint4(0, 0, 0, 0);
+  if (tok_rows) {
+    for (int i = threadIdx.x; i < f8; i += blockDim.x) o[i] = live ? f[i] : zero;
+    if (threadIdx.x == 0) tok_rows[blockIdx.x] = t;
+    return;
+  }
   for (int i = threadIdx.x; i < n8; i += blockDim.x) {
     o[i] = live ? f[i] : zero;
     o[n8 + i] = live ? e[i] : zero;
@@ -345,11 +353,13 @@ __global__ void sx_commit_advance_kernel(int B, const int32_t *accept_len, int32
 
 void sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
                              const int32_t *path, int path_stride, const int32_t *accept_len, const int32_t *recover,
-                             const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0, int32_t *status, cudaStream_t st) {
+                             const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0, int32_t *status, cudaStream_t st,
+                             int32_t *tok_rows) {
   int threads = ((sh.H / 8 + 31) / 32) * 32;
   if (threads > 512) threads = 512;
-  sx_launch(sx_commit_gather_kernel, dim3(B * M + B), dim3(threads), 0, st, B, M, P, sh.H, sh.V, th, cand, path,
-            path_stride, accept_len, recover, embed, u, feat0, tok0, status);
+  const int FW = tok_rows ? 3 * sh.H : sh.H;
+  sx_launch(sx_commit_gather_kernel, dim3(B * M + B), dim3(threads), 0, st, B, M, P, sh.H, FW, sh.V, th, cand, path,
+            path_stride, accept_len, recover, embed, u, tok_rows, feat0, tok0, status);
 }
 
 void sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st) {

@@ -40,7 +40,7 @@ void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const floa
 void sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
                              const int32_t *path, int path_stride, const int32_t *accept_len,
                              const int32_t *recover, const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0,
-                             int32_t *status, cudaStream_t st);
+                             int32_t *status, cudaStream_t st, int32_t *tok_rows = nullptr);
 void sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st);
 
 void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits,

@@ -30,15 +30,18 @@ def _random_paths(B, P, M, gen, tree):
 
 @pytest.mark.parametrize("tree", [False, True])
 @pytest.mark.parametrize("shape_kw,B,K", [(dict(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16), 5, 4),
-                                          (dict(H=256, n_q=4, n_kv=2, d=64, F=688, V=4096, page=64), 3, 6)])
+                                          (dict(H=256, n_q=4, n_kv=2, d=64, F=688, V=4096, page=64), 3, 6),
+                                          (dict(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16, arch=1), 5, 4),
+                                          (dict(H=256, n_q=4, n_kv=2, d=64, F=688, V=4096, page=64, arch=1), 3, 6)])
 def test_commit_matches_oracle(shape_kw, B, K, tree):
+    # with the three-feature layer (arch=1) the rows handed to the commit are [.., 3H] target features
     sh = synth.ModelShape(**shape_kw)
     wl = synth.Workload("cm", sh, B=B, mode=synth.TREE if tree else synth.CHAIN, K=K, topk=2 if tree else 1,
                         max_nodes=9 if tree else 0, len_lo=3, len_hi=70, seed=17)
     case = harness.build_case(wl)
     P = wl.P
     g = torch.Generator().manual_seed(23)
-    th = torch.randn(B, P, sh.H, generator=g).to(torch.bfloat16)
+    th = torch.randn(B, P, (3 if sh.arch else 1) * sh.H, generator=g).to(torch.bfloat16)
     cand = torch.randint(0, sh.V, (B, P), generator=g, dtype=torch.int32)
     rec = torch.randint(0, sh.V, (B,), generator=g, dtype=torch.int32)
     L, path = _random_paths(B, P, K, g, tree)
@@ -72,8 +75,9 @@ def test_commit_matches_oracle(shape_kw, B, K, tree):
     assert bool(same[keep].all())
 
 
-def test_three_iterations_with_commit_on_the_gpu():
-    wl = synth.Workload("loop", synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16), B=3,
+@pytest.mark.parametrize("arch", [0, 1])
+def test_three_iterations_with_commit_on_the_gpu(arch):
+    wl = synth.Workload("loop", synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16, arch=arch), B=3,
                         mode=synth.CHAIN, K=3, len_lo=5, len_hi=20, seed=3)
     case = harness.build_case(wl, poison_tail=False)
     # room for three iterations of K + 1 new tokens each
@@ -88,6 +92,8 @@ def test_three_iterations_with_commit_on_the_gpu():
     for it in range(3):
         th = torch.randn(wl.B, wl.P, wl.shape.H, generator=g).to(torch.bfloat16).to(dev)
         sx.sx_spec_exit_iter(params, state, feat, tok, th, out)
+        if arch:                                   # the target's three features of every verify slot
+            th = torch.randn(wl.B, wl.P, 3 * wl.shape.H, generator=g).to(torch.bfloat16).to(dev)
         feat, tok = sx.sx_commit(th, out["cand_tok_d"], out["path_d"], out["accept_len_out_d"], out["recover_tok_out_d"])
         torch.cuda.synchronize()
         sx.check_status()

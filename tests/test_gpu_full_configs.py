@@ -33,3 +33,15 @@ def test_chain_config1_with_a_32k_draft_vocabulary():
     print(f"C1/Vd=32768: accept_len {rep.accept_len} exempt {rep.exempt} "
           f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
     assert len(rep.exempt) <= 2
+
+
+def test_chain_config1_with_the_three_feature_layer_and_a_32k_draft_vocabulary():
+    """C1's shapes in the EAGLE-3-like configuration: three-feature fusion, concatenated attention
+    input, draft head over 32768 ids."""
+    import dataclasses
+    wl = synth.workload("C1")
+    wl = dataclasses.replace(wl, shape=dataclasses.replace(wl.shape, Vd=32768, arch=1))
+    rep = parity.run_chain(harness.build_case(wl, poison_tail=True))
+    print(f"C1/fused3/Vd=32768: accept_len {rep.accept_len} exempt {rep.exempt} "
+          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
+    assert len(rep.exempt) <= 2

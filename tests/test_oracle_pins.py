@@ -1025,3 +1025,29 @@ def test_fused3_tree_with_one_child_per_node_is_the_chain():
     c = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 3)
     assert torch.equal(t.cand_tok, c.cand_tok)
     assert torch.equal(t.hidden, c.hidden)
+
+
+def test_fused3_commit_rekeys_from_the_three_target_features():
+    wl = synth.Workload("f3c", _SH_F3, B=2, mode=synth.CHAIN, K=2, len_lo=9, len_hi=30, seed=53)
+    case = harness.build_case(wl, poison_tail=False)
+    case.kv.update(synth.make_kv(wl.shape, synth.cache_lengths(wl), wl.K + 2, wl.seed, poison_tail=False))
+    model = harness.oracle_model(case)
+    kv = harness.oracle_kv(case)
+    n0 = list(kv.len)
+    g = torch.Generator().manual_seed(2)
+    tf = torch.randn(wl.B, wl.P, 3 * _SH_F3.H, generator=g).to(torch.bfloat16)
+    cand = torch.randint(0, _SH_F3.V, (wl.B, wl.P), generator=g)
+    path = torch.tensor([[0, 1, 2], [0, 1, -1]])
+    L, rec = torch.tensor([2, 1]), torch.tensor([7, 8])
+    oc = orc.commit(model, kv, tf, cand, path, L, rec)
+    assert oc.cache_len == [n0[0] + 3, n0[1] + 2] and oc.feat0.shape == (2, 3 * _SH_F3.H)
+    assert torch.equal(oc.feat0[0], tf[0, 2].to(torch.float64)) and torch.equal(oc.feat0[1], tf[1, 1].to(torch.float64))
+    # the K/V of accepted token j: the restatement fed (features of path slot j - 1, token of slot j)
+    for b, j in ((0, 1), (0, 2), (1, 1)):
+        f = tf[b, j - 1].to(torch.float64).numpy()
+        extra_k = [kv.read(b, n0[b] + i)[0].numpy()[None] for i in range(0, j)]
+        extra_v = [kv.read(b, n0[b] + i)[1].numpy()[None] for i in range(0, j)]
+        _, _, k1, v1, _ = _np_forward(case, f, int(cand[b, j]), b, extra_k, extra_v, fused3=True)
+        kk, vv = kv.read(b, n0[b] + j)
+        assert np.linalg.norm(kk.numpy() - k1[0]) / np.linalg.norm(k1[0]) < 1e-2
+        assert np.linalg.norm(vv.numpy() - v1[0]) / np.linalg.norm(v1[0]) < 1e-2
