@@ -100,3 +100,40 @@ def test_three_iterations_with_commit_on_the_gpu(arch):
         n = n + out["accept_len_out_d"].cpu() + 1
         assert sx.kv["cache_len"].cpu().tolist() == n.tolist()
         assert tok.cpu().tolist() == out["recover_tok_out_d"].cpu().tolist()
+
+
+@pytest.mark.parametrize("arch", [0, 1])
+def test_second_iteration_after_a_commit_matches_the_oracle(arch):
+    """Iteration 1 and its commit run on the GPU; iteration 2 then starts from the committed cache
+    and the returned first row, and is compared with the oracle element by element."""
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16, arch=arch)
+    wl = synth.Workload("it2", sh, B=3, mode=synth.CHAIN, K=3, len_lo=5, len_hi=40, seed=9,
+                        sigma_lo=0.0, sigma_hi=0.0)
+    case = harness.build_case(wl, poison_tail=False)
+    case.kv.update(synth.make_kv(sh, synth.cache_lengths(wl), 2 * (wl.K + 1) + wl.K, wl.seed, poison_tail=False))
+    w = dict(case.weights)
+    w["head"] = (w["head"].to(torch.float32) * 30.0).to(torch.bfloat16)       # peaked: some drafts get accepted
+    case = harness.Case(wl, w, case.kv, case.f0, case.t0, case.sigma)
+    sx = parity.make_gpu(case)
+    dev = sx.dev
+    params = parity.to_params(sx, harness.default_exit_cfg(wl, thr=(0.99, 0.0, 0.0)))
+    state, out = sx.new_state(wl.B), sx.new_outputs(wl.B)
+    # iteration 1 on the oracle gives the target hiddens the harness would use; the GPU runs on them
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    th = harness.chain_target_hidden(case, d)
+    sx.sx_spec_exit_iter(params, state, case.f0.to(dev), case.t0.to(dev), th.to(dev), out)
+    g = torch.Generator().manual_seed(10)
+    tf = th if not arch else torch.randn(wl.B, wl.P, 3 * sh.H, generator=g).to(torch.bfloat16)
+    feat, tok = sx.sx_commit(tf.to(dev), out["cand_tok_d"], out["path_d"], out["accept_len_out_d"],
+                             out["recover_tok_out_d"])
+    torch.cuda.synchronize()
+    sx.check_status()
+    assert int(out["accept_len_out_d"].sum()) > 0
+    kv2 = {"k_pages": sx.kv["k_pages"].cpu(), "v_pages": sx.kv["v_pages"].cpu(),
+           "page_table": sx.kv["page_table"].cpu(), "cache_len": sx.kv["cache_len"].cpu(),
+           "max_pages": case.kv["max_pages"]}
+    case2 = harness.Case(wl, w, kv2, feat.cpu(), tok.cpu(), case.sigma)
+    sx.close()
+    rep = parity.run_chain(case2)
+    print("iteration 2 accept:", rep.accept_len, "hidden rel:", rep.max_hidden_rel)
