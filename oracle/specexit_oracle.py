@@ -322,11 +322,12 @@ class ChainDraft:
     #                             position of slot j's token (round j+1); slot K: NaN
     gap: torch.Tensor           # [B, K] relative top-2 gap at each draft argmax
     z: torch.Tensor             # [B, K, S] raw signal rows per round
+    logits: Optional[torch.Tensor] = None   # [B, K, Vd] draft logits, kept when drafts are sampled
 
 
 def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, K: int,
                 forced: Optional[Dict[Tuple[int, int], int]] = None, chooser=None,
-                before_round=None, head_input=None) -> ChainDraft:
+                before_round=None, head_input=None, sample=None) -> ChainDraft:
     """K autoregressive draft rounds per sequence.  ``forced[(b, k)]`` (k = 1..K) replaces
     the k-th draft token of sequence b (used to replay a near-tie the other way);
     ``chooser("tok", (b, k), logits, 1, [tok]) -> [tok]`` may do the same on the fly."""
@@ -338,6 +339,11 @@ def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tens
     zz = torch.empty(B, K, S, dtype=F64)
     gap = torch.empty(B, K, dtype=F64)
     feat = f0.to(F64)
+    # sampled drafts: token k of sequence b is a Gumbel-max draw from softmax(logits / tau), with
+    # the draws of verify slot k - 1 of the draft stream (see speculative_sample)
+    sampling = sample is not None and sample.sample_drafts and sample.temperature > 0.0
+    kept = torch.empty(B, K, model.Vd, dtype=F64) if sampling else None
+    tau = float(torch.tensor(sample.temperature, dtype=torch.float32)) if sampling else 0.0
     for k in range(1, K + 1):
         if before_round is not None and k > 1:
             # replay hook: lets a test restart round k from another implementation's state
@@ -349,18 +355,22 @@ def draft_chain(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tens
                     visible=[kv.len[b] + j for j in range(k)]) for b in range(B)]
         g, ho = model.round(kv, rows, head_input)
         for b in range(B):
-            tok = argmax_low(ho.logits[b])
-            gap[b, k - 1] = top_gap(ho.logits[b])
+            score = ho.logits[b]
+            if sampling:
+                kept[b, k - 1] = ho.logits[b]
+                score = score + tau * gumbel_noise(sample, b, DRAFT_STREAM + k - 1, model.Vd)
+            tok = argmax_low(score)
+            gap[b, k - 1] = top_gap(score)
             if forced and (b, k) in forced:
                 tok = int(forced[(b, k)])
             if chooser is not None:
-                tok = int(chooser("tok", (b, k), ho.logits[b], 1, [tok])[0])
+                tok = int(chooser("tok", (b, k), score, 1, [tok])[0])
             cand[b, k] = model.to_token(tok)      # decisions are taken on draft ids, tokens are stored
         hidden[:, k - 1] = g
         sig[:, k - 1] = ho.s
         zz[:, k - 1] = ho.z
         feat = g
-    return ChainDraft(cand, hidden, sig, gap, zz)
+    return ChainDraft(cand, hidden, sig, gap, zz, kept)
 
 
 # --------------------------------------------------------------------------------------
@@ -587,6 +597,13 @@ class SampleCfg:
     temperature: float = 0.0
     seed: int = 0
     offset: int = 0          # e.g. the iteration number: a fresh set of draws per iteration
+    sample_drafts: bool = False   # chain drafts are drawn from the draft's softmax as well
+
+
+# The slot word of the counter separates three streams of draws: verify slot j itself (the
+# target-side Gumbel noise), ACCEPT_STREAM + j (the uniform of the accept test) and
+# DRAFT_STREAM + j (the Gumbel noise that draws the draft token proposed at slot j).
+ACCEPT_STREAM, DRAFT_STREAM = 0x20000000, 0x40000000
 
 
 def gumbel_noise(cfg: SampleCfg, b: int, j: int, V: int) -> torch.Tensor:
@@ -617,6 +634,65 @@ def target_sample(model: DraftModel, target_hidden: torch.Tensor, cfg: SampleCfg
     return tok.view(B, P), gap.view(B, P)
 
 
+@dataclass
+class SpecSampleOut:
+    target_tok: torch.Tensor   # [B, P] the kept draft token where the test passed, else the residual draw
+    accepted: torch.Tensor     # [B, P] bool
+    margin: torch.Tensor       # [B, P] |u - min(1, p(x)/q(x))| of the accept test (inf at the last slot)
+    gap: torch.Tensor          # [B, P] relative top-2 gap of the residual draw (inf where accepted)
+
+
+def speculative_sample(model: DraftModel, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
+                       draft_logits: torch.Tensor, cfg: SampleCfg) -> SpecSampleOut:
+    """Speculative sampling with sampled drafts, slot by slot (chain).  The draft token x
+    proposed at slot j (cand_tok[b, j + 1], drawn from q_j = softmax(draft_logits[b, j] / tau)) is
+    kept when u_j < min(1, p_j(x) / q_j(x)), p_j = softmax(target logits / tau); otherwise the slot's
+    token is drawn from the normalised max(0, p_j - q_j).  The last slot has no draft: its token is
+    drawn from p itself.  Draws: u_j from word 0 of the block with counter (0, ACCEPT_STREAM + j, b,
+    offset); the residual draw is a Gumbel-max over log max(0, p - q) with the noise of slot j.
+    Probabilities are float64 functions of the float32 logits."""
+    import numpy as np
+    B, P, H = target_hidden.shape
+    K = P - 1
+    assert model.map is None and draft_logits.shape[-1] == model.sh.V, "needs a full-vocabulary draft head"
+    logits = f32r(linear(target_hidden.reshape(B * P, H).to(F64), model.target_head)).view(B, P, -1)
+    tau = float(torch.tensor(cfg.temperature, dtype=torch.float32))
+    key = (cfg.seed & 0xFFFFFFFF, (cfg.seed >> 32) & 0xFFFFFFFF)
+    tok = torch.zeros(B, P, dtype=torch.int64)
+    acc = torch.zeros(B, P, dtype=torch.bool)
+    margin = torch.full((B, P), float("inf"), dtype=F64)
+    gap = torch.full((B, P), float("inf"), dtype=F64)
+    for b in range(B):
+        for j in range(P):
+            lp = logits[b, j] / tau
+            logp = lp - torch.logsumexp(lp, dim=0)
+            p = torch.exp(logp)
+            q = torch.zeros_like(p)
+            x = -1
+            if j < K:
+                lq = draft_logits[b, j].to(F64) / tau
+                logq = lq - torch.logsumexp(lq, dim=0)
+                q = torch.exp(logq)
+                x = int(cand_tok[b, j + 1])
+                ratio = min(1.0, math.exp(float(logp[x] - logq[x])))
+                u = float(uniform_open(philox4x32_10((0, ACCEPT_STREAM + j, b, cfg.offset), key)[0]))
+                margin[b, j] = abs(u - ratio)
+                if u < ratio:
+                    acc[b, j] = True
+                    tok[b, j] = x
+                    continue
+            r = p - q
+            if not bool((r > 0).any()):
+                tok[b, j] = x              # p == q: nothing is left to draw from (x >= 0 here)
+                continue
+            g = gumbel_noise(cfg, b, j, r.numel())
+            s = torch.where(r > 0, torch.log(r.clamp_min(1e-300)) + g, torch.full_like(r, -float("inf")))
+            tok[b, j] = argmax_low(s)
+            t2 = torch.topk(s, 2).values
+            gap[b, j] = float(t2[0] - t2[1])          # absolute: the scores are logarithms
+    return SpecSampleOut(tok, acc, margin, gap)
+
+
 def accept_chain(cand_tok: Sequence[int], target_tok: Sequence[int]) -> Tuple[int, List[int], int]:
     """Longest prefix of draft tokens that equal the target's greedy choice one slot
     earlier; the recover token is the target's choice after the last accepted slot."""
@@ -645,9 +721,15 @@ def accept_tree(cand_tok: Sequence[int], parent: Sequence[int], target_tok: Sequ
 def verify(model: DraftModel, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
            parent: Optional[torch.Tensor] = None,
            forced_target: Optional[Dict[Tuple[int, int], int]] = None,
-           sample: Optional[SampleCfg] = None) -> VerifyOut:
-    """Greedy verification, or (``sample`` with a positive temperature) speculative sampling."""
-    if sample is not None and sample.temperature > 0.0:
+           sample: Optional[SampleCfg] = None, draft_logits: Optional[torch.Tensor] = None) -> VerifyOut:
+    """Greedy verification, or (``sample`` with a positive temperature) speculative sampling:
+    with deterministic drafts through one draw per slot, with sampled drafts (chain only,
+    ``draft_logits`` given) through the accept test and the residual draw."""
+    if sample is not None and sample.temperature > 0.0 and sample.sample_drafts:
+        assert parent is None and draft_logits is not None
+        so = speculative_sample(model, target_hidden, cand_tok, draft_logits, sample)
+        tt, gap = so.target_tok, so.gap
+    elif sample is not None and sample.temperature > 0.0:
         tt, gap = target_sample(model, target_hidden, sample)
     else:
         tt, gap = target_argmax(model, target_hidden)

@@ -1051,3 +1051,80 @@ def test_fused3_commit_rekeys_from_the_three_target_features():
         kk, vv = kv.read(b, n0[b] + j)
         assert np.linalg.norm(kk.numpy() - k1[0]) / np.linalg.norm(k1[0]) < 1e-2
         assert np.linalg.norm(vv.numpy() - v1[0]) / np.linalg.norm(v1[0]) < 1e-2
+
+
+# ---------------------------------------------------------------------------------------
+# speculative sampling with sampled drafts (accept test + residual draw)
+# ---------------------------------------------------------------------------------------
+class _IdentityModel(_IdentityHead):
+    def __init__(self, V):
+        super().__init__(V)
+        self.map = None
+        self.sh = synth.ModelShape(H=V, n_q=1, n_kv=1, d=8, F=8, V=V)
+
+
+def test_speculative_sampling_emits_the_target_distribution_whatever_the_draft_distribution():
+    # the defining property of the rule: x ~ q, kept with min(1, p/q), else a draw from norm(max(0, p - q))
+    # gives a token distributed as p; the acceptance rate is sum_i min(p_i, q_i)
+    lp = [1.0, -0.5, 2.0, 0.25, 1.5, -2.0]
+    lq = [0.5, 1.0, 0.0, 2.0, -1.0, 0.25]
+    V, n = 6, 20000
+    for tau in (1.0, 0.5):
+        cfg = orc.SampleCfg(tau, 99, 5, True)
+        p = np.exp(np.array(lp) / tau)
+        p /= p.sum()
+        q = np.exp(np.array(lq) / tau)
+        q /= q.sum()
+        cand = torch.zeros(n, 2, dtype=torch.int64)
+        for b in range(n):          # one draft draw per sequence, as draft_chain makes it
+            s = torch.tensor(lq, dtype=F64) + tau * orc.gumbel_noise(cfg, b, orc.DRAFT_STREAM, V)
+            cand[b, 1] = orc.argmax_low(s)
+        fq = np.bincount(cand[:, 1].numpy(), minlength=V) / n
+        assert np.all(np.abs(fq - q) < 5 * np.sqrt(q * (1 - q) / n))
+        dl = torch.tensor(lq, dtype=F64).view(1, 1, V).repeat(n, 1, 1)
+        hid = torch.tensor(lp, dtype=torch.bfloat16).view(1, 1, V).repeat(n, 2, 1)
+        so = orc.speculative_sample(_IdentityModel(V), hid, cand, dl, cfg)
+        f = np.bincount(so.target_tok[:, 0].numpy(), minlength=V) / n
+        assert np.all(np.abs(f - p) < 5 * np.sqrt(p * (1 - p) / n)), (tau, f, p)
+        rate = float(so.accepted[:, 0].float().mean())
+        want = float(np.minimum(p, q).sum())
+        assert abs(rate - want) < 5 * math.sqrt(want * (1 - want) / n)
+        # the last slot has no draft: a plain draw from p
+        f1 = np.bincount(so.target_tok[:, 1].numpy(), minlength=V) / n
+        assert np.all(np.abs(f1 - p) < 5 * np.sqrt(p * (1 - p) / n))
+        assert not bool(so.accepted[:, 1].any())
+        # a refused draft token is never drawn again when q exceeds p there
+        refused = ~so.accepted[:, 0]
+        over = torch.tensor(q > p)[cand[:, 1]]
+        assert not bool((so.target_tok[:, 0] == cand[:, 1])[refused & over].any())
+
+
+def test_speculative_sampling_keeps_every_draft_when_draft_and_target_agree():
+    lp = [1.0, -0.5, 2.0, 0.25]
+    V, n = 4, 300
+    cfg = orc.SampleCfg(0.7, 3, 1, True)
+    cand = torch.zeros(n, 2, dtype=torch.int64)
+    cand[:, 1] = torch.arange(n) % V
+    dl = torch.tensor(lp, dtype=F64).view(1, 1, V).repeat(n, 1, 1)
+    hid = torch.tensor(lp, dtype=torch.bfloat16).view(1, 1, V).repeat(n, 2, 1)
+    so = orc.speculative_sample(_IdentityModel(V), hid, cand, dl, cfg)
+    assert bool(so.accepted[:, 0].all()) and torch.equal(so.target_tok[:, 0], cand[:, 1])
+
+
+def test_sampled_chain_drafts_and_their_verification_run_end_to_end():
+    wl = harness.tiny_workload(B=2, K=3, len_lo=6, len_hi=20)
+    case = harness.build_case(wl, poison_tail=False)
+    model = harness.oracle_model(case)
+    smp = orc.SampleCfg(0.8, 21, 2, True)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, sample=smp)
+    g = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    assert d.logits.shape == (2, 3, wl.shape.V) and g.logits is None
+    assert torch.equal(d.hidden[:, 0], g.hidden[:, 0])               # round 1 does not depend on a draw
+    assert not torch.equal(d.cand_tok, g.cand_tok)
+    th = harness.chain_target_hidden(case, d)
+    v = orc.verify(model, th, d.cand_tok, sample=smp, draft_logits=d.logits)
+    for b in range(wl.B):
+        L = int(v.accept_len[b])
+        assert all(int(v.target_tok[b, j]) == int(d.cand_tok[b, j + 1]) for j in range(L))
+        assert L == wl.K or int(v.target_tok[b, L]) != int(d.cand_tok[b, L + 1])
+        assert int(v.recover_tok[b]) == int(v.target_tok[b, L])
