@@ -63,6 +63,14 @@ def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
     return {"total": total, "head_launch": 2 * head, "w_round": w_round, "kv_round": kv_round}
 
 
+def _oracle_sample(args):
+    """Sampling settings of the CPU legs (None: greedy)."""
+    from oracle import specexit_oracle as orc
+    if args.temperature <= 0.0:
+        return None
+    return orc.SampleCfg(args.temperature, 1234, 1, bool(args.sample_drafts))
+
+
 def max_over_ranks(ms_local: float, dist, device) -> float:
     """Replicas share nothing on the data path; the job's time is the slowest rank's."""
     if dist is None:
@@ -204,13 +212,13 @@ def run_reference(args, wl):
     def one():
         kv = harness.oracle_kv(case)
         if wl.mode == synth.CHAIN:
-            d = orc.draft_chain(model, kv, case.f0, case.t0, wl.K)
+            d = orc.draft_chain(model, kv, case.f0, case.t0, wl.K, sample=_oracle_sample(args))
             th = harness.chain_target_hidden(case, d)
-            v = orc.verify(model, th, d.cand_tok, sample=orc.SampleCfg(args.temperature, 1234, 1))
+            v = orc.verify(model, th, d.cand_tok, sample=_oracle_sample(args), draft_logits=d.logits)
         else:
             d = orc.draft_tree(model, kv, case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
             th = harness.tree_target_hidden(case, d)
-            v = orc.verify(model, th, d.cand_tok, d.parent, sample=orc.SampleCfg(args.temperature, 1234, 1))
+            v = orc.verify(model, th, d.cand_tok, d.parent, sample=_oracle_sample(args))
         e = orc.exit_update(cfg, orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path, v.accept_len,
                             v.recover_tok)
         return int((e.accept_len + 1).sum())
@@ -245,6 +253,9 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="verify with stochastic acceptance at this temperature (0 = greedy, the headline setting)")
+    ap.add_argument("--sample-drafts", action="store_true",
+                    help="with --temperature: draw the chain's draft tokens too and verify with the accept "
+                         "test min(1, p/q) and the residual draw")
     ap.add_argument("--layer", choices=["concat", "fused3"], default="concat",
                     help="draft layer: fc over [hidden ; embedding] every round (the headline setting), or "
                          "three-feature fusion in round 1 with [norm(embedding) ; norm(hidden)] as attention input")
@@ -266,7 +277,7 @@ def main():
                                  shape=dataclasses.replace(wl.shape, Vd=args.draft_vocab))
     if args.temperature > 0.0:
         import dataclasses
-        wl = dataclasses.replace(wl, name=f"{wl.name}+tau{args.temperature:g}")
+        wl = dataclasses.replace(wl, name=f"{wl.name}+tau{args.temperature:g}" + ("+sampled-drafts" if args.sample_drafts else ""))
     if args.layer == "fused3":
         import dataclasses
         wl = dataclasses.replace(wl, name=f"{wl.name}+fused3", shape=dataclasses.replace(wl.shape, arch=1))
@@ -290,7 +301,7 @@ def main():
 
     lens, kv, weights, f0, t0 = build_inputs(wl)
     sx = binding.SpecExit(wl.shape, weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
-                          wl.max_nodes, device=str(dev))
+                          wl.max_nodes, device=str(dev), sample_drafts=args.sample_drafts)
     sx.set_kv(kv)
     del weights
     P, H, S = wl.P, wl.shape.H, wl.shape.S
@@ -444,13 +455,13 @@ def main():
         model = harness.oracle_model(case)
         t2 = time.perf_counter()
         if wl.mode == synth.CHAIN:
-            d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+            d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, sample=_oracle_sample(args))
             v = orc.verify(model, harness.chain_target_hidden(case, d), d.cand_tok,
-                           sample=orc.SampleCfg(args.temperature, 1234, 1))
+                           sample=_oracle_sample(args), draft_logits=d.logits)
         else:
             d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
             v = orc.verify(model, harness.tree_target_hidden(case, d), d.cand_tok, d.parent,
-                           sample=orc.SampleCfg(args.temperature, 1234, 1))
+                           sample=_oracle_sample(args))
         orc.exit_update(harness.default_exit_cfg(wl), orc.ExitState.fresh(wl.B), d.slot_signal, d.cand_tok, v.path,
                         v.accept_len, v.recover_tok)
         dt = time.perf_counter() - t2

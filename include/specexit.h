@@ -132,6 +132,7 @@ typedef struct {
   int32_t K;           /* chain length, or tree depth */
   int32_t topk;        /* tree: children per expanded node (<= SX_MAX_TOPK); chain: 1 */
   int32_t max_nodes;   /* tree: nodes kept for verification, root excluded (< SX_MAX_VERIFY_SLOTS) */
+  int32_t sample_drafts; /* chain only, 0 or 1: reserve workspace for sampled drafts, see sx_set_sampling */
 } sx_draft_cfg;
 
 /* Exit rule.  Signal i passes when smoothed_i > thr[i] (SX_DIR_GT) or < thr[i] (SX_DIR_LT),
@@ -246,7 +247,19 @@ sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hi
  * Philox4x32-10 block with counter (i div 4, slot, sequence, offset) and key (seed mod 2^32,
  * seed div 2^32).  Give every iteration its own offset.  temperature = 0 (the state of a new
  * context) is greedy verification.  Host-side state, read when a call is issued; returns
- * SX_ERR_INVALID_ARG for a negative or non-finite temperature. */
+ * SX_ERR_INVALID_ARG for a negative or non-finite temperature.
+ *
+ * Sampled drafts.  In a context created with sx_draft_cfg.sample_drafts = 1 (chain mode, full
+ * draft vocabulary without an id map) a positive temperature makes sx_spec_exit_iter apply the
+ * rule in its general form: draft token k of a sequence is drawn from q = softmax(draft logits /
+ * temperature) (a Gumbel-max draw with slot word 0x40000000 + k - 1); at verify slot j the token
+ * x proposed there is kept when u_j < min(1, p(x) / q(x)), u_j from word 0 of the block with
+ * counter (0, 0x20000000 + j, sequence, offset); otherwise the slot's token is a Gumbel-max draw
+ * over log max(0, p - q) with the noise of slot j; the last slot, which has no draft, draws from
+ * p.  target_tok_d then holds the kept or drawn token of every slot, and acceptance walks it as
+ * before.  For this the draft and target logits of the iteration are written to the workspace
+ * (fp32, (batch * K + batch * (K + 1)) * vocab values) and one extra kernel evaluates the rule in
+ * float64.  The standalone sx_draft_step / sx_verify calls keep deterministic drafts. */
 sx_status sx_set_sampling(sx_ctx *ctx, float temperature, uint64_t seed, uint32_t offset);
 
 /* Exit decision (Section 3.3; Appendix A.1).  Walks path slots 0..accept_len; each slot that

@@ -59,7 +59,8 @@ class KV(C.Structure):
 
 
 class DraftCfg(C.Structure):
-    _fields_ = [("mode", C.c_int32), ("K", C.c_int32), ("topk", C.c_int32), ("max_nodes", C.c_int32)]
+    _fields_ = [("mode", C.c_int32), ("K", C.c_int32), ("topk", C.c_int32), ("max_nodes", C.c_int32),
+                ("sample_drafts", C.c_int32)]
 
 
 class ExitCfg(C.Structure):
@@ -198,7 +199,7 @@ class SpecExit:
     def __init__(self, shape: synth.ModelShape, weights: Dict[str, torch.Tensor], max_batch: int,
                  mode: int, K: int, topk: int = 1, max_nodes: int = 0,
                  act=(ACT_SIGMOID, ACT_SIGMOID, ACT_SIGMOID), device: str = "cuda:0",
-                 max_verify_rows: int = 0):
+                 max_verify_rows: int = 0, sample_drafts: bool = False):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise SxError("a CUDA device is required (there is no CPU fallback)")
@@ -221,7 +222,7 @@ class SpecExit:
                                                        "wgate_up", "wdown", "normf", "head", "target_head")],
                      d2t.data_ptr() if d2t is not None else None,
                      self.w["norm_e"].data_ptr() if "norm_e" in self.w else None)
-        dc = DraftCfg(mode, K, topk, max_nodes)
+        dc = DraftCfg(mode, K, topk, max_nodes, 1 if sample_drafts else 0)
         h = C.c_void_p()
         _check(self.lib.sx_create(C.byref(mc), C.byref(ws), max_batch, C.byref(dc), max_verify_rows,
                                   C.byref(h)), "sx_create")

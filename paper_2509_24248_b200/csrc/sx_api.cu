@@ -17,9 +17,13 @@ struct sx_ctx {
   int max_splits, part_N, head_G, head_rows;
   // workspace offsets (bytes)
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
-      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, total;
+      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, off_dlogits, off_tlogits, total;
   int commit_rows, commit_N;
   SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
+  // set around a draft round whose head samples its token and leaves its logits (sampled drafts)
+  bool round_sampled;
+  SxSample round_smp;
+  SxLogitsOut round_lo;
   // tree sub-offsets relative to off_tree
   size_t t_tok, t_par, t_src, t_row, t_score, t_rmask, t_selcid, t_seltok, t_fidx, t_hidx, t_nmask, t_rsig;
   // optional per-class event timing
@@ -114,6 +118,9 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (m->arch != SX_ARCH_CONCAT && m->arch != SX_ARCH_FUSED3) return SX_ERR_UNSUPPORTED;
   if (m->arch == SX_ARCH_FUSED3 && (!w->norm_e_d || ((uintptr_t)w->norm_e_d & 15))) return SX_ERR_INVALID_ARG;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
+  if (dc->sample_drafts != 0 && dc->sample_drafts != 1) return SX_ERR_INVALID_ARG;
+  if (dc->sample_drafts && (dc->mode != SX_MODE_CHAIN || Vd != m->vocab || w->draft_to_token_d))
+    return SX_ERR_UNSUPPORTED;        // sampled drafts: chain, full draft vocabulary, no id map
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
@@ -192,6 +199,10 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->off_cu = take((size_t)c->commit_rows * (s.arch == SX_ARCH_FUSED3 ? 3 : 2) * s.H * 2);
   c->off_cn = take((size_t)c->commit_rows * s.H * 2);
   c->off_cpart = take((size_t)SX_COMMIT_MAX_SPLITS * c->commit_rows * c->commit_N * 4);
+  if (dc->sample_drafts) {
+    c->off_dlogits = take((size_t)max_batch * dc->K * s.V * 4);
+    c->off_tlogits = take((size_t)max_batch * c->P * s.V * 4);
+  }
   if (s.arch == SX_ARCH_FUSED3) {
     c->off_cu2 = take((size_t)c->commit_rows * 2 * s.H * 2);
     c->off_ctok = take((size_t)c->commit_rows * 4);
@@ -275,7 +286,8 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
 static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S, const bf16 *X, int R, int T, int lse,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
                       int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
-                      const int32_t *map = nullptr, const SxSample *smp = nullptr) {
+                      const int32_t *map = nullptr, const SxSample *smp = nullptr,
+                      SxLogitsOut lo = SxLogitsOut{nullptr, 0}) {
   const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
@@ -286,7 +298,8 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     SxSample sm2;
     if (smp) { sm2 = *smp; sm2.row0 = r0; }
     SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
-                          c->head_rows, &G, z, S, c->sm_count, status, st, smp ? &sm2 : nullptr));
+                          c->head_rows, &G, z, S, c->sm_count, status, st, smp ? &sm2 : nullptr,
+                          SxLogitsOut{lo.out ? lo.out + (size_t)r0 * lo.ld : nullptr, lo.ld}));
     prof_mark(c, cls, false, st);
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
@@ -357,7 +370,8 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
               status, st,
               (prepare_next && !fused3) ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
                            : SxNextInput{nullptr, nullptr, nullptr, 0, 0},
-              c->w.draft_to_token_d));
+              c->w.draft_to_token_d, c->round_sampled ? &c->round_smp : nullptr,
+              c->round_sampled ? c->round_lo : SxLogitsOut{nullptr, 0}));
   return SX_OK;
 }
 
@@ -455,15 +469,41 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
     c->launches += 1;
     // one head launch per round: its merge can write the next input (concat layer only)
     const bool fuse = B <= sx_head_max_rows(1, 0) && c->sh.arch == SX_ARCH_CONCAT;
+    // sampled drafts: every draft head draws its token and leaves its logits for the accept test
+    const bool sampled = c->dc.sample_drafts && c->smp.temp > 0.f;
+    float *dlogits = sampled ? (float *)(ws + c->off_dlogits) : nullptr;
+    const int V = c->sh.V;
     for (int k = 1; k <= K; ++k) {
       const bf16 *feat = (k == 1) ? (const bf16 *)feat0_d : hid;
       SxIndex fi = (k == 1) ? SxIndex{nullptr, 1, 0} : SxIndex{nullptr, K, k - 2};
-      SX_TRY(draft_round(c, kv, k, B, feat, fi, o->cand_tok_d, SxIndex{nullptr, P, k - 1}, nullptr, hid,
-                         SxIndex{nullptr, K, k - 1}, o->cand_tok_d, SxIndex{nullptr, P, k}, nullptr,
-                         o->slot_signal_d, SxIndex{nullptr, P, k - 1}, ws, status_d, st, k > 1 && fuse, k < K && fuse));
+      if (sampled) {
+        c->round_sampled = true;
+        c->round_smp = c->smp;
+        c->round_smp.P = 1;
+        c->round_smp.slot_base = 0x40000000u + (uint32_t)(k - 1);
+        c->round_lo = SxLogitsOut{dlogits + (size_t)(k - 1) * V, (size_t)K * V};
+      }
+      const sx_status rc = draft_round(c, kv, k, B, feat, fi, o->cand_tok_d, SxIndex{nullptr, P, k - 1}, nullptr, hid,
+                                       SxIndex{nullptr, K, k - 1}, o->cand_tok_d, SxIndex{nullptr, P, k}, nullptr,
+                                       o->slot_signal_d, SxIndex{nullptr, P, k - 1}, ws, status_d, st, k > 1 && fuse,
+                                       k < K && fuse);
+      c->round_sampled = false;
+      SX_TRY(rc);
     }
-    SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
-                     K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+    if (sampled) {
+      // target logits of every slot, then the accept test / residual draw, then the usual walk
+      float *tlogits = (float *)(ws + c->off_tlogits);
+      SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, V, V, 0, (const bf16 *)target_hidden_d, B * P, 1, 0, ws,
+                  o->target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
+                  SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr, SxLogitsOut{tlogits, (size_t)V}));
+      sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, o->target_tok_d, status_d, st);
+      sx_launch_accept(B, P, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d, K + 1,
+                       o->recover_tok_d, st);
+      c->launches += 2;
+    } else {
+      SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
+                       K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+    }
   } else {
     if (!o->parent_d) return SX_ERR_INVALID_ARG;
     SxTree t = tree_view(c, ws);

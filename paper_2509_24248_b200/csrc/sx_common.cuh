@@ -101,3 +101,29 @@ struct SxHeadPartial {       // what a CTA leaves behind for the merge, per row
   unsigned long long top[SX_MAX_TOPK];   // packed (value, index), best first; 0 = empty
   float m, l;                            // running max and sum of exp(v - m)
 };
+// ---- counter-based random numbers for sampled verification ---------------------------------
+// Philox4x32 with 10 rounds (Salmon et al., SC'11), written from its definition: two 32x32->64
+// multiplies per round on counter words 0 and 2, the high halves xored with words 1 and 3 and
+// the round key, the key advanced by the Weyl constants between rounds.
+__device__ __forceinline__ void sx_philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                 uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+// standard Gumbel draw from a 32-bit word: u = (top 23 bits + 1/2) / 2^23 lies strictly inside (0, 1)
+__device__ __forceinline__ float sx_gumbel(uint32_t w) {
+  const float u = (float)((w >> 9) * 2u + 1u) * 5.9604644775390625e-8f;      // exact: odd / 2^24
+  // inner logarithm at full accuracy (u close to 1 gives the largest draws, the likely winners);
+  // the outer one only needs absolute accuracy: its argument lies in [6e-8, 17]
+  return -__logf(-logf(u));
+}
+
+

@@ -42,32 +42,8 @@ struct SxTcParams {
   float *z;
   int32_t *status;
   SxSample smp;                  // temp > 0: the argmax epilogue draws a Gumbel-max sample instead
+  SxLogitsOut lo;                // argmax epilogue: also leave the logits in global memory
 };
-
-// ---- counter-based random numbers for sampled verification ---------------------------------
-// Philox4x32 with 10 rounds (Salmon et al., SC'11), written from its definition: two 32x32->64
-// multiplies per round on counter words 0 and 2, the high halves xored with words 1 and 3 and
-// the round key, the key advanced by the Weyl constants between rounds.
-__device__ __forceinline__ void sx_philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
-                                                 uint32_t k1, uint32_t out[4]) {
-#pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
-    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
-  }
-  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
-}
-// standard Gumbel draw from a 32-bit word: u = (top 23 bits + 1/2) / 2^23 lies strictly inside (0, 1)
-__device__ __forceinline__ float sx_gumbel(uint32_t w) {
-  const float u = (float)((w >> 9) * 2u + 1u) * 5.9604644775390625e-8f;      // exact: odd / 2^24
-  // inner logarithm at full accuracy (u close to 1 gives the largest draws, the likely winners);
-  // the outer one only needs absolute accuracy: its argument lies in [6e-8, 17]
-  return -__logf(-logf(u));
-}
 
 // ---- PTX wrappers -------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -339,6 +315,11 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
               for (int j = 0; j < 32; ++j)
                 if (ch * 32 + j < p.R) p.z[(size_t)(ch * 32 + j) * p.S + (n - p.V)] = v[j];
             }
+            if (p.lo.out && in_vocab) {                           // lanes hold consecutive vocabulary rows
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (ch * 32 + j < p.R) p.lo.out[(size_t)(ch * 32 + j) * p.lo.ld + n] = v[j];
+            }
             epi_bar();
             if (ch * 32 + col < p.R) {
               float bv = bestv[ch];
@@ -349,7 +330,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
                 // sampled verification: score = logit + temperature * Gumbel(sequence, slot, token id);
                 // one generator block serves four consecutive token ids
                 const int row = p.smp.row0 + ch * 32 + col;
-                const uint32_t sb = (uint32_t)(row / p.smp.P), sj = (uint32_t)(row % p.smp.P);
+                const uint32_t sb = (uint32_t)(row / p.smp.P), sj = (uint32_t)(row % p.smp.P) + p.smp.slot_base;
 #pragma unroll 2
                 for (int r4 = 0; r4 < 8; ++r4) {
                   uint32_t w[4];
@@ -697,9 +678,10 @@ int sx_head_max_rows(int T, int lse) { return (T == 1 && !lse) ? 256 : 64; }
 
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
-                         cudaStream_t st, const SxSample *smp) {
+                         cudaStream_t st, const SxSample *smp, SxLogitsOut lo) {
   if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T, lse)) return SX_ERR_UNSUPPORTED;
   if (smp && smp->temp > 0.f && (T != 1 || lse || smp->P < 1)) return SX_ERR_UNSUPPORTED;
+  if (lo.out && (T != 1 || lse)) return SX_ERR_UNSUPPORTED;
   SxTcParams p;
   memset(&p, 0, sizeof(p));
   const size_t epi = (T == 1 && !lse) ? SX_ARGMAX_SMEM : SX_TOPK_SMEM;
@@ -708,6 +690,7 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
   p.kb_per_split = p.num_kb;
   p.V = V; p.S = S; p.T = T; p.lse = lse; p.parts = parts; p.part_stride = part_stride; p.z = z; p.status = status;
   if (smp) p.smp = *smp;
+  p.lo = lo;
   CUtensorMap mw, mx;
   if (!get_map(W, Ntot, K, SX_TILE_M, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
   const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;

@@ -801,3 +801,126 @@ void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, c
                            cudaStream_t st) {
   sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)2 * t.NC * sizeof(int), st, t, S, tok0, o);
 }
+
+// ---------------------------------------------------------------------------------------
+// Speculative sampling with sampled drafts: accept test and residual draw of one verify slot.
+// One CTA per (sequence, slot); probabilities are float64 functions of the fp32 logits.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ double sx_block_sum(double v, double *red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];       // same order in every thread
+  return t;
+}
+__device__ __forceinline__ float sx_block_max(float v, double *red) {
+  v = sx_warp_max(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = (double)v;
+  __syncthreads();
+  double t = -INFINITY;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t = fmax(t, red[w]);
+  return (float)t;
+}
+
+__global__ void __launch_bounds__(1024)
+sx_spec_sample_kernel(int P, int V, const float *target_logits, const float *draft_logits, const int32_t *cand_tok,
+                      SxSample smp, int32_t *target_tok, int32_t *status) {
+  __shared__ double red[32];
+  __shared__ int red_i[32];
+  __shared__ int s_accept;
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int row = blockIdx.x, b = row / P, j = row % P, K = P - 1, tid = threadIdx.x;
+  const float *lp = target_logits + (size_t)row * V;
+  const float *lq = (j < K) ? draft_logits + ((size_t)b * K + j) * V : nullptr;
+  const double tau = (double)smp.temp;
+  // maxima, then the two partition sums
+  float mp = -INFINITY, mq = -INFINITY;
+  for (int i = tid; i < V; i += blockDim.x) {
+    mp = fmaxf(mp, lp[i]);
+    if (lq) mq = fmaxf(mq, lq[i]);
+  }
+  mp = sx_block_max(mp, red);
+  mq = sx_block_max(mq, red);
+  double sp = 0.0, sq = 0.0;
+  for (int i = tid; i < V; i += blockDim.x) {
+    sp += exp(((double)lp[i] - (double)mp) / tau);
+    if (lq) sq += exp(((double)lq[i] - (double)mq) / tau);
+  }
+  sp = sx_block_sum(sp, red);
+  sq = sx_block_sum(sq, red);
+  const double lsp = log(sp), lsq = lq ? log(sq) : 0.0;
+  int x = -1;
+  if (j < K) {
+    x = cand_tok[(size_t)b * P + j + 1];
+    if (x < 0 || x >= V) {
+      if (tid == 0) sx_set_status(status, SX_ERR_CAPACITY);
+      x = 0;
+    }
+    if (tid == 0) {
+      // keep the draft token with probability min(1, p(x) / q(x))
+      const double logpx = ((double)lp[x] - (double)mp) / tau - lsp;
+      const double logqx = ((double)lq[x] - (double)mq) / tau - lsq;
+      const double ratio = fmin(1.0, exp(logpx - logqx));
+      uint32_t w[4];
+      sx_philox4x32_10(0u, 0x20000000u + (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+      const double u = ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+      s_accept = (u < ratio) ? 1 : 0;
+    }
+    __syncthreads();
+    if (s_accept) {
+      if (tid == 0) target_tok[row] = x;
+      return;
+    }
+  }
+  // a draw from the normalised max(0, p - q): Gumbel-max over log(p_i - q_i), lower index among equals
+  double best = -INFINITY;
+  int besti = -1;
+  for (int i0 = tid * 4; i0 < V; i0 += blockDim.x * 4) {
+    uint32_t w[4];
+    sx_philox4x32_10((uint32_t)(i0 >> 2), (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = i0 + e;
+      if (i < V) {
+        const double p = exp(((double)lp[i] - (double)mp) / tau - lsp);
+        const double q = lq ? exp(((double)lq[i] - (double)mq) / tau - lsq) : 0.0;
+        const double r = p - q;
+        if (r > 0.0) {
+          const double u = ((double)(w[e] >> 9) + 0.5) * (1.0 / 8388608.0);
+          const double s = log(r) - log(-log(u));
+          if (s > best) { best = s; besti = i; }
+        }
+      }
+    }
+  }
+  // block arg max; among equal scores the lower index
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+    if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+  }
+  __syncthreads();
+  if ((tid & 31) == 0) { red[tid >> 5] = best; red_i[tid >> 5] = besti; }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+      const double ob = red[w];
+      const int oi = red_i[w];
+      if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+    }
+    target_tok[row] = besti >= 0 ? besti : (x >= 0 ? x : 0);      // nothing left to draw from: p == q
+  }
+}
+
+void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
+                           const int32_t *cand_tok, SxSample smp, int32_t *target_tok, int32_t *status,
+                           cudaStream_t st) {
+  sx_launch(sx_spec_sample_kernel, dim3(B * P), dim3(1024), 0, st, P, V, target_logits, draft_logits, cand_tok, smp,
+            target_tok, status);
+}

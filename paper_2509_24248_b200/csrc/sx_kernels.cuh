@@ -112,9 +112,23 @@ struct SxSample {
   float temp;
   uint32_t k0, k1, offset;
   int P, row0;
+  uint32_t slot_base;            // added to the slot word (separates the draft stream from the verify stream)
+};
+// Optional copy of the head's logits: row r of the launch goes to out[r * ld + 0 .. V) (fp32).
+struct SxLogitsOut {
+  float *out;
+  size_t ld;
 };
 // head: per-CTA partial results out[cta][row]; returns the number of CTAs used in *G
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
-                         int32_t *status, cudaStream_t st, const SxSample *smp = nullptr);
+                         int32_t *status, cudaStream_t st, const SxSample *smp = nullptr,
+                         SxLogitsOut lo = SxLogitsOut{nullptr, 0});
+
+// Speculative sampling with sampled drafts, one CTA per (sequence, verify slot): writes the kept draft
+// token or the residual draw of every slot to target_tok [B, P].  target_logits [B * P, V],
+// draft_logits [B, K, V] (K = P - 1), both fp32.
+void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
+                           const int32_t *cand_tok, SxSample smp, int32_t *target_tok, int32_t *status,
+                           cudaStream_t st);
 int sx_head_max_rows(int T, int lse);

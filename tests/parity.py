@@ -145,10 +145,10 @@ def _kv_replay(sx: binding.SpecExit, case: harness.Case):
     return f
 
 
-def make_gpu(case: harness.Case, act=(0, 0, 0)) -> binding.SpecExit:
+def make_gpu(case: harness.Case, act=(0, 0, 0), sample_drafts: bool = False) -> binding.SpecExit:
     wl = case.wl
     sx = binding.SpecExit(wl.shape, case.weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
-                          wl.max_nodes, act=act)
+                          wl.max_nodes, act=act, sample_drafts=sample_drafts)
     sx.set_kv(case.kv)
     return sx
 
@@ -169,11 +169,20 @@ def _set_sampling(sx: binding.SpecExit, sample) -> None:
 
 
 def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, parent, slot_signal,
-                  out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int, sample=None):
+                  out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int, sample=None,
+                  draft_logits=None):
     """verify + exit comparison, shared by chain and tree."""
     B, P = cand_tok.shape
     sampling = sample is not None and sample.temperature > 0.0
-    tt, gap = orc.target_sample(model, th, sample) if sampling else orc.target_argmax(model, th)
+    full_rule = sampling and sample.sample_drafts
+    if full_rule:
+        so = orc.speculative_sample(model, th, cand_tok, draft_logits, sample)
+        tt = so.target_tok
+        # a slot may fall the other way when the accept test is within 1e-4 of its threshold, or
+        # when the two best residual scores (logarithms) lie within 1e-3 of each other
+        gap = torch.where((so.margin < 1e-4) | (so.gap < 1e-3), torch.zeros_like(so.gap), torch.ones_like(so.gap))
+    else:
+        tt, gap = orc.target_sample(model, th, sample) if sampling else orc.target_argmax(model, th)
     g_tt = out["target_tok_d"].cpu().to(torch.int64)
     forced = {}
     for b in range(B):
@@ -185,7 +194,7 @@ def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, 
                 else:
                     raise ParityError(f"target token b={b} slot={j}: gpu {int(g_tt[b, j])} vs {int(tt[b, j])} "
                                       f"gap {float(gap[b, j]):.3e}")
-    v = orc.verify(model, th, cand_tok, parent, forced_target=forced, sample=sample)
+    v = orc.verify(model, th, cand_tok, parent, forced_target=forced, sample=sample, draft_logits=draft_logits)
     g_L = out["accept_len_d"].cpu().to(torch.int64)
     g_path = out["path_d"].cpu().to(torch.int64)
     g_rec = out["recover_tok_d"].cpu().to(torch.int64)
@@ -252,10 +261,12 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     rep = Report()
     cfg = cfg or harness.default_exit_cfg(wl)
     model = harness.oracle_model(case, act=act)
-    d0 = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K)
+    sampled_drafts = sample is not None and sample.sample_drafts and sample.temperature > 0.0
+    dsample = sample if sampled_drafts else None
+    d0 = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, sample=dsample)
     th = harness.chain_target_hidden(case, d0)             # inputs of the verify step, fixed from here
     own = sx is None
-    sx = sx or make_gpu(case, act)
+    sx = sx or make_gpu(case, act, sample_drafts=sampled_drafts)
     out = sx.new_outputs(wl.B)
     gst = sx.new_state(wl.B)
     state0 = state0 or orc.ExitState.fresh(wl.B, wl.shape.S)
@@ -289,7 +300,7 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
         return torch.stack([g_hid[r.b, r.slot - lens[r.b]].to(torch.float64) for r in rows])
 
     d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, chooser=chooser,
-                        before_round=before_round, head_input=head_input)
+                        before_round=before_round, head_input=head_input, sample=dsample)
     if not torch.equal(g_tok, d.cand_tok):
         raise ParityError("draft tokens differ after adopting near-ties")
     rep.free_running_hidden_rel = max(_rel_l2(g_hid[b, wl.K - 1].to(torch.float64), d0.hidden[b, wl.K - 1])
@@ -302,7 +313,7 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     if not torch.equal(out["parent_d"].cpu().to(torch.int64), want_par):
         raise ParityError("chain parents")
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, None, d.slot_signal, out,
-                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample)
+                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample, draft_logits=d.logits)
     if own:
         sx.close()
     return rep

@@ -84,3 +84,60 @@ def test_set_sampling_rejects_bad_temperatures():
     assert sx.lib.sx_set_sampling(sx.h, float("nan"), 0, 0) == -1
     assert sx.lib.sx_set_sampling(sx.h, float("inf"), 0, 0) == -1
     sx.close()
+
+
+# ---------------------------------------------------------------------------------------
+# sampled drafts: the rule in its general form (accept test min(1, p/q), residual draw)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("tau,seed,offset,scale", [(0.3, 1, 0, 30.0), (1.0, 2, 5, 30.0), (1.0, (7 << 32) + 1, 9, 100.0),
+                                                   (2.5, 3, 1, 100.0)])
+def test_chain_sampled_drafts(tau, seed, offset, scale):
+    wl = harness.tiny_workload(B=4, K=5, len_lo=5, len_hi=50, sigma_lo=0.0, sigma_hi=0.02)
+    case = _peaked(harness.build_case(wl), scale)
+    rep = parity.run_chain(case, sample=orc.SampleCfg(tau, seed, offset, True))
+    print("tau", tau, "accept:", rep.accept_len, "exempt:", rep.exempt)
+
+
+def test_sampled_drafts_are_all_kept_when_target_and_draft_distributions_coincide():
+    # noise-free target hiddens: p == q at every slot, so the accept test passes whatever the temperature
+    wl = harness.tiny_workload(B=4, K=4, len_lo=5, len_hi=50, sigma_lo=0.0, sigma_hi=0.0)
+    case = _peaked(harness.build_case(wl), 60.0)
+    cfg = harness.default_exit_cfg(wl, thr=(2.0, 0.0, 0.0))          # the exit rule never fires
+    sx = parity.make_gpu(case, sample_drafts=True)
+    for tau in (0.05, 1.0, 20.0):
+        for it in range(3):
+            rep = parity.run_chain(case, cfg, sx=sx, sample=orc.SampleCfg(tau, 31, it, True))
+            assert rep.accept_len == [wl.K] * wl.B
+    # zero temperature on the same context is plain greedy verification
+    parity.run_chain(case, cfg, sx=sx)
+    # with noisy target hiddens some drafts are refused
+    sx.close()
+    wl2 = harness.tiny_workload(B=4, K=4, len_lo=5, len_hi=50, sigma_lo=0.5, sigma_hi=1.0)
+    case2 = _peaked(harness.build_case(wl2), 60.0)
+    cfg2 = harness.default_exit_cfg(wl2, thr=(2.0, 0.0, 0.0))
+    sx = parity.make_gpu(case2, sample_drafts=True)
+    n = 0
+    for it in range(5):
+        n += sum(parity.run_chain(case2, cfg2, sx=sx, sample=orc.SampleCfg(0.5, 32, it, True)).accept_len)
+    sx.close()
+    print("accepted with noisy targets:", n, "of", 5 * wl2.B * wl2.K)
+    assert 0 < n < 5 * wl2.B * wl2.K
+
+
+def test_sampled_drafts_on_an_odd_vocabulary_and_the_three_feature_layer():
+    sh = synth.ModelShape(H=128, n_q=8, n_kv=1, d=16, F=200, V=333, page=16, arch=1)
+    wl = synth.Workload("sd", sh, B=3, mode=synth.CHAIN, K=3, len_lo=3, len_hi=90, seed=71, sigma_lo=0.0, sigma_hi=0.05)
+    case = _peaked(harness.build_case(wl), 40.0)
+    parity.run_chain(case, sample=orc.SampleCfg(0.8, 5, 3, True))
+
+
+def test_sampled_drafts_need_chain_mode_and_a_full_draft_vocabulary():
+    from paper_2509_24248_b200 import binding
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
+    wl = synth.Workload("sdt", sh, B=1, mode=synth.TREE, K=3, topk=2, max_nodes=5, len_lo=9, len_hi=9, seed=72)
+    with pytest.raises(binding.SxError):
+        parity.make_gpu(harness.build_case(wl), sample_drafts=True)
+    sh2 = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16, Vd=100)
+    wl2 = synth.Workload("sdv", sh2, B=1, mode=synth.CHAIN, K=3, len_lo=9, len_hi=9, seed=73)
+    with pytest.raises(binding.SxError):
+        parity.make_gpu(harness.build_case(wl2), sample_drafts=True)

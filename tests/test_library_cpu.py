@@ -43,7 +43,7 @@ def test_struct_layouts_match_header():
     from paper_2509_24248_b200 import binding as b
     assert ctypes.sizeof(b.ModelCfg) == 4 * 15
     assert ctypes.sizeof(b.Weights) == 8 * 13
-    assert ctypes.sizeof(b.DraftCfg) == 16
+    assert ctypes.sizeof(b.DraftCfg) == 20
     assert ctypes.sizeof(b.IterOut) == 8 * 18
     assert b.ExitCfg.split_bitmap_d.offset % 8 == 0
 
