@@ -258,8 +258,7 @@ sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hi
  * over log max(0, p - q) with the noise of slot j; the last slot, which has no draft, draws from
  * p.  target_tok_d then holds the kept or drawn token of every slot, and acceptance walks it as
  * before.  For this the draft and target logits of the iteration are written to the workspace
- * (fp32, (batch * K + batch * (K + 1)) * vocab values) and one extra kernel evaluates the rule in
- * float64.  The standalone sx_draft_step / sx_verify calls keep deterministic drafts. */
+ * (fp32, (batch * K + batch * (K + 1)) * vocab values) and three small kernels evaluate the rule.  The standalone sx_draft_step / sx_verify calls keep deterministic drafts. */
 sx_status sx_set_sampling(sx_ctx *ctx, float temperature, uint64_t seed, uint32_t offset);
 
 /* Exit decision (Section 3.3; Appendix A.1).  Walks path slots 0..accept_len; each slot that

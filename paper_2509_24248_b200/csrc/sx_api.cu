@@ -17,7 +17,7 @@ struct sx_ctx {
   int max_splits, part_N, head_G, head_rows;
   // workspace offsets (bytes)
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
-      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, off_dlogits, off_tlogits, total;
+      off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, off_dlogits, off_tlogits, off_spec, total;
   int commit_rows, commit_N;
   SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
   // set around a draft round whose head samples its token and leaves its logits (sampled drafts)
@@ -202,6 +202,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (dc->sample_drafts) {
     c->off_dlogits = take((size_t)max_batch * dc->K * s.V * 4);
     c->off_tlogits = take((size_t)max_batch * c->P * s.V * 4);
+    c->off_spec = take(sx_spec_sample_ws_bytes(max_batch * c->P));
   }
   if (s.arch == SX_ARCH_FUSED3) {
     c->off_cu2 = take((size_t)c->commit_rows * 2 * s.H * 2);
@@ -496,10 +497,11 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
       SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, V, V, 0, (const bf16 *)target_hidden_d, B * P, 1, 0, ws,
                   o->target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
                   SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr, SxLogitsOut{tlogits, (size_t)V}));
-      sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, o->target_tok_d, status_d, st);
+      sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, ws + c->off_spec, c->sm_count,
+                            o->target_tok_d, status_d, st);
       sx_launch_accept(B, P, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d, K + 1,
                        o->recover_tok_d, st);
-      c->launches += 2;
+      c->launches += 4;
     } else {
       SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
                        K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));

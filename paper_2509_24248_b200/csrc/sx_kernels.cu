@@ -826,101 +826,173 @@ __device__ __forceinline__ float sx_block_max(float v, double *red) {
   return (float)t;
 }
 
-__global__ void __launch_bounds__(1024)
-sx_spec_sample_kernel(int P, int V, const float *target_logits, const float *draft_logits, const int32_t *cand_tok,
-                      SxSample smp, int32_t *target_tok, int32_t *status) {
+// Slice s of a row covers token ids [s * len, min(V, (s + 1) * len)), len a multiple of 4.
+struct SxSpecPartial {
+  double mp, sp, mq, sq;      // slice maxima and sums of exp((logit - max) / tau), target and draft
+  double best;                // best residual score of the slice (phase 2)
+  int besti, accept;
+};
+
+// Phase 1: per (row, slice) the pieces of the two log-partition sums.
+__global__ void __launch_bounds__(512)
+sx_spec_partials_kernel(int P, int V, int len, const float *target_logits, const float *draft_logits, float temp,
+                        SxSpecPartial *parts) {
   __shared__ double red[32];
-  __shared__ int red_i[32];
-  __shared__ int s_accept;
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int row = blockIdx.x, b = row / P, j = row % P, K = P - 1, tid = threadIdx.x;
+  const int row = blockIdx.x, sl = blockIdx.y, S = gridDim.y, b = row / P, j = row % P, K = P - 1, tid = threadIdx.x;
+  const int i0 = sl * len, i1 = min(V, i0 + len);
   const float *lp = target_logits + (size_t)row * V;
   const float *lq = (j < K) ? draft_logits + ((size_t)b * K + j) * V : nullptr;
-  const double tau = (double)smp.temp;
-  // maxima, then the two partition sums
+  // the exponentials are fp32 (their rounding is below the fp32 logits' own), the sums float64
+  const float inv_tau = 1.0f / temp;
   float mp = -INFINITY, mq = -INFINITY;
-  for (int i = tid; i < V; i += blockDim.x) {
+  for (int i = i0 + tid; i < i1; i += blockDim.x) {
     mp = fmaxf(mp, lp[i]);
     if (lq) mq = fmaxf(mq, lq[i]);
   }
   mp = sx_block_max(mp, red);
   mq = sx_block_max(mq, red);
   double sp = 0.0, sq = 0.0;
-  for (int i = tid; i < V; i += blockDim.x) {
-    sp += exp(((double)lp[i] - (double)mp) / tau);
-    if (lq) sq += exp(((double)lq[i] - (double)mq) / tau);
+  for (int i = i0 + tid; i < i1; i += blockDim.x) {
+    sp += (double)expf((lp[i] - mp) * inv_tau);
+    if (lq) sq += (double)expf((lq[i] - mq) * inv_tau);
   }
   sp = sx_block_sum(sp, red);
   sq = sx_block_sum(sq, red);
-  const double lsp = log(sp), lsq = lq ? log(sq) : 0.0;
-  int x = -1;
-  if (j < K) {
-    x = cand_tok[(size_t)b * P + j + 1];
-    if (x < 0 || x >= V) {
-      if (tid == 0) sx_set_status(status, SX_ERR_CAPACITY);
-      x = 0;
-    }
-    if (tid == 0) {
-      // keep the draft token with probability min(1, p(x) / q(x))
-      const double logpx = ((double)lp[x] - (double)mp) / tau - lsp;
-      const double logqx = ((double)lq[x] - (double)mq) / tau - lsq;
-      const double ratio = fmin(1.0, exp(logpx - logqx));
-      uint32_t w[4];
-      sx_philox4x32_10(0u, 0x20000000u + (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
-      const double u = ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
-      s_accept = (u < ratio) ? 1 : 0;
-    }
-    __syncthreads();
-    if (s_accept) {
-      if (tid == 0) target_tok[row] = x;
-      return;
-    }
-  }
-  // a draw from the normalised max(0, p - q): Gumbel-max over log(p_i - q_i), lower index among equals
-  double best = -INFINITY;
-  int besti = -1;
-  for (int i0 = tid * 4; i0 < V; i0 += blockDim.x * 4) {
-    uint32_t w[4];
-    sx_philox4x32_10((uint32_t)(i0 >> 2), (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int i = i0 + e;
-      if (i < V) {
-        const double p = exp(((double)lp[i] - (double)mp) / tau - lsp);
-        const double q = lq ? exp(((double)lq[i] - (double)mq) / tau - lsq) : 0.0;
-        const double r = p - q;
-        if (r > 0.0) {
-          const double u = ((double)(w[e] >> 9) + 0.5) * (1.0 / 8388608.0);
-          const double s = log(r) - log(-log(u));
-          if (s > best) { best = s; besti = i; }
-        }
-      }
-    }
-  }
-  // block arg max; among equal scores the lower index
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-    if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
-  }
-  __syncthreads();
-  if ((tid & 31) == 0) { red[tid >> 5] = best; red_i[tid >> 5] = besti; }
-  __syncthreads();
   if (tid == 0) {
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
-      const double ob = red[w];
-      const int oi = red_i[w];
-      if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
-    }
-    target_tok[row] = besti >= 0 ? besti : (x >= 0 ? x : 0);      // nothing left to draw from: p == q
+    SxSpecPartial &o = parts[(size_t)row * S + sl];
+    o.mp = (double)mp; o.sp = sp; o.mq = (double)mq; o.sq = sq;
   }
 }
 
+// Phase 2: every CTA of a row rebuilds the row's normalisers (slice order, so all agree), takes the
+// accept test, and - for a refused or draft-less slot - leaves the best residual score of its slice.
+__global__ void __launch_bounds__(512)
+sx_spec_draw_kernel(int P, int V, int len, const float *target_logits, const float *draft_logits,
+                    const int32_t *cand_tok, SxSample smp, SxSpecPartial *parts, int32_t *status) {
+  __shared__ double red[32];
+  __shared__ int red_i[32];
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int row = blockIdx.x, sl = blockIdx.y, S = gridDim.y, b = row / P, j = row % P, K = P - 1, tid = threadIdx.x;
+  const float *lp = target_logits + (size_t)row * V;
+  const float *lq = (j < K) ? draft_logits + ((size_t)b * K + j) * V : nullptr;
+  const double tau = (double)smp.temp;
+  SxSpecPartial *pr = parts + (size_t)row * S;
+  double mp = -INFINITY, mq = -INFINITY;
+  for (int s = 0; s < S; ++s) {
+    if (pr[s].sp > 0.0) mp = fmax(mp, pr[s].mp);
+    if (pr[s].sq > 0.0) mq = fmax(mq, pr[s].mq);
+  }
+  double sp = 0.0, sq = 0.0;
+  for (int s = 0; s < S; ++s) {
+    if (pr[s].sp > 0.0) sp += pr[s].sp * exp((pr[s].mp - mp) / tau);
+    if (pr[s].sq > 0.0) sq += pr[s].sq * exp((pr[s].mq - mq) / tau);
+  }
+  const double lsp = log(sp), lsq = lq ? log(sq) : 0.0;
+  int x = -1, accept = 0;
+  if (j < K) {
+    x = cand_tok[(size_t)b * P + j + 1];
+    if (x < 0 || x >= V) {
+      if (tid == 0 && sl == 0) sx_set_status(status, SX_ERR_CAPACITY);
+      x = 0;
+    }
+    // keep the draft token with probability min(1, p(x) / q(x)); every thread takes the same decision
+    const double logpx = ((double)lp[x] - mp) / tau - lsp;
+    const double logqx = ((double)lq[x] - mq) / tau - lsq;
+    const double ratio = fmin(1.0, exp(logpx - logqx));
+    uint32_t w[4];
+    sx_philox4x32_10(0u, 0x20000000u + (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+    const double u = ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+    accept = (u < ratio) ? 1 : 0;
+  }
+  double best = -INFINITY;
+  int besti = -1;
+  if (!accept) {
+    // a draw from the normalised max(0, p - q): Gumbel-max over log(p_i - q_i), lower index among equals
+    const int i0 = sl * len, i1 = min(V, i0 + len);
+    const float inv_tau = 1.0f / smp.temp, fmp = (float)mp, fmq = (float)mq, flsp = (float)lsp, flsq = (float)lsq;
+    for (int a = i0 + tid * 4; a < i1; a += blockDim.x * 4) {
+      uint32_t w[4];
+      sx_philox4x32_10((uint32_t)(a >> 2), (uint32_t)j, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int i = a + e;
+        if (i < i1) {
+          const float p = expf((lp[i] - fmp) * inv_tau - flsp);
+          const float q = lq ? expf((lq[i] - fmq) * inv_tau - flsq) : 0.f;
+          const float r = p - q;
+          if (r > 0.f) {
+            const float u = (float)((w[e] >> 9) * 2u + 1u) * 5.9604644775390625e-8f;
+            const double sc = (double)(logf(r) - logf(-logf(u)));
+            if (sc > best) { best = sc; besti = i; }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+      if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+    }
+    if ((tid & 31) == 0) { red[tid >> 5] = best; red_i[tid >> 5] = besti; }
+    __syncthreads();
+    if (tid == 0) {
+      best = -INFINITY;
+      besti = -1;
+      for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+        const double ob = red[w];
+        const int oi = red_i[w];
+        if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+      }
+    }
+  }
+  if (tid == 0) {
+    pr[sl].best = best;
+    pr[sl].besti = besti;
+    pr[sl].accept = accept;
+  }
+}
+
+// Phase 3: the slot's token - the kept draft token, or the best residual score over the slices.
+__global__ void sx_spec_pick_kernel(int P, int V, int S, int rows, const int32_t *cand_tok, const SxSpecPartial *parts,
+                                    int32_t *target_tok) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const int b = row / P, j = row % P;
+  const SxSpecPartial *pr = parts + (size_t)row * S;
+  int x = (j < P - 1) ? cand_tok[(size_t)b * P + j + 1] : -1;
+  if (j < P - 1 && (x < 0 || x >= V)) x = 0;
+  if (pr[0].accept) { target_tok[row] = x; return; }
+  double best = -INFINITY;
+  int besti = -1;
+  for (int s = 0; s < S; ++s)                       // slices in index order: a strict compare keeps the lower index
+    if (pr[s].besti >= 0 && (besti < 0 || pr[s].best > best)) { best = pr[s].best; besti = pr[s].besti; }
+  target_tok[row] = besti >= 0 ? besti : (x >= 0 ? x : 0);      // nothing left to draw from: p == q
+}
+
+int sx_spec_sample_slices(int rows, int V, int sm_count) {
+  int S = (2 * sm_count + rows - 1) / rows;
+  const int cap = (V + 2047) / 2048;
+  if (S > cap) S = cap;
+  if (S > SX_SPEC_MAX_SLICES) S = SX_SPEC_MAX_SLICES;
+  return S < 1 ? 1 : S;
+}
+size_t sx_spec_sample_ws_bytes(int rows) { return (size_t)rows * SX_SPEC_MAX_SLICES * sizeof(SxSpecPartial); }
+
 void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
-                           const int32_t *cand_tok, SxSample smp, int32_t *target_tok, int32_t *status,
-                           cudaStream_t st) {
-  sx_launch(sx_spec_sample_kernel, dim3(B * P), dim3(1024), 0, st, P, V, target_logits, draft_logits, cand_tok, smp,
-            target_tok, status);
+                           const int32_t *cand_tok, SxSample smp, void *parts_ws, int sm_count, int32_t *target_tok,
+                           int32_t *status, cudaStream_t st) {
+  const int rows = B * P, S = sx_spec_sample_slices(rows, V, sm_count);
+  const int len = (((V + S - 1) / S + 3) / 4) * 4;
+  SxSpecPartial *parts = (SxSpecPartial *)parts_ws;
+  sx_launch(sx_spec_partials_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits, smp.temp,
+            parts);
+  sx_launch(sx_spec_draw_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits, cand_tok, smp,
+            parts, status);
+  sx_launch(sx_spec_pick_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, P, V, S, rows, cand_tok, parts, target_tok);
 }

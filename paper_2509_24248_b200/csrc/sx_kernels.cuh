@@ -125,10 +125,13 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
                          int32_t *status, cudaStream_t st, const SxSample *smp = nullptr,
                          SxLogitsOut lo = SxLogitsOut{nullptr, 0});
 
-// Speculative sampling with sampled drafts, one CTA per (sequence, verify slot): writes the kept draft
-// token or the residual draw of every slot to target_tok [B, P].  target_logits [B * P, V],
-// draft_logits [B, K, V] (K = P - 1), both fp32.
+// Speculative sampling with sampled drafts: writes the kept draft token or the residual draw of every
+// verify slot to target_tok [B, P].  target_logits [B * P, V], draft_logits [B, K, V] (K = P - 1), both
+// fp32.  Three small launches (partition sums per slice, accept test + best residual score per slice,
+// pick); parts_ws holds sx_spec_sample_ws_bytes(B * P) bytes.
+#define SX_SPEC_MAX_SLICES 64
+size_t sx_spec_sample_ws_bytes(int rows);
 void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
-                           const int32_t *cand_tok, SxSample smp, int32_t *target_tok, int32_t *status,
-                           cudaStream_t st);
+                           const int32_t *cand_tok, SxSample smp, void *parts_ws, int sm_count, int32_t *target_tok,
+                           int32_t *status, cudaStream_t st);
 int sx_head_max_rows(int T, int lse);
