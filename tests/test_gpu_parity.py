@@ -225,3 +225,26 @@ def test_errors_are_reported_not_fatal():
     sx.status.zero_()
     # the context is still usable
     parity.run_chain(case, sx=sx)
+
+
+def test_chain_of_maximum_length():
+    """K = 63 draft rounds (64 verify slots): the limit of the per-sequence slot masks."""
+    wl = _wl(B=2, K=63, len_lo=1, len_hi=30, sigma_lo=0.0, sigma_hi=0.05)
+    rep = parity.run_chain(harness.build_case(wl))
+    print("K=63 accept:", rep.accept_len, "exempt:", len(rep.exempt))
+
+
+@pytest.mark.parametrize("topk,depth", [(8, 8), (7, 10), (1, 64)])
+def test_tree_at_the_row_and_slot_limits(topk, depth):
+    """1 + topk (depth - 1) drafted rows per sequence up to the 64-row limit, 63 kept nodes (64 slots)."""
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
+    rows = 1 + topk * (depth - 1)
+    assert rows <= 64
+    nodes = min(63, topk + (depth - 1) * topk * topk)
+    wl = synth.Workload("tmax", sh, B=2, mode=synth.TREE, K=depth, topk=topk, max_nodes=nodes, len_lo=3, len_hi=40,
+                        seed=81, sigma_lo=0.0, sigma_hi=0.1)
+    case = harness.build_case(wl)
+    w = dict(case.weights)
+    w["head"] = (w["head"].to(torch.float32) * 20.0).to(torch.bfloat16)
+    rep = parity.run_tree(dataclasses.replace(case, weights=w))
+    print("tree", topk, depth, "accept:", rep.accept_len, "exempt:", len(rep.exempt))
