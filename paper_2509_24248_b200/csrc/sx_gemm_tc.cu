@@ -667,7 +667,8 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
     CUtensorMap mw, mx;
     if (!get_map(W, N, K, SX_TILE_M, &mw) || !get_map(X + (size_t)r0 * K, rc, K, p.nmma, &mx)) return SX_ERR_CUDA;
     const int items = p.num_tiles * p.splits;
-    const int grid = items < sm_count ? items : sm_count;
+    const int per_cta = (items + sm_count - 1) / sm_count;          // the same number of items for every CTA
+    const int grid = (items + per_cta - 1) / per_cta;
     if (sx_launch(sx_tc_gemm_kernel<false>, dim3(grid), dim3(192), smem_bytes(p, 0), st, mw, mx, p) != cudaSuccess)
       return SX_ERR_CUDA;
   }
@@ -693,7 +694,10 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
   p.lo = lo;
   CUtensorMap mw, mx;
   if (!get_map(W, Ntot, K, SX_TILE_M, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
-  const int grid = p.num_tiles < sm_count ? p.num_tiles : sm_count;
+  // every CTA gets the same number of tiles (no CTA is left alone with one more 1 MB tile at the end):
+  // with w = ceil(tiles / SMs) tiles per CTA, ceil(tiles / w) CTAs cover the matrix
+  const int per_cta = (p.num_tiles + sm_count - 1) / sm_count;
+  const int grid = (p.num_tiles + per_cta - 1) / per_cta;
   if (sx_launch(sx_tc_gemm_kernel<true>, dim3(grid), dim3(192), smem_bytes(p, epi), st, mw, mx, p) != cudaSuccess)
     return SX_ERR_CUDA;
   *G = grid;
