@@ -210,10 +210,12 @@ int64_t sx_launch_count(const sx_ctx *ctx);
  * (r - 2) * topk + j, attending to the cache plus the drafted rows whose bit is set in
  * row_mask_d[row] (bit i = drafted row i of the same sequence; the own bit included).
  * The rows' K/V are written into the cache at those slots; cache_len is not advanced.
- *   feat_d        [R, H] bf16   hidden state of the previous position
+ *   feat_d        [R, H] bf16   hidden state of the previous position (SX_ARCH_FUSED3, round 1:
+ *                               [R, 3H], the three target features)
  *   tok_d         [R]           token at this position
  *   row_mask_d    [R] or NULL   tree rounds >= 2 only
- *   hidden_out_d  [R, H] bf16   final-normed hidden (feeds the head and the next round)
+ *   hidden_out_d  [R, H] bf16   final-normed hidden (feeds the head and the next round);
+ *                               SX_ARCH_FUSED3: the layer output before the final norm
  *   tok_out_d     [R, topk]     chain: argmax (topk = 1); tree: the topk best ids, best first,
  *                               lower id first among equal logits
  *   logp_out_d    [R, topk]     tree: log-probabilities of those ids; may be NULL in chain mode
@@ -275,7 +277,9 @@ sx_status sx_exit_update(sx_ctx *ctx, int32_t batch, int32_t P, const sx_exit_cf
 
 /* The whole iteration in one enqueue: all draft rounds, (tree) candidate selection and
  * layout, verification and the exit decision.  target_hidden_d [B, P, H] stands in for the
- * target trunk's output at the verify slots; it is read only after the draft has finished. */
+ * target trunk's output at the verify slots; it is read only after the draft has finished.
+ * feat0_d is [B, H] bf16, the target feature of the last accepted token ([B, 3H] with
+ * SX_ARCH_FUSED3); tok0_d [B] is that token. */
 sx_status sx_spec_exit_iter(sx_ctx *ctx, const sx_kv *kv, const sx_exit_cfg *cfg,
                             const sx_exit_state *state, const void *feat0_d, const int32_t *tok0_d,
                             const void *target_hidden_d, const sx_iter_out *out, void *ws_d,
