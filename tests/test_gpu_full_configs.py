@@ -45,3 +45,16 @@ def test_chain_config1_with_the_three_feature_layer_and_a_32k_draft_vocabulary()
     print(f"C1/fused3/Vd=32768: accept_len {rep.accept_len} exempt {rep.exempt} "
           f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
     assert len(rep.exempt) <= 2
+
+
+@pytest.mark.parametrize("sample_drafts", [False, True])
+def test_chain_config1_with_stochastic_acceptance(sample_drafts):
+    """C1's shapes with speculative sampling at temperature 1: the verify head's draws over the
+    151936-token vocabulary (deterministic drafts), and the accept test with the residual draw
+    (sampled drafts)."""
+    from oracle import specexit_oracle as orc
+    wl = synth.workload("C1")
+    rep = parity.run_chain(harness.build_case(wl, poison_tail=True),
+                           sample=orc.SampleCfg(1.0, 20250924, 3, sample_drafts))
+    print(f"C1/tau=1/sampled drafts {sample_drafts}: accept_len {rep.accept_len} exempt {rep.exempt}")
+    assert len(rep.exempt) <= 2
