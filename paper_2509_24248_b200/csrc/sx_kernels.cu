@@ -753,14 +753,16 @@ void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok
 __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_iter_out o) {
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  extern __shared__ int sx_tl[];           // kept[NC], slot_of[NC]
+  extern __shared__ int sx_tl[];           // kept[NC], slot_of[NC], score[NC]
   const int b = blockIdx.x, tid = threadIdx.x;
   const int NC = t.NC, P = 1 + t.max_nodes, T = t.T;
   int *kept = sx_tl, *slot_of = sx_tl + NC;
+  float *csc = reinterpret_cast<float *>(sx_tl + 2 * NC);
   const int32_t *ctok = t.cand_tok + (size_t)b * NC, *cpar = t.cand_parent + (size_t)b * NC;
   const int32_t *csrc = t.cand_src_row + (size_t)b * NC, *crow = t.cand_row + (size_t)b * NC;
-  const float *csc = t.cand_score + (size_t)b * NC;
-  for (int i = tid; i < NC; i += blockDim.x) {
+  for (int i = tid; i < NC; i += blockDim.x) csc[i] = t.cand_score[(size_t)b * NC + i];
+  __syncthreads();
+  for (int i = tid; i < NC; i += blockDim.x) {      // rank of candidate i among all scores (shared-memory broadcast reads)
     const float s = csc[i];
     int rank = 0;
     for (int k = 0; k < NC; ++k) rank += sx_better(csc[k], k, s, i) ? 1 : 0;
@@ -799,7 +801,7 @@ __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_i
 
 void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
                            cudaStream_t st) {
-  sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)2 * t.NC * sizeof(int), st, t, S, tok0, o);
+  sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)3 * t.NC * sizeof(int), st, t, S, tok0, o);
 }
 
 // ---------------------------------------------------------------------------------------
