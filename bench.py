@@ -253,6 +253,9 @@ def main():
     ap.add_argument("--impl", default="b200")
     ap.add_argument("--temperature", type=float, default=0.0,
                     help="verify with stochastic acceptance at this temperature (0 = greedy, the headline setting)")
+    ap.add_argument("--weights", choices=["tiled", "rowmajor"], default="tiled",
+                    help="layout of the GEMM weights in HBM: repacked tile by tile at load (sx_tile_weight) or "
+                         "row-major as handed in")
     ap.add_argument("--sample-drafts", action="store_true",
                     help="with --temperature: draw the chain's draft tokens too and verify with the accept "
                          "test min(1, p/q) and the residual draw")
@@ -301,7 +304,8 @@ def main():
 
     lens, kv, weights, f0, t0 = build_inputs(wl)
     sx = binding.SpecExit(wl.shape, weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
-                          wl.max_nodes, device=str(dev), sample_drafts=args.sample_drafts)
+                          wl.max_nodes, device=str(dev), sample_drafts=args.sample_drafts,
+                          tiled=args.weights == "tiled")
     sx.set_kv(kv)
     del weights
     P, H, S = wl.P, wl.shape.H, wl.shape.S
@@ -434,6 +438,7 @@ def main():
         "ms_per_step_percentiles": {"p10": pct(0.10), "p50": pct(0.50), "p90": pct(0.90)},
         "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree",
                    "cached_tokens": int(sum(int(n) for n in lens)),
+                   "weights": "tiled at load (sx_tile_weight)" if args.weights == "tiled" else "row-major",
                    "l2": "no flush: each iteration streams %.2f GB of weights and KV, far beyond the 126 MB L2"
                          % (ab["total"] / 1e9)},
         "step_roofline": {"bytes_per_iteration": ab["total"], "hbm_bound_ms": ab["total"] / (peak * 1e9) * 1e3,

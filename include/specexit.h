@@ -79,6 +79,9 @@ typedef struct {
                                        draft vocabulary (draft_vocab < vocab) scores draft ids
                                        0..draft_vocab-1, see sx_weights.draft_to_token_d */
   int32_t arch;                     /* SX_ARCH_CONCAT (0) or SX_ARCH_FUSED3, see below */
+  int32_t tiled_weights;            /* 0: the GEMM weights are row-major [out, in]; 1: they were repacked with
+                                       sx_tile_weight (fc, wqkv, wo, wgate_up, wdown, head, target_head; the
+                                       embedding table and the gains stay as they are) */
 } sx_model_cfg;
 
 /* Shape of the draft layer.
@@ -235,6 +238,16 @@ sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hi
                     int32_t *accept_len_d, int32_t *path_d, int32_t path_stride,
                     int32_t *recover_tok_d, void *ws_d, size_t ws_bytes, int32_t *status_d,
                     void *stream);
+
+/* Weight layout for the GEMM kernels (a deployment choice; the paper describes no kernels).  A
+ * row-major [N, K] matrix is read in boxes of 128 rows x 64 columns, 128 pieces of 128 bytes that lie
+ * K * 2 bytes apart; stored tile by tile - [ceil(N / 128)][ceil(K / 64)][128][64], zero padded - the
+ * same box is one contiguous 16 KB block and the weight stream runs about 4 % faster.
+ * sx_tiled_weight_bytes gives the size of that layout; sx_tile_weight repacks src_d ([N, K] bf16,
+ * K a multiple of 8, 16-byte aligned) into dst_d (16-byte aligned, not overlapping src_d) on `stream`.
+ * A context created with sx_model_cfg.tiled_weights = 1 expects every GEMM weight in that layout. */
+size_t sx_tiled_weight_bytes(int32_t N, int32_t K);
+sx_status sx_tile_weight(const void *src_d, int32_t N, int32_t K, void *dst_d, void *stream);
 
 /* Stochastic acceptance: speculative sampling, the acceptance rule of the speculative-decoding
  * scheme the method builds on (Section 2, background on speculative decoding; Algorithm 1,

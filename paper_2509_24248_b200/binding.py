@@ -29,7 +29,7 @@ HIST = 16
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
            "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit",
-           "sx_set_sampling"]
+           "sx_set_sampling", "sx_tiled_weight_bytes", "sx_tile_weight"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -43,7 +43,7 @@ class ModelCfg(C.Structure):
                 ("head_dim", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
                 ("n_signals", C.c_int32), ("rms_eps", C.c_float), ("rope_theta", C.c_float),
                 ("page_size", C.c_int32), ("act", C.c_int32 * SX_MAX_SIGNALS), ("draft_vocab", C.c_int32),
-                ("arch", C.c_int32)]
+                ("arch", C.c_int32), ("tiled_weights", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -107,6 +107,10 @@ def load_library() -> C.CDLL:
     lib.sx_workspace_bytes.argtypes = [vp]
     lib.sx_strerror.restype = C.c_char_p
     lib.sx_strerror.argtypes = [i32]
+    lib.sx_tiled_weight_bytes.restype = sz
+    lib.sx_tiled_weight_bytes.argtypes = [i32, i32]
+    lib.sx_tile_weight.restype = i32
+    lib.sx_tile_weight.argtypes = [vp, i32, i32, vp, vp]
     lib.sx_set_sampling.restype = i32
     lib.sx_set_sampling.argtypes = [vp, C.c_float, C.c_uint64, C.c_uint32]
     lib.sx_launch_count.restype = C.c_int64
@@ -176,6 +180,22 @@ class ExitParams:
 NOALLOC_MAX_ROWS = 64
 
 
+GEMM_WEIGHTS = ("fc", "wqkv", "wo", "wgate_up", "wdown", "head", "target_head")
+
+
+def sx_tile_weight(w: torch.Tensor) -> torch.Tensor:
+    """Repacks a row-major bf16 ``[N, K]`` device matrix tile by tile (``[ceil(N/128)][ceil(K/64)][128][64]``,
+    zero padded), the layout a context created with ``tiled=True`` expects.  Returns a flat bf16 tensor."""
+    lib = load_library()
+    N, K = int(w.shape[0]), int(w.shape[1])
+    if w.dtype != torch.bfloat16 or not w.is_cuda or not w.is_contiguous():
+        raise SxError("sx_tile_weight wants a contiguous bf16 matrix on the device")
+    out = torch.empty(int(lib.sx_tiled_weight_bytes(N, K)) // 2, dtype=torch.bfloat16, device=w.device)
+    _check(lib.sx_tile_weight(w.data_ptr(), N, K, out.data_ptr(), torch.cuda.current_stream(w.device).cuda_stream),
+           "sx_tile_weight")
+    return out
+
+
 def sx_verify_noalloc(target_head: torch.Tensor, target_hidden: torch.Tensor, cand_tok: torch.Tensor,
                       parent: Optional[torch.Tensor], out: Dict[str, torch.Tensor], status: torch.Tensor) -> None:
     """Verification without a context or a workspace, for callers that may not allocate device
@@ -199,7 +219,7 @@ class SpecExit:
     def __init__(self, shape: synth.ModelShape, weights: Dict[str, torch.Tensor], max_batch: int,
                  mode: int, K: int, topk: int = 1, max_nodes: int = 0,
                  act=(ACT_SIGMOID, ACT_SIGMOID, ACT_SIGMOID), device: str = "cuda:0",
-                 max_verify_rows: int = 0, sample_drafts: bool = False):
+                 max_verify_rows: int = 0, sample_drafts: bool = False, tiled: bool = False):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise SxError("a CUDA device is required (there is no CPU fallback)")
@@ -212,9 +232,19 @@ class SpecExit:
         self.w = {k: (v.to(self.dev).contiguous() if v.device != self.dev else v) for k, v in weights.items()}
         if "target_head" not in self.w:
             self.w["target_head"] = self.w["head"]      # rows [0, V) of the shared head
+        self.tiled = bool(tiled)
+        if self.tiled:
+            # every GEMM weight is repacked on the device (sx_tile_weight); the row-major copies are dropped
+            done = {}
+            for name in GEMM_WEIGHTS:
+                src = self.w[name]
+                if src.data_ptr() not in done:
+                    done[src.data_ptr()] = sx_tile_weight(src)
+                self.w[name] = done[src.data_ptr()]
+            del done, src
         mc = ModelCfg(shape.H, shape.n_q, shape.n_kv, shape.d, shape.F, shape.V, shape.S, shape.eps,
                       shape.theta, shape.page, (C.c_int32 * 3)(*act), getattr(shape, "Vd", 0),
-                      getattr(shape, "arch", 0))
+                      getattr(shape, "arch", 0), 1 if self.tiled else 0)
         d2t = self.w.get("draft_to_token")
         if d2t is not None and (d2t.dtype != torch.int32 or d2t.numel() != (shape.Vd or shape.V)):
             raise SxError("draft_to_token must be int32 with one entry per draft id")

@@ -19,6 +19,7 @@ struct sx_ctx {
   size_t off_u, off_x, off_n, off_q, off_o, off_a, off_m, off_g, off_part, off_attn, off_hparts, off_z,
       off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, off_dlogits, off_tlogits, off_spec, total;
   int commit_rows, commit_N;
+  bool tiled;                    // GEMM weights are stored tile by tile (sx_tile_weight)
   SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
   // set around a draft round whose head samples its token and leaves its logits (sampled drafts)
   bool round_sampled;
@@ -116,6 +117,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (Vd < 1 || Vd > m->vocab) return SX_ERR_INVALID_ARG;
   if (Vd < m->vocab && !w->draft_to_token_d) return SX_ERR_INVALID_ARG;   // a reduced vocabulary needs its id map
   if (m->arch != SX_ARCH_CONCAT && m->arch != SX_ARCH_FUSED3) return SX_ERR_UNSUPPORTED;
+  if (m->tiled_weights != 0 && m->tiled_weights != 1) return SX_ERR_INVALID_ARG;
   if (m->arch == SX_ARCH_FUSED3 && (!w->norm_e_d || ((uintptr_t)w->norm_e_d & 15))) return SX_ERR_INVALID_ARG;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   if (dc->sample_drafts != 0 && dc->sample_drafts != 1) return SX_ERR_INVALID_ARG;
@@ -132,6 +134,7 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   for (int i = 0; i < SX_MAX_SIGNALS; ++i) c->sh.act[i] = m->act[i];
   c->w = *w;
   c->dc = *dc;
+  c->tiled = m->tiled_weights == 1;
   c->max_batch = max_batch;
   int T = 1;
   if (dc->mode == SX_MODE_TREE) {
@@ -278,7 +281,8 @@ static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf1
   *stride = (size_t)R * N;
   c->launches += 1;
   prof_mark(c, cls, true, st);
-  sx_status rc = sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, c->sm_count, status, st);
+  sx_status rc = sx_launch_gemm_partial((const bf16 *)W, N, K, X, R, (float *)(ws + c->off_part), sp, *stride, c->sm_count, status, st,
+                                        c->tiled);
   prof_mark(c, cls, false, st);
   return rc;
 }
@@ -300,7 +304,7 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     if (smp) { sm2 = *smp; sm2.row0 = r0; }
     SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
                           c->head_rows, &G, z, S, c->sm_count, status, st, smp ? &sm2 : nullptr,
-                          SxLogitsOut{lo.out ? lo.out + (size_t)r0 * lo.ld : nullptr, lo.ld}));
+                          SxLogitsOut{lo.out ? lo.out + (size_t)r0 * lo.ld : nullptr, lo.ld}, c->tiled));
     prof_mark(c, cls, false, st);
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
@@ -395,6 +399,16 @@ extern "C" sx_status sx_draft_step(sx_ctx *c, const sx_kv *kv, int32_t round, in
                      (tree && round > 1) ? row_mask_d : nullptr, (bf16 *)hidden_out_d, SxIndex{nullptr, 1, 0},
                      tok_out_d, SxIndex{nullptr, T, 0}, logp_out_d, signals_out_d, SxIndex{nullptr, 1, 0},
                      (char *)ws_d, status_d, (cudaStream_t)stream);
+}
+
+extern "C" size_t sx_tiled_weight_bytes(int32_t N, int32_t K) {
+  if (N < 1 || K < 1) return 0;
+  return sx_tiled_elems(N, K) * sizeof(bf16);
+}
+
+extern "C" sx_status sx_tile_weight(const void *src_d, int32_t N, int32_t K, void *dst_d, void *stream) {
+  if (!src_d || !dst_d || ((uintptr_t)src_d & 15) || ((uintptr_t)dst_d & 15)) return SX_ERR_INVALID_ARG;
+  return sx_launch_tile_weight((const bf16 *)src_d, N, K, (bf16 *)dst_d, (cudaStream_t)stream);
 }
 
 extern "C" sx_status sx_set_sampling(sx_ctx *c, float temperature, uint64_t seed, uint32_t offset) {
@@ -567,7 +581,7 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
       int sp = sx_gemm_pick_splits(s.H, 3 * s.H, c->sm_count);
       if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
       SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 3 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
-                                    status_d, st));
+                                    status_d, st, c->tiled));
       sx_launch_fused_input(s, R, part, sp, (size_t)R * s.H, nullptr, SxIndex{nullptr, 1, 0}, trow, SxIndex{nullptr, 1, 0},
                             (const bf16 *)c->w.embed_d, (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, n, u2,
                             status_d, st);
@@ -575,7 +589,7 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
       sp = sx_gemm_pick_splits(N, 2 * s.H, c->sm_count);
       if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
       SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, 2 * s.H, u2, R, part, sp, (size_t)R * N, c->sm_count,
-                                    status_d, st));
+                                    status_d, st, c->tiled));
       SxRowMap rm;
       memset(&rm, 0, sizeof(rm));
       rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
@@ -594,14 +608,14 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
     int sp = sx_gemm_pick_splits(s.H, 2 * s.H, c->sm_count);
     if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
     SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 2 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
-                                  status_d, st));
+                                  status_d, st, c->tiled));
     sx_launch_finish_norm(s, R, part, sp, (size_t)R * s.H, nullptr, (const bf16 *)c->w.norm1_d, nullptr, n, nullptr,
                           SxIndex{nullptr, 1, 0}, st);
     const int N = (s.nq + 2 * s.nkv) * s.d;
     sp = sx_gemm_pick_splits(N, s.H, c->sm_count);
     if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
     SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, s.H, n, R, part, sp, (size_t)R * N, c->sm_count, status_d,
-                                  st));
+                                  st, c->tiled));
     SxRowMap rm;
     memset(&rm, 0, sizeof(rm));
     rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;

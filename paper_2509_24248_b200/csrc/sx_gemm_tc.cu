@@ -43,6 +43,7 @@ struct SxTcParams {
   int32_t *status;
   SxSample smp;                  // temp > 0: the argmax epilogue draws a Gumbel-max sample instead
   SxLogitsOut lo;                // argmax epilogue: also leave the logits in global memory
+  int w_tiled;                   // weights stored tile by tile: [row tile][k-block][128 rows][64 columns]
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -222,13 +223,15 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             const uint32_t dst = smem_u32(smem + (size_t)stage * stage_bytes);
             if (pass == 0) {
               mbar_expect_tx(fb, stage_bytes);
-              tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
+              tma_load_2d(dst, &tmW, fb, p.w_tiled ? 0 : kb * SX_BK,
+                          p.w_tiled ? (tile * p.num_kb + kb) * SX_TILE_M : tile * SX_TILE_M, pol_w);
             } else if (pass == 1) {
               tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
             } else if (cnt >= p.stages) {
               if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
               mbar_expect_tx(fb, stage_bytes);
-              tma_load_2d(dst, &tmW, fb, kb * SX_BK, tile * SX_TILE_M, pol_w);
+              tma_load_2d(dst, &tmW, fb, p.w_tiled ? 0 : kb * SX_BK,
+                          p.w_tiled ? (tile * p.num_kb + kb) * SX_TILE_M : tile * SX_TILE_M, pol_w);
               tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
             }
             if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -650,8 +653,17 @@ int sx_gemm_pick_splits(int N, int K, int sm_count) {
   return best;
 }
 
+// Tensor map of a weight matrix.  Row-major [N, K]: a box is 128 rows x 64 columns, i.e. 128 pieces of
+// 128 bytes that lie K * 2 bytes apart.  Tiled ([row tile][k-block][128][64], zero padded): the same box
+// is one contiguous 16 KB block, which keeps the DRAM pages it touches open for the whole transfer.
+static bool weight_map(const bf16 *W, int N, int K, bool tiled, CUtensorMap *out) {
+  if (!tiled) return get_map(W, N, K, SX_TILE_M, out);
+  const int tiles = (N + SX_TILE_M - 1) / SX_TILE_M, kbs = (K + SX_BK - 1) / SX_BK;
+  return get_map(W, tiles * kbs * SX_TILE_M, SX_BK, SX_TILE_M, out);
+}
+
 sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part, int splits,
-                                 size_t split_stride, int sm_count, int32_t *status, cudaStream_t st) {
+                                 size_t split_stride, int sm_count, int32_t *status, cudaStream_t st, bool tiled) {
   if ((K % 8) != 0 || R < 1) return SX_ERR_UNSUPPORTED;
   for (int r0 = 0; r0 < R; r0 += 256) {
     const int rc = (R - r0 < 256) ? R - r0 : 256;
@@ -665,7 +677,8 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
     p.split_stride = split_stride;
     p.status = status;
     CUtensorMap mw, mx;
-    if (!get_map(W, N, K, SX_TILE_M, &mw) || !get_map(X + (size_t)r0 * K, rc, K, p.nmma, &mx)) return SX_ERR_CUDA;
+    p.w_tiled = tiled ? 1 : 0;
+    if (!weight_map(W, N, K, tiled, &mw) || !get_map(X + (size_t)r0 * K, rc, K, p.nmma, &mx)) return SX_ERR_CUDA;
     const int items = p.num_tiles * p.splits;
     const int per_cta = (items + sm_count - 1) / sm_count;          // the same number of items for every CTA
     const int grid = (items + per_cta - 1) / per_cta;
@@ -679,7 +692,7 @@ int sx_head_max_rows(int T, int lse) { return (T == 1 && !lse) ? 256 : 64; }
 
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count, int32_t *status,
-                         cudaStream_t st, const SxSample *smp, SxLogitsOut lo) {
+                         cudaStream_t st, const SxSample *smp, SxLogitsOut lo, bool tiled) {
   if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T, lse)) return SX_ERR_UNSUPPORTED;
   if (smp && smp->temp > 0.f && (T != 1 || lse || smp->P < 1)) return SX_ERR_UNSUPPORTED;
   if (lo.out && (T != 1 || lse)) return SX_ERR_UNSUPPORTED;
@@ -693,7 +706,8 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
   if (smp) p.smp = *smp;
   p.lo = lo;
   CUtensorMap mw, mx;
-  if (!get_map(W, Ntot, K, SX_TILE_M, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
+  p.w_tiled = tiled ? 1 : 0;
+  if (!weight_map(W, Ntot, K, tiled, &mw) || !get_map(X, R, K, p.nmma, &mx)) return SX_ERR_CUDA;
   // every CTA gets the same number of tiles (no CTA is left alone with one more 1 MB tile at the end):
   // with w = ceil(tiles / SMs) tiles per CTA, ceil(tiles / w) CTAs cover the matrix
   const int per_cta = (p.num_tiles + sm_count - 1) / sm_count;
@@ -702,4 +716,30 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
     return SX_ERR_CUDA;
   *G = grid;
   return SX_OK;
+}
+
+// ---- weight tiling ------------------------------------------------------------------------
+// dst[tile][kb][r][c] = src[tile * 128 + r][kb * 64 + c], zero outside the matrix.  One CTA per
+// (k-block, row tile); a thread moves 16 bytes at a time.
+__global__ void sx_tile_weight_kernel(const bf16 *__restrict__ src, int N, int K, bf16 *__restrict__ dst) {
+  const int kb = blockIdx.x, tile = blockIdx.y, kbs = gridDim.x;
+  uint4 *out = reinterpret_cast<uint4 *>(dst + ((size_t)tile * kbs + kb) * SX_TILE_M * SX_BK);
+  for (int i = threadIdx.x; i < SX_TILE_M * SX_BK / 8; i += blockDim.x) {
+    const int r = i / (SX_BK / 8), c8 = i % (SX_BK / 8);
+    const int row = tile * SX_TILE_M + r, col = kb * SX_BK + c8 * 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (row < N && col < K) v = *reinterpret_cast<const uint4 *>(src + (size_t)row * K + col);   // K % 8 == 0
+    out[i] = v;
+  }
+}
+
+size_t sx_tiled_elems(int N, int K) {
+  return (size_t)((N + SX_TILE_M - 1) / SX_TILE_M) * ((K + SX_BK - 1) / SX_BK) * SX_TILE_M * SX_BK;
+}
+
+sx_status sx_launch_tile_weight(const bf16 *src, int N, int K, bf16 *dst, cudaStream_t st) {
+  if (N < 1 || K < 8 || (K % 8) != 0) return SX_ERR_UNSUPPORTED;
+  dim3 grid((K + SX_BK - 1) / SX_BK, (N + SX_TILE_M - 1) / SX_TILE_M);
+  sx_tile_weight_kernel<<<grid, 256, 0, st>>>(src, N, K, dst);
+  return cudaGetLastError() == cudaSuccess ? SX_OK : SX_ERR_CUDA;
 }

@@ -102,7 +102,10 @@ void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, c
 int sx_gemm_pick_splits(int N, int K, int sm_count);
 sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int R, float *part,
                                  int splits, size_t split_stride, int sm_count, int32_t *status,
-                                 cudaStream_t st);
+                                 cudaStream_t st, bool tiled = false);
+// weights tile by tile ([row tile][k-block][128][64], zero padded): elements of that layout, and the repack
+size_t sx_tiled_elems(int N, int K);
+sx_status sx_launch_tile_weight(const bf16 *src, int N, int K, bf16 *dst, cudaStream_t st);
 void sx_gemm_init(int device);
 // Sampled verification: with temp > 0 the plain-argmax head returns, per row, the arg max of
 // logit + temp * Gumbel noise, i.e. a draw from softmax(logits / temp).  Row r of the launch is
@@ -123,7 +126,7 @@ struct SxLogitsOut {
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
                          int32_t *status, cudaStream_t st, const SxSample *smp = nullptr,
-                         SxLogitsOut lo = SxLogitsOut{nullptr, 0});
+                         SxLogitsOut lo = SxLogitsOut{nullptr, 0}, bool tiled = false);
 
 // Speculative sampling with sampled drafts: writes the kept draft token or the residual draw of every
 // verify slot to target_tok [B, P].  target_logits [B * P, V], draft_logits [B, K, V] (K = P - 1), both

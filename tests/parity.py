@@ -145,10 +145,13 @@ def _kv_replay(sx: binding.SpecExit, case: harness.Case):
     return f
 
 
+TILED = False      # tests of the tiled weight layout switch this on for the contexts they build
+
+
 def make_gpu(case: harness.Case, act=(0, 0, 0), sample_drafts: bool = False) -> binding.SpecExit:
     wl = case.wl
     sx = binding.SpecExit(wl.shape, case.weights, wl.B, wl.mode, wl.K, wl.topk if wl.mode == synth.TREE else 1,
-                          wl.max_nodes, act=act, sample_drafts=sample_drafts)
+                          wl.max_nodes, act=act, sample_drafts=sample_drafts, tiled=TILED)
     sx.set_kv(case.kv)
     return sx
 

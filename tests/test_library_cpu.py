@@ -41,7 +41,7 @@ def test_strerror_and_null_checks_without_a_device(lib):
 
 def test_struct_layouts_match_header():
     from paper_2509_24248_b200 import binding as b
-    assert ctypes.sizeof(b.ModelCfg) == 4 * 15
+    assert ctypes.sizeof(b.ModelCfg) == 4 * 16
     assert ctypes.sizeof(b.Weights) == 8 * 13
     assert ctypes.sizeof(b.DraftCfg) == 20
     assert ctypes.sizeof(b.IterOut) == 8 * 18
