@@ -15,8 +15,14 @@
  * Conventions for every entry point
  *   - Pointers named *_d are DEVICE pointers, 16-byte aligned, owned by the caller, and
  *     borrowed until the enqueued work has finished.  Everything else is host memory.
- *   - All work is enqueued on the given stream; no entry point synchronises, allocates
- *     device memory or frees it (sx_create / sx_destroy only touch host memory).
+ *   - All work is enqueued on the given stream; no entry point allocates or frees device
+ *     memory (sx_create / sx_destroy only touch host memory), and none synchronises except
+ *     sx_spec_exit_iter_host, which waits for the stream before it returns (its results are
+ *     host buffers) and sx_profile_end's event queries.
+ *   - Weight buffers must be completely written and visible to the device (stream-ordered
+ *     work that produced them finished: an event wait or a synchronisation) BEFORE a call
+ *     that reads them is enqueued: the GEMM kernels request their first weight tiles while
+ *     the preceding kernel of the stream is still running.
  *   - Host-detectable problems (NULL, unsupported shape, workspace too small) return a
  *     negative sx_status and launch nothing.  Problems only the device can see (a page
  *     table too short for a write, a token id outside the vocabulary, a bounded wait that
@@ -122,7 +128,8 @@ typedef struct {
  * page_table_d[b * max_pages + s / page_size] at offset s % page_size.  K is stored rotated. */
 typedef struct {
   int32_t batch;
-  const int32_t *cache_len_d;   /* [batch] valid slots per sequence (not advanced by this library) */
+  int32_t *cache_len_d;         /* [batch] valid slots per sequence; read by every call, advanced only by
+                                   sx_commit */
   const int32_t *page_table_d;  /* [batch, max_pages] */
   int32_t max_pages;
   int32_t num_pages;            /* physical pages in k_pages_d / v_pages_d */
@@ -344,6 +351,17 @@ enum {
 sx_status sx_profile_begin(sx_ctx *ctx);
 sx_status sx_profile_end(sx_ctx *ctx, float *ms_out, int32_t *count_out);
 
+/* Diagnostic (the paper has no counterpart).  Every wait of the GEMM kernels on a shared-memory barrier is
+ * bounded: after `wait_limit` polls the waiting role raises an abort flag, the CTA's other roles leave
+ * at their next poll, SX_ERR_TIMEOUT goes to the status word, copies in flight are given time to land,
+ * the CTA frees its tensor memory and returns - the context stays usable.  This call runs that path on
+ * its own: `ctas` CTAs (1..1024) with the GEMM kernel's thread layout allocate tensor memory and wait, with
+ * `limit` polls (1..2^20), on barriers nothing arrives at; no copy is issued.  Afterwards *status_d is
+ * SX_ERR_TIMEOUT, reached_d[0] == 0 (no wait reported success) and reached_d[1] == ctas (every CTA
+ * returned through the tear-down).  reached_d: two int32 on the device, zeroed by the caller. */
+sx_status sx_selftest_bounded_wait(uint32_t limit, int32_t ctas, int32_t *status_d, int32_t *reached_d,
+                                   void *stream);
+
 /* Verification for callers that cannot allocate device memory (the paper has no counterpart;
  * this is a deployment convenience).  Some hosts of this library hold no allocator at the point
  * where a draft is verified: an inference server whose memory pool owns the whole device and
@@ -357,7 +375,9 @@ sx_status sx_profile_end(sx_ctx *ctx, float *ms_out, int32_t *count_out);
  * library until the process exits).  The call allocates and frees no device memory.
  *   - Limit: batch * P <= SX_NOALLOC_MAX_ROWS; beyond it the call returns SX_ERR_STATIC_LIMIT and
  *     launches nothing.  Tree mode (parent_d != NULL) also needs P <= SX_MAX_VERIFY_SLOTS.
- *   - target_head_d is the [vocab, H] bf16 head; the other arguments are those of sx_verify.
+ *   - target_head_d is the [vocab, H] bf16 head, ROW-MAJOR as handed in (not a matrix repacked with
+ *     sx_tile_weight: there is no context here to say so, and a tiled head would be misread); the other
+ *     arguments are those of sx_verify.
  *   - The first call on a device resolves the array's device address and sets kernel attributes
  *     for that device (which must be current); make that first call outside any stream capture.
  *   - All calls on a device share the array and it keeps the previous call's contents.  Nothing

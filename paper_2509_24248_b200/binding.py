@@ -29,7 +29,7 @@ HIST = 16
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
            "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit",
-           "sx_set_sampling", "sx_tiled_weight_bytes", "sx_tile_weight"]
+           "sx_set_sampling", "sx_tiled_weight_bytes", "sx_tile_weight", "sx_selftest_bounded_wait"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -134,6 +134,8 @@ def load_library() -> C.CDLL:
     lib.sx_profile_end.argtypes = [vp, vp, vp]
     lib.sx_commit.restype = i32
     lib.sx_commit.argtypes = [vp, C.POINTER(KV), i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.sx_selftest_bounded_wait.restype = i32
+    lib.sx_selftest_bounded_wait.argtypes = [C.c_uint32, i32, vp, vp, vp]
     lib.sx_verify_noalloc.restype = i32
     lib.sx_verify_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp]
     _lib = lib
@@ -242,6 +244,9 @@ class SpecExit:
                     done[src.data_ptr()] = sx_tile_weight(src)
                 self.w[name] = done[src.data_ptr()]
             del done, src
+            # weights must be complete before any call that reads them is enqueued (the GEMM kernels
+            # fetch their first weight tiles ahead of stream order)
+            torch.cuda.synchronize(self.dev)
         mc = ModelCfg(shape.H, shape.n_q, shape.n_kv, shape.d, shape.F, shape.V, shape.S, shape.eps,
                       shape.theta, shape.page, (C.c_int32 * 3)(*act), getattr(shape, "Vd", 0),
                       getattr(shape, "arch", 0), 1 if self.tiled else 0)

@@ -169,8 +169,10 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   }
   c->device = dev;
   c->sm_count = prop.multiProcessorCount;
-  sx_gemm_init(dev);
-  sx_attn_init(dev);
+  if (sx_gemm_init(dev) != SX_OK || sx_attn_init(dev) != SX_OK || sx_kernels_init(dev) != SX_OK) {
+    delete c;
+    return SX_ERR_CUDA;
+  }
 
   const SxShape &s = c->sh;
   const int R = c->Rmax;
@@ -270,8 +272,6 @@ static SxTree tree_view(const sx_ctx *c, char *ws) {
   return t;
 }
 
-#define SX_TRY(e) do { sx_status _s = (e); if (_s != SX_OK) return _s; } while (0)
-
 // GEMM + its split-K buffer; returns the split count used
 static sx_status gemm(sx_ctx *c, int cls, const void *W, int N, int K, const bf16 *X, int R, char *ws, int *splits,
                       size_t *stride, int32_t *status, cudaStream_t st) {
@@ -309,9 +309,9 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
     if (s2.idx) s2.idx += r0; else s2.add += r0 * s2.mul;
-    sx_launch_head_finalize(c->sh, rc, parts, G, c->head_rows, T, lse, z, S, tok_out, t2,
+    SX_TRY(sx_launch_head_finalize(c->sh, rc, parts, G, c->head_rows, T, lse, z, S, tok_out, t2,
                             logp_out ? logp_out + (size_t)r0 * T : nullptr, sig_out, s2, st,
-                            (R <= cap) ? nx : SxNextInput{nullptr, nullptr, nullptr, 0, 0}, map, V);
+                            (R <= cap) ? nx : SxNextInput{nullptr, nullptr, nullptr, 0, 0}, map, V));
     c->launches += 2;
   }
   return SX_OK;
@@ -338,37 +338,37 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
     if (round == 1) {
       if (fi.idx || fi.mul != 1 || fi.add != 0) return SX_ERR_UNSUPPORTED;      // the GEMM reads the rows in place
       SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 3 * s.H, feat, R, ws, &sp, &stride, status, st));
-      sx_launch_fused_input(s, R, part, sp, stride, nullptr, fi, tok, ti, (const bf16 *)c->w.embed_d,
-                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st);
+      SX_TRY(sx_launch_fused_input(s, R, part, sp, stride, nullptr, fi, tok, ti, (const bf16 *)c->w.embed_d,
+                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st));
     } else {
-      sx_launch_fused_input(s, R, nullptr, 0, 0, feat, fi, tok, ti, (const bf16 *)c->w.embed_d,
-                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st);
+      SX_TRY(sx_launch_fused_input(s, R, nullptr, 0, 0, feat, fi, tok, ti, (const bf16 *)c->w.embed_d,
+                            (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, x, u, status, st));
     }
     SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, 2 * s.H, u, R, ws, &sp, &stride, status, st));
   } else {
     // input_ready: the previous round's merge kernel has already written u (chain drafting)
     if (!input_ready) {
-      sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st);
+      SX_TRY(sx_launch_embed_concat(s, R, feat, fi, tok, ti, (const bf16 *)c->w.embed_d, u, status, st));
       c->launches += 1;
     }
     SX_TRY(gemm(c, SX_PROF_GEMM_FC, c->w.fc_d, s.H, 2 * s.H, u, R, ws, &sp, &stride, status, st));
-    sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st);
+    SX_TRY(sx_launch_finish_norm(s, R, part, sp, stride, nullptr, (const bf16 *)c->w.norm1_d, x, n, nullptr, SxIndex{nullptr, 1, 0}, st));
     SX_TRY(gemm(c, SX_PROF_GEMM_QKV, c->w.wqkv_d, (s.nq + 2 * s.nkv) * s.d, s.H, n, R, ws, &sp, &stride, status, st));
   }
-  sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st);
+  SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st));
   const int B = kv->batch, nr = R / B;
   const int E = (c->dc.mode == SX_MODE_CHAIN) ? round : (round == 1 ? 1 : 1 + (round - 1) * c->dc.topk);
   const int nsplit = sx_attn_splits(s, B, nr, kv->max_pages * s.page, c->sm_count);
   prof_mark(c, SX_PROF_ATTENTION, true, st);
-  sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st);
+  SX_TRY(sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st));
   prof_mark(c, SX_PROF_ATTENTION, false, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_O, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
-  sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st);
+  SX_TRY(sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st));
   SX_TRY(gemm(c, SX_PROF_GEMM_GATE_UP, c->w.wgate_up_d, 2 * s.F, s.H, n, R, ws, &sp, &stride, status, st));
-  sx_launch_finish_swiglu(s, R, part, sp, stride, m, st);
+  SX_TRY(sx_launch_finish_swiglu(s, R, part, sp, stride, m, st));
   SX_TRY(gemm(c, SX_PROF_GEMM_DOWN, c->w.wdown_d, s.H, s.F, m, R, ws, &sp, &stride, status, st));
   // the hidden handed to the caller (and to the next round) is g, or y for the fused layer
-  sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st, fused3 ? 1 : 0);
+  SX_TRY(sx_launch_finish_norm(s, R, part, sp, stride, a, (const bf16 *)c->w.normf_d, nullptr, g, hid_user, ui, st, fused3 ? 1 : 0));
   c->launches += 7;   // 3 norms, rope, attention x2, swiglu
   const int T = c->dc.mode == SX_MODE_TREE ? c->dc.topk : 1;
   SX_TRY(head(c, SX_PROF_HEAD_DRAFT, c->w.head_d, s.Vd + s.S, s.Vd, s.S, g, R, T, c->dc.mode == SX_MODE_TREE ? 1 : 0, ws, tok_out, toi, logp_out, sig_out, si,
@@ -411,6 +411,12 @@ extern "C" sx_status sx_tile_weight(const void *src_d, int32_t N, int32_t K, voi
   return sx_launch_tile_weight((const bf16 *)src_d, N, K, (bf16 *)dst_d, (cudaStream_t)stream);
 }
 
+extern "C" sx_status sx_selftest_bounded_wait(uint32_t limit, int32_t ctas, int32_t *status_d, int32_t *reached_d,
+                                              void *stream) {
+  if (!status_d || !reached_d) return SX_ERR_INVALID_ARG;
+  return sx_launch_wait_selftest(limit, ctas, status_d, reached_d, (cudaStream_t)stream);
+}
+
 extern "C" sx_status sx_set_sampling(sx_ctx *c, float temperature, uint64_t seed, uint32_t offset) {
   if (!c || !(temperature >= 0.f) || !(temperature < INFINITY)) return SX_ERR_INVALID_ARG;
   c->smp.temp = temperature;
@@ -435,7 +441,7 @@ extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *
   SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, c->sh.V, c->sh.V, 0, (const bf16 *)target_hidden_d, batch * P, 1, 0, (char *)ws_d,
               target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
               SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, smp.temp > 0.f ? &smp : nullptr));
-  sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st);
+  SX_TRY(sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st));
   c->launches += 1;
   return SX_OK;
 }
@@ -456,9 +462,9 @@ extern "C" sx_status sx_exit_update(sx_ctx *c, int32_t batch, int32_t P, const s
       (!state->hist_d || cfg->window < 2 || cfg->window >= SX_HIST))
     return SX_ERR_INVALID_ARG;
   if (cfg->smoothing == SX_SMOOTH_PARAGRAPH && (!state->par_sum_d || !state->par_n_d)) return SX_ERR_INVALID_ARG;
-  sx_launch_exit(batch, P, c->sh.S, *cfg, *state, slot_signal_d, cand_tok_d, path_d, path_stride, accept_len_d,
+  SX_TRY(sx_launch_exit(batch, P, c->sh.S, *cfg, *state, slot_signal_d, cand_tok_d, path_d, path_stride, accept_len_d,
                  recover_tok_d, exit_flag_d, accept_len_out_d, recover_tok_out_d, smoothed_out_d, c->sh.V, status_d,
-                 (cudaStream_t)stream);
+                 (cudaStream_t)stream));
   c->launches += 1;
   return SX_OK;
 }
@@ -480,7 +486,7 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
   const int B = kv->batch, K = c->dc.K, P = c->P, S = c->sh.S;
   bf16 *hid = (bf16 *)o->hidden_d;
   if (c->dc.mode == SX_MODE_CHAIN) {
-    sx_launch_chain_layout(B, K, S, tok0_d, *o, st);
+    SX_TRY(sx_launch_chain_layout(B, K, S, tok0_d, *o, st));
     c->launches += 1;
     // one head launch per round: its merge can write the next input (concat layer only)
     const bool fuse = B <= sx_head_max_rows(1, 0) && c->sh.arch == SX_ARCH_CONCAT;
@@ -511,10 +517,10 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
       SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, V, V, 0, (const bf16 *)target_hidden_d, B * P, 1, 0, ws,
                   o->target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
                   SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr, SxLogitsOut{tlogits, (size_t)V}));
-      sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, ws + c->off_spec, c->sm_count,
-                            o->target_tok_d, status_d, st);
-      sx_launch_accept(B, P, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d, K + 1,
-                       o->recover_tok_d, st);
+      SX_TRY(sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, ws + c->off_spec, c->sm_count,
+                            o->target_tok_d, status_d, st));
+      SX_TRY(sx_launch_accept(B, P, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d, K + 1,
+                       o->recover_tok_d, st));
       c->launches += 4;
     } else {
       SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d,
@@ -532,16 +538,16 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
     SX_TRY(draft_round(c, kv, 1, B, (const bf16 *)feat0_d, SxIndex{nullptr, 1, 0}, tok0_d, SxIndex{nullptr, 1, 0},
                        nullptr, hid, SxIndex{nullptr, rows, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt, t.row_sig,
                        SxIndex{nullptr, rows, 0}, ws, status_d, st));
-    sx_launch_tree_expand(t, B, 1, tok_rt, logp_rt, st);
+    SX_TRY(sx_launch_tree_expand(t, B, 1, tok_rt, logp_rt, st));
     c->launches += 1;
     for (int r = 2; r <= K; ++r) {
       SX_TRY(draft_round(c, kv, r, B * T, hid, SxIndex{t.feat_idx, 0, 0}, t.sel_tok, SxIndex{nullptr, 1, 0},
                          t.next_mask, hid, SxIndex{t.hid_idx, 0, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt,
                          t.row_sig, SxIndex{t.hid_idx, 0, 0}, ws, status_d, st));
-      sx_launch_tree_expand(t, B, r, tok_rt, logp_rt, st);
+      SX_TRY(sx_launch_tree_expand(t, B, r, tok_rt, logp_rt, st));
       c->launches += 1;
     }
-    sx_launch_tree_layout(t, B, S, tok0_d, *o, st);
+    SX_TRY(sx_launch_tree_layout(t, B, S, tok0_d, *o, st));
     c->launches += 1;
     SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, o->parent_d, o->target_tok_d, o->accept_len_d,
                      o->path_d, K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
@@ -573,18 +579,18 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
     // catch-up rows go through fc (3H -> H), the two input norms and the K/V part of the projection
     bf16 *u2 = (bf16 *)(ws + c->off_cu2);
     int32_t *trow = (int32_t *)(ws + c->off_ctok);
-    sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
+    SX_TRY(sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
                             recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d,
-                            st, trow);
+                            st, trow));
     c->launches += 1;
     if (R > 0) {
       int sp = sx_gemm_pick_splits(s.H, 3 * s.H, c->sm_count);
       if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
       SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 3 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
                                     status_d, st, c->tiled));
-      sx_launch_fused_input(s, R, part, sp, (size_t)R * s.H, nullptr, SxIndex{nullptr, 1, 0}, trow, SxIndex{nullptr, 1, 0},
+      SX_TRY(sx_launch_fused_input(s, R, part, sp, (size_t)R * s.H, nullptr, SxIndex{nullptr, 1, 0}, trow, SxIndex{nullptr, 1, 0},
                             (const bf16 *)c->w.embed_d, (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, n, u2,
-                            status_d, st);
+                            status_d, st));
       const int N = (s.nq + 2 * s.nkv) * s.d;
       sp = sx_gemm_pick_splits(N, 2 * s.H, c->sm_count);
       if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
@@ -594,23 +600,23 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
       memset(&rm, 0, sizeof(rm));
       rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
       rm.valid_len = accept_len_out_d; rm.per_seq = M;
-      sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st);
+      SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st));
       c->launches += 4;
     }
-    sx_launch_commit_advance(B, accept_len_out_d, const_cast<int32_t *>(kv->cache_len_d), st);
+    SX_TRY(sx_launch_commit_advance(B, accept_len_out_d, kv->cache_len_d, st));
     c->launches += 1;
     return SX_OK;
   }
-  sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
-                          recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d, st);
+  SX_TRY(sx_launch_commit_gather(s, B, M, P, (const bf16 *)target_hidden_d, cand_tok_d, path_d, path_stride, accept_len_out_d,
+                          recover_tok_out_d, (const bf16 *)c->w.embed_d, u, (bf16 *)feat0_next_d, tok0_next_d, status_d, st));
   c->launches += 1;
   if (R > 0) {
     int sp = sx_gemm_pick_splits(s.H, 2 * s.H, c->sm_count);
     if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
     SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.fc_d, s.H, 2 * s.H, u, R, part, sp, (size_t)R * s.H, c->sm_count,
                                   status_d, st, c->tiled));
-    sx_launch_finish_norm(s, R, part, sp, (size_t)R * s.H, nullptr, (const bf16 *)c->w.norm1_d, nullptr, n, nullptr,
-                          SxIndex{nullptr, 1, 0}, st);
+    SX_TRY(sx_launch_finish_norm(s, R, part, sp, (size_t)R * s.H, nullptr, (const bf16 *)c->w.norm1_d, nullptr, n, nullptr,
+                          SxIndex{nullptr, 1, 0}, st));
     const int N = (s.nq + 2 * s.nkv) * s.d;
     sp = sx_gemm_pick_splits(N, s.H, c->sm_count);
     if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
@@ -620,10 +626,10 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
     memset(&rm, 0, sizeof(rm));
     rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
     rm.valid_len = accept_len_out_d; rm.per_seq = M;
-    sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st);
+    SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st));
     c->launches += 4;
   }
-  sx_launch_commit_advance(B, accept_len_out_d, const_cast<int32_t *>(kv->cache_len_d), st);
+  SX_TRY(sx_launch_commit_advance(B, accept_len_out_d, kv->cache_len_d, st));
   c->launches += 1;
   return SX_OK;
 }
@@ -646,10 +652,11 @@ extern "C" sx_status sx_spec_exit_iter_host(sx_ctx *c, const sx_kv *kv, const sx
     return SX_ERR_CUDA;
   SX_TRY(sx_spec_exit_iter(c, kv, cfg, state, stage_feat0_d, stage_tok0_d, stage_target_hidden_d, o, ws_d, ws_bytes,
                            status_d, stream));
-  cudaMemcpyAsync(accept_len_out_h, o->accept_len_out_d, B * 4, cudaMemcpyDeviceToHost, st);
-  cudaMemcpyAsync(recover_tok_out_h, o->recover_tok_out_d, B * 4, cudaMemcpyDeviceToHost, st);
-  cudaMemcpyAsync(exit_flag_h, o->exit_flag_d, B * 4, cudaMemcpyDeviceToHost, st);
-  cudaMemcpyAsync(smoothed_h, o->smoothed_d, B * c->sh.S * 4, cudaMemcpyDeviceToHost, st);
+  if (cudaMemcpyAsync(accept_len_out_h, o->accept_len_out_d, B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(recover_tok_out_h, o->recover_tok_out_d, B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(exit_flag_h, o->exit_flag_d, B * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(smoothed_h, o->smoothed_d, B * c->sh.S * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return SX_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return SX_ERR_CUDA;
   return SX_OK;
 }

@@ -425,18 +425,17 @@ static int attn_tiles(const SxShape &sh, int nr) {          // warps per group
 static int attn_groups_per_cta(int NT) { return NT >= 4 ? 1 : 4 / NT; }
 
 template <int D>
-static void attn_init_d() {
+static bool attn_init_d() {
   const int smem = SX_ATTN_SMEM_BUDGET;
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  cudaFuncSetAttribute(sx_attn_mma_kernel<D, 4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const cudaFuncAttribute at = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  return cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 1>, at, smem) == cudaSuccess &&
+         cudaFuncSetAttribute(sx_attn_mma_kernel<D, 1, 2>, at, smem) == cudaSuccess &&
+         cudaFuncSetAttribute(sx_attn_mma_kernel<D, 2, 2>, at, smem) == cudaSuccess &&
+         cudaFuncSetAttribute(sx_attn_mma_kernel<D, 4, 2>, at, smem) == cudaSuccess;
 }
-void sx_attn_init(int device) {
-  attn_init_d<16>();
-  attn_init_d<32>();
-  attn_init_d<64>();
-  attn_init_d<128>();
+sx_status sx_attn_init(int device) {
+  (void)device;
+  return (attn_init_d<16>() && attn_init_d<32>() && attn_init_d<64>() && attn_init_d<128>()) ? SX_OK : SX_ERR_CUDA;
 }
 
 // Key chunks per (sequence, KV head): enough warp groups to fill the machine a few times over,
@@ -468,7 +467,7 @@ bool sx_attn_supported(const SxShape &sh) {
          attn_qtiles(sh, SX_MAX_TOPK) <= SX_ATTN_MAX_TILES;
 }
 
-void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q, const sx_kv &kv,
+sx_status sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q, const sx_kv &kv,
                          int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st) {
   const int R = B * nr;
   const int G = sh.nq / sh.nkv;
@@ -489,9 +488,10 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
   const size_t smem = (size_t)gpc * stages * stage_bytes;
-#define SX_ATTN_NT(DD, NN, QQ)                                                                                    \
-  sx_launch(sx_attn_mma_kernel<DD, NN, QQ>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, rm, \
-            nr, E, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status)
+  cudaError_t err = cudaSuccess;
+#define SX_ATTN_NT(DD, NN, QQ)                                                                                          \
+  err = sx_launch(sx_attn_mma_kernel<DD, NN, QQ>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, scale_log2, \
+                  rm, nr, E, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status)
 #define SX_ATTN(DD)                                  \
   switch (attn_qtiles(sh, nr)) {                     \
     case 1: SX_ATTN_NT(DD, 1, 1); break;             \
@@ -507,6 +507,7 @@ void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, i
   }
 #undef SX_ATTN_NT
 #undef SX_ATTN
-  sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3((nsplit > 64 && sh.nq * R <= 296) ? 1024 : 256), 0, st, sh.nq, sh.d, nsplit,
-            (const float2 *)ws_ml, (const float *)ws_o, o_out);
+  if (err != cudaSuccess) return SX_ERR_CUDA;
+  return sx_rc(sx_launch(sx_attn_merge_kernel, dim3(sh.nq, R), dim3((nsplit > 64 && sh.nq * R <= 296) ? 1024 : 256), 0, st, sh.nq, sh.d, nsplit,
+            (const float2 *)ws_ml, (const float *)ws_o, o_out));
 }

@@ -44,6 +44,7 @@ struct SxTcParams {
   SxSample smp;                  // temp > 0: the argmax epilogue draws a Gumbel-max sample instead
   SxLogitsOut lo;                // argmax epilogue: also leave the logits in global memory
   int w_tiled;                   // weights stored tile by tile: [row tile][k-block][128 rows][64 columns]
+  uint32_t wait_limit;           // polls of an mbarrier before a wait gives up
 };
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -70,8 +71,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // bounded wait; false = gave up (or another role already did)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-  for (uint32_t i = 0; i < SX_WAIT_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 255u && *abort_flag) return false;
   }
@@ -164,6 +165,21 @@ __device__ __forceinline__ bool epi_all(bool ok) {
   return out != 0;
 }
 
+// Common exit of a CTA.  After a wait ran out (abort flag set): report it, give copies that are already
+// in flight time to land in shared memory, then free TMEM like a normal exit does.
+__device__ __forceinline__ void tc_teardown(volatile int *abort_flag, int32_t *status, uint32_t tmem_base, uint32_t cols) {
+  if (*abort_flag) {
+    if (threadIdx.x == 0) sx_set_status(status, SX_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if ((threadIdx.x >> 5) == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, cols);
+  }
+}
+
 template <bool HEAD>
 __global__ void __launch_bounds__(192, 1)
 sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, SxTcParams p) {
@@ -228,7 +244,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             } else if (pass == 1) {
               tma_load_2d(dst + SX_A_BYTES, &tmX, fb, kb * SX_BK, 0, pol_x);
             } else if (cnt >= p.stages) {
-              if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+              if (!mbar_wait(smem_u32(&empty[stage]), phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
               mbar_expect_tx(fb, stage_bytes);
               tma_load_2d(dst, &tmW, fb, p.w_tiled ? 0 : kb * SX_BK,
                           p.w_tiled ? (tile * p.num_kb + kb) * SX_TILE_M : tile * SX_TILE_M, pol_w);
@@ -252,11 +268,11 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         const int sp = HEAD ? 0 : item % p.splits;
         const int kb0 = sp * p.kb_per_split;
         const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
-        if (!mbar_wait(smem_u32(&tempty[acc]), acc_phase ^ 1u, abort_flag)) break;
+        if (!mbar_wait(smem_u32(&tempty[acc]), acc_phase ^ 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * p.acc_cols);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(smem_u32(&full[stage]), phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&full[stage]), phase, abort_flag, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a = smem_u32(smem + (size_t)stage * stage_bytes);
           const uint32_t b = a + SX_A_BYTES;
@@ -290,7 +306,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
       for (int ch = 0; ch < SX_ARGMAX_CHUNKS; ++ch) { bestv[ch] = -INFINITY; besti[ch] = -1; }
       for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag, p.wait_limit))) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
         const int n = item * SX_TILE_M + et;
@@ -359,7 +375,9 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      // merge the four row quarters per token row (quarter order = index order) and leave the result
+      // Merge the four row quarters per token row.  A quarter's best may come from any tile of this CTA,
+      // so quarter order is not index order: the merge ranks (value, then lower index) through the
+      // packed key.
       epi_bar();
       int *ci = reinterpret_cast<int *>(tb + 4 * 256);
 #pragma unroll
@@ -368,12 +386,13 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       epi_bar();
       SxHeadPartial *out = p.parts + (size_t)blockIdx.x * p.part_stride;
       for (int r = tid; r < p.R; r += 128) {
-        float bv = tb[r];
-        int bi = ci[r];
-        for (int w = 1; w < 4; ++w)
-          if (tb[w * 256 + r] > bv) { bv = tb[w * 256 + r]; bi = ci[w * 256 + r]; }
+        unsigned long long best = 0ull;
+        for (int w = 0; w < 4; ++w) {
+          const int xi = ci[w * 256 + r];
+          if (xi >= 0) best = max(best, sx_pack(tb[w * 256 + r], (uint32_t)xi));
+        }
         SxHeadPartial hp;
-        hp.top[0] = (bi >= 0) ? sx_pack(bv, (uint32_t)bi) : 0ull;
+        hp.top[0] = best;
 #pragma unroll
         for (int tt = 1; tt < SX_MAX_TOPK; ++tt) hp.top[tt] = 0ull;
         hp.m = -INFINITY;
@@ -397,7 +416,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         for (int k = 0; k < 8; ++k) { tv[ch][k] = -INFINITY; ti[ch][k] = -1; }
       }
       for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag, p.wait_limit))) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
         const int n = item * SX_TILE_M + et;
@@ -472,7 +491,8 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      // merge the four row quarters per token row, in quarter (= index) order
+      // Merge the four row quarters per token row.  A quarter's list may hold entries of any tile of this
+      // CTA, so the lists are merged on the packed key: larger value first, then the lower index.
       epi_bar();
       int *tbi = reinterpret_cast<int *>(tb);
 #pragma unroll
@@ -488,26 +508,24 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       SxHeadPartial *out = p.parts + (size_t)blockIdx.x * p.part_stride;
       if (tid < p.R) {
         const int r = tid;
-        float bv[8], M = tb[r * 18 + 16];
-        int bi[8];
+        unsigned long long bk[8];                  // 0 = empty (below every real entry)
+        float M = -INFINITY;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { bv[k] = tb[r * 18 + k]; bi[k] = tbi[r * 18 + 8 + k]; }
-        for (int w = 1; w < 4; ++w) {
+        for (int k = 0; k < 8; ++k) bk[k] = 0ull;
+        for (int w = 0; w < 4; ++w) {
           const int at = (w * 64 + r) * 18;
           M = fmaxf(M, tb[at + 16]);
           for (int e = 0; e < 8; ++e) {
-            const float xv = tb[at + e];
             const int xi = tbi[at + 8 + e];
-            if (xv > bv[7]) {
-              bool ge[8];
+            if (xi < 0) break;                     // a list is filled from the front
+            const unsigned long long xk = sx_pack(tb[at + e], (uint32_t)xi);
+            if (xk > bk[7]) {
+              bool gt[8];
 #pragma unroll
-              for (int k = 0; k < 8; ++k) ge[k] = bv[k] >= xv;
+              for (int k = 0; k < 8; ++k) gt[k] = bk[k] > xk;
 #pragma unroll
-              for (int k = 7; k >= 1; --k) {
-                bv[k] = ge[k] ? bv[k] : (ge[k - 1] ? xv : bv[k - 1]);
-                bi[k] = ge[k] ? bi[k] : (ge[k - 1] ? xi : bi[k - 1]);
-              }
-              if (!ge[0]) { bv[0] = xv; bi[0] = xi; }
+              for (int k = 7; k >= 1; --k) bk[k] = gt[k] ? bk[k] : (gt[k - 1] ? xk : bk[k - 1]);
+              if (!gt[0]) bk[0] = xk;
             }
           }
         }
@@ -519,7 +537,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
         SxHeadPartial hp;
 #pragma unroll
         for (int k = 0; k < SX_MAX_TOPK; ++k)
-          hp.top[k] = (k < p.T && bi[k] >= 0) ? sx_pack(bv[k], (uint32_t)bi[k]) : 0ull;
+          hp.top[k] = (k < p.T) ? bk[k] : 0ull;
         hp.m = (L > 0.f) ? M * 0.6931471805599453f : -INFINITY;
         hp.l = L;
         out[r] = hp;
@@ -529,7 +547,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int tile = item / p.splits;
         const int sp = item % p.splits;
-        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag))) break;
+        if (!epi_all(mbar_wait(smem_u32(&tfull[acc]), acc_phase, abort_flag, p.wait_limit))) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * p.acc_cols);
         const int n = tile * SX_TILE_M + et;
@@ -550,17 +568,50 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
       }
     }
   }
-  if (*abort_flag) {
-    // a wait ran out: report, give copies already in flight time to land, then tear down
-    if (threadIdx.x == 0) sx_set_status(p.status, SX_ERR_TIMEOUT);
-    for (int i = 0; i < 64; ++i) __nanosleep(20000);
+  tc_teardown(abort_flag, p.status, tmem_base, (uint32_t)p.tmem_cols);
+}
+
+// Give-up path of the bounded waits, on its own: a CTA with the GEMM kernel's thread layout allocates
+// TMEM, then every role waits on a barrier that nothing ever arrives at (no copy is in flight).  The
+// first wait to run out raises the abort flag, the others see it at their next poll, and the CTA leaves
+// through the same tear-down as the GEMM kernel: SX_ERR_TIMEOUT in the status word, TMEM freed, a
+// normal return.  Used by the tests; `limit` is small there.
+__global__ void __launch_bounds__(192, 1) sx_wait_selftest_kernel(uint32_t limit, int32_t *status, int32_t *reached) {
+  __shared__ __align__(8) uint64_t bars[3];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_word;
+  volatile int *abort_flag = &abort_word;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 3; ++i) mbar_init(smem_u32(&bars[i]), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    tc_alloc(smem_u32(&tmem_slot), 32u);
+    tc_relinquish();
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    tc_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  bool ok = false;
+  if (warp == 0) {
+    if (lane == 0) ok = mbar_wait(smem_u32(&bars[0]), 0u, abort_flag, limit);                 // producer's wait
+  } else if (warp == 1) {
+    if (lane == 0) ok = mbar_wait(smem_u32(&bars[1]), 0u, abort_flag, limit * 4u);            // MMA issuer's wait
+  } else {
+    ok = epi_all(mbar_wait(smem_u32(&bars[2]), 0u, abort_flag, limit * 4u));                  // epilogue's wait
   }
+  if (ok) atomicAdd(reached, 1);           // stays 0: no wait may report success
+  tc_teardown(abort_flag, status, tmem_base, 32u);
+  if (threadIdx.x == 0) atomicAdd(reached + 1, 1);      // CTAs that returned through the tear-down
+}
+
+sx_status sx_launch_wait_selftest(uint32_t limit, int ctas, int32_t *status, int32_t *reached, cudaStream_t st) {
+  if (limit < 1 || limit > (1u << 20) || ctas < 1 || ctas > 1024) return SX_ERR_INVALID_ARG;
+  sx_wait_selftest_kernel<<<ctas, 192, 0, st>>>(limit, status, reached);
+  return sx_rc(cudaGetLastError());
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -613,6 +664,7 @@ static bool fill_common(SxTcParams &p, int n_rows, int K, int R, size_t epi_byte
   if (p.nmma > 256) return false;
   p.num_tiles = (n_rows + SX_TILE_M - 1) / SX_TILE_M;
   p.acc_cols = p.nmma;
+  p.wait_limit = SX_WAIT_LIMIT;
   p.tmem_cols = pow2_at_least(2 * p.nmma);
   const size_t stage_bytes = SX_A_BYTES + (size_t)p.nmma * 128;
   const size_t fixed = 1024 + 256 + 64 + epi_bytes + 64;
@@ -627,9 +679,12 @@ static size_t smem_bytes(const SxTcParams &p, size_t epi_bytes) {
   return 1024 + (size_t)p.stages * (SX_A_BYTES + (size_t)p.nmma * 128) + (size_t)(2 * p.stages + 4) * 8 + 16 + epi_bytes + 64;
 }
 
-void sx_gemm_init(int device) {
-  cudaFuncSetAttribute(sx_tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
-  cudaFuncSetAttribute(sx_tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX);
+sx_status sx_gemm_init(int device) {
+  (void)device;
+  if (cudaFuncSetAttribute(sx_tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX) != cudaSuccess ||
+      cudaFuncSetAttribute(sx_tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_SMEM_MAX) != cudaSuccess)
+    return SX_ERR_CUDA;
+  return SX_OK;
 }
 
 // Choose the K split: fill the SMs in whole waves, keep at least 4 k-blocks per item, and use at

@@ -32,11 +32,11 @@ __global__ void sx_embed_concat_kernel(int H, int V, const bf16 *feat, SxIndex f
   }
 }
 
-void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
+sx_status sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
                             SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status, cudaStream_t st) {
   int threads = ((sh.H / 8 + 31) / 32) * 32;
   if (threads > 512) threads = 512;
-  sx_launch(sx_embed_concat_kernel, dim3(R), dim3(threads), 0, st, sh.H, sh.V, feat, fi, tok, ti, embed, u, status);
+  return sx_rc(sx_launch(sx_embed_concat_kernel, dim3(R), dim3(threads), 0, st, sh.H, sh.V, feat, fi, tok, ti, embed, u, status));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -117,15 +117,13 @@ sx_finish_norm_kernel(int H, float eps, const float *part, int splits, size_t sp
   }
 }
 
-void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+sx_status sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
                            bf16 *out_user, SxIndex ui, cudaStream_t st, int user_gets_v) {
   int threads = ((sh.H / 4 + 31) / 32) * 32;
   if (threads > 1024) threads = 1024;
-  if (sh.H * 6 > 48 * 1024)
-    cudaFuncSetAttribute(sx_finish_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.H * 6);
-  sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * (sizeof(float) + sizeof(bf16)), st, sh.H, sh.eps, part,
-            splits, split_stride, residual, gamma, out_v, out_n, out_user, ui, user_gets_v);
+  return sx_rc(sx_launch(sx_finish_norm_kernel, dim3(R), dim3(threads), sh.H * (sizeof(float) + sizeof(bf16)), st, sh.H, sh.eps, part,
+            splits, split_stride, residual, gamma, out_v, out_n, out_user, ui, user_gets_v));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -205,16 +203,24 @@ sx_fused_input_kernel(int H, int V, float eps, const float *part, int splits, si
   }
 }
 
-void sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+sx_status sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *feat, SxIndex fi, const int32_t *tok, SxIndex ti, const bf16 *embed,
                            const bf16 *gamma_e, const bf16 *gamma_h, bf16 *x_out, bf16 *u, int32_t *status,
                            cudaStream_t st) {
   int threads = ((sh.H / 4 + 31) / 32) * 32;
   if (threads > 1024) threads = 1024;
-  if (sh.H * 8 > 48 * 1024)
-    cudaFuncSetAttribute(sx_fused_input_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, sh.H * 8);
-  sx_launch(sx_fused_input_kernel, dim3(R), dim3(threads), (size_t)sh.H * 8, st, sh.H, sh.V, sh.eps, part, splits,
-            split_stride, feat, fi, tok, ti, embed, gamma_e, gamma_h, x_out, u, status);
+  return sx_rc(sx_launch(sx_fused_input_kernel, dim3(R), dim3(threads), (size_t)sh.H * 8, st, sh.H, sh.V, sh.eps, part, splits,
+            split_stride, feat, fi, tok, ti, embed, gamma_e, gamma_h, x_out, u, status));
+}
+
+// The two row kernels above keep a row (and its gain, or the embedding row) in shared memory: opt in,
+// once per device, to the size the largest supported hidden width needs.
+sx_status sx_kernels_init(int device) {
+  (void)device;
+  if (cudaFuncSetAttribute(sx_finish_norm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_MAX_H * 6) != cudaSuccess ||
+      cudaFuncSetAttribute(sx_fused_input_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SX_MAX_H * 8) != cudaSuccess)
+    return SX_ERR_CUDA;
+  return SX_OK;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -277,14 +283,14 @@ __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, 
   dst[i + half] = y2;
 }
 
-void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
+sx_status sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
                                cudaStream_t st) {
   int threads = ((sh.d / 2 + 31) / 32) * 32;
   // q_out == nullptr: only the K and V heads (commit)
   const int head_begin = q_out ? 0 : sh.nq;
-  sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv - head_begin, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv,
-            sh.d, (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, head_begin, status);
+  return sx_rc(sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv - head_begin, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv,
+            sh.d, (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, head_begin, status));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -351,19 +357,19 @@ __global__ void sx_commit_advance_kernel(int B, const int32_t *accept_len, int32
   if (b < B) cache_len[b] += accept_len[b] + 1;
 }
 
-void sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
+sx_status sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
                              const int32_t *path, int path_stride, const int32_t *accept_len, const int32_t *recover,
                              const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0, int32_t *status, cudaStream_t st,
                              int32_t *tok_rows) {
   int threads = ((sh.H / 8 + 31) / 32) * 32;
   if (threads > 512) threads = 512;
   const int FW = tok_rows ? 3 * sh.H : sh.H;
-  sx_launch(sx_commit_gather_kernel, dim3(B * M + B), dim3(threads), 0, st, B, M, P, sh.H, FW, sh.V, th, cand, path,
-            path_stride, accept_len, recover, embed, u, tok_rows, feat0, tok0, status);
+  return sx_rc(sx_launch(sx_commit_gather_kernel, dim3(B * M + B), dim3(threads), 0, st, B, M, P, sh.H, FW, sh.V, th, cand, path,
+            path_stride, accept_len, recover, embed, u, tok_rows, feat0, tok0, status));
 }
 
-void sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st) {
-  sx_launch(sx_commit_advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, B, accept_len, cache_len);
+sx_status sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st) {
+  return sx_rc(sx_launch(sx_commit_advance_kernel, dim3((B + 127) / 128), dim3(128), 0, st, B, accept_len, cache_len));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -387,10 +393,10 @@ __global__ void sx_finish_swiglu_kernel(int F, const float *part, int splits, si
   *reinterpret_cast<uint2 *>(m_out + (size_t)r * F + i) = w;
 }
 
-void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+sx_status sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                              bf16 *m_out, cudaStream_t st) {
   dim3 grid((sh.F / 4 + 127) / 128, R);
-  sx_launch(sx_finish_swiglu_kernel, grid, dim3(128), 0, st, sh.F, part, splits, split_stride, m_out);
+  return sx_rc(sx_launch(sx_finish_swiglu_kernel, grid, dim3(128), 0, st, sh.F, part, splits, split_stride, m_out));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -479,14 +485,14 @@ sx_head_finalize_kernel(const SxHeadPartial *parts, int G, int part_stride, int 
   }
 }
 
-void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
+sx_status sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
                              float *logp_out, float *sig_out, SxIndex si, cudaStream_t st, SxNextInput nx,
                              const int32_t *map, int Vd) {
   int threads = ((G + 31) / 32) * 32;              // one thread per CTA of the head kernel (G <= SM count)
   if (threads < 128) threads = 128;
-  sx_launch(sx_head_finalize_kernel, dim3(R), dim3(threads), 0, st, parts, G, part_stride, T, lse, z, S, sh.act[0],
-            sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx, map, Vd);
+  return sx_rc(sx_launch(sx_head_finalize_kernel, dim3(R), dim3(threads), 0, st, parts, G, part_stride, T, lse, z, S, sh.act[0],
+            sh.act[1], sh.act[2], tok_out, toi, logp_out, sig_out, si, nx, map, Vd));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -508,9 +514,9 @@ __global__ void sx_chain_layout_kernel(int B, int K, int S, const int32_t *tok0,
     for (int s = 0; s < S; ++s) o.slot_signal_d[(size_t)i * S + s] = __int_as_float(0x7fc00000);
 }
 
-void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st) {
+sx_status sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st) {
   const int n = B * (K + 1);
-  sx_launch(sx_chain_layout_kernel, dim3((n + 127) / 128), dim3(128), 0, st, B, K, S, tok0, o);
+  return sx_rc(sx_launch(sx_chain_layout_kernel, dim3((n + 127) / 128), dim3(128), 0, st, B, K, S, tok0, o));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -563,10 +569,10 @@ __global__ void sx_accept_kernel(int B, int P, const int32_t *cand, const int32_
   }
 }
 
-void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
+sx_status sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                       int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st) {
-  sx_launch(sx_accept_kernel, dim3((B + 3) / 4), dim3(128), 0, st, B, P, cand, parent, target, accept_len, path,
-            path_stride, recover);
+  return sx_rc(sx_launch(sx_accept_kernel, dim3((B + 3) / 4), dim3(128), 0, st, B, P, cand, parent, target, accept_len, path,
+            path_stride, recover));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -666,7 +672,7 @@ __global__ void sx_exit_kernel(int B, int P, int S, int V, SxExitParams p, float
   for (int i = 0; i < S; ++i) smoothed[(size_t)b * S + i] = x[i];
 }
 
-void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
+sx_status sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
                     const float *slot_signal, const int32_t *cand, const int32_t *path, int path_stride,
                     const int32_t *accept_len, const int32_t *recover, int32_t *exit_flag,
                     int32_t *accept_out, int32_t *recover_out, float *smoothed, int V, int32_t *status,
@@ -680,9 +686,9 @@ void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_s
   p.stop_tok = cfg.stop_think_token;
   p.smoothing = cfg.smoothing; p.window = cfg.window;
   p.hist = state.hist_d; p.par_sum = state.par_sum_d; p.par_n = state.par_n_d;
-  sx_launch(sx_exit_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, S, V, p, state.x_d, state.n_updates_d,
+  return sx_rc(sx_launch(sx_exit_kernel, dim3((B + 31) / 32), dim3(32), 0, st, B, P, S, V, p, state.x_d, state.n_updates_d,
             state.thinking_d, slot_signal, cand, path, path_stride, accept_len, recover, exit_flag, accept_out,
-            recover_out, smoothed, status);
+            recover_out, smoothed, status));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -745,9 +751,9 @@ __global__ void sx_tree_expand_kernel(SxTree t, int round, const int32_t *tok_rt
   }
 }
 
-void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
+sx_status sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
                            cudaStream_t st) {
-  sx_launch(sx_tree_expand_kernel, dim3(B), dim3(64), 0, st, t, round, tok_rt, logp_rt);
+  return sx_rc(sx_launch(sx_tree_expand_kernel, dim3(B), dim3(64), 0, st, t, round, tok_rt, logp_rt));
 }
 
 __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_iter_out o) {
@@ -799,9 +805,9 @@ __global__ void sx_tree_layout_kernel(SxTree t, int S, const int32_t *tok0, sx_i
   }
 }
 
-void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
+sx_status sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
                            cudaStream_t st) {
-  sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)3 * t.NC * sizeof(int), st, t, S, tok0, o);
+  return sx_rc(sx_launch(sx_tree_layout_kernel, dim3(B), dim3(256), (size_t)3 * t.NC * sizeof(int), st, t, S, tok0, o));
 }
 
 // ---------------------------------------------------------------------------------------
@@ -986,15 +992,15 @@ int sx_spec_sample_slices(int rows, int V, int sm_count) {
 }
 size_t sx_spec_sample_ws_bytes(int rows) { return (size_t)rows * SX_SPEC_MAX_SLICES * sizeof(SxSpecPartial); }
 
-void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
+sx_status sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
                            const int32_t *cand_tok, SxSample smp, void *parts_ws, int sm_count, int32_t *target_tok,
                            int32_t *status, cudaStream_t st) {
   const int rows = B * P, S = sx_spec_sample_slices(rows, V, sm_count);
   const int len = (((V + S - 1) / S + 3) / 4) * 4;
   SxSpecPartial *parts = (SxSpecPartial *)parts_ws;
-  sx_launch(sx_spec_partials_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits, smp.temp,
-            parts);
-  sx_launch(sx_spec_draw_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits, cand_tok, smp,
-            parts, status);
-  sx_launch(sx_spec_pick_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, P, V, S, rows, cand_tok, parts, target_tok);
+  SX_TRY(sx_rc(sx_launch(sx_spec_partials_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits,
+                         smp.temp, parts)));
+  SX_TRY(sx_rc(sx_launch(sx_spec_draw_kernel, dim3(rows, S), dim3(512), 0, st, P, V, len, target_logits, draft_logits,
+                         cand_tok, smp, parts, status)));
+  return sx_rc(sx_launch(sx_spec_pick_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, P, V, S, rows, cand_tok, parts, target_tok));
 }

@@ -9,6 +9,11 @@ struct SxIndex {
   int mul, add;
 };
 
+#define SX_MAX_H 16384           // widest hidden state the row kernels hold in shared memory
+#define SX_TRY(e) do { sx_status _s = (e); if (_s != SX_OK) return _s; } while (0)
+static inline sx_status sx_rc(cudaError_t e) { return e == cudaSuccess ? SX_OK : SX_ERR_CUDA; }
+sx_status sx_kernels_init(int device);
+
 struct SxShape {
   int H, nq, nkv, d, F, V, S, page;
   int arch;                    // SX_ARCH_CONCAT | SX_ARCH_FUSED3
@@ -17,42 +22,42 @@ struct SxShape {
   int act[SX_MAX_SIGNALS];
 };
 
-void sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
+sx_status sx_launch_embed_concat(const SxShape &sh, int R, const bf16 *feat, SxIndex fi, const int32_t *tok,
                             SxIndex ti, const bf16 *embed, bf16 *u, int32_t *status, cudaStream_t st);
 
 // v = sum_s part[s][r][:] (+ residual); out_v = bf16(v); out_n = bf16(rmsnorm(out_v) * gamma);
 // out_user (optional) receives out_n at row index ui(r).
-void sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+sx_status sx_launch_finish_norm(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *residual, const bf16 *gamma, bf16 *out_v, bf16 *out_n,
                            bf16 *out_user, SxIndex ui, cudaStream_t st, int user_gets_v = 0);
 
 // Layer with three-feature fusion: x_out[r] = bf16(sum of the fc partials) (part != nullptr) or the
 // hidden of row fi(r) of `feat`; u[r] = [rmsnorm(E[token]) * gamma_e ; rmsnorm(x) * gamma_h].
-void sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
+sx_status sx_launch_fused_input(const SxShape &sh, int R, const float *part, int splits, size_t split_stride,
                            const bf16 *feat, SxIndex fi, const int32_t *tok, SxIndex ti, const bf16 *embed,
                            const bf16 *gamma_e, const bf16 *gamma_h, bf16 *x_out, bf16 *u, int32_t *status,
                            cudaStream_t st);
 
-void sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
+sx_status sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
                                cudaStream_t st);
 
-void sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
+sx_status sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
                              const int32_t *path, int path_stride, const int32_t *accept_len,
                              const int32_t *recover, const bf16 *embed, bf16 *u, bf16 *feat0, int32_t *tok0,
                              int32_t *status, cudaStream_t st, int32_t *tok_rows = nullptr);
-void sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st);
+sx_status sx_launch_commit_advance(int B, const int32_t *accept_len, int32_t *cache_len, cudaStream_t st);
 
-void sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits,
+sx_status sx_launch_finish_swiglu(const SxShape &sh, int R, const float *part, int splits,
                              size_t split_stride, bf16 *m_out, cudaStream_t st);
 
 // decode attention (sx_attention.cu).  B sequences with nr rows each this round, E drafted slots
 // behind the cached prefix (this round's rows included).
 bool sx_attn_supported(const SxShape &sh);
-void sx_attn_init(int device);
+sx_status sx_attn_init(int device);
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count);
 size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_count);
-void sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
+sx_status sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
                          const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
 
 // Optional fusion for chain drafting: the merge kernel also writes the next round's input row
@@ -62,18 +67,18 @@ struct SxNextInput {
   bf16 *u;
   int H, V;
 };
-void sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
+sx_status sx_launch_head_finalize(const SxShape &sh, int R, const SxHeadPartial *parts, int G, int part_stride,
                              int T, int lse, const float *z, int S, int32_t *tok_out, SxIndex toi,
                              float *logp_out, float *sig_out, SxIndex si, cudaStream_t st,
                              SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
                              const int32_t *map = nullptr, int Vd = 0);   // map: draft id -> token id
 
-void sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st);
+sx_status sx_launch_chain_layout(int B, int K, int S, const int32_t *tok0, const sx_iter_out &o, cudaStream_t st);
 
-void sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
+sx_status sx_launch_accept(int B, int P, const int32_t *cand, const int32_t *parent, const int32_t *target,
                       int32_t *accept_len, int32_t *path, int path_stride, int32_t *recover, cudaStream_t st);
 
-void sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
+sx_status sx_launch_exit(int B, int P, int S, const sx_exit_cfg &cfg, const sx_exit_state &state,
                     const float *slot_signal, const int32_t *cand, const int32_t *path, int path_stride,
                     const int32_t *accept_len, const int32_t *recover, int32_t *exit_flag,
                     int32_t *accept_out, int32_t *recover_out, float *smoothed, int V, int32_t *status,
@@ -91,9 +96,9 @@ struct SxTree {
   uint64_t *next_mask;                                         // [B*T]
   float *row_sig;                                              // [B, rows, S]
 };
-void sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
+sx_status sx_launch_tree_expand(const SxTree &t, int B, int round, const int32_t *tok_rt, const float *logp_rt,
                            cudaStream_t st);
-void sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
+sx_status sx_launch_tree_layout(const SxTree &t, int B, int S, const int32_t *tok0, const sx_iter_out &o,
                            cudaStream_t st);
 
 // ---- GEMMs (sx_gemm_tc.cu) ----------------------------------------------------------------
@@ -106,7 +111,9 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
 // weights tile by tile ([row tile][k-block][128][64], zero padded): elements of that layout, and the repack
 size_t sx_tiled_elems(int N, int K);
 sx_status sx_launch_tile_weight(const bf16 *src, int N, int K, bf16 *dst, cudaStream_t st);
-void sx_gemm_init(int device);
+sx_status sx_gemm_init(int device);
+// give-up path of the bounded mbarrier waits on its own (see sx_selftest_bounded_wait)
+sx_status sx_launch_wait_selftest(uint32_t limit, int ctas, int32_t *status, int32_t *reached, cudaStream_t st);
 // Sampled verification: with temp > 0 the plain-argmax head returns, per row, the arg max of
 // logit + temp * Gumbel noise, i.e. a draw from softmax(logits / temp).  Row r of the launch is
 // verify slot (row0 + r) % P of sequence (row0 + r) / P; the noise of (sequence, slot, token id)
@@ -134,7 +141,7 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
 // pick); parts_ws holds sx_spec_sample_ws_bytes(B * P) bytes.
 #define SX_SPEC_MAX_SLICES 64
 size_t sx_spec_sample_ws_bytes(int rows);
-void sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
+sx_status sx_launch_spec_sample(int B, int P, int V, const float *target_logits, const float *draft_logits,
                            const int32_t *cand_tok, SxSample smp, void *parts_ws, int sm_count, int32_t *target_tok,
                            int32_t *status, cudaStream_t st);
 int sx_head_max_rows(int T, int lse);

@@ -43,7 +43,7 @@ static sx_status noalloc_setup(int dev, void **scratch, int *sm) {
     if (cudaGetSymbolAddress(&p, sx_noalloc_scratch) != cudaSuccess || p == nullptr) return SX_ERR_CUDA;
     int n = 0;
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return SX_ERR_CUDA;
-    sx_gemm_init(dev);
+    if (sx_gemm_init(dev) != SX_OK) return SX_ERR_CUDA;
     g_scratch_ptr[dev] = p;
     g_sm_count[dev] = n;
     g_ready[dev] = true;
@@ -71,7 +71,9 @@ extern "C" sx_status sx_verify_noalloc(const void *target_head_d, int32_t vocab,
   int sm = 0;
   sx_status rc = noalloc_setup(dev, &scratch, &sm);
   if (rc != SX_OK) return rc;
-  if (sm > SX_NOALLOC_MAX_CTAS) sm = SX_NOALLOC_MAX_CTAS;      // fewer CTAs, each takes more tiles
+  // The head kernel never uses more CTAs than the SM count it is given (a CTA takes several tiles instead),
+  // and every CTA leaves one slice: capping that count here keeps the launch inside the array.
+  if (sm > SX_NOALLOC_MAX_CTAS) sm = SX_NOALLOC_MAX_CTAS;
   cudaStream_t st = (cudaStream_t)stream;
   const int R = batch * P;
   SxHeadPartial *parts = reinterpret_cast<SxHeadPartial *>(scratch);
@@ -79,12 +81,11 @@ extern "C" sx_status sx_verify_noalloc(const void *target_head_d, int32_t vocab,
   rc = sx_launch_head((const bf16 *)target_head_d, vocab, vocab, H, (const bf16 *)target_hidden_d, R, 1, 0, parts,
                       SX_NOALLOC_MAX_ROWS, &G, nullptr, 0, sm, status_d, st);
   if (rc != SX_OK) return rc;
-  if (G > SX_NOALLOC_MAX_CTAS) return SX_ERR_STATIC_LIMIT;
   SxShape sh;
   memset(&sh, 0, sizeof(sh));
   sh.H = H; sh.V = vocab;
-  sx_launch_head_finalize(sh, R, parts, G, SX_NOALLOC_MAX_ROWS, 1, 0, nullptr, 0, target_tok_d, SxIndex{nullptr, 1, 0},
-                          nullptr, nullptr, SxIndex{nullptr, 1, 0}, st);
-  sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st);
+  SX_TRY(sx_launch_head_finalize(sh, R, parts, G, SX_NOALLOC_MAX_ROWS, 1, 0, nullptr, 0, target_tok_d, SxIndex{nullptr, 1, 0},
+                          nullptr, nullptr, SxIndex{nullptr, 1, 0}, st));
+  SX_TRY(sx_launch_accept(batch, P, cand_tok_d, parent_d, target_tok_d, accept_len_d, path_d, path_stride, recover_tok_d, st));
   return SX_OK;
 }

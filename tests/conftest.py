@@ -12,7 +12,10 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
 
 
-def pytest_collection_modifyitems(config, items):
-    # a GPU-marked test on a box without a device is an error, not a silent skip,
-    # unless the run deselected the marker
-    pass
+def pytest_runtest_setup(item):
+    # a GPU-marked test that was selected on a box without a device fails loudly instead of
+    # passing on some fallback or being skipped silently (deselect with -m "not gpu")
+    if "gpu" in item.keywords:
+        import torch
+        if not torch.cuda.is_available():
+            pytest.fail("this test needs a CUDA device; deselect it with -m \"not gpu\"", pytrace=False)

@@ -18,8 +18,9 @@ hiddens fed to verification, and its drift from the GPU is reported).
 """
 from __future__ import annotations
 
+import dataclasses
 from dataclasses import dataclass, field
-from typing import Dict, List
+from typing import Dict, List, Optional
 
 import torch
 
@@ -37,14 +38,35 @@ class ParityError(AssertionError):
 
 
 @dataclass
+class FreeRun:
+    """The GPU against the oracle's own free-running pass (no hook of any kind): per draft round (chain) or
+    tree depth, over the sequences whose decisions have all agreed so far ("in step")."""
+    hidden_rel: List[float] = field(default_factory=list)    # max relative L2 over the rows in step
+    signal_err: List[float] = field(default_factory=list)    # max absolute signal difference over them
+    in_step: List[int] = field(default_factory=list)         # sequences compared in that round
+    diverged: List[str] = field(default_factory=list)        # first differing decision per sequence, with its margin
+    tail_equal: Optional[bool] = None                        # verify + exit outputs equal the free-running oracle's
+
+    def table(self, name: str) -> str:
+        rows = [f"{name}: free-running comparison (oracle pass without hooks)",
+                "  round  sequences-in-step  hidden rel-L2 (max)  signal |err| (max)"]
+        for k, (h, e, n) in enumerate(zip(self.hidden_rel, self.signal_err, self.in_step), start=1):
+            rows.append(f"  {k:5d}  {n:17d}  {h:19.3e}  {e:18.3e}")
+        rows.append("  first differing decision per sequence: " + ("none" if not self.diverged else ""))
+        rows += [f"    {d}" for d in self.diverged]
+        rows.append(f"  verify + exit outputs equal the free-running oracle's: {self.tail_equal}")
+        return "\n".join(rows)
+
+
+@dataclass
 class Report:
-    exempt: List[str] = field(default_factory=list)
+    exempt: List[str] = field(default_factory=list)          # near-tie decisions adopted from the GPU
+    exit_near_threshold: List[str] = field(default_factory=list)   # exit flags that differ with a smoothed value at its threshold
     max_signal_err: float = 0.0
     max_hidden_rel: float = 0.0
     accept_len: List[int] = field(default_factory=list)
     exit_flag: List[int] = field(default_factory=list)
-    free_running_tokens_equal: bool = True
-    free_running_hidden_rel: float = 0.0
+    free: FreeRun = field(default_factory=FreeRun)
 
 
 def _rel_l2(a: torch.Tensor, b: torch.Tensor) -> float:
@@ -225,7 +247,7 @@ def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, 
                        for i in range(slot_signal.shape[2]))
             if not near:
                 raise ParityError(f"exit flag b={b}: gpu {int(g_flag[b])} vs {int(e.exit_flag[b])}")
-            rep.exempt.append(f"exit flag b={b} (smoothed value at threshold)")
+            rep.exit_near_threshold.append(f"exit flag b={b} (smoothed value within 1e-3 of its threshold)")
             continue
         if int(g_Lo[b]) != int(e.accept_len[b]) or int(g_ro[b]) != int(e.recover_tok[b]):
             raise ParityError(f"exit outputs b={b}")
@@ -258,8 +280,64 @@ def _compare_signals(rep: Report, g: torch.Tensor, o: torch.Tensor):
         raise ParityError(f"signals differ by {err}")
 
 
+def _free_fail(strict: bool, k: int, msg: str):
+    """Round 1 sees identical inputs on both sides, so the stated tolerances bind there without any hook;
+    later rounds bind only where the caller asks for the whole free-running pass (strict)."""
+    if strict or k == 1:
+        raise ParityError("free-running " + msg)
+
+
+def _free_chain(rep: Report, wl, d0, g_tok, g_hid, g_sig, strict: bool) -> None:
+    fr = rep.free
+    live = [True] * wl.B
+    for k in range(1, wl.K + 1):
+        hr, se, n = 0.0, 0.0, 0
+        for b in range(wl.B):
+            if not live[b]:
+                continue
+            n += 1
+            hr = max(hr, _rel_l2(g_hid[b, k - 1].to(torch.float64), d0.hidden[b, k - 1]))
+            se = max(se, float((g_sig[b, k - 1] - d0.slot_signal[b, k - 1]).abs().max()))
+            if int(g_tok[b, k]) != int(d0.cand_tok[b, k]):
+                gap = float(d0.gap[b, k - 1])
+                fr.diverged.append(f"b={b} round={k}: gpu token {int(g_tok[b, k])} vs oracle {int(d0.cand_tok[b, k])}, "
+                                   f"oracle top-2 gap {gap:.3e}")
+                live[b] = False
+                if gap >= REL_GAP:
+                    _free_fail(strict, k, f"draft token b={b} round={k} differs with gap {gap:.3e}")
+        fr.hidden_rel.append(hr)
+        fr.signal_err.append(se)
+        fr.in_step.append(n)
+        if hr > HIDDEN_REL_L2:
+            _free_fail(strict, k, f"hidden round {k}: rel L2 {hr:.3e}")
+        if se > SIGNAL_ATOL:
+            _free_fail(strict, k, f"signals round {k}: {se:.3e}")
+
+
+def _free_tail(rep: Report, model, cfg, state0, th, d0, parent, out, K: int, strict: bool) -> None:
+    """With every draft decision in step, the verify and exit outputs are compared with the free-running
+    oracle's directly (its own tokens, its own signals)."""
+    fr = rep.free
+    if fr.diverged:
+        return
+    v = orc.verify(model, th, d0.cand_tok, parent)
+    e = orc.exit_update(cfg, state0.clone(), d0.slot_signal, d0.cand_tok, v.path, v.accept_len, v.recover_tok)
+    same = (torch.equal(out["target_tok_d"].cpu().to(torch.int64), v.target_tok)
+            and out["accept_len_d"].cpu().tolist() == v.accept_len.tolist()
+            and out["exit_flag_d"].cpu().tolist() == e.exit_flag.tolist()
+            and out["accept_len_out_d"].cpu().tolist() == e.accept_len.tolist()
+            and out["recover_tok_out_d"].cpu().tolist() == e.recover_tok.tolist())
+    fr.tail_equal = bool(same)
+    if strict and not same:
+        raise ParityError("free-running verify / exit outputs differ")
+    if strict:
+        err = float((out["smoothed_d"].cpu().to(torch.float64) - e.smoothed).abs().max())
+        if err > SIGNAL_ATOL:
+            raise ParityError(f"free-running smoothed signals differ by {err}")
+
+
 def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0: orc.ExitState = None,
-              sx: binding.SpecExit = None, sample=None) -> Report:
+              sx: binding.SpecExit = None, sample=None, strict_free: bool = False) -> Report:
     wl = case.wl
     rep = Report()
     cfg = cfg or harness.default_exit_cfg(wl)
@@ -283,7 +361,7 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     sx.check_status("sx_spec_exit_iter")
     g_tok = out["cand_tok_d"].cpu().to(torch.int64)
     g_hid = out["hidden_d"].cpu()
-    rep.free_running_tokens_equal = bool(torch.equal(g_tok, d0.cand_tok))
+    _free_chain(rep, wl, d0, g_tok, g_hid, out["slot_signal_d"].cpu().to(torch.float64), strict_free)
     # Replay: every round of the oracle restarts from the GPU's state (its previous hidden and the
     # K/V rows it appended), so each round is compared on identical inputs.  Without this the two
     # runs drift apart round by round: bf16 re-rounding turns summation-order noise into ulp-level
@@ -306,8 +384,6 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
                         before_round=before_round, head_input=head_input, sample=dsample)
     if not torch.equal(g_tok, d.cand_tok):
         raise ParityError("draft tokens differ after adopting near-ties")
-    rep.free_running_hidden_rel = max(_rel_l2(g_hid[b, wl.K - 1].to(torch.float64), d0.hidden[b, wl.K - 1])
-                                      for b in range(wl.B))
     for b in range(wl.B):
         _compare_rows(rep, f"b={b}", g_hid[b], d.hidden[b])
     _compare_signals(rep, out["slot_signal_d"].cpu(), d.slot_signal)
@@ -315,6 +391,8 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     want_par = torch.arange(-1, wl.K).repeat(wl.B, 1)
     if not torch.equal(out["parent_d"].cpu().to(torch.int64), want_par):
         raise ParityError("chain parents")
+    if sample is None:
+        _free_tail(rep, model, cfg, state0, th, d0, None, out, wl.K, strict_free)
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, None, d.slot_signal, out,
                   {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample, draft_logits=d.logits)
     if own:
@@ -322,8 +400,58 @@ def run_chain(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), state0
     return rep
 
 
+def _free_tree(rep: Report, wl, d0, o, strict: bool) -> None:
+    """Depth by depth: hiddens and signals of the rows drafted at that depth, then the decisions taken from
+    them (each row's top-k children, the candidates chosen for expansion), for the sequences whose
+    decisions have all agreed so far; last the kept set."""
+    fr = rep.free
+    T, D = wl.topk, wl.K
+    live = [True] * wl.B
+    g_hid = o["hidden_d"]
+    g_tok, g_row = o["tree_cand_tok_d"], o["tree_cand_row_d"]
+
+    def lost(b, r, what, margin):
+        fr.diverged.append(f"b={b} depth={r}: {what}, oracle margin {margin:.3e}")
+        live[b] = False
+        if margin >= REL_GAP:
+            _free_fail(strict, r, f"tree decision b={b} depth={r} ({what}) differs with margin {margin:.3e}")
+
+    for r in range(1, D + 1):
+        rows = [0] if r == 1 else list(range(1 + (r - 2) * T, 1 + (r - 1) * T))
+        base, cnt = (0, T) if r == 1 else (T + (r - 2) * T * T, T * T)
+        hr, se, n = 0.0, 0.0, 0
+        for b in range(wl.B):
+            if not live[b]:
+                continue
+            n += 1
+            for i in rows:
+                hr = max(hr, _rel_l2(g_hid[b, i].to(torch.float64), d0.hidden[b, i]))
+            by_cid = d0.cands[b]
+            for j, i in enumerate(rows):                                   # the children each row emitted
+                ids = range(base + j * T, base + (j + 1) * T)
+                if [int(g_tok[b, c]) for c in ids] != [by_cid[c].tok for c in ids]:
+                    lost(b, r, f"top-{T} of row {i}", d0.margins.get(("topk", b, i), 0.0))
+                    break
+            if live[b] and r < D:                                          # who gets expanded next
+                ids = range(base, base + cnt)
+                if [int(g_row[b, c]) for c in ids] != [by_cid[c].row for c in ids]:
+                    lost(b, r, "candidates chosen for expansion", d0.margins.get(("expand", b, r), 0.0))
+        fr.hidden_rel.append(hr)
+        fr.in_step.append(n)
+        if hr > HIDDEN_REL_L2:
+            _free_fail(strict, r, f"hidden depth {r}: rel L2 {hr:.3e}")
+    for b in range(wl.B):
+        if live[b] and not torch.equal(o["cand_tok_d"][b].to(torch.int64), d0.cand_tok[b]):
+            lost(b, D, "kept set", d0.margins.get(("keep", b), 0.0))
+    # the root's signal (round 1); deeper rows' signals are compared in the per-round pass
+    se = max(float((o["slot_signal_d"][b, 0].to(torch.float64) - d0.slot_signal[b, 0]).abs().max()) for b in range(wl.B))
+    fr.signal_err = [se] + [float("nan")] * (len(fr.hidden_rel) - 1)
+    if se > SIGNAL_ATOL:
+        _free_fail(strict, 1, f"root signals differ by {se}")
+
+
 def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: binding.SpecExit = None,
-             sample=None) -> Report:
+             sample=None, strict_free: bool = False) -> Report:
     wl = case.wl
     rep = Report()
     cfg = cfg or harness.default_exit_cfg(wl)
@@ -361,6 +489,7 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
                 raise ParityError(f"tree slot b={b} s={s} does not name a generated candidate")
             ks.append(lut[key])
         kept.append(ks)
+    _free_tree(rep, wl, d0, o, strict_free)
     chooser = GpuChooser(rep, tree={"tok": o["tree_cand_tok_d"], "row": o["tree_cand_row_d"], "kept": kept}, T=T, id_map=model.map)
     replay = _kv_replay(sx, case)
     g_hid = o["hidden_d"]
@@ -392,8 +521,33 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
     for b in range(wl.B):
         _compare_rows(rep, f"b={b}", o["hidden_d"][b], d.hidden[b])
     _compare_signals(rep, o["slot_signal_d"], d.slot_signal)
+    if sample is None:
+        _free_tail(rep, model, cfg, state0, th, d0, d0.parent, out, wl.K, strict_free)
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, d.parent, d.slot_signal, out,
                   {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample)
     if own:
         sx.close()
     return rep
+
+
+def periodic_head_case(mode, B, K, topk=1, max_nodes=0, seed=31, scale=20.0):
+    """H = 64 and a vocabulary of 2 SMs + 1 tiles whose head rows repeat with period 128 G - 32."""
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    tiles = 2 * sm + 1
+    per_cta = (tiles + sm - 1) // sm
+    G = (tiles + per_cta - 1) // per_cta
+    M = 128 * G - 32
+    V = tiles * 128 - 3 - 20                       # V + 3 signal rows end 20 rows short of a full tile
+    assert per_cta >= 2 and V > 2 * M
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=V, page=16)
+    wl = synth.Workload("ties", sh, B=B, mode=mode, K=K, topk=topk, max_nodes=max_nodes, len_lo=5, len_hi=30,
+                        seed=seed)
+    case = harness.build_case(wl)
+    w = dict(case.weights)
+    head = w["head"].clone()
+    base = (head[:M].to(torch.float32) * scale).to(torch.bfloat16)
+    for i0 in range(0, V, M):
+        n = min(M, V - i0)
+        head[i0:i0 + n] = base[:n]
+    w["head"] = head
+    return dataclasses.replace(case, weights=w), M

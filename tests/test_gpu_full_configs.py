@@ -1,5 +1,13 @@
-"""Full-size benchmark configurations: CUDA path vs the CPU oracle on the same seeded inputs,
-in the launch configuration bench.py times."""
+"""Full-size benchmark configurations: CUDA path vs the CPU oracle on the same seeded inputs, in both
+weight layouts: tile by tile (what bench.py times by default) and row-major.
+
+Per configuration two comparisons are made and printed (run with -s to see the tables):
+  * round by round on identical inputs (the oracle restarts each round from the GPU's state): every
+    decision exact, hiddens within 2e-2 relative L2, signals within 1e-2; no decision may need the
+    near-tie exemption and no exit flag may sit at its threshold;
+  * against the oracle's own free-running pass, with no hook: round 1 (identical inputs) must meet the same
+    tolerances; later rounds are recorded - drift per round, first differing decision with its margin.
+"""
 import pytest
 
 from paper_2509_24248_b200 import synth
@@ -8,20 +16,40 @@ from tests import harness, parity
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["tiled", "rowmajor"])
+def layout(request):
+    parity.TILED = request.param == "tiled"
+    yield request.param
+    parity.TILED = False
+
+
+DRIFT_PER_ROUND = 7e-3     # envelope of the free-running drift, k * 7e-3 at round k: a regression guard taken from
+#                            the measured growth (which the oracle shows against itself, tests/test_drift_cpu.py),
+#                            not a tolerance of the method
+
+
+def _show(name, layout, rep):
+    for k, h in enumerate(rep.free.hidden_rel, start=1):
+        assert h <= DRIFT_PER_ROUND * k, f"free-running drift at round {k}: {h:.3e}"
+    print(f"\n{name} [{layout}]: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
+          f"at-threshold {rep.exit_near_threshold} signal err {rep.max_signal_err:.2e} "
+          f"hidden rel-L2 (per round, identical inputs) {rep.max_hidden_rel:.2e}")
+    print(rep.free.table(f"{name} [{layout}]"))
+
+
 @pytest.mark.parametrize("name", ["C1", "C2", "C3"])
-def test_chain_config(name):
+def test_chain_config(name, layout):
     wl = synth.workload(name)
     rep = parity.run_chain(harness.build_case(wl, poison_tail=True))
-    print(f"{name}: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
-          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
-    assert len(rep.exempt) <= max(2, wl.B * (wl.K + 1) // 10)
+    _show(name, layout, rep)
+    assert rep.exempt == [] and rep.exit_near_threshold == []
 
 
-def test_tree_config4():
+def test_tree_config4(layout):
     wl = synth.workload("C4")
     rep = parity.run_tree(harness.build_case(wl, poison_tail=True))
-    print(f"C4: accept_len {rep.accept_len} exit {rep.exit_flag} exempt {rep.exempt} "
-          f"signal err {rep.max_signal_err:.2e} hidden rel-L2 {rep.max_hidden_rel:.2e}")
+    _show("C4", layout, rep)
+    assert rep.exempt == [] and rep.exit_near_threshold == []
 
 
 def test_chain_config1_with_a_32k_draft_vocabulary():

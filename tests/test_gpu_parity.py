@@ -25,11 +25,21 @@ def test_chain_zero_cached_tokens():
     parity.run_chain(harness.build_case(_wl(B=2, K=3, len_lo=0, len_hi=0)))
 
 
-def test_chain_config0_exact():
+@pytest.mark.parametrize("tiled", [False, True])
+def test_chain_config0_exact(tiled):
+    """The tiny exactness configuration, held to the whole free-running pass: the oracle runs all K rounds
+    on its own (no hook) and every draft token, accepted length, exit flag and recover token must be equal,
+    every hidden within 2e-2 relative L2 and every signal within 1e-2."""
     wl = synth.workload("C0")
-    rep = parity.run_chain(harness.build_case(wl))
-    print("C0 exempt:", rep.exempt, "accept:", rep.accept_len, "sig err:", rep.max_signal_err,
-          "hid rel:", rep.max_hidden_rel)
+    parity.TILED = tiled
+    try:
+        rep = parity.run_chain(harness.build_case(wl), strict_free=True)
+    finally:
+        parity.TILED = False
+    print(rep.free.table("C0"))
+    assert rep.exempt == [] and rep.exit_near_threshold == []
+    assert rep.free.diverged == [] and rep.free.tail_equal is True
+    assert rep.free.in_step == [wl.B] * wl.K
 
 
 @pytest.mark.parametrize("shape_kw", [dict(H=128, n_q=8, n_kv=1, d=16, F=200, V=333),

@@ -547,11 +547,20 @@ def test_tree_top1_degenerates_to_chain():
 
 
 # ---------------------------------------------------------------- whole forward vs an independent restatement
-def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False):
-    """float64 numpy restatement of one draft position without any intermediate rounding,
-    written against the logical (un-paged) cache.  ``fused3``: the layer with three-feature
-    fusion (f of length 3H goes through fc, f of length H is the residual stream itself) and
-    [norm(embedding) ; norm(x)] as the attention input; then y is returned as well."""
+def _np_bf16(v):
+    """Round-to-nearest-even to bf16 on the bit pattern of the fp32 value (numpy only)."""
+    u = np.asarray(v, dtype=np.float64).astype(np.float32).view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False, rnd=lambda v: v):
+    """float64 numpy restatement of one draft position, written against the logical (un-paged) cache.
+    By default nothing is rounded on the way; ``rnd`` is applied at the points where the method stores a
+    bf16 activation (x, the normed inputs, q / k / v, the attention output, a, m, y, the final hidden).
+    ``fused3``: the layer with three-feature fusion (f of length 3H goes through fc, f of length H is the
+    residual stream itself) and [norm(embedding) ; norm(x)] as the attention input; then y is returned as
+    well."""
     sh, w = case.wl.shape, {k: v.to(torch.float64).numpy() for k, v in case.weights.items()}
     page = sh.page
     n = int(case.kv["cache_len"][b])
@@ -571,8 +580,8 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False):
         x = w["fc"] @ f if f.size == 3 * sh.H else f
         att_in = np.concatenate([norm(w["embed"][tok], w["norm_e"]), norm(x, w["norm1"])])
     else:
-        x = w["fc"] @ np.concatenate([f, w["embed"][tok]])
-        att_in = norm(x, w["norm1"])
+        x = rnd(w["fc"] @ np.concatenate([f, w["embed"][tok]]))
+        att_in = rnd(norm(x, w["norm1"]))
 
     def rot(v):
         out = v.copy()
@@ -584,9 +593,9 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False):
         return out
 
     qkv = w["wqkv"] @ att_in
-    q = rot(qkv[:sh.n_q * sh.d].reshape(sh.n_q, sh.d))
-    k = rot(qkv[sh.n_q * sh.d:(sh.n_q + sh.n_kv) * sh.d].reshape(sh.n_kv, sh.d))
-    v = qkv[(sh.n_q + sh.n_kv) * sh.d:].reshape(sh.n_kv, sh.d)
+    q = rnd(rot(qkv[:sh.n_q * sh.d].reshape(sh.n_q, sh.d)))
+    k = rnd(rot(qkv[sh.n_q * sh.d:(sh.n_q + sh.n_kv) * sh.d].reshape(sh.n_kv, sh.d)))
+    v = rnd(qkv[(sh.n_q + sh.n_kv) * sh.d:].reshape(sh.n_kv, sh.d))
     K = np.concatenate([K, k[None]], axis=0)
     Vv = np.concatenate([Vv, v[None]], axis=0)
     o = np.zeros((sh.n_q, sh.d))
@@ -595,11 +604,12 @@ def _np_forward(case, f, tok, b, n_extra_k, n_extra_v, fused3=False):
         sc = K[:, kvh] @ q[h] / math.sqrt(sh.d)
         p = np.exp(sc - sc.max())
         o[h] = (p / p.sum()) @ Vv[:, kvh]
-    a = x + w["wo"] @ o.reshape(-1)
-    gu = w["wgate_up"] @ norm(a, w["norm2"])
+    o = rnd(o)
+    a = rnd(x + w["wo"] @ o.reshape(-1))
+    gu = w["wgate_up"] @ rnd(norm(a, w["norm2"]))
     gate, up = gu[:sh.F], gu[sh.F:]
-    y = a + w["wdown"] @ (gate / (1 + np.exp(-gate)) * up)
-    g = norm(y, w["normf"])
+    y = rnd(a + w["wdown"] @ rnd(gate / (1 + np.exp(-gate)) * up))
+    g = rnd(norm(y, w["normf"]))
     if fused3:
         return g, w["head"] @ g, k[None], v[None], y
     return g, w["head"] @ g, k[None], v[None]
@@ -621,6 +631,53 @@ def test_full_forward_against_float64_restatement():
     g2, _, _, _ = _np_forward(case, g1, int(d.cand_tok[0, 1]), 0, [k1], [v1])
     rel = np.linalg.norm(d.hidden[0, 1].numpy() - g2) / np.linalg.norm(g2)
     assert rel < 2e-2
+
+
+def test_full_forward_against_float64_restatement_with_the_rounding_points():
+    """The same restatement with bf16 rounding (its own bit-level implementation) at exactly the points
+    where an activation is stored: now the two agree to float64 noise except where a value sits on a
+    rounding boundary, so a misplaced, missing or extra rounding point (an error of a bf16 ulp, 4e-3, on
+    every element of a row) fails, as does any wrong operand."""
+    wl = synth.workload("C0")
+    case = harness.build_case(wl)
+    model = harness.oracle_model(case)
+    d = orc.draft_chain(model, harness.oracle_kv(case), case.f0, case.t0, 3)
+    f, tok, ks, vs = case.f0[0].to(torch.float64).numpy(), int(case.t0[0]), [], []
+    for k in range(3):
+        g, logits, k1, v1 = _np_forward(case, f, tok, 0, ks, vs, rnd=_np_bf16)
+        got = d.hidden[0, k].numpy()
+        rel = np.linalg.norm(got - g) / np.linalg.norm(g)
+        assert rel < 1e-3, (k, rel)
+        assert np.mean(got == g) > 0.97, (k, np.mean(got == g))    # nearly every element bit-identical
+        lg = logits[:wl.shape.V].astype(np.float32)
+        assert int(np.argmax(lg)) == int(d.cand_tok[0, k + 1]) or float(d.gap[0, k]) < 1e-3
+        s1 = 1 / (1 + np.exp(-logits[wl.shape.V:]))
+        assert np.abs(s1 - d.slot_signal[0, k].numpy()).max() < 1e-3
+        # continue from the oracle's own state so that each position is checked on identical inputs
+        f, tok = got, int(d.cand_tok[0, k + 1])
+        ks.append(k1)
+        vs.append(v1)
+
+
+def test_top_gap_is_the_kth_margin_over_the_largest_value():
+    """The margin that decides whether a differing decision is exempt: (k-th largest - (k+1)-th largest) /
+    |largest|, checked for k = 1 and k = 8 against a sorted list, on values with a known answer and on random
+    ones; an off-by-one in k or another denominator fails."""
+    v = torch.tensor([0.5, -4.0, 2.0, 1.0, 8.0, 7.5, 3.0, 2.5, 6.0, 5.0, 4.0, 0.0], dtype=F64)
+    # sorted: 8, 7.5, 6, 5, 4, 3, 2.5, 2, 1, 0.5, 0, -4
+    assert orc.top_gap(v) == pytest.approx((8.0 - 7.5) / 8.0)
+    assert orc.top_gap(v, 1) == pytest.approx(0.0625)
+    assert orc.top_gap(v, 8) == pytest.approx((2.0 - 1.0) / 8.0)
+    assert orc.top_gap(v, 3) == pytest.approx((6.0 - 5.0) / 8.0)
+    assert orc.top_gap(-v) == pytest.approx((4.0 - 0.0) / 4.0)          # largest is 4, runner-up 0
+    g = torch.Generator().manual_seed(77)
+    for _ in range(20):
+        x = torch.randn(500, generator=g, dtype=F64) * 3 - 1.0
+        srt = sorted((float(t) for t in x), reverse=True)
+        for k in (1, 8):
+            assert orc.top_gap(x, k) == pytest.approx((srt[k - 1] - srt[k]) / abs(srt[0]), rel=1e-12)
+    assert orc.top_gap(torch.tensor([2.0, 2.0, 1.0], dtype=F64)) == 0.0
+    assert orc.top_gap(torch.tensor([2.0, 2.0, 1.0], dtype=F64), 2) == pytest.approx(0.5)
 
 
 def test_chain_iteration_end_to_end_properties():

@@ -68,6 +68,51 @@ def test_noalloc_verify_matches_sx_verify_twice_in_a_row():
     assert L2.cpu().tolist() == [2] * B2 or min(L2.cpu().tolist()) >= 2
 
 
+def test_noalloc_many_tiles_per_cta_then_a_smaller_call_against_the_oracle():
+    """A vocabulary with more tiles than SMs (every CTA owns three tiles, equal logits across them must go
+    to the lower index), then a small vocabulary that uses fewer CTAs, so that slices of the shared
+    scratch beyond the second call's CTAs still hold the first call's results.  Both are checked against
+    the oracle's target argmax, not only against sx_verify."""
+    from oracle import specexit_oracle as orc
+    case, M = parity.periodic_head_case(synth.CHAIN, B=8, K=7)
+    wl = case.wl
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(12)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    # call 1: 64 rows over 2 * SMs + 1 tiles
+    head1 = case.weights["head"][: wl.shape.V].contiguous().to(dev)
+    th1 = torch.randn(wl.B, wl.P, wl.shape.H, generator=g).to(torch.bfloat16)
+    cand1 = torch.randint(0, wl.shape.V, (wl.B, wl.P), generator=g, dtype=torch.int32)
+    want1, _ = orc.target_argmax(harness.oracle_model(case), th1)
+    cand1[:, 1] = want1[:, 0].to(torch.int32)
+    out1 = _outputs(wl.B, wl.P, wl.P, dev)
+    binding.sx_verify_noalloc(head1, th1.to(dev), cand1.to(dev), None, out1, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert int(((want1 % 128) >= 32).sum()) > wl.B * wl.P // 2 and int(want1.max()) < M
+    assert torch.equal(out1["target_tok"].cpu().to(torch.int64), want1)
+    v1 = orc.verify(harness.oracle_model(case), th1, cand1.to(torch.int64))
+    assert out1["accept_len"].cpu().tolist() == v1.accept_len.tolist() and min(v1.accept_len.tolist()) >= 1
+    assert out1["recover_tok"].cpu().tolist() == v1.recover_tok.tolist()
+    # call 2: 4096 ids = 32 tiles = 32 CTAs; the slices of CTAs 32.. keep call 1's partial results
+    sh = synth.ModelShape(H=256, n_q=4, n_kv=2, d=64, F=688, V=4096, page=64)
+    case2 = harness.build_case(synth.Workload("na2", sh, B=3, mode=synth.CHAIN, K=4, len_lo=8, len_hi=8, seed=43))
+    head2 = case2.weights["head"][: sh.V].contiguous().to(dev)
+    th2 = torch.randn(3, 5, sh.H, generator=g).to(torch.bfloat16)
+    cand2 = torch.randint(0, sh.V, (3, 5), generator=g, dtype=torch.int32)
+    want2, gap2 = orc.target_argmax(harness.oracle_model(case2), th2)
+    out2 = _outputs(3, 5, 5, dev)
+    binding.sx_verify_noalloc(head2, th2.to(dev), cand2.to(dev), None, out2, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    diff = out2["target_tok"].cpu().to(torch.int64) != want2
+    assert bool((gap2[diff] < parity.REL_GAP).all())
+    if not bool(diff.any()):
+        v2 = orc.verify(harness.oracle_model(case2), th2, cand2.to(torch.int64))
+        assert out2["accept_len"].cpu().tolist() == v2.accept_len.tolist()
+        assert out2["recover_tok"].cpu().tolist() == v2.recover_tok.tolist()
+
+
 def test_noalloc_rejects_more_rows_than_the_built_in_scratch_holds():
     lib = binding.load_library()
     dev = torch.device("cuda:0")
