@@ -557,6 +557,23 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
                         status_d, stream);
 }
 
+// K/V part of the q/k/v projection for a commit: the rows behind the n_q * d query rows.  Row-major weights
+// are entered at that row; tiled weights at that row tile (when the query rows end on a tile boundary,
+// otherwise the whole projection is computed and the query part ignored).
+static sx_status commit_kv_projection(sx_ctx *c, int Kin, const bf16 *X, int R, float *part, int *sp_out,
+                                      bool *kv_only, int32_t *status, cudaStream_t st) {
+  const SxShape &s = c->sh;
+  const int Nq = s.nq * s.d, Nkv = 2 * s.nkv * s.d, N = Nq + Nkv;
+  const bf16 *W = (const bf16 *)c->w.wqkv_d;
+  *kv_only = !c->tiled || (Nq % SX_TILE_M) == 0;
+  const int n = *kv_only ? Nkv : N;
+  if (*kv_only) W += c->tiled ? sx_tiled_elems(Nq, Kin) : (size_t)Nq * Kin;
+  int sp = sx_gemm_pick_splits(n, Kin, c->sm_count);
+  if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
+  *sp_out = sp;
+  return sx_launch_gemm_partial(W, n, Kin, X, R, part, sp, (size_t)R * n, c->sm_count, status, st, c->tiled);
+}
+
 extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void *target_hidden_d,
                                const int32_t *cand_tok_d, const int32_t *path_d, int32_t path_stride,
                                const int32_t *accept_len_out_d, const int32_t *recover_tok_out_d, void *feat0_next_d,
@@ -591,16 +608,14 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
       SX_TRY(sx_launch_fused_input(s, R, part, sp, (size_t)R * s.H, nullptr, SxIndex{nullptr, 1, 0}, trow, SxIndex{nullptr, 1, 0},
                             (const bf16 *)c->w.embed_d, (const bf16 *)c->w.norm_e_d, (const bf16 *)c->w.norm1_d, n, u2,
                             status_d, st));
-      const int N = (s.nq + 2 * s.nkv) * s.d;
-      sp = sx_gemm_pick_splits(N, 2 * s.H, c->sm_count);
-      if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
-      SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, 2 * s.H, u2, R, part, sp, (size_t)R * N, c->sm_count,
-                                    status_d, st, c->tiled));
+      bool kv_only;
+      SX_TRY(commit_kv_projection(c, 2 * s.H, u2, R, part, &sp, &kv_only, status_d, st));
+      const int N = kv_only ? 2 * s.nkv * s.d : (s.nq + 2 * s.nkv) * s.d;
       SxRowMap rm;
       memset(&rm, 0, sizeof(rm));
       rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
       rm.valid_len = accept_len_out_d; rm.per_seq = M;
-      SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st));
+      SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st, kv_only));
       c->launches += 4;
     }
     SX_TRY(sx_launch_commit_advance(B, accept_len_out_d, kv->cache_len_d, st));
@@ -617,16 +632,14 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
                                   status_d, st, c->tiled));
     SX_TRY(sx_launch_finish_norm(s, R, part, sp, (size_t)R * s.H, nullptr, (const bf16 *)c->w.norm1_d, nullptr, n, nullptr,
                           SxIndex{nullptr, 1, 0}, st));
-    const int N = (s.nq + 2 * s.nkv) * s.d;
-    sp = sx_gemm_pick_splits(N, s.H, c->sm_count);
-    if (sp > SX_COMMIT_MAX_SPLITS) sp = 1;
-    SX_TRY(sx_launch_gemm_partial((const bf16 *)c->w.wqkv_d, N, s.H, n, R, part, sp, (size_t)R * N, c->sm_count, status_d,
-                                  st, c->tiled));
+    bool kv_only;
+    SX_TRY(commit_kv_projection(c, s.H, n, R, part, &sp, &kv_only, status_d, st));
+    const int N = kv_only ? 2 * s.nkv * s.d : (s.nq + 2 * s.nkv) * s.d;
     SxRowMap rm;
     memset(&rm, 0, sizeof(rm));
     rm.mode = SX_MODE_COMMIT; rm.round = 1; rm.topk = 1; rm.R = R; rm.cache_len = kv->cache_len_d;
     rm.valid_len = accept_len_out_d; rm.per_seq = M;
-    SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st));
+    SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, (size_t)R * N, nullptr, *kv, status_d, st, kv_only));
     c->launches += 4;
   }
   SX_TRY(sx_launch_commit_advance(B, accept_len_out_d, kv->cache_len_d, st));

@@ -229,7 +229,7 @@ sx_status sx_kernels_init(int device) {
 // ---------------------------------------------------------------------------------------
 __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, SxRowMap rm, const float *part,
                                           int splits, size_t split_stride, bf16 *q_out, sx_kv kv, int page,
-                                          int head_begin, int32_t *status) {
+                                          int head_begin, int part_head0, int part_heads, int32_t *status) {
   sx_pdl_launch_dependents();
   const int hh = head_begin + blockIdx.x, r = blockIdx.y;
   const int i = threadIdx.x;
@@ -248,8 +248,8 @@ __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, 
   sx_pdl_wait();
   if (i >= half) return;
   if (rm.mode == SX_MODE_COMMIT && (ri.rel - 1) >= rm.valid_len[ri.b]) return;   // row does not exist
-  const int N = (nq + 2 * nkv) * d;
-  const float *row = part + (size_t)r * N + hh * d;
+  // the partial sums hold heads [part_head0, part_head0 + part_heads) of the projection
+  const float *row = part + ((size_t)r * part_heads + (hh - part_head0)) * d;
   float x1 = 0.f, x2 = 0.f;
   for (int sp = 0; sp < splits; ++sp) {
     x1 += row[sp * split_stride + i];
@@ -285,12 +285,16 @@ __global__ void sx_finish_qkv_rope_kernel(int nq, int nkv, int d, double theta, 
 
 sx_status sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool kv_only_partials) {
   int threads = ((sh.d / 2 + 31) / 32) * 32;
-  // q_out == nullptr: only the K and V heads (commit)
+  // q_out == nullptr: only the K and V heads (commit); the partial sums then hold either the whole
+  // projection or just its K and V rows
   const int head_begin = q_out ? 0 : sh.nq;
+  const int part_head0 = kv_only_partials ? sh.nq : 0;
+  const int part_heads = kv_only_partials ? 2 * sh.nkv : sh.nq + 2 * sh.nkv;
   return sx_rc(sx_launch(sx_finish_qkv_rope_kernel, dim3(sh.nq + 2 * sh.nkv - head_begin, rm.R), dim3(threads), 0, st, sh.nq, sh.nkv,
-            sh.d, (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, head_begin, status));
+            sh.d, (double)sh.theta, rm, part, splits, split_stride, q_out, kv, sh.page, head_begin, part_head0,
+            part_heads, status));
 }
 
 // ---------------------------------------------------------------------------------------

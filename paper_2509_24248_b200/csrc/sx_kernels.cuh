@@ -40,7 +40,7 @@ sx_status sx_launch_fused_input(const SxShape &sh, int R, const float *part, int
 
 sx_status sx_launch_finish_qkv_rope(const SxShape &sh, const SxRowMap &rm, const float *part, int splits,
                                size_t split_stride, bf16 *q_out, const sx_kv &kv, int32_t *status,
-                               cudaStream_t st);
+                               cudaStream_t st, bool kv_only_partials = false);
 
 sx_status sx_launch_commit_gather(const SxShape &sh, int B, int M, int P, const bf16 *th, const int32_t *cand,
                              const int32_t *path, int path_stride, const int32_t *accept_len,
