@@ -284,6 +284,7 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
                           wl.max_nodes, device=str(dev), sample_drafts=args.sample_drafts,
                           tiled=args.weights == "tiled")
     sx.set_kv(kv)
+    sx.sx_set_attention({"auto": binding.ATTN_AUTO, "split": binding.ATTN_SPLIT, "tc": binding.ATTN_TC}[args.attention])
     del weights
     P, H, S = wl.P, wl.shape.H, wl.shape.S
     FW = (3 if wl.shape.arch else 1) * H
@@ -554,6 +555,8 @@ def main():
                          "three-feature fusion in round 1 with [norm(embedding) ; norm(hidden)] as attention input")
     ap.add_argument("--draft-vocab", type=int, default=0, metavar="VD",
                     help="reduce the draft head to VD ids (id map + the target's own head); 0 = the workload as defined")
+    ap.add_argument("--attention", choices=["auto", "split", "tc"], default="auto",
+                    help="decode-attention kernel: the library's own choice, the split kernel, or the tensor-memory kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-one-thread", action="store_true", help="skip the single-thread figure of the CPU baseline")
     ap.add_argument("--timeline", default=None, metavar="FILE",

@@ -256,6 +256,18 @@ sx_status sx_verify(sx_ctx *ctx, int32_t batch, int32_t P, const void *target_hi
 size_t sx_tiled_weight_bytes(int32_t N, int32_t K);
 sx_status sx_tile_weight(const void *src_d, int32_t N, int32_t K, void *dst_d, void *stream);
 
+/* Choice of the decode-attention kernel (a deployment choice; the paper describes no kernels).  Two kernels
+ * compute the same attention over the paged cache: SX_ATTN_SPLIT cuts the keys into chunks, one warp per
+ * (sequence, KV head, 8 queries, chunk), on the warp-level tensor-core path; SX_ATTN_TC streams 128-key
+ * blocks through tcgen05 tensor memory, which is faster on long caches but needs head_dim = 128, a page
+ * size that is a multiple of 64 and at most 32 queries per (sequence, KV head) (group size * rows drafted
+ * per sequence in the round).  SX_ATTN_AUTO (the state of a new context) takes SX_ATTN_TC where it is
+ * supported and the cache capacity is at least four 128-key blocks per SM, else SX_ATTN_SPLIT.  Forcing
+ * SX_ATTN_TC makes a draft call return SX_ERR_UNSUPPORTED where the shape does not allow it.  Host-side
+ * state, read when a call is issued. */
+enum { SX_ATTN_AUTO = 0, SX_ATTN_SPLIT = 1, SX_ATTN_TC = 2 };
+sx_status sx_set_attention(sx_ctx *ctx, int32_t kernel);
+
 /* Stochastic acceptance: speculative sampling, the acceptance rule of the speculative-decoding
  * scheme the method builds on (Section 2, background on speculative decoding; Algorithm 1,
  * "accept tokens").  A draft token x is kept with probability min(1, p(x) / q(x)), else a token is

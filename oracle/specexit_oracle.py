@@ -121,6 +121,16 @@ def top_gap(v: torch.Tensor, k: int = 1) -> float:
     return float(t[k - 1] - t[k]) / den if den > 0 else 0.0
 
 
+def order_gap(v: torch.Tensor, k: int) -> float:
+    """Smallest gap between neighbours among the k + 1 largest values, over |largest|: the margin by which
+    an ordered top-k list (its order and its cut) is decided."""
+    t = torch.topk(v, min(k + 1, v.numel())).values
+    den = abs(float(t[0]))
+    if t.numel() < 2 or den == 0:
+        return 0.0 if den == 0 else 1.0
+    return float((t[:-1] - t[1:]).min()) / den
+
+
 def topk_low(v: torch.Tensor, k: int) -> List[int]:
     """The k largest entries, larger value first, lower index first among equals."""
     order = sorted(range(v.numel()), key=lambda i: (-float(v[i]), i)) if v.numel() <= 4096 else None
@@ -426,7 +436,7 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
 
     def emit(b, row, par_cid, par_score, dep, logits):
         ids = topk_low(logits, topk)
-        margins[("topk", b, row)] = top_gap(logits, topk) if topk < logits.numel() else 1.0
+        margins[("topk", b, row)] = order_gap(logits, topk)      # order of the k children and the cut behind them
         if ("topk", b, row) in ov:
             ids = list(ov[("topk", b, row)])
         if chooser is not None:
@@ -457,10 +467,9 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
         for b in range(B):
             level = [c for c in cands[b] if c.depth == r - 1]
             level.sort(key=lambda c: (-c.score, c.cid))
-            if len(level) > topk:
-                den = abs(level[0].score)
-                margins[("expand", b, r - 1)] = (
-                    (level[topk - 1].score - level[topk].score) / den if den > 0 else 0.0)
+            if len(level) > 1:
+                # the chosen candidates take their rows in rank order: order and cut both decide
+                margins[("expand", b, r - 1)] = order_gap(torch.tensor([c.score for c in level], dtype=F64), topk)
             chosen = level[:topk]
             if ("expand", b, r - 1) in ov:
                 byid = {c.cid: c for c in cands[b]}

@@ -23,13 +23,14 @@ MODE_CHAIN, MODE_TREE = 0, 1
 ACT_SIGMOID, ACT_EXPM1, ACT_IDENTITY = 0, 1, 2
 DIR_GT, DIR_LT = 0, 1
 EMA_VERIFIED_CONTEXT, EMA_FIRST_ONLY = 0, 1
+ATTN_AUTO, ATTN_SPLIT, ATTN_TC = 0, 1, 2
 SMOOTH_EWMA, SMOOTH_NONE, SMOOTH_WINDOW, SMOOTH_MOMENTUM, SMOOTH_PARAGRAPH = 0, 1, 2, 3, 4
 HIST = 16
 
 EXPORTS = ["sx_create", "sx_destroy", "sx_workspace_bytes", "sx_strerror", "sx_launch_count",
            "sx_draft_step", "sx_verify", "sx_exit_update", "sx_spec_exit_iter",
            "sx_spec_exit_iter_host", "sx_profile_begin", "sx_profile_end", "sx_verify_noalloc", "sx_commit",
-           "sx_set_sampling", "sx_tiled_weight_bytes", "sx_tile_weight", "sx_selftest_bounded_wait"]
+           "sx_set_sampling", "sx_tiled_weight_bytes", "sx_tile_weight", "sx_selftest_bounded_wait", "sx_set_attention"]
 PROF_CLASSES = ["head_draft", "head_verify", "gemm_fc", "gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down",
                 "attention"]
 
@@ -134,6 +135,8 @@ def load_library() -> C.CDLL:
     lib.sx_profile_end.argtypes = [vp, vp, vp]
     lib.sx_commit.restype = i32
     lib.sx_commit.argtypes = [vp, C.POINTER(KV), i32, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+    lib.sx_set_attention.restype = i32
+    lib.sx_set_attention.argtypes = [vp, i32]
     lib.sx_selftest_bounded_wait.restype = i32
     lib.sx_selftest_bounded_wait.argtypes = [C.c_uint32, i32, vp, vp, vp]
     lib.sx_verify_noalloc.restype = i32
@@ -369,6 +372,10 @@ class SpecExit:
                                       logp.data_ptr(), sig.data_ptr(), self.ws_ptr, self.ws_bytes,
                                       self.status.data_ptr(), self._stream()), "sx_draft_step")
         return hid, tok_out, logp, sig
+
+    def sx_set_attention(self, kernel: int) -> None:
+        """Decode-attention kernel of the draft calls that follow: ATTN_AUTO, ATTN_SPLIT or ATTN_TC."""
+        _check(self.lib.sx_set_attention(self.h, int(kernel)), "sx_set_attention")
 
     def sx_set_sampling(self, temperature: float, seed: int = 0, offset: int = 0) -> None:
         """Stochastic acceptance for the verify calls that follow (0 = greedy)."""

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspecexit.so")
-SOURCES = ["sx_api.cu", "sx_kernels.cu", "sx_attention.cu", "sx_gemm_tc.cu", "sx_noalloc.cu"]
+SOURCES = ["sx_api.cu", "sx_kernels.cu", "sx_attention.cu", "sx_attention_tc.cu", "sx_gemm_tc.cu", "sx_noalloc.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Wno-deprecated-gpu-targets",
               "-Xcompiler", "-fPIC"]
 

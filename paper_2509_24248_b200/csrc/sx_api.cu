@@ -20,6 +20,7 @@ struct sx_ctx {
       off_tok_rt, off_logp_rt, off_tree, off_cu, off_cn, off_cpart, off_cu2, off_ctok, off_dlogits, off_tlogits, off_spec, total;
   int commit_rows, commit_N;
   bool tiled;                    // GEMM weights are stored tile by tile (sx_tile_weight)
+  int attn_kernel;               // SX_ATTN_AUTO / _SPLIT / _TC (sx_set_attention)
   SxSample smp;                  // sampled verification (sx_set_sampling); temp == 0: greedy
   // set around a draft round whose head samples its token and leaves its logits (sampled drafts)
   bool round_sampled;
@@ -169,7 +170,8 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   }
   c->device = dev;
   c->sm_count = prop.multiProcessorCount;
-  if (sx_gemm_init(dev) != SX_OK || sx_attn_init(dev) != SX_OK || sx_kernels_init(dev) != SX_OK) {
+  if (sx_gemm_init(dev) != SX_OK || sx_attn_init(dev) != SX_OK || sx_attn_tc_init(dev) != SX_OK ||
+      sx_kernels_init(dev) != SX_OK) {
     delete c;
     return SX_ERR_CUDA;
   }
@@ -193,7 +195,10 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->off_m = take((size_t)R * s.F * 2);
   c->off_g = take((size_t)R * s.H * 2);
   c->off_part = take((size_t)c->max_splits * R * c->part_N * 4);
-  c->off_attn = take(sx_attn_ws_bytes(s, max_batch, T, c->sm_count));
+  {
+    const size_t a = sx_attn_ws_bytes(s, max_batch, T, c->sm_count), b = sx_attn_tc_ws_bytes(s, max_batch, c->sm_count);
+    c->off_attn = take(a > b ? a : b);
+  }
   c->off_hparts = take((size_t)c->head_G * c->head_rows * sizeof(SxHeadPartial));
   c->off_z = take((size_t)R * SX_MAX_SIGNALS * 4);
   c->off_tok_rt = take((size_t)R * SX_MAX_TOPK * 4);
@@ -358,9 +363,20 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st));
   const int B = kv->batch, nr = R / B;
   const int E = (c->dc.mode == SX_MODE_CHAIN) ? round : (round == 1 ? 1 : 1 + (round - 1) * c->dc.topk);
-  const int nsplit = sx_attn_splits(s, B, nr, kv->max_pages * s.page, c->sm_count);
+  // Which attention kernel: the tensor-core one streams long caches faster; below a few blocks of keys per
+  // SM its set-up outweighs that and the split kernel is used (the host knows capacities, not lengths).
+  bool tc = sx_attn_tc_supported(s, nr, *kv);
+  if (c->attn_kernel == SX_ATTN_SPLIT) tc = false;
+  else if (c->attn_kernel == SX_ATTN_AUTO)
+    tc = tc && (long long)B * s.nkv * ((kv->max_pages * s.page + 127) / 128) >= 4ll * c->sm_count;
+  else if (!tc) return SX_ERR_UNSUPPORTED;
   prof_mark(c, SX_PROF_ATTENTION, true, st);
-  SX_TRY(sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st));
+  if (tc) {
+    SX_TRY(sx_launch_attention_tc(s, rm, B, nr, E, q, *kv, (float *)(ws + c->off_attn), o, c->sm_count, status, st));
+  } else {
+    const int nsplit = sx_attn_splits(s, B, nr, kv->max_pages * s.page, c->sm_count);
+    SX_TRY(sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st));
+  }
   prof_mark(c, SX_PROF_ATTENTION, false, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_O, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));
   SX_TRY(sx_launch_finish_norm(s, R, part, sp, stride, x, (const bf16 *)c->w.norm2_d, a, n, nullptr, SxIndex{nullptr, 1, 0}, st));
@@ -415,6 +431,12 @@ extern "C" sx_status sx_selftest_bounded_wait(uint32_t limit, int32_t ctas, int3
                                               void *stream) {
   if (!status_d || !reached_d) return SX_ERR_INVALID_ARG;
   return sx_launch_wait_selftest(limit, ctas, status_d, reached_d, (cudaStream_t)stream);
+}
+
+extern "C" sx_status sx_set_attention(sx_ctx *c, int32_t kernel) {
+  if (!c || kernel < SX_ATTN_AUTO || kernel > SX_ATTN_TC) return SX_ERR_INVALID_ARG;
+  c->attn_kernel = kernel;
+  return SX_OK;
 }
 
 extern "C" sx_status sx_set_sampling(sx_ctx *c, float temperature, uint64_t seed, uint32_t offset) {

@@ -60,6 +60,15 @@ size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_cou
 sx_status sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
                          const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
 
+// The same attention on tcgen05 (sx_attention_tc.cu): head dimension 128, pages of a multiple of 64 slots,
+// at most 32 queries per (sequence, KV head).
+bool sx_attn_tc_supported(const SxShape &sh, int nr, const sx_kv &kv);
+sx_status sx_attn_tc_init(int device);
+size_t sx_attn_tc_ws_bytes(const SxShape &sh, int max_batch, int sm_count);
+sx_status sx_launch_attention_tc(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
+                                 const sx_kv &kv, float *ws, bf16 *o_out, int sm_count, int32_t *status,
+                                 cudaStream_t st);
+
 // Optional fusion for chain drafting: the merge kernel also writes the next round's input row
 // u[r] = [feat[r] ; embed[token chosen for row r]] (u == nullptr: off).
 struct SxNextInput {
@@ -112,6 +121,9 @@ sx_status sx_launch_gemm_partial(const bf16 *W, int N, int K, const bf16 *X, int
 size_t sx_tiled_elems(int N, int K);
 sx_status sx_launch_tile_weight(const bf16 *src, int N, int K, bf16 *dst, cudaStream_t st);
 sx_status sx_gemm_init(int device);
+// cached 2-D tensor map of a bf16 matrix [rows, cols], box = box_rows x 64 columns, 128-byte swizzle
+struct CUtensorMap_st;
+bool sx_tma_map_2d(const void *ptr, long long rows, int cols, int box_rows, CUtensorMap_st *out);
 // give-up path of the bounded mbarrier waits on its own (see sx_selftest_bounded_wait)
 sx_status sx_launch_wait_selftest(uint32_t limit, int ctas, int32_t *status, int32_t *reached, cudaStream_t st);
 // Sampled verification: with temp > 0 the plain-argmax head returns, per row, the arg max of

@@ -680,6 +680,25 @@ def test_top_gap_is_the_kth_margin_over_the_largest_value():
     assert orc.top_gap(torch.tensor([2.0, 2.0, 1.0], dtype=F64), 2) == pytest.approx(0.5)
 
 
+def test_order_gap_is_the_smallest_neighbour_gap_among_the_first_k_plus_one():
+    v = torch.tensor([0.5, -4.0, 2.0, 1.0, 8.0, 7.5, 3.0, 2.5, 6.0, 5.0, 4.0, 0.0], dtype=F64)
+    # sorted: 8, 7.5, 6, 5, 4, 3, 2.5, 2, 1 | 0.5, 0, -4
+    assert orc.order_gap(v, 1) == pytest.approx(0.5 / 8.0)
+    assert orc.order_gap(v, 3) == pytest.approx(0.5 / 8.0)            # 8 - 7.5 is the smallest among 8, 7.5, 6, 5
+    assert orc.order_gap(v, 8) == pytest.approx(0.5 / 8.0)
+    w = torch.tensor([10.0, 7.0, 6.9, 1.0, 0.0], dtype=F64)
+    assert orc.order_gap(w, 1) == pytest.approx(0.3)                  # cut between 10 and 7
+    assert orc.order_gap(w, 2) == pytest.approx(0.01)                 # 7 vs 6.9 decides the cut
+    assert orc.order_gap(w, 3) == pytest.approx(0.01)                 # ... and then the order inside the list
+    assert orc.order_gap(torch.tensor([3.0, 3.0, 1.0], dtype=F64), 2) == 0.0
+    g = torch.Generator().manual_seed(78)
+    for _ in range(10):
+        x = torch.randn(300, generator=g, dtype=F64)
+        srt = sorted((float(t) for t in x), reverse=True)
+        want = min(srt[i] - srt[i + 1] for i in range(8)) / abs(srt[0])
+        assert orc.order_gap(x, 8) == pytest.approx(want, rel=1e-12)
+
+
 def test_chain_iteration_end_to_end_properties():
     wl = harness.tiny_workload(B=3, K=4)
     case = harness.build_case(wl)
