@@ -3,26 +3,31 @@
 // the group's query heads times the rows the sequence drafts this round (1 in a chain, the sibling
 // rows in a tree).
 //
-// Both products of a block of 128 keys run as tcgen05.mma with the queries on the M side:
-//     S[q][key]  = sum_d Q[q][d] K[key][d]       A = Q (shared memory), B = K block (as stored: K-major)
-//     O[q][d]   += sum_key P[q][key] V[key][d]   A = P (shared memory), B = V block (as stored: N-major)
-// M is 128: the (at most 32) queries are laid out four times, rows 32 w + q (w = 0..3), and replica w
-// owns the keys 32 w .. 32 w + 31 of every block: its softmax threads read only those 32 columns of S
-// and write only those 32 columns of P (the rest of a P row stays zero), so each of the 128 softmax
-// threads owns one row (one TMEM lane) and one quarter of the keys, keeps a running (max, sum) of its
-// own, and never exchanges anything with another thread inside the loop.  The four replicas of a query
-// are four independent partial results over disjoint keys; they are merged once, when the CTA leaves
-// the (sequence, KV head) pair.  The tensor pipe does four times the useful work - it has the time:
-// the kernel is bound by the K/V stream.
+// Both products of a block of 128 keys run as tcgen05.mma with the 128-wide side of the data on M, so
+// that no tensor-core work is spent on padding:
+//     S^T[key][q] = sum_d K[key][d] Q[q][d]         A = K block (as stored: K-major), B = Q         M = keys, N = 32
+//     O^T[d][q]  += sum_key V[key][d] P[key][q]     A = V block (as stored: M-major), B = P^T       M = d,    N = 32
+// A softmax thread owns one TMEM lane: one key of S^T (its scores against all 32 queries), one head-dimension
+// row of O^T.  The softmax of a query runs over keys, i.e. across threads; what makes that cheap is that the
+// reference maximum m_q only has to keep the exponentials in range, not be the maximum: all threads hold
+// the same m_q in registers and change it only when some score exceeds it by more than 2^8 - an event the
+// 128 threads detect with one barrier vote per block - and the sums l_q are kept as per-thread partial sums
+// (one per query) that are added up once, when the CTA leaves the (sequence, KV head) pair.  The rare
+// update (always the first block of a pair) goes through shared memory: block maximum per query, rescale
+// of O^T and of the partial sums.
 //
 // Work is cut "stream-K" style: all 128-key blocks of all (sequence, KV head) pairs form one list, CTA c
 // takes the c-th run of ceil(total / CTAs) consecutive blocks, so every CTA streams the same number of
 // bytes whatever the sequence lengths, and leaves one partial result per pair it touched (a pair is
 // shared by the few CTAs whose runs meet inside it).  A merge kernel combines those.
 //
-// Warp roles (192 threads): warp 0 = TMA producer (K and V blocks of 32 KB through a ring of five),
-// warp 1 = MMA issuer (owns TMEM: two S accumulators and O), warps 2-5 = softmax / epilogue.
-// Every mbarrier wait is bounded (see sx_tc_ptx.cuh).
+// Warp roles (384 threads): warps 0 and 11 = TMA producers (K blocks and V blocks of 32 KB, a ring of three
+// slots each), warp 1 = issuer of the first product (owns TMEM: two S^T accumulators and O^T, 32 columns each), warp 10 =
+// issuer of the second product, warps 2-9 = softmax / epilogue: two warps per TMEM lane quarter, each taking half of the query columns, so that every
+// scheduler has two softmax warps to interleave.  P^T is double-buffered: the softmax of a block does not
+// wait for the second product of the block before it.  The kernel is compiled for 16 and for 32 query
+// columns (a chain with a group of at most 16 query heads takes the narrow one).  Every mbarrier wait is
+// bounded (see sx_tc_ptx.cuh).
 #include <cuda.h>
 
 #include "sx_kernels.cuh"
@@ -32,13 +37,20 @@
 #define AT_D 128
 #define AT_KEYS 128                         // keys per block
 #define AT_SLAB 64                          // keys per TMA box (a page holds a multiple of this)
-#define AT_NS 5                             // ring slots, one K block or one V block each
+#define AT_NS 6                             // ring slots of 32 KB in all
+#define AT_NR 3                             // ... three for K blocks, three for V blocks: two rings
 #define AT_BLK_BYTES (AT_KEYS * AT_D * 2)   // 32 KB
 #define AT_HALF_BYTES (128 * 128)           // a 128-row tile of 64 columns (one swizzle row per matrix row)
 #define AT_SLAB_BYTES (AT_SLAB * 128)
-#define AT_TMEM_COLS 512                    // S0 | S1 | O (128 columns each), rounded to a power of two
-#define AT_O_COL 256
-#define AT_SMEM_BYTES (1024 + 2 * 32768 + AT_NS * AT_BLK_BYTES + 256 + 1024)
+#define AT_NQ 32                            // query columns of the accumulators
+#define AT_TMEM_COLS 128                    // S^T 0 | S^T 1 | O^T (32 columns each), rounded to a power of two
+#define AT_O_COL 64
+#define AT_QP_BYTES (AT_NQ * AT_D * 2)      // Q, and P^T: 32 rows of 128 elements
+#define AT_SMEM_BYTES (1024 + 3 * AT_QP_BYTES + AT_NS * AT_BLK_BYTES + 256 + 512 + 256 + 128)
+#define AT_EPI_THREADS 256
+#define AT_MMA2_WARP 10                     // warps 0, 1: producer, first product; 2-9: softmax; 10: second product
+#define AT_VPROD_WARP 11                    // producer of the V ring
+#define AT_THREADS (64 + AT_EPI_THREADS + 64)
 
 struct SxAtParams {
   int nq, nkv, G, page, nr, E, NQ, B, tree_masks;
@@ -97,23 +109,37 @@ __device__ __forceinline__ void at_next(const SxAtParams &p, AtCursor &c) {
   }
 }
 
-// position of a block's K and V loads in the ring order K0, V0, K1, V1, ...  (requesting V one block later,
-// when the MMA issuer gets to it, was tried: the second product then waits for the V block to land and the
-// softmax of the next block behind it - 36 % slower)
-__device__ __forceinline__ int at_k_entry(int li) { return 2 * li; }
-__device__ __forceinline__ int at_v_entry(int li, int n) { (void)n; return 2 * li + 1; }
+__device__ __forceinline__ void at_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier over the 256 softmax threads that also ANDs a flag, so that they all take the same branch
+__device__ __forceinline__ bool at_all(bool ok) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred pi, po;\n\t"
+      "setp.ne.u32 pi, %1, 0;\n\t"
+      "bar.red.and.pred po, 1, 256, pi;\n\t"
+      "selp.u32 %0, 1, 0, po;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return out != 0;
+}
 
-__global__ void __launch_bounds__(192, 1)
+template <int NQT>       // query columns of the accumulators: 16 or 32
+__global__ void __launch_bounds__(AT_THREADS, 1)
 sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, SxAtParams p) {
+  constexpr int QH = NQT / 2;                 // query columns per softmax thread
   extern __shared__ uint8_t sx_at_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>(((uintptr_t)sx_at_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t *sQ = smem, *sP = smem + 32768, *ring = smem + 65536;
+  uint8_t *sQ = smem, *sPT = smem + AT_QP_BYTES, *ring = smem + 3 * AT_QP_BYTES;      // P^T: two buffers
   uint64_t *bars = reinterpret_cast<uint64_t *>(ring + AT_NS * AT_BLK_BYTES);
+  // K ring: full[0..2] / empty[0..2]; V ring: full[3..5] / empty[3..5]
   uint64_t *full = bars, *empty = bars + AT_NS, *sfull = bars + 2 * AT_NS, *sempty = sfull + 2;
-  uint64_t *pfull = sempty + 2, *pempty = pfull + 1, *qfull = pempty + 1, *ofull = qfull + 1, *oempty = ofull + 1;
+  uint64_t *pfull = sempty + 2, *pempty = pfull + 2, *qfull = pempty + 2, *ofull = qfull + 1, *oempty = ofull + 1;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(oempty + 1);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-  float *cm = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(bars) + 256), *cl = cm + 128;
+  float *red = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(bars) + 256);  // [4 lane quarters][32 queries]
+  uint64_t *vis_sh = reinterpret_cast<uint64_t *>(red + 128);                       // [32] visibility of the drafted rows
+  float *m_sh = reinterpret_cast<float *>(vis_sh + 32);                             // [32]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   sx_pdl_launch_dependents();
@@ -127,18 +153,21 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < AT_NS; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sfull[i]), 1); mbar_init(smem_u32(&sempty[i]), 4); }
-    mbar_init(smem_u32(pfull), 4);
-    mbar_init(smem_u32(pempty), 1);
-    mbar_init(smem_u32(qfull), 4);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&sfull[i]), 1);
+      mbar_init(smem_u32(&sempty[i]), 8);
+      mbar_init(smem_u32(&pempty[i]), 1);
+      // one barrier per P^T buffer: a buffer is refilled only after the second product that read it has
+      // completed, so its barrier can never run a whole phase ahead of the MMA issuer (a single barrier
+      // for both buffers could: the softmax may be a block ahead)
+      mbar_init(smem_u32(&pfull[i]), 8);
+    }
+    mbar_init(smem_u32(qfull), 8);
     mbar_init(smem_u32(ofull), 1);
-    mbar_init(smem_u32(oempty), 4);
+    mbar_init(smem_u32(oempty), 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Q and P start as zeros: the parts of a P row outside its owner's 32 keys are never written
-  for (int i = threadIdx.x; i < 65536 / 16; i += blockDim.x) reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
-  fence_async_smem();
   if (warp == 1) {
     tc_alloc(smem_u32(tmem_slot), AT_TMEM_COLS);
     tc_relinquish();
@@ -148,8 +177,14 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ---- producer ------------------------------------------------------------------------------------
+  if (warp == 0 || warp == AT_VPROD_WARP) {
+    // ---- producers: warp 0 streams the K blocks of the run through ring slots 0-2, warp 11 the V blocks
+    // through slots 3-5.  Two rings, because the two streams are consumed at different points of a block's
+    // life (K at once, V only after the scores have been through the softmax): in one ring a landed V block
+    // would hold a slot the K stream could have in flight.
+    const bool is_v = warp != 0;
+    const int base_slot = is_v ? AT_NR : 0;
+    const CUtensorMap *map = is_v ? &tmV : &tmK;
     const uint64_t pol = policy_evict_first();
     AtCursor c = at_seek(p, g0);
     bool waited = false, ok = true, bad = false;
@@ -167,16 +202,23 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
       return row;
     };
-    auto load = [&](int entry, bool is_v, int row) {
-      const int row0 = __shfl_sync(0xffffffffu, row, 0), row1 = __shfl_sync(0xffffffffu, row, 1);
-      if (lane == 0 && ok) {
-        const int slot = entry % AT_NS;
-        const uint32_t ph = (uint32_t)(entry / AT_NS) & 1u;
-        if (entry >= AT_NS && !mbar_wait(smem_u32(&empty[slot]), ph ^ 1u, abort_flag, p.wait_limit)) ok = false;
+    int row_cur = rows_of(c);
+    // (Asking L2 for blocks further ahead with cp.async.bulk.prefetch.tensor, to have more than the rings'
+    // 64 KB per stream on its way, was tried with 6 blocks of lead: 100 -> 157 us on the tree rounds.)
+    for (int li = 0; li < nblk && ok; ++li) {
+      // cached keys are inputs of the iteration; the rows drafted in it come from the preceding kernel
+      if (!waited && (c.blk + 1) * AT_KEYS > p.cache_len[c.b]) { sx_pdl_wait(); waited = true; }
+      AtCursor nx = c;
+      at_next(p, nx);
+      const int row_next = (li + 1 < nblk) ? rows_of(nx) : p.pool_rows;      // looked up while this block's loads wait
+      const int row0 = __shfl_sync(0xffffffffu, row_cur, 0), row1 = __shfl_sync(0xffffffffu, row_cur, 1);
+      if (lane == 0) {
+        const int slot = base_slot + li % AT_NR;
+        const uint32_t ph = (uint32_t)(li / AT_NR) & 1u;
+        if (li >= AT_NR && !mbar_wait(smem_u32(&empty[slot]), ph ^ 1u, abort_flag, p.wait_limit)) ok = false;
         if (ok) {
           const uint32_t fb = smem_u32(&full[slot]);
           const uint32_t dst = smem_u32(ring + (size_t)slot * AT_BLK_BYTES);
-          const CUtensorMap *map = is_v ? &tmV : &tmK;
           mbar_expect_tx(fb, AT_BLK_BYTES);
 #pragma unroll
           for (int s = 0; s < 2; ++s)
@@ -186,118 +228,113 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         }
       }
       ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-    };
-    int row_cur = rows_of(c);
-    for (int li = 0; li < nblk && ok; ++li) {
-      // cached keys are inputs of the iteration; the rows drafted in it come from the preceding kernel
-      if (!waited && (c.blk + 1) * AT_KEYS > p.cache_len[c.b]) { sx_pdl_wait(); waited = true; }
-      AtCursor nx = c;
-      at_next(p, nx);
-      const int row_next = (li + 1 < nblk) ? rows_of(nx) : p.pool_rows;      // looked up while this block's loads wait
-      load(at_k_entry(li), false, row_cur);
-      load(at_v_entry(li, nblk), true, row_cur);
       row_cur = row_next;
       c = nx;
     }
-    if (__any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(p.status, SX_ERR_CAPACITY);
+    if (!is_v && __any_sync(0xffffffffu, bad) && lane == 0) sx_set_status(p.status, SX_ERR_CAPACITY);
   } else if (warp == 1) {
-    // ---- MMA issuer -----------------------------------------------------------------------------------
+    // ---- issuer of the first product (S^T = K.Q^T); owns the TMEM allocation -----------------------------
     if (lane == 0) {
-      // fp32 accumulate, bf16 A and B, M = 128, N = 128; the second product reads V along its rows (N-major B)
-      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-      const uint32_t idesc_o = idesc_s | (1u << 16);
-      const uint32_t q_addr = smem_u32(sQ), p_addr = smem_u32(sP);
-      AtCursor c1 = at_seek(p, g0);              // cursor of the next first product
-      int li1 = 0, item1 = 0;                    // blocks whose first product has been issued; their item index
-      bool ok = true;
-      auto mma1 = [&]() {
-        const bool first = (li1 == 0) || (c1.blk == 0);
-        if (first && li1 > 0) ++item1;
-        if (first && !mbar_wait(smem_u32(qfull), (uint32_t)item1 & 1u, abort_flag, p.wait_limit)) { ok = false; return; }
-        const int cnt = at_k_entry(li1), slot = cnt % AT_NS, sb = li1 & 1, u = li1 >> 1;
-        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(cnt / AT_NS) & 1u, abort_flag, p.wait_limit)) { ok = false; return; }
-        if (u >= 1 && !mbar_wait(smem_u32(&sempty[sb]), (uint32_t)(u - 1) & 1u, abort_flag, p.wait_limit)) { ok = false; return; }
+      // fp32 accumulate, bf16 A and B, both K-major, M = 128, N = NQT
+      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NQT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t q_addr = smem_u32(sQ);
+      AtCursor c1 = at_seek(p, g0);
+      int item1 = 0;
+      for (int li = 0; li < nblk; ++li) {
+        const bool first = (li == 0) || (c1.blk == 0);
+        if (first && li > 0) ++item1;
+        if (first && !mbar_wait(smem_u32(qfull), (uint32_t)item1 & 1u, abort_flag, p.wait_limit)) break;
+        const int slot = li % AT_NR, sb = li & 1, u = li >> 1;
+        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit)) break;
+        if (u >= 1 && !mbar_wait(smem_u32(&sempty[sb]), (uint32_t)(u - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t kb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES);
 #pragma unroll
-        for (int k = 0; k < AT_D / 16; ++k) {
-          const uint32_t o = (uint32_t)(k >> 2) * AT_HALF_BYTES + (uint32_t)(k & 3) * 32u;
-          tc_mma(tmem_base + (uint32_t)sb * 128u, smem_desc(q_addr + o), smem_desc(kb + o), idesc_s, k > 0 ? 1u : 0u);
-        }
+        for (int k = 0; k < AT_D / 16; ++k)
+          tc_mma(tmem_base + (uint32_t)sb * AT_NQ, smem_desc(kb + (uint32_t)(k >> 2) * AT_HALF_BYTES + (uint32_t)(k & 3) * 32u),
+                 smem_desc(q_addr + (uint32_t)(k >> 2) * (AT_NQ * 128) + (uint32_t)(k & 3) * 32u), idesc_s, k > 0 ? 1u : 0u);
         tc_commit(smem_u32(&empty[slot]));
         tc_commit(smem_u32(&sfull[sb]));
-        ++li1;
         at_next(p, c1);
-      };
-      AtCursor c2 = at_seek(p, g0);              // cursor of the next second product
+      }
+    }
+  } else if (warp == AT_MMA2_WARP) {
+    // ---- issuer of the second product (O^T += V^T.P^T): its own thread, so that its waits (probabilities
+    // written, V block landed) do not hold up the first products of the blocks behind --------------------
+    if (lane == 0) {
+      // the second product reads V along its rows: M-major A
+      const uint32_t idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(NQT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t pt_addr = smem_u32(sPT);
+      AtCursor c2 = at_seek(p, g0);
       int item2 = 0;
-      mma1();
-      for (int li = 0; li < nblk && ok; ++li) {
-        if (li + 1 < nblk) mma1();               // keeps the tensor pipe busy while block li's softmax runs
-        if (!ok) break;
+      for (int li = 0; li < nblk; ++li) {
         const bool first = (li == 0) || (c2.blk == 0);
         const bool last = (li == nblk - 1) || (c2.blk == c2.nb - 1);
         if (first && li > 0) ++item2;
-        const int cnt = at_v_entry(li, nblk), slot = cnt % AT_NS;
-        if (!mbar_wait(smem_u32(pfull), (uint32_t)li & 1u, abort_flag, p.wait_limit)) break;
-        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(cnt / AT_NS) & 1u, abort_flag, p.wait_limit)) break;
+        const int slot = AT_NR + li % AT_NR, pb = li & 1;
+        if (!mbar_wait(smem_u32(&pfull[pb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit)) break;
+        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit)) break;
         if (first && item2 > 0 && !mbar_wait(smem_u32(oempty), (uint32_t)(item2 - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
-        const uint32_t vb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES);
+        const uint32_t vb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES), pt = pt_addr + (uint32_t)pb * AT_QP_BYTES;
 #pragma unroll
-        for (int k = 0; k < AT_KEYS / 16; ++k) {
-          const uint32_t o = (uint32_t)(k >> 2) * AT_HALF_BYTES + (uint32_t)(k & 3) * 32u;
-          tc_mma(tmem_base + AT_O_COL, smem_desc(p_addr + o), smem_desc_mn(vb + (uint32_t)k * 2048u, AT_HALF_BYTES, 1024u),
-                 idesc_o, (first && k == 0) ? 0u : 1u);
-        }
+        for (int k = 0; k < AT_KEYS / 16; ++k)
+          tc_mma(tmem_base + AT_O_COL, smem_desc_mn(vb + (uint32_t)k * 2048u, AT_HALF_BYTES, 1024u),
+                 smem_desc(pt + (uint32_t)(k >> 2) * (AT_NQ * 128) + (uint32_t)(k & 3) * 32u), idesc_o,
+                 (first && k == 0) ? 0u : 1u);
         tc_commit(smem_u32(&empty[slot]));
-        tc_commit(smem_u32(pempty));
+        tc_commit(smem_u32(&pempty[pb]));
         if (last) tc_commit(smem_u32(ofull));
         at_next(p, c2);
       }
     }
   } else {
-    // ---- softmax / epilogue: thread = (replica w, query `lane`), TMEM lane 32 w + lane ---------------------
-    const int w = warp & 3, tid = threadIdx.x - 64, row = w * 32 + lane;
+    // ---- softmax / epilogue: thread = (TMEM lane i, half hq of the query columns).  Lane i is key i of a
+    // block's S^T and row i (of the head dimension) of O^T.
+    const int w = warp & 3, etid = threadIdx.x - 64, hq = (warp - 2) >> 2, i = w * 32 + lane, q0 = hq * QH;
     const uint32_t lane_base = tmem_base + ((uint32_t)(w * 32) << 16);
-    uint8_t *q_row = sQ + row * 128, *p_row = sP + (w >> 1) * AT_HALF_BYTES + row * 128;
-    float *scratch = reinterpret_cast<float *>(sP);     // [64 columns][128 rows] at the end of a pair
+    // this key's column in P^T: 64-key half, 16-byte chunk (XORed with the query row's low bits), byte in the chunk
+    const uint32_t pt_col = (uint32_t)((i >> 6) * (AT_NQ * 128) + (i & 7) * 2);
+    const int pt_chunk = (i & 63) >> 3;
     sx_pdl_wait();
     AtCursor c = at_seek(p, g0);
     int item = 0;
-    float m = -INFINITY, l = 0.f;
-    uint64_t vis = 0;
-    bool ok = true;
-    // the queries of a pair into shared memory, each laid out four times (rows 32 w + q)
+    float m[QH], lsum[QH];
+    // the queries of a pair into shared memory (row = query, 128-byte swizzle); rows beyond the pair's queries are zero
     auto load_q = [&](const AtCursor &cc) {
-      const bool valid = lane < p.NQ;
-      const int j = valid ? lane / p.G : 0, r = cc.b * p.nr + j;
-      const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)r * p.nq + cc.h * p.G + (valid ? lane - j * p.G : 0)) * AT_D);
+      const int q = etid >> 3, c8 = etid & 7;
+      const bool valid = q < p.NQ;
+      const int j = valid ? q / p.G : 0, r = cc.b * p.nr + j;
+      const uint4 *src = reinterpret_cast<const uint4 *>(p.q + ((size_t)r * p.nq + cc.h * p.G + (valid ? q - j * p.G : 0)) * AT_D);
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
+      for (int jj = 0; jj < 2; ++jj) {
+        const int ch = c8 * 2 + jj;
         const uint4 v = valid ? src[ch] : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4 *>(q_row + (ch >> 3) * AT_HALF_BYTES + (((ch & 7) ^ (row & 7)) << 4)) = v;
+        *reinterpret_cast<uint4 *>(sQ + (ch >> 3) * (AT_NQ * 128) + q * 128 + (((ch & 7) ^ (q & 7)) << 4)) = v;
       }
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(qfull));
     };
     auto pair_state = [&](const AtCursor &cc) {
-      const int j = lane < p.NQ ? lane / p.G : 0, r = cc.b * p.nr + j;
-      vis = p.tree_masks ? p.row_mask[r] : (p.E >= 64 ? ~0ull : ((1ull << p.E) - 1ull));
-      m = -INFINITY;
-      l = 0.f;
+      if (etid < AT_NQ) {
+        const int j = etid < p.NQ ? etid / p.G : 0, r = cc.b * p.nr + j;
+        vis_sh[etid] = p.tree_masks ? p.row_mask[r] : (p.E >= 64 ? ~0ull : ((1ull << p.E) - 1ull));
+      }
+#pragma unroll
+      for (int q = 0; q < QH; ++q) { m[q] = -INFINITY; lsum[q] = 0.f; }
     };
     load_q(c);
     pair_state(c);
     for (int li = 0; li < nblk; ++li) {
       const bool first = (li == 0) || (c.blk == 0);
       const bool last = (li == nblk - 1) || (c.blk == c.nb - 1);
-      const int sb = li & 1, n = p.cache_len[c.b], ntot = n + p.E;
-      if (!epi_all(mbar_wait(smem_u32(&sfull[sb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit))) { ok = false; break; }
+      const int sb = li & 1, pb = li & 1, n = p.cache_len[c.b], ntot = n + p.E;
+      if (!at_all(mbar_wait(smem_u32(&sfull[sb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit))) break;
       tc_fence_after();
-      float s[32];
-      tc_ld32(lane_base + (uint32_t)(sb * 128 + w * 32), s);
+      float s[QH];
+      if (QH == 16) tc_ld16(lane_base + (uint32_t)(sb * AT_NQ + q0), s);
+      else tc_ld8(lane_base + (uint32_t)(sb * AT_NQ + q0), s);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&sempty[sb]));
@@ -305,127 +342,121 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       at_next(p, nx);
       // every first product of this pair has completed: the next pair's queries may replace this pair's
       if (last && li + 1 < nblk) load_q(nx);
-      // scores in base 2, visibility, block maximum
-      const int key0 = c.blk * AT_KEYS + w * 32;
-      float mx = -INFINITY;
+      // scores in base 2; a slot this thread's key may not be seen from gives -inf (a select: whatever the
+      // slot holds stays out)
+      const int slot = c.blk * AT_KEYS + i;
+      bool exceed = false;
       if ((c.blk + 1) * AT_KEYS <= n) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) { s[i] *= p.scale_log2; mx = fmaxf(mx, s[i]); }
+        for (int q = 0; q < QH; ++q) { s[q] *= p.scale_log2; exceed |= s[q] > m[q] + 8.0f; }
       } else {
+        const bool cached = slot < n, drafted = slot >= n && slot < ntot;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int slot = key0 + i;
-          const bool seen = slot < n || (slot < ntot && ((vis >> (slot - n)) & 1ull));
-          s[i] = seen ? s[i] * p.scale_log2 : -INFINITY;      // a select: whatever an unseen slot holds stays out
-          mx = fmaxf(mx, s[i]);
+        for (int q = 0; q < QH; ++q) {
+          const bool seen = cached || (drafted && ((vis_sh[q0 + q] >> (slot - n)) & 1ull));
+          s[q] = seen ? s[q] * p.scale_log2 : -INFINITY;
+          exceed |= s[q] > m[q] + 8.0f;
         }
       }
-      // the reference maximum moves only when it is exceeded by more than 2^8 (P stays below 256)
-      const float mnew = (mx > m + 8.0f) ? mx : m;
-      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
-      const float corr = (mnew == m) ? 1.0f : sx_ex2f(m - msafe);
-      // the second product of the previous block has completed: P is free again and O is at rest
-      if (li >= 1 && !epi_all(mbar_wait(smem_u32(pempty), (uint32_t)(li - 1) & 1u, abort_flag, p.wait_limit))) { ok = false; break; }
-      if (!first && __any_sync(0xffffffffu, corr != 1.0f)) {
-        tc_fence_after();
-#pragma unroll 1
-        for (int c0 = 0; c0 < AT_D; c0 += 16) {
-          float v[16];
-          tc_ld16(lane_base + AT_O_COL + c0, v);
+      // the second product of the block before the previous one has completed: this P^T buffer is free again
+      if (li >= 2 && !at_all(mbar_wait(smem_u32(&pempty[pb]), (uint32_t)((li >> 1) - 1) & 1u, abort_flag, p.wait_limit))) break;
+      if (first || !at_all(!exceed)) {
+        // ---- a reference maximum moves: block maximum per query over the 128 keys -------------------------
+        // O^T must be at rest for the rescale: the second product of the previous block has completed
+        if (li >= 1 && !at_all(mbar_wait(smem_u32(&pempty[pb ^ 1]), (uint32_t)((li - 1) >> 1) & 1u, abort_flag, p.wait_limit))) break;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] *= corr;
-          tc_st16(lane_base + AT_O_COL + c0, v);
+        for (int q = 0; q < QH; ++q) {
+          float bm = s[q];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+          if (lane == 0) red[w * 32 + q0 + q] = bm;
         }
-        tc_wait_st();
-        tc_fence_before();
-      }
-      float sum = 0.f;
-      uint32_t pk[16];
+        at_bar();
+        float corr[QH];
+        bool any = false;
 #pragma unroll
-      for (int i = 0; i < 32; i += 2) {
-        const float a = sx_ex2f(s[i] - msafe), b2 = sx_ex2f(s[i + 1] - msafe);
-        sum += a + b2;
-        __nv_bfloat162 t2 = __floats2bfloat162_rn(a, b2);
-        pk[i >> 1] = *reinterpret_cast<uint32_t *>(&t2);
-      }
-      l = (first ? 0.f : l * corr) + sum;
-      m = mnew;
+        for (int q = 0; q < QH; ++q) {
+          const int qa = q0 + q;
+          const float bm = fmaxf(fmaxf(red[qa], red[32 + qa]), fmaxf(red[64 + qa], red[96 + qa]));
+          const float mold = m[q];
+          const float mnew = (first || bm > mold + 8.0f) ? bm : mold;
+          corr[q] = (first || mnew == mold) ? 1.0f : sx_ex2f(mold - mnew);      // mnew > mold is finite here
+          any |= corr[q] != 1.0f;
+          m[q] = mnew;
+          lsum[q] = first ? 0.f : lsum[q] * corr[q];
+        }
+        if (__any_sync(0xffffffffu, any)) {                   // the same in every lane of the warp: same inputs
+          float v[QH];
+          tc_fence_after();
+          if (QH == 16) tc_ld16(lane_base + AT_O_COL + q0, v);
+          else tc_ld8(lane_base + AT_O_COL + q0, v);
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch)
-        *reinterpret_cast<uint4 *>(p_row + ((((w & 1) * 4 + ch) ^ (row & 7)) << 4)) =
-            make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+          for (int q = 0; q < QH; ++q) v[q] *= corr[q];
+          if (QH == 16) tc_st16(lane_base + AT_O_COL + q0, v);
+          else tc_st8(lane_base + AT_O_COL + q0, v);
+          tc_wait_st();
+          tc_fence_before();
+        }
+        at_bar();                                              // red may be rewritten from here on
+      }
+      // probabilities (below 2^8), their partial sums, and this key's column of P^T
+      {
+        uint8_t *col = sPT + pb * AT_QP_BYTES + pt_col;
+#pragma unroll
+        for (int q = 0; q < QH; ++q) {
+          const int qa = q0 + q;
+          const float pq = sx_ex2f(s[q] - ((m[q] == -INFINITY) ? 0.f : m[q]));
+          lsum[q] += pq;
+          *reinterpret_cast<__nv_bfloat16 *>(col + qa * 128 + ((pt_chunk ^ (qa & 7)) << 4)) = __float2bfloat16_rn(pq);
+        }
+      }
       if ((c.blk + 1) * AT_KEYS > ntot) {
         // the block runs past the last slot: what the V rows behind it hold (anything, NaN included) must not
         // meet even a zero probability - clear them once the block has landed
-        const int cnt = at_v_entry(li, nblk), slot = cnt % AT_NS, nv = ntot - c.blk * AT_KEYS;
-        if (!epi_all(mbar_wait(smem_u32(&full[slot]), (uint32_t)(cnt / AT_NS) & 1u, abort_flag, p.wait_limit))) { ok = false; break; }
-        uint8_t *vb = ring + (size_t)slot * AT_BLK_BYTES;
-        for (int i = tid; i < (AT_KEYS - nv) * 16; i += 128) {
-          const int rr = nv + (i >> 4), ch = i & 15;
+        const int vslot = AT_NR + li % AT_NR, nv = ntot - c.blk * AT_KEYS;
+        if (!at_all(mbar_wait(smem_u32(&full[vslot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit))) break;
+        uint8_t *vb = ring + (size_t)vslot * AT_BLK_BYTES;
+        for (int e = etid; e < (AT_KEYS - nv) * 16; e += AT_EPI_THREADS) {
+          const int rr = nv + (e >> 4), ch = e & 15;
           *reinterpret_cast<uint4 *>(vb + (ch >> 3) * AT_HALF_BYTES + rr * 128 + ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
         }
       }
       fence_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(pfull));
+      if (lane == 0) mbar_arrive(smem_u32(&pfull[pb]));
       if (last) {
-        // ---- leave the pair: merge the four replicas of every query, write one partial result ------------
-        if (!epi_all(mbar_wait(smem_u32(ofull), (uint32_t)item & 1u, abort_flag, p.wait_limit))) { ok = false; break; }
+        // ---- leave the pair: add up the partial sums, write one partial result (m, l, O) per query -------
+        if (!at_all(mbar_wait(smem_u32(ofull), (uint32_t)item & 1u, abort_flag, p.wait_limit))) break;
         tc_fence_after();
-        cm[row] = m;
-        cl[row] = l;
-        epi_bar();
-        const float M = fmaxf(fmaxf(cm[lane], cm[32 + lane]), fmaxf(cm[64 + lane], cm[96 + lane]));
-        const float wgt = (m == -INFINITY) ? 0.f : sx_ex2f(m - M);
-        const int qq = tid & 31, seg = tid >> 5;                   // reduction role: query qq, 16 columns of a half
-        const size_t ps = (size_t)blockIdx.x + (size_t)(c.b * p.nkv + c.h);
-        if (seg == 0 && qq < p.NQ) {
-          float L = 0.f;
 #pragma unroll
-          for (int ww = 0; ww < 4; ++ww) {
-            const float mw = cm[ww * 32 + qq];
-            if (mw != -INFINITY) L += cl[ww * 32 + qq] * sx_ex2f(mw - M);
-          }
-          p.ws_ml[ps * 32 + qq] = make_float2(M, L);
+        for (int q = 0; q < QH; ++q) {
+          float a = lsum[q];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0) red[w * 32 + q0 + q] = a;
+          if (lane == 0 && w == 0) m_sh[q0 + q] = m[q];
         }
-#pragma unroll 1
-        for (int hf = 0; hf < 2; ++hf) {
-#pragma unroll 1
-          for (int c0 = 0; c0 < 64; c0 += 16) {
-            float v[16];
-            tc_ld16(lane_base + AT_O_COL + hf * 64 + c0, v);
+        at_bar();
+        const size_t ps = (size_t)blockIdx.x + (size_t)(c.b * p.nkv + c.h);
+        if (etid < p.NQ)
+          p.ws_ml[ps * 32 + etid] = make_float2(m_sh[etid], (red[etid] + red[32 + etid]) + (red[64 + etid] + red[96 + etid]));
+        {
+          float v[QH];
+          if (QH == 16) tc_ld16(lane_base + AT_O_COL + q0, v);
+          else tc_ld8(lane_base + AT_O_COL + q0, v);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) scratch[(c0 + i) * 128 + row] = v[i] * wgt;
-          }
-          epi_bar();
-          if (qq < p.NQ) {
-            float *dst = p.ws_o + (ps * 32 + qq) * AT_D + hf * 64 + seg * 16;
-#pragma unroll
-            for (int i = 0; i < 16; i += 4) {
-              float4 a;
-              const float *sc = scratch + (seg * 16 + i) * 128 + qq;
-              a.x = sc[0] + sc[32] + sc[64] + sc[96];
-              a.y = sc[128] + sc[160] + sc[192] + sc[224];
-              a.z = sc[256] + sc[288] + sc[320] + sc[352];
-              a.w = sc[384] + sc[416] + sc[448] + sc[480];
-              *reinterpret_cast<float4 *>(dst + i) = a;
-            }
-          }
-          epi_bar();
+          for (int q = 0; q < QH; ++q)
+            if (q0 + q < p.NQ) p.ws_o[(ps * 32 + q0 + q) * AT_D + i] = v[q];     // a warp: 32 consecutive floats
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(oempty));
-        // P served as scratch: back to zeros before the next block's probabilities go in
-        for (int i = tid; i < 32768 / 16; i += 128) reinterpret_cast<uint4 *>(sP)[i] = make_uint4(0, 0, 0, 0);
-        fence_async_smem();
-        epi_bar();
+        at_bar();                                              // red / m_sh / vis_sh are rewritten from here on
         ++item;
         if (li + 1 < nblk) pair_state(nx);
       }
       c = nx;
     }
-    (void)ok;
   }
   tc_teardown(abort_flag, p.status, tmem_base, AT_TMEM_COLS);
 }
@@ -469,7 +500,10 @@ bool sx_attn_tc_supported(const SxShape &sh, int nr, const sx_kv &kv) {
 
 sx_status sx_attn_tc_init(int device) {
   (void)device;
-  return sx_rc(cudaFuncSetAttribute(sx_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES));
+  if (cudaFuncSetAttribute(sx_attn_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sx_attn_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM_BYTES) != cudaSuccess)
+    return SX_ERR_CUDA;
+  return SX_OK;
 }
 
 size_t sx_attn_tc_ws_bytes(const SxShape &sh, int max_batch, int sm_count) {
@@ -500,6 +534,7 @@ sx_status sx_launch_attention_tc(const SxShape &sh, const SxRowMap &rm, int B, i
   CUtensorMap mk, mv;
   if (!sx_tma_map_2d(kv.k_pages_d, p.pool_rows, AT_D, AT_SLAB, &mk) || !sx_tma_map_2d(kv.v_pages_d, p.pool_rows, AT_D, AT_SLAB, &mv))
     return SX_ERR_CUDA;
-  SX_TRY(sx_rc(sx_launch(sx_attn_tc_kernel, dim3(sm_count), dim3(192), AT_SMEM_BYTES, st, mk, mv, p)));
+  if (p.NQ <= 16) SX_TRY(sx_rc(sx_launch(sx_attn_tc_kernel<16>, dim3(sm_count), dim3(AT_THREADS), AT_SMEM_BYTES, st, mk, mv, p)));
+  else SX_TRY(sx_rc(sx_launch(sx_attn_tc_kernel<32>, dim3(sm_count), dim3(AT_THREADS), AT_SMEM_BYTES, st, mk, mv, p)));
   return sx_rc(sx_launch(sx_attn_tc_merge_kernel, dim3(B * sh.nkv, p.NQ), dim3(AT_D), 0, st, p, sm_count, o_out));
 }
