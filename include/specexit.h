@@ -33,6 +33,8 @@
  *   - Matrices are bf16, row-major [out, in].  Activations handed between layers are
  *     bf16; accumulation, normalisation, softmax, rotary and signal math are fp32.
  *   - One sx_ctx per stream: a context is not thread-safe.
+ *   - With the environment variable SX_NVTX=1 the entry points open NVTX ranges ("sx spec exit iteration",
+ *     "sx draft round k", "sx verify", "sx exit update", "sx commit") for timeline tools.
  */
 #ifndef SPECEXIT_H
 #define SPECEXIT_H

@@ -5,7 +5,26 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <stdlib.h>
+
+#include <nvtx3/nvToolsExt.h>
+
 #include "sx_kernels.cuh"
+
+// Named ranges for timeline tools (the header-only NVTX v3: nothing is linked, and without a tool attached a
+// range costs a function-pointer test).  Off unless the environment variable SX_NVTX is set to 1.
+static bool sx_nvtx_on() {
+  static const bool on = [] { const char *e = getenv("SX_NVTX"); return e && e[0] == '1'; }();
+  return on;
+}
+struct SxRange {
+  bool on;
+  explicit SxRange(const char *name) : on(sx_nvtx_on()) { if (on) nvtxRangePushA(name); }
+  SxRange(const char *fmt, int k) : on(sx_nvtx_on()) {
+    if (on) { char buf[48]; snprintf(buf, sizeof(buf), fmt, k); nvtxRangePushA(buf); }
+  }
+  ~SxRange() { if (on) nvtxRangePop(); }
+};
 
 struct sx_ctx {
   SxShape sh;
@@ -326,6 +345,7 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
                              const int32_t *tok, SxIndex ti, const uint64_t *row_mask, bf16 *hid_user, SxIndex ui,
                              int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si, char *ws,
                              int32_t *status, cudaStream_t st, bool input_ready = false, bool prepare_next = false) {
+  SxRange range("sx draft round %d", round);
   const SxShape &s = c->sh;
   bf16 *u = (bf16 *)(ws + c->off_u), *x = (bf16 *)(ws + c->off_x), *n = (bf16 *)(ws + c->off_n);
   bf16 *q = (bf16 *)(ws + c->off_q), *o = (bf16 *)(ws + c->off_o), *a = (bf16 *)(ws + c->off_a);
@@ -457,6 +477,7 @@ extern "C" sx_status sx_verify(sx_ctx *c, int32_t batch, int32_t P, const void *
   if (batch < 1 || P < 1 || path_stride < 1 || ((uintptr_t)target_hidden_d & 15)) return SX_ERR_INVALID_ARG;
   if (parent_d && P > SX_MAX_VERIFY_SLOTS) return SX_ERR_UNSUPPORTED;
   SX_TRY(check_ws(c, ws_d, ws_bytes));
+  SxRange range("sx verify");
   cudaStream_t st = (cudaStream_t)stream;
   SxSample smp = c->smp;
   smp.P = P;
@@ -484,6 +505,7 @@ extern "C" sx_status sx_exit_update(sx_ctx *c, int32_t batch, int32_t P, const s
       (!state->hist_d || cfg->window < 2 || cfg->window >= SX_HIST))
     return SX_ERR_INVALID_ARG;
   if (cfg->smoothing == SX_SMOOTH_PARAGRAPH && (!state->par_sum_d || !state->par_n_d)) return SX_ERR_INVALID_ARG;
+  SxRange range("sx exit update");
   SX_TRY(sx_launch_exit(batch, P, c->sh.S, *cfg, *state, slot_signal_d, cand_tok_d, path_d, path_stride, accept_len_d,
                  recover_tok_d, exit_flag_d, accept_len_out_d, recover_tok_out_d, smoothed_out_d, c->sh.V, status_d,
                  (cudaStream_t)stream));
@@ -503,6 +525,7 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
     return SX_ERR_INVALID_ARG;
   if (((uintptr_t)feat0_d & 15) || ((uintptr_t)o->hidden_d & 15) || ((uintptr_t)target_hidden_d & 15))
     return SX_ERR_INVALID_ARG;
+  SxRange range("sx spec exit iteration");
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)ws_d;
   const int B = kv->batch, K = c->dc.K, P = c->P, S = c->sh.S;
@@ -607,6 +630,7 @@ extern "C" sx_status sx_commit(sx_ctx *c, const sx_kv *kv, int32_t P, const void
   SX_TRY(check_ws(c, ws_d, ws_bytes));
   if (P < 1 || path_stride < 1 || path_stride - 1 > c->dc.K) return SX_ERR_INVALID_ARG;
   if (((uintptr_t)target_hidden_d & 15) || ((uintptr_t)feat0_next_d & 15)) return SX_ERR_INVALID_ARG;
+  SxRange range("sx commit");
   cudaStream_t st = (cudaStream_t)stream;
   char *ws = (char *)ws_d;
   const SxShape &s = c->sh;

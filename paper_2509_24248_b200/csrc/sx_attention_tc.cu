@@ -38,7 +38,10 @@
 #define AT_KEYS 128                         // keys per block
 #define AT_SLAB 64                          // keys per TMA box (a page holds a multiple of this)
 #define AT_NS 6                             // ring slots of 32 KB in all
-#define AT_NR 3                             // ... three for K blocks, three for V blocks: two rings
+#ifndef AT_NK
+#define AT_NK 3                             // ... of them for K blocks,
+#endif
+#define AT_NV (AT_NS - AT_NK)               // the rest for V blocks: two rings
 #define AT_BLK_BYTES (AT_KEYS * AT_D * 2)   // 32 KB
 #define AT_HALF_BYTES (128 * 128)           // a 128-row tile of 64 columns (one swizzle row per matrix row)
 #define AT_SLAB_BYTES (AT_SLAB * 128)
@@ -183,7 +186,7 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     // life (K at once, V only after the scores have been through the softmax): in one ring a landed V block
     // would hold a slot the K stream could have in flight.
     const bool is_v = warp != 0;
-    const int base_slot = is_v ? AT_NR : 0;
+    const int base_slot = is_v ? AT_NK : 0, nring = is_v ? AT_NV : AT_NK;
     const CUtensorMap *map = is_v ? &tmV : &tmK;
     const uint64_t pol = policy_evict_first();
     AtCursor c = at_seek(p, g0);
@@ -213,9 +216,9 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       const int row_next = (li + 1 < nblk) ? rows_of(nx) : p.pool_rows;      // looked up while this block's loads wait
       const int row0 = __shfl_sync(0xffffffffu, row_cur, 0), row1 = __shfl_sync(0xffffffffu, row_cur, 1);
       if (lane == 0) {
-        const int slot = base_slot + li % AT_NR;
-        const uint32_t ph = (uint32_t)(li / AT_NR) & 1u;
-        if (li >= AT_NR && !mbar_wait(smem_u32(&empty[slot]), ph ^ 1u, abort_flag, p.wait_limit)) ok = false;
+        const int slot = base_slot + li % nring;
+        const uint32_t ph = (uint32_t)(li / nring) & 1u;
+        if (li >= nring && !mbar_wait(smem_u32(&empty[slot]), ph ^ 1u, abort_flag, p.wait_limit)) ok = false;
         if (ok) {
           const uint32_t fb = smem_u32(&full[slot]);
           const uint32_t dst = smem_u32(ring + (size_t)slot * AT_BLK_BYTES);
@@ -244,8 +247,8 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const bool first = (li == 0) || (c1.blk == 0);
         if (first && li > 0) ++item1;
         if (first && !mbar_wait(smem_u32(qfull), (uint32_t)item1 & 1u, abort_flag, p.wait_limit)) break;
-        const int slot = li % AT_NR, sb = li & 1, u = li >> 1;
-        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit)) break;
+        const int slot = li % AT_NK, sb = li & 1, u = li >> 1;
+        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NK) & 1u, abort_flag, p.wait_limit)) break;
         if (u >= 1 && !mbar_wait(smem_u32(&sempty[sb]), (uint32_t)(u - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t kb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES);
@@ -271,9 +274,9 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const bool first = (li == 0) || (c2.blk == 0);
         const bool last = (li == nblk - 1) || (c2.blk == c2.nb - 1);
         if (first && li > 0) ++item2;
-        const int slot = AT_NR + li % AT_NR, pb = li & 1;
+        const int slot = AT_NK + li % AT_NV, pb = li & 1;
         if (!mbar_wait(smem_u32(&pfull[pb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit)) break;
-        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit)) break;
+        if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NV) & 1u, abort_flag, p.wait_limit)) break;
         if (first && item2 > 0 && !mbar_wait(smem_u32(oempty), (uint32_t)(item2 - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t vb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES), pt = pt_addr + (uint32_t)pb * AT_QP_BYTES;
@@ -413,8 +416,8 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       if ((c.blk + 1) * AT_KEYS > ntot) {
         // the block runs past the last slot: what the V rows behind it hold (anything, NaN included) must not
         // meet even a zero probability - clear them once the block has landed
-        const int vslot = AT_NR + li % AT_NR, nv = ntot - c.blk * AT_KEYS;
-        if (!at_all(mbar_wait(smem_u32(&full[vslot]), (uint32_t)(li / AT_NR) & 1u, abort_flag, p.wait_limit))) break;
+        const int vslot = AT_NK + li % AT_NV, nv = ntot - c.blk * AT_KEYS;
+        if (!at_all(mbar_wait(smem_u32(&full[vslot]), (uint32_t)(li / AT_NV) & 1u, abort_flag, p.wait_limit))) break;
         uint8_t *vb = ring + (size_t)vslot * AT_BLK_BYTES;
         for (int e = etid; e < (AT_KEYS - nv) * 16; e += AT_EPI_THREADS) {
           const int rr = nv + (e >> 4), ch = e & 15;
