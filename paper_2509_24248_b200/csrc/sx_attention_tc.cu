@@ -46,7 +46,7 @@
 #define AT_HALF_BYTES (128 * 128)           // a 128-row tile of 64 columns (one swizzle row per matrix row)
 #define AT_SLAB_BYTES (AT_SLAB * 128)
 #define AT_NQ 32                            // query columns of the accumulators
-#define AT_TMEM_COLS 128                    // S^T 0 | S^T 1 | O^T (32 columns each), rounded to a power of two
+#define AT_TMEM_COLS 128                    // S^T 0 | S^T 1 | O^T 0 | O^T 1 (32 columns each)
 #define AT_O_COL 64
 #define AT_QP_BYTES (AT_NQ * AT_D * 2)      // Q, and P^T: 32 rows of 128 elements
 #define AT_SMEM_BYTES (1024 + 3 * AT_QP_BYTES + AT_NS * AT_BLK_BYTES + 256 + 512 + 256 + 128)
@@ -137,8 +137,8 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   uint64_t *bars = reinterpret_cast<uint64_t *>(ring + AT_NS * AT_BLK_BYTES);
   // K ring: full[0..2] / empty[0..2]; V ring: full[3..5] / empty[3..5]
   uint64_t *full = bars, *empty = bars + AT_NS, *sfull = bars + 2 * AT_NS, *sempty = sfull + 2;
-  uint64_t *pfull = sempty + 2, *pempty = pfull + 2, *qfull = pempty + 2, *ofull = qfull + 1, *oempty = ofull + 1;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(oempty + 1);
+  uint64_t *pfull = sempty + 2, *pempty = pfull + 2, *qfull = pempty + 2, *ofull = qfull + 1, *oempty = ofull + 2;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(oempty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   float *red = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(bars) + 256);  // [4 lane quarters][32 queries]
   uint64_t *vis_sh = reinterpret_cast<uint64_t *>(red + 128);                       // [32] visibility of the drafted rows
@@ -166,8 +166,10 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       mbar_init(smem_u32(&pfull[i]), 8);
     }
     mbar_init(smem_u32(qfull), 8);
-    mbar_init(smem_u32(ofull), 1);
-    mbar_init(smem_u32(oempty), 8);
+    for (int i = 0; i < 2; ++i) {            // O^T of consecutive pairs alternates between two accumulators
+      mbar_init(smem_u32(&ofull[i]), 1);
+      mbar_init(smem_u32(&oempty[i]), 8);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -277,17 +279,19 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const int slot = AT_NK + li % AT_NV, pb = li & 1;
         if (!mbar_wait(smem_u32(&pfull[pb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit)) break;
         if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NV) & 1u, abort_flag, p.wait_limit)) break;
-        if (first && item2 > 0 && !mbar_wait(smem_u32(oempty), (uint32_t)(item2 - 1) & 1u, abort_flag, p.wait_limit)) break;
+        const int ob = item2 & 1;
+        // the accumulator was last used two pairs ago: its result has been read out
+        if (first && item2 >= 2 && !mbar_wait(smem_u32(&oempty[ob]), (uint32_t)((item2 >> 1) - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
         const uint32_t vb = smem_u32(ring + (size_t)slot * AT_BLK_BYTES), pt = pt_addr + (uint32_t)pb * AT_QP_BYTES;
 #pragma unroll
         for (int k = 0; k < AT_KEYS / 16; ++k)
-          tc_mma(tmem_base + AT_O_COL, smem_desc_mn(vb + (uint32_t)k * 2048u, AT_HALF_BYTES, 1024u),
+          tc_mma(tmem_base + AT_O_COL + (uint32_t)ob * AT_NQ, smem_desc_mn(vb + (uint32_t)k * 2048u, AT_HALF_BYTES, 1024u),
                  smem_desc(pt + (uint32_t)(k >> 2) * (AT_NQ * 128) + (uint32_t)(k & 3) * 32u), idesc_o,
                  (first && k == 0) ? 0u : 1u);
         tc_commit(smem_u32(&empty[slot]));
         tc_commit(smem_u32(&pempty[pb]));
-        if (last) tc_commit(smem_u32(ofull));
+        if (last) tc_commit(smem_u32(&ofull[ob]));
         at_next(p, c2);
       }
     }
@@ -326,6 +330,24 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       }
 #pragma unroll
       for (int q = 0; q < QH; ++q) { m[q] = -INFINITY; lsum[q] = 0.f; }
+    };
+    int pend_item = -1;
+    size_t pend_ps = 0;
+    auto flush_pending = [&]() -> bool {
+      const int ob = pend_item & 1;
+      if (!at_all(mbar_wait(smem_u32(&ofull[ob]), (uint32_t)(pend_item >> 1) & 1u, abort_flag, p.wait_limit))) return false;
+      tc_fence_after();
+      float v[QH];
+      if (QH == 16) tc_ld16(lane_base + AT_O_COL + (uint32_t)ob * AT_NQ + q0, v);
+      else tc_ld8(lane_base + AT_O_COL + (uint32_t)ob * AT_NQ + q0, v);
+#pragma unroll
+      for (int q = 0; q < QH; ++q)
+        if (q0 + q < p.NQ) p.ws_o[(pend_ps * 32 + q0 + q) * AT_D + i] = v[q];     // a warp: 32 consecutive floats
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&oempty[ob]));
+      pend_item = -1;
+      return true;
     };
     load_q(c);
     pair_state(c);
@@ -391,12 +413,13 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         if (__any_sync(0xffffffffu, any)) {                   // the same in every lane of the warp: same inputs
           float v[QH];
           tc_fence_after();
-          if (QH == 16) tc_ld16(lane_base + AT_O_COL + q0, v);
-          else tc_ld8(lane_base + AT_O_COL + q0, v);
+          const uint32_t ocol = lane_base + AT_O_COL + (uint32_t)(item & 1) * AT_NQ + q0;
+          if (QH == 16) tc_ld16(ocol, v);
+          else tc_ld8(ocol, v);
 #pragma unroll
           for (int q = 0; q < QH; ++q) v[q] *= corr[q];
-          if (QH == 16) tc_st16(lane_base + AT_O_COL + q0, v);
-          else tc_st8(lane_base + AT_O_COL + q0, v);
+          if (QH == 16) tc_st16(ocol, v);
+          else tc_st8(ocol, v);
           tc_wait_st();
           tc_fence_before();
         }
@@ -427,10 +450,11 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
       fence_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&pfull[pb]));
+      // The O^T of a pair that ended one block ago: its last second product has surely completed by now, so
+      // reading it out here costs no wait, and the pair that follows it was not held up (two accumulators).
+      if (pend_item >= 0 && !flush_pending()) break;
       if (last) {
-        // ---- leave the pair: add up the partial sums, write one partial result (m, l, O) per query -------
-        if (!at_all(mbar_wait(smem_u32(ofull), (uint32_t)item & 1u, abort_flag, p.wait_limit))) break;
-        tc_fence_after();
+        // ---- leave the pair: add up the partial sums, write (m, l) per query; O^T follows one block later ----
 #pragma unroll
         for (int q = 0; q < QH; ++q) {
           float a = lsum[q];
@@ -443,23 +467,15 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const size_t ps = (size_t)blockIdx.x + (size_t)(c.b * p.nkv + c.h);
         if (etid < p.NQ)
           p.ws_ml[ps * 32 + etid] = make_float2(m_sh[etid], (red[etid] + red[32 + etid]) + (red[64 + etid] + red[96 + etid]));
-        {
-          float v[QH];
-          if (QH == 16) tc_ld16(lane_base + AT_O_COL + q0, v);
-          else tc_ld8(lane_base + AT_O_COL + q0, v);
-#pragma unroll
-          for (int q = 0; q < QH; ++q)
-            if (q0 + q < p.NQ) p.ws_o[(ps * 32 + q0 + q) * AT_D + i] = v[q];     // a warp: 32 consecutive floats
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(oempty));
+        pend_item = item;
+        pend_ps = ps;
         at_bar();                                              // red / m_sh / vis_sh are rewritten from here on
         ++item;
         if (li + 1 < nblk) pair_state(nx);
       }
       c = nx;
     }
+    if (pend_item >= 0) flush_pending();
   }
   tc_teardown(abort_flag, p.status, tmem_base, AT_TMEM_COLS);
 }
