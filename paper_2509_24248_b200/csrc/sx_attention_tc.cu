@@ -46,8 +46,9 @@
 #define AT_HALF_BYTES (128 * 128)           // a 128-row tile of 64 columns (one swizzle row per matrix row)
 #define AT_SLAB_BYTES (AT_SLAB * 128)
 #define AT_NQ 32                            // query columns of the accumulators
-#define AT_TMEM_COLS 128                    // S^T 0 | S^T 1 | O^T 0 | O^T 1 (32 columns each)
-#define AT_O_COL 64
+#define AT_NSB 4                            // S^T accumulators: the first products run up to four blocks ahead of the softmax
+#define AT_TMEM_COLS 256                    // S^T 0..3 | O^T 0 | O^T 1 (32 columns each), rounded to a power of two
+#define AT_O_COL (AT_NSB * 32)
 #define AT_QP_BYTES (AT_NQ * AT_D * 2)      // Q, and P^T: 32 rows of 128 elements
 #define AT_SMEM_BYTES (1024 + 3 * AT_QP_BYTES + AT_NS * AT_BLK_BYTES + 256 + 512 + 256 + 128)
 #define AT_EPI_THREADS 256
@@ -136,8 +137,8 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
   uint8_t *sQ = smem, *sPT = smem + AT_QP_BYTES, *ring = smem + 3 * AT_QP_BYTES;      // P^T: two buffers
   uint64_t *bars = reinterpret_cast<uint64_t *>(ring + AT_NS * AT_BLK_BYTES);
   // K ring: full[0..2] / empty[0..2]; V ring: full[3..5] / empty[3..5]
-  uint64_t *full = bars, *empty = bars + AT_NS, *sfull = bars + 2 * AT_NS, *sempty = sfull + 2;
-  uint64_t *pfull = sempty + 2, *pempty = pfull + 2, *qfull = pempty + 2, *ofull = qfull + 1, *oempty = ofull + 2;
+  uint64_t *full = bars, *empty = bars + AT_NS, *sfull = bars + 2 * AT_NS, *sempty = sfull + AT_NSB;
+  uint64_t *pfull = sempty + AT_NSB, *pempty = pfull + 2, *qfull = pempty + 2, *ofull = qfull + 1, *oempty = ofull + 2;
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(oempty + 2);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
   float *red = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(bars) + 256);  // [4 lane quarters][32 queries]
@@ -156,9 +157,11 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < AT_NS; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < AT_NSB; ++i) {
       mbar_init(smem_u32(&sfull[i]), 1);
       mbar_init(smem_u32(&sempty[i]), 8);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&pempty[i]), 1);
       // one barrier per P^T buffer: a buffer is refilled only after the second product that read it has
       // completed, so its barrier can never run a whole phase ahead of the MMA issuer (a single barrier
@@ -249,7 +252,7 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
         const bool first = (li == 0) || (c1.blk == 0);
         if (first && li > 0) ++item1;
         if (first && !mbar_wait(smem_u32(qfull), (uint32_t)item1 & 1u, abort_flag, p.wait_limit)) break;
-        const int slot = li % AT_NK, sb = li & 1, u = li >> 1;
+        const int slot = li % AT_NK, sb = li % AT_NSB, u = li / AT_NSB;
         if (!mbar_wait(smem_u32(&full[slot]), (uint32_t)(li / AT_NK) & 1u, abort_flag, p.wait_limit)) break;
         if (u >= 1 && !mbar_wait(smem_u32(&sempty[sb]), (uint32_t)(u - 1) & 1u, abort_flag, p.wait_limit)) break;
         tc_fence_after();
@@ -354,8 +357,8 @@ sx_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant
     for (int li = 0; li < nblk; ++li) {
       const bool first = (li == 0) || (c.blk == 0);
       const bool last = (li == nblk - 1) || (c.blk == c.nb - 1);
-      const int sb = li & 1, pb = li & 1, n = p.cache_len[c.b], ntot = n + p.E;
-      if (!at_all(mbar_wait(smem_u32(&sfull[sb]), (uint32_t)(li >> 1) & 1u, abort_flag, p.wait_limit))) break;
+      const int sb = li % AT_NSB, pb = li & 1, n = p.cache_len[c.b], ntot = n + p.E;
+      if (!at_all(mbar_wait(smem_u32(&sfull[sb]), (uint32_t)(li / AT_NSB) & 1u, abort_flag, p.wait_limit))) break;
       tc_fence_after();
       float s[QH];
       if (QH == 16) tc_ld16(lane_base + (uint32_t)(sb * AT_NQ + q0), s);
