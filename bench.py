@@ -65,6 +65,17 @@ def algorithmic_bytes(wl: synth.Workload, lens) -> dict:
     return {"total": total, "head_launch": 2 * head, "w_round": w_round, "kv_round": kv_round}
 
 
+def workload_config(args, wl: synth.Workload, lens) -> dict:
+    """The `config` entry of the JSON line: what was run.  Both arms print the same dictionary for the same
+    command-line options."""
+    ab = algorithmic_bytes(wl, lens)
+    return {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree",
+            "cached_tokens": int(sum(int(n) for n in lens)),
+            "weights": "tiled at load (sx_tile_weight)" if args.weights == "tiled" else "row-major",
+            "l2": "no flush: each iteration streams %.2f GB of weights and KV, far beyond the 126 MB L2"
+                  % (ab["total"] / 1e9)}
+
+
 def _oracle_sample(args):
     """Sampling settings of the CPU legs (None: greedy)."""
     from oracle import specexit_oracle as orc
@@ -231,7 +242,7 @@ def run_reference(args, wl):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "verified_tokens_per_s": toks / dt,
-            "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree"},
+            "config": workload_config(args, wl, synth.cache_lengths(wl)),
             "cpu_baseline": {"value": val, "unit": "iterations/s", "cores": cores, "kind": "oracle",
                              "sample": f"{args.steps} whole iteration(s) of {wl.name} (draft rounds + verify + exit)"},
             "e2e": {"value": val, "unit": "iterations/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -464,11 +475,7 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
         "value": value, "ms_per_step": ms, "steps": steps, "warmup": max(3, warmup),
         "verified_tokens_per_s": vtok, "sequence_iterations_per_s": value * wl.B,
         "ms_per_step_percentiles": {"p10": pct(0.10), "p50": pct(0.50), "p90": pct(0.90)},
-        "config": {"workload": wl.name, "batch": wl.B, "K": wl.K, "mode": "chain" if wl.mode == synth.CHAIN else "tree",
-                   "cached_tokens": int(sum(int(n) for n in lens)),
-                   "weights": "tiled at load (sx_tile_weight)" if args.weights == "tiled" else "row-major",
-                   "l2": "no flush: each iteration streams %.2f GB of weights and KV, far beyond the 126 MB L2"
-                         % (ab["total"] / 1e9)},
+        "config": workload_config(args, wl, lens),
         # the step's bound is the slower of its bytes at the HBM bandwidth and its flops at the bf16 tensor peak
         "step_roofline": {"bytes_per_iteration": ab["total"], "flops_per_iteration": fl,
                           "hbm_bound_ms": hbm_ms, "flop_bound_ms": flop_ms, "bound": "hbm" if hbm_ms >= flop_ms else "tensor",
