@@ -410,11 +410,12 @@ class TreeDraft:
     slot_signal: torch.Tensor       # [B, P, S], NaN where the slot was never expanded
     margins: Dict[Tuple, float] = field(default_factory=dict)  # deciding margin per decision
     slot_cid: Optional[torch.Tensor] = None
+    row_logits: Optional[Dict[Tuple[int, int], torch.Tensor]] = None   # (b, row) -> draft logits, when children are sampled
 
 
 def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tensor, depth: int,
                topk: int, max_nodes: int, override: Optional[Dict[Tuple, List[int]]] = None,
-               chooser=None, before_round=None, head_input=None) -> TreeDraft:
+               chooser=None, before_round=None, head_input=None, sample=None) -> TreeDraft:
     """Tree drafting.  Round 1 drafts the root; round r >= 2 expands the `topk` best
     candidates of depth r-1 (score = sum of log-probabilities; ties: lower candidate id).
     After the last round the `max_nodes` best candidates overall are kept and laid out in
@@ -426,6 +427,14 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
     sh = model.sh
     B, H, S = f0.shape[0], sh.H, sh.S
     ov = override or {}
+    # Sampled children (``sample.sample_drafts`` with a positive temperature): the children of a drafted row
+    # are the topk largest of logit + tau * Gumbel noise, best first, which is a draw of topk tokens WITHOUT
+    # replacement, in order, from softmax(logits / tau) (the Gumbel-top-k identity).  The noise of the
+    # children of drafted row `row` of sequence b is the stream with slot word TREE_STREAM + row.  Scores
+    # stay sums of (unperturbed) log-probabilities.  The rows' logits are kept for the verification walk.
+    sampling = sample is not None and sample.sample_drafts and sample.temperature > 0.0
+    tau = float(torch.tensor(sample.temperature, dtype=torch.float32)) if sampling else 0.0
+    row_logits: Dict[Tuple[int, int], torch.Tensor] = {}
     n_rows = 1 + topk * (depth - 1)
     P = 1 + max_nodes
     hidden = torch.empty(B, n_rows, H, dtype=F64)
@@ -435,12 +444,17 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
     row_vis: List[Dict[int, List[int]]] = [dict() for _ in range(B)]
 
     def emit(b, row, par_cid, par_score, dep, logits):
-        ids = topk_low(logits, topk)
-        margins[("topk", b, row)] = order_gap(logits, topk)      # order of the k children and the cut behind them
+        rank_by = logits
+        if sampling:
+            assert model.map is None, "sampled children need a full-vocabulary draft head"
+            row_logits[(b, row)] = logits
+            rank_by = logits + tau * gumbel_noise(sample, b, TREE_STREAM + row, logits.numel())
+        ids = topk_low(rank_by, topk)
+        margins[("topk", b, row)] = order_gap(rank_by, topk)     # order of the k children and the cut behind them
         if ("topk", b, row) in ov:
             ids = list(ov[("topk", b, row)])
         if chooser is not None:
-            ids = list(chooser("topk", (b, row), logits, topk, ids))
+            ids = list(chooser("topk", (b, row), rank_by, topk, ids))
         lse = torch.logsumexp(logits, dim=0)
         for t in ids:
             lp = f32r(logits[t] - lse)
@@ -527,7 +541,7 @@ def draft_tree(model: DraftModel, kv: PagedKV, f0: torch.Tensor, t0: torch.Tenso
             if c.row >= 0:
                 slot_sig[b, s] = row_sig[b, c.row]
     return TreeDraft(cands, cand_tok, parent, dep, slot_row, slot_src, hidden, slot_sig, margins,
-                     slot_cid)
+                     slot_cid, row_logits if sampling else None)
 
 
 # --------------------------------------------------------------------------------------
@@ -613,6 +627,8 @@ class SampleCfg:
 # target-side Gumbel noise), ACCEPT_STREAM + j (the uniform of the accept test) and
 # DRAFT_STREAM + j (the Gumbel noise that draws the draft token proposed at slot j).
 ACCEPT_STREAM, DRAFT_STREAM = 0x20000000, 0x40000000
+# TREE_STREAM + r: the Gumbel noise that draws the children of drafted row r of a tree
+TREE_STREAM = 0x50000000
 
 
 def gumbel_noise(cfg: SampleCfg, b: int, j: int, V: int) -> torch.Tensor:
@@ -700,6 +716,92 @@ def speculative_sample(model: DraftModel, target_hidden: torch.Tensor, cand_tok:
             t2 = torch.topk(s, 2).values
             gap[b, j] = float(t2[0] - t2[1])          # absolute: the scores are logarithms
     return SpecSampleOut(tok, acc, margin, gap)
+
+
+@dataclass
+class TreeWalkOut:
+    target_tok: torch.Tensor   # [B, P] at a visited slot: the accepted child's token, or the token drawn there; else -1
+    accept_len: torch.Tensor   # [B]
+    path: List[List[int]]      # accepted slots, starting with slot 0
+    recover_tok: torch.Tensor  # [B]
+    exempt: List[str]          # decisions adopted from `decide` (see below)
+
+
+def tree_speculative_walk(model: DraftModel, target_hidden: torch.Tensor, draft: "TreeDraft", cfg: SampleCfg,
+                          decide=None) -> TreeWalkOut:
+    """Speculative sampling down a tree whose children were drawn from the draft (see draft_tree).
+
+    At the current slot, with p = softmax(target logits / tau) and q = softmax(the logits of the drafted row
+    that produced the slot's children / tau), the kept children are tried in the order they were drawn:
+    child token x is accepted when u < min(1, p(x) / q(x)); a refusal replaces p by the normalised
+    max(0, p - q) and takes x out of q (renormalised), which is the law of the next draw without replacement.
+    When a child is accepted the walk continues from it; when all are refused (or the slot has none) the
+    recover token is drawn from the p that is left, and the walk ends.  The emitted token then follows the
+    target's distribution exactly as long as every child drawn at a visited slot is still in the tree (a
+    child pruned away for its score is simply not tried: with pruning the rule is approximate).
+    Draws: u of slot s from word 0 of the block with counter (0, ACCEPT_STREAM + s, b, offset); the final draw
+    at slot s is a Gumbel-max over the logarithm of what is left of p, with the noise of slot s - for a
+    slot where nothing was refused that is argmax(logit + tau g), the draw of `target_sample`.
+    ``decide(kind, key, default, margin)`` may replace a decision whose margin is small (tests): kind
+    "accept" with key (b, slot) and a bool, kind "draw" with key (b, slot) and a token."""
+    B, P, H = target_hidden.shape
+    assert draft.row_logits is not None and model.map is None
+    logits = f32r(linear(target_hidden.reshape(B * P, H).to(F64), model.target_head)).view(B, P, -1)
+    tau = float(torch.tensor(cfg.temperature, dtype=torch.float32))
+    key = (cfg.seed & 0xFFFFFFFF, (cfg.seed >> 32) & 0xFFFFFFFF)
+    tt = torch.full((B, P), -1, dtype=torch.int64)
+    L = torch.zeros(B, dtype=torch.int64)
+    rec = torch.zeros(B, dtype=torch.int64)
+    paths, exempt = [], []
+    for b in range(B):
+        cur, path = 0, [0]
+        while True:
+            lp = logits[b, cur] / tau
+            p = torch.exp(lp - torch.logsumexp(lp, dim=0))
+            kids = [s for s in range(cur + 1, P) if int(draft.parent[b, s]) == cur]
+            row = int(draft.slot_row[b, cur])
+            nxt = -1
+            if kids:
+                lq = draft.row_logits[(b, row)].to(F64) / tau
+                q = torch.exp(lq - torch.logsumexp(lq, dim=0))
+                for s in kids:
+                    x = int(draft.cand_tok[b, s])
+                    ratio = min(1.0, float(p[x]) / float(q[x]))
+                    u = float(uniform_open(philox4x32_10((0, ACCEPT_STREAM + s, b, cfg.offset), key)[0]))
+                    ok = u < ratio
+                    if decide is not None:
+                        ok2 = bool(decide("accept", (b, s), ok, abs(u - ratio)))
+                        if ok2 != ok:
+                            exempt.append(f"accept test b={b} slot={s}")
+                        ok = ok2
+                    if ok:
+                        nxt = s
+                        break
+                    p = (p - q).clamp_min(0.0)
+                    p = p / p.sum()
+                    q = q.clone()
+                    q[x] = 0.0
+                    q = q / q.sum()
+            if nxt >= 0:
+                tt[b, cur] = int(draft.cand_tok[b, nxt])
+                cur = nxt
+                path.append(cur)
+                continue
+            g = gumbel_noise(cfg, b, cur, p.numel())
+            sc = torch.where(p > 0, torch.log(p.clamp_min(1e-300)) + g, torch.full_like(p, -float("inf")))
+            t = argmax_low(sc)
+            if decide is not None:
+                t2 = torch.topk(sc, 2).values
+                tnew = int(decide("draw", (b, cur), t, float(t2[0] - t2[1])))
+                if tnew != t:
+                    exempt.append(f"draw b={b} slot={cur}")
+                t = tnew
+            tt[b, cur] = t
+            rec[b] = t
+            break
+        L[b] = len(path) - 1
+        paths.append(path)
+    return TreeWalkOut(tt, L, paths, rec, exempt)
 
 
 def accept_chain(cand_tok: Sequence[int], target_tok: Sequence[int]) -> Tuple[int, List[int], int]:

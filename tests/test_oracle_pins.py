@@ -1187,6 +1187,120 @@ def test_speculative_sampling_keeps_every_draft_when_draft_and_target_agree():
     assert bool(so.accepted[:, 0].all()) and torch.equal(so.target_tok[:, 0], cand[:, 1])
 
 
+# ---------------------------------------------------------------------------------------
+# sampled children in a tree: draws without replacement, the sequential accept / residual rule
+# ---------------------------------------------------------------------------------------
+def _one_level_tree(n, V, k, lq, cfg):
+    """n sequences, each a root (slot 0) with k children drawn from softmax(lq / tau) the way draft_tree
+    draws them: the k best of lq + tau * Gumbel noise of the stream TREE_STREAM + 0, best first."""
+    tau = cfg.temperature
+    cand = torch.zeros(n, 1 + k, dtype=torch.int64)
+    rl = {}
+    for b in range(n):
+        sc = torch.tensor(lq, dtype=F64) + tau * orc.gumbel_noise(cfg, b, orc.TREE_STREAM, V)
+        cand[b, 1:] = torch.tensor(orc.topk_low(sc, k))
+        rl[(b, 0)] = torch.tensor(lq, dtype=F64)
+    parent = torch.tensor([[-1] + [0] * k] * n)
+    slot_row = torch.tensor([[0] + [-1] * k] * n)
+    return orc.TreeDraft(cands=None, cand_tok=cand, parent=parent, depth=None, slot_row=slot_row, slot_src_row=None,
+                         hidden=None, slot_signal=None, row_logits=rl)
+
+
+def test_children_drawn_with_the_gumbel_top_k_are_a_draw_without_replacement():
+    # P(first = i, second = j) = q_i q_j / (1 - q_i): the law of sequential draws without replacement
+    lq, V, n, tau = [0.5, 1.0, 0.0, 2.0, -1.0], 5, 20000, 0.8
+    cfg = orc.SampleCfg(tau, 17, 3, True)
+    d = _one_level_tree(n, V, 2, lq, cfg)
+    q = np.exp(np.array(lq) / tau)
+    q /= q.sum()
+    pair = np.zeros((V, V))
+    for a, b2 in d.cand_tok[:, 1:].numpy():
+        pair[a, b2] += 1
+    pair /= n
+    for i in range(V):
+        assert pair[i, i] == 0.0
+        for j in range(V):
+            if i != j:
+                want = q[i] * q[j] / (1 - q[i])
+                assert abs(pair[i, j] - want) < 5 * math.sqrt(want * (1 - want) / n), (i, j)
+
+
+def test_tree_walk_with_sampled_children_emits_the_target_distribution():
+    # the defining property of the sequential rule: whatever q is and however many children are tried, the
+    # token emitted at the root (an accepted child or the final draw) follows p; one child = the chain's rule
+    lp = [1.0, -0.5, 2.0, 0.25, 1.5, -2.0]
+    lq = [0.5, 1.0, 0.0, 2.0, -1.0, 0.25]
+    V, n = 6, 12000
+    model = _IdentityModel(V)
+    for tau, k in ((1.0, 1), (1.0, 3), (0.6, 2), (1.3, 5)):
+        cfg = orc.SampleCfg(tau, 1234, 7, True)
+        p = np.exp(np.array(lp) / tau)
+        p /= p.sum()
+        q = np.exp(np.array(lq) / tau)
+        q /= q.sum()
+        d = _one_level_tree(n, V, k, lq, cfg)
+        hid = torch.tensor(lp, dtype=torch.bfloat16).view(1, 1, V).repeat(n, 1 + k, 1)
+        w = orc.tree_speculative_walk(model, hid, d, cfg)
+        f = np.bincount(w.target_tok[:, 0].numpy(), minlength=V) / n
+        assert np.all(np.abs(f - p) < 5 * np.sqrt(p * (1 - p) / n)), (tau, k, f, p)
+        # an accepted child is the root's emitted token and the walk moved there; its own draw follows p again
+        moved = w.accept_len == 1
+        for b in range(0, n, 97):
+            if moved[b]:
+                s = w.path[b][1]
+                assert int(w.target_tok[b, 0]) == int(d.cand_tok[b, s]) and int(w.target_tok[b, s]) == int(w.recover_tok[b])
+            else:
+                assert w.path[b] == [0] and int(w.recover_tok[b]) == int(w.target_tok[b, 0])
+        if k == 1:
+            rate, want = float(moved.float().mean()), float(np.minimum(p, q).sum())
+            assert abs(rate - want) < 5 * math.sqrt(want * (1 - want) / n)
+        leaf = torch.stack([w.target_tok[b, w.path[b][-1]] for b in range(n) if w.accept_len[b] == 1])
+        f2 = np.bincount(leaf.numpy(), minlength=V) / max(1, leaf.numel())
+        assert np.all(np.abs(f2 - p) < 5 * np.sqrt(p * (1 - p) / max(1, leaf.numel())) + 1e-9)
+
+
+def test_tree_walk_accepts_the_first_child_when_draft_and_target_agree_and_can_be_steered():
+    lp = [1.0, -0.5, 2.0, 0.25]
+    V, n, k = 4, 200, 2
+    cfg = orc.SampleCfg(0.7, 3, 1, True)
+    d = _one_level_tree(n, V, k, lp, cfg)
+    hid = torch.tensor(lp, dtype=torch.bfloat16).view(1, 1, V).repeat(n, 1 + k, 1)
+    w = orc.tree_speculative_walk(_IdentityModel(V), hid, d, cfg)
+    assert bool((w.accept_len == 1).all()) and all(pth == [0, 1] for pth in w.path)      # p / q = 1 for every token
+    # the decision hook (used by the GPU comparison at near-ties) replaces single decisions and is recorded
+    w2 = orc.tree_speculative_walk(_IdentityModel(V), hid[:3], d, cfg,
+                                   decide=lambda kind, key, default, margin: (False if (kind == "accept" and key == (1, 1)) else default))
+    assert w2.path[0] == [0, 1] and w2.path[1] == [0, 2] and w2.exempt == ["accept test b=1 slot=1"]
+
+
+def test_sampled_tree_children_run_through_the_draft_model():
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
+    wl = synth.Workload("st", sh, B=2, mode=synth.TREE, K=3, topk=3, max_nodes=3 + 2 * 9, len_lo=9, len_hi=40, seed=5)
+    case = harness.build_case(wl, poison_tail=False)
+    w = dict(case.weights)
+    w["head"] = (w["head"].to(torch.float32) * 20.0).to(torch.bfloat16)
+    case = dataclasses.replace(case, weights=w)
+    model = harness.oracle_model(case)
+    smp = orc.SampleCfg(1.0, 8, 4, True)
+    d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes, sample=smp)
+    g = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, wl.K, wl.topk, wl.max_nodes)
+    assert g.row_logits is None and len(d.row_logits) == wl.B * (1 + wl.topk * (wl.K - 1))
+    assert torch.equal(d.hidden[:, 0], g.hidden[:, 0])               # the root row does not depend on a draw
+    assert not torch.equal(d.cand_tok, g.cand_tok)                   # ... its children do
+    for b in range(wl.B):                                            # siblings are distinct tokens; scores stay log-probabilities
+        for c in d.cands[b]:
+            sib = [x.tok for x in d.cands[b] if x.parent == c.parent and x.src_row == c.src_row]
+            assert len(set(sib)) == len(sib)
+            lg = d.row_logits[(b, c.src_row)]
+            assert abs(c.logp - float(lg[c.tok] - torch.logsumexp(lg, dim=0))) < 1e-5
+    th = harness.tree_target_hidden(case, d)
+    v = orc.tree_speculative_walk(model, th, d, smp)
+    for b in range(wl.B):
+        pth = v.path[b]
+        assert pth[0] == 0 and all(int(d.parent[b, pth[i + 1]]) == pth[i] for i in range(len(pth) - 1))
+        assert int(v.accept_len[b]) == len(pth) - 1 and int(v.recover_tok[b]) == int(v.target_tok[b, pth[-1]])
+
+
 def test_sampled_chain_drafts_and_their_verification_run_end_to_end():
     wl = harness.tiny_workload(B=2, K=3, len_lo=6, len_hi=20)
     case = harness.build_case(wl, poison_tail=False)
