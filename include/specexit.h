@@ -144,7 +144,8 @@ typedef struct {
   int32_t K;           /* chain length, or tree depth */
   int32_t topk;        /* tree: children per expanded node (<= SX_MAX_TOPK); chain: 1 */
   int32_t max_nodes;   /* tree: nodes kept for verification, root excluded (< SX_MAX_VERIFY_SLOTS) */
-  int32_t sample_drafts; /* chain only, 0 or 1: reserve workspace for sampled drafts, see sx_set_sampling */
+  int32_t sample_drafts; /* 0 or 1: reserve workspace for sampled drafts (chain) / sampled children (tree), see
+                            sx_set_sampling; needs the full draft vocabulary without an id map */
 } sx_draft_cfg;
 
 /* Exit rule.  Signal i passes when smoothed_i > thr[i] (SX_DIR_GT) or < thr[i] (SX_DIR_LT),
@@ -294,7 +295,22 @@ sx_status sx_set_attention(sx_ctx *ctx, int32_t kernel);
  * over log max(0, p - q) with the noise of slot j; the last slot, which has no draft, draws from
  * p.  target_tok_d then holds the kept or drawn token of every slot, and acceptance walks it as
  * before.  For this the draft and target logits of the iteration are written to the workspace
- * (fp32, (batch * K + batch * (K + 1)) * vocab values) and three small kernels evaluate the rule.  The standalone sx_draft_step / sx_verify calls keep deterministic drafts. */
+ * (fp32, (batch * K + batch * (K + 1)) * vocab values) and three small kernels evaluate the rule.  The standalone sx_draft_step / sx_verify calls keep deterministic drafts.
+ *
+ * Sampled children.  In a TREE context created with sample_drafts = 1 a positive temperature makes
+ * sx_spec_exit_iter draw the children of every drafted row instead of taking its top-k: the topk largest of
+ * logit_i + temperature * g_i, best first, with the noise stream of slot word 0x50000000 + r for drafted row
+ * r - a draw of topk tokens without replacement, in order, from q = softmax(draft logits / temperature).
+ * Scores (for expansion and for the kept set) stay sums of log-probabilities.  Verification walks from slot 0:
+ * with p the target's softmax at the current slot and q that of the row which produced the slot's children,
+ * the kept children are tried in slot order; token x of child slot s is accepted when u_s < min(1, p(x) /
+ * q(x)) (u_s as above, slot word 0x20000000 + s), a refusal replaces p by the normalised max(0, p - q) and
+ * takes x out of q; when none is accepted the slot's token is drawn from what is left of p (Gumbel-max with
+ * the noise of that slot) and becomes the recover token.  target_tok_d then holds, at every visited slot,
+ * the accepted child's token or that draw, and -1 elsewhere; the iteration's out->slot_row_d must be given.
+ * The token emitted at a slot follows the target's distribution exactly when no child drawn at that slot
+ * was pruned from the tree (max_nodes = all candidates); a pruned child is simply not tried.  The logits of
+ * every drafted row and verify slot are written to the workspace (fp32, batch * (rows + P) * vocab values). */
 sx_status sx_set_sampling(sx_ctx *ctx, float temperature, uint64_t seed, uint32_t offset);
 
 /* Exit decision (Section 3.3; Appendix A.1).  Walks path slots 0..accept_len; each slot that

@@ -141,8 +141,8 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   if (m->arch == SX_ARCH_FUSED3 && (!w->norm_e_d || ((uintptr_t)w->norm_e_d & 15))) return SX_ERR_INVALID_ARG;
   if (dc->K < 1) return SX_ERR_INVALID_ARG;
   if (dc->sample_drafts != 0 && dc->sample_drafts != 1) return SX_ERR_INVALID_ARG;
-  if (dc->sample_drafts && (dc->mode != SX_MODE_CHAIN || Vd != m->vocab || w->draft_to_token_d))
-    return SX_ERR_UNSUPPORTED;        // sampled drafts: chain, full draft vocabulary, no id map
+  if (dc->sample_drafts && (Vd != m->vocab || w->draft_to_token_d))
+    return SX_ERR_UNSUPPORTED;        // sampled drafts: full draft vocabulary, no id map
   sx_ctx *c = new (std::nothrow) sx_ctx();
   if (!c) return SX_ERR_INVALID_ARG;
   memset(c, 0, sizeof(*c));
@@ -229,9 +229,11 @@ extern "C" sx_status sx_create(const sx_model_cfg *m, const sx_weights *w, int32
   c->off_cn = take((size_t)c->commit_rows * s.H * 2);
   c->off_cpart = take((size_t)SX_COMMIT_MAX_SPLITS * c->commit_rows * c->commit_N * 4);
   if (dc->sample_drafts) {
-    c->off_dlogits = take((size_t)max_batch * dc->K * s.V * 4);
+    // logits of every drafted row and of every verify slot (fp32), and the scratch of the accept / residual step
+    c->off_dlogits = take((size_t)max_batch * c->rows_per_seq * s.V * 4);
     c->off_tlogits = take((size_t)max_batch * c->P * s.V * 4);
-    c->off_spec = take(sx_spec_sample_ws_bytes(max_batch * c->P));
+    const size_t a = sx_spec_sample_ws_bytes(max_batch * c->P), b = sx_tree_spec_ws_bytes(max_batch, s.V);
+    c->off_spec = take(dc->mode == SX_MODE_TREE ? b : a);
   }
   if (s.arch == SX_ARCH_FUSED3) {
     c->off_cu2 = take((size_t)c->commit_rows * 2 * s.H * 2);
@@ -316,7 +318,7 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
                       char *ws, int32_t *tok_out, SxIndex toi, float *logp_out, float *sig_out, SxIndex si,
                       int32_t *status, cudaStream_t st, SxNextInput nx = SxNextInput{nullptr, nullptr, nullptr, 0, 0},
                       const int32_t *map = nullptr, const SxSample *smp = nullptr,
-                      SxLogitsOut lo = SxLogitsOut{nullptr, 0}) {
+                      SxLogitsOut lo = SxLogitsOut{nullptr, 0, SxIndex{nullptr, 1, 0}}) {
   const int cap = sx_head_max_rows(T, lse);
   SxHeadPartial *parts = (SxHeadPartial *)(ws + c->off_hparts);
   float *z = (float *)(ws + c->off_z);
@@ -326,9 +328,11 @@ static sx_status head(sx_ctx *c, int cls, const void *W, int Ntot, int V, int S,
     prof_mark(c, cls, true, st);
     SxSample sm2;
     if (smp) { sm2 = *smp; sm2.row0 = r0; }
+    SxLogitsOut lo2 = lo;                           // the chunk's rows go to the rows ri(r0 + r)
+    if (lo2.ri.idx) lo2.ri.idx += r0; else lo2.ri.add += r0 * lo2.ri.mul;
     SX_TRY(sx_launch_head((const bf16 *)W, Ntot, V, c->sh.H, X + (size_t)r0 * c->sh.H, rc, T, lse, parts,
                           c->head_rows, &G, z, S, c->sm_count, status, st, smp ? &sm2 : nullptr,
-                          SxLogitsOut{lo.out ? lo.out + (size_t)r0 * lo.ld : nullptr, lo.ld}, c->tiled));
+                          lo2, c->tiled));
     prof_mark(c, cls, false, st);
     SxIndex t2 = toi, s2 = si;
     if (t2.idx) t2.idx += r0; else t2.add += r0 * t2.mul;
@@ -411,8 +415,15 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
               status, st,
               (prepare_next && !fused3) ? SxNextInput{g, (const bf16 *)c->w.embed_d, u, s.H, s.V}
                            : SxNextInput{nullptr, nullptr, nullptr, 0, 0},
-              c->w.draft_to_token_d, c->round_sampled ? &c->round_smp : nullptr,
-              c->round_sampled ? c->round_lo : SxLogitsOut{nullptr, 0}));
+              c->w.draft_to_token_d, (c->round_sampled && c->dc.mode == SX_MODE_CHAIN) ? &c->round_smp : nullptr,
+              c->round_sampled ? c->round_lo : SxLogitsOut{nullptr, 0, SxIndex{nullptr, 1, 0}}));
+  if (c->round_sampled && c->dc.mode == SX_MODE_TREE) {
+    // sampled children: the head above left the rows' logits in memory; the children are the T best of
+    // logit + temperature * Gumbel noise (a draw without replacement), with their raw log-probabilities
+    SX_TRY(sx_launch_gumbel_topk(R, s.V, T, c->round_lo.out, c->round_lo.ld, c->round_lo.ri, c->round_smp, tok_out,
+                                 logp_out, st));
+    c->launches += 1;
+  }
   return SX_OK;
 }
 
@@ -547,7 +558,7 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
         c->round_smp = c->smp;
         c->round_smp.P = 1;
         c->round_smp.slot_base = 0x40000000u + (uint32_t)(k - 1);
-        c->round_lo = SxLogitsOut{dlogits + (size_t)(k - 1) * V, (size_t)K * V};
+        c->round_lo = SxLogitsOut{dlogits + (size_t)(k - 1) * V, (size_t)K * V, SxIndex{nullptr, 1, 0}};
       }
       const sx_status rc = draft_round(c, kv, k, B, feat, fi, o->cand_tok_d, SxIndex{nullptr, P, k - 1}, nullptr, hid,
                                        SxIndex{nullptr, K, k - 1}, o->cand_tok_d, SxIndex{nullptr, P, k}, nullptr,
@@ -561,7 +572,7 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
       float *tlogits = (float *)(ws + c->off_tlogits);
       SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, V, V, 0, (const bf16 *)target_hidden_d, B * P, 1, 0, ws,
                   o->target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
-                  SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr, SxLogitsOut{tlogits, (size_t)V}));
+                  SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr, SxLogitsOut{tlogits, (size_t)V, SxIndex{nullptr, 1, 0}}));
       SX_TRY(sx_launch_spec_sample(B, P, V, tlogits, dlogits, o->cand_tok_d, c->smp, ws + c->off_spec, c->sm_count,
                             o->target_tok_d, status_d, st));
       SX_TRY(sx_launch_accept(B, P, o->cand_tok_d, nullptr, o->target_tok_d, o->accept_len_d, o->path_d, K + 1,
@@ -580,22 +591,62 @@ extern "C" sx_status sx_spec_exit_iter(sx_ctx *c, const sx_kv *kv, const sx_exit
     const int T = t.T, rows = t.rows;
     int32_t *tok_rt = (int32_t *)(ws + c->off_tok_rt);
     float *logp_rt = (float *)(ws + c->off_logp_rt);
-    SX_TRY(draft_round(c, kv, 1, B, (const bf16 *)feat0_d, SxIndex{nullptr, 1, 0}, tok0_d, SxIndex{nullptr, 1, 0},
-                       nullptr, hid, SxIndex{nullptr, rows, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt, t.row_sig,
-                       SxIndex{nullptr, rows, 0}, ws, status_d, st));
+    // sampled children: every draft head leaves its rows' logits (row b * rows + drafted row) and the children
+    // are drawn from them; the noise of the children of drafted row r is the stream 0x50000000 + r
+    const bool sampled = c->dc.sample_drafts && c->smp.temp > 0.f;
+    float *dlogits = sampled ? (float *)(ws + c->off_dlogits) : nullptr;
+    const int V = c->sh.V;
+    auto round_sampling = [&](int r) {
+      if (!sampled) return;
+      c->round_sampled = true;
+      c->round_smp = c->smp;
+      c->round_smp.row0 = 0;
+      c->round_smp.P = (r == 1) ? 1 : T;
+      c->round_smp.slot_base = 0x50000000u + (uint32_t)(r == 1 ? 0 : 1 + (r - 2) * T);
+      SxLogitsOut lo;
+      lo.out = dlogits;
+      lo.ld = (size_t)V;
+      lo.ri.idx = (r == 1) ? nullptr : t.hid_idx;
+      lo.ri.mul = (r == 1) ? rows : 0;
+      lo.ri.add = 0;
+      c->round_lo = lo;
+    };
+    round_sampling(1);
+    sx_status rc1 = draft_round(c, kv, 1, B, (const bf16 *)feat0_d, SxIndex{nullptr, 1, 0}, tok0_d, SxIndex{nullptr, 1, 0},
+                                nullptr, hid, SxIndex{nullptr, rows, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt, t.row_sig,
+                                SxIndex{nullptr, rows, 0}, ws, status_d, st);
+    c->round_sampled = false;
+    SX_TRY(rc1);
     SX_TRY(sx_launch_tree_expand(t, B, 1, tok_rt, logp_rt, st));
     c->launches += 1;
     for (int r = 2; r <= K; ++r) {
-      SX_TRY(draft_round(c, kv, r, B * T, hid, SxIndex{t.feat_idx, 0, 0}, t.sel_tok, SxIndex{nullptr, 1, 0},
-                         t.next_mask, hid, SxIndex{t.hid_idx, 0, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt,
-                         t.row_sig, SxIndex{t.hid_idx, 0, 0}, ws, status_d, st));
+      round_sampling(r);
+      const sx_status rcr = draft_round(c, kv, r, B * T, hid, SxIndex{t.feat_idx, 0, 0}, t.sel_tok, SxIndex{nullptr, 1, 0},
+                                        t.next_mask, hid, SxIndex{t.hid_idx, 0, 0}, tok_rt, SxIndex{nullptr, T, 0}, logp_rt,
+                                        t.row_sig, SxIndex{t.hid_idx, 0, 0}, ws, status_d, st);
+      c->round_sampled = false;
+      SX_TRY(rcr);
       SX_TRY(sx_launch_tree_expand(t, B, r, tok_rt, logp_rt, st));
       c->launches += 1;
     }
     SX_TRY(sx_launch_tree_layout(t, B, S, tok0_d, *o, st));
     c->launches += 1;
-    SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, o->parent_d, o->target_tok_d, o->accept_len_d,
-                     o->path_d, K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+    if (sampled) {
+      // target logits of every slot, then the walk with the accept tests and residual draws
+      if (!o->slot_row_d) return SX_ERR_INVALID_ARG;
+      float *tlogits = (float *)(ws + c->off_tlogits);
+      SX_TRY(head(c, SX_PROF_HEAD_VERIFY, c->w.target_head_d, V, V, 0, (const bf16 *)target_hidden_d, B * P, 1, 0, ws,
+                  o->target_tok_d, SxIndex{nullptr, 1, 0}, nullptr, nullptr, SxIndex{nullptr, 1, 0}, status_d, st,
+                  SxNextInput{nullptr, nullptr, nullptr, 0, 0}, nullptr, nullptr,
+                  SxLogitsOut{tlogits, (size_t)V, SxIndex{nullptr, 1, 0}}));
+      SX_TRY(sx_launch_tree_spec_walk(B, P, V, rows, K + 1, tlogits, dlogits, o->cand_tok_d, o->parent_d, o->slot_row_d,
+                                      c->smp, ws + c->off_spec, o->target_tok_d, o->accept_len_d, o->path_d,
+                                      o->recover_tok_d, status_d, st));
+      c->launches += 1;
+    } else {
+      SX_TRY(sx_verify(c, B, P, target_hidden_d, o->cand_tok_d, o->parent_d, o->target_tok_d, o->accept_len_d,
+                       o->path_d, K + 1, o->recover_tok_d, ws_d, ws_bytes, status_d, stream));
+    }
   }
   return sx_exit_update(c, B, P, cfg, state, o->slot_signal_d, o->cand_tok_d, o->path_d, K + 1, o->accept_len_d,
                         o->recover_tok_d, o->exit_flag_d, o->accept_len_out_d, o->recover_tok_out_d, o->smoothed_d,

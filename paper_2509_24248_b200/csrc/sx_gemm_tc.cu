@@ -47,6 +47,8 @@ struct SxTcParams {
   uint32_t wait_limit;           // polls of an mbarrier before a wait gives up
 };
 
+__device__ __forceinline__ int sx_lo_row(const SxLogitsOut &lo, int r) { return lo.ri.idx ? lo.ri.idx[r] : r * lo.ri.mul + lo.ri.add; }
+
 template <bool HEAD>
 __global__ void __launch_bounds__(192, 1)
 sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, SxTcParams p) {
@@ -204,7 +206,7 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
             if (p.lo.out && in_vocab) {                           // lanes hold consecutive vocabulary rows
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (ch * 32 + j < p.R) p.lo.out[(size_t)(ch * 32 + j) * p.lo.ld + n] = v[j];
+                if (ch * 32 + j < p.R) p.lo.out[(size_t)sx_lo_row(p.lo, ch * 32 + j) * p.lo.ld + n] = v[j];
             }
             epi_bar();
             if (ch * 32 + col < p.R) {
@@ -311,6 +313,11 @@ sx_tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
                   if (ch * 32 + j < p.R) p.z[(size_t)(ch * 32 + j) * p.S + (n - p.V)] = v[j];
+              }
+              if (p.lo.out && in_vocab) {                         // lanes hold consecutive vocabulary rows
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (ch * 32 + j < p.R) p.lo.out[(size_t)sx_lo_row(p.lo, ch * 32 + j) * p.lo.ld + n] = v[j];
               }
             }
             epi_bar();
@@ -617,7 +624,7 @@ sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, i
                          cudaStream_t st, const SxSample *smp, SxLogitsOut lo, bool tiled) {
   if ((K % 8) != 0 || R < 1 || R > sx_head_max_rows(T, lse)) return SX_ERR_UNSUPPORTED;
   if (smp && smp->temp > 0.f && (T != 1 || lse || smp->P < 1)) return SX_ERR_UNSUPPORTED;
-  if (lo.out && (T != 1 || lse)) return SX_ERR_UNSUPPORTED;
+  if (lo.out && smp && smp->temp > 0.f && lse) return SX_ERR_UNSUPPORTED;
   SxTcParams p;
   memset(&p, 0, sizeof(p));
   const size_t epi = (T == 1 && !lse) ? SX_ARGMAX_SMEM : SX_TOPK_SMEM;

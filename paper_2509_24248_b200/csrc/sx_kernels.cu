@@ -1008,3 +1008,250 @@ sx_status sx_launch_spec_sample(int B, int P, int V, const float *target_logits,
                          cand_tok, smp, parts, status)));
   return sx_rc(sx_launch(sx_spec_pick_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, P, V, S, rows, cand_tok, parts, target_tok));
 }
+
+// ---------------------------------------------------------------------------------------
+// Sampled children in a draft tree
+// ---------------------------------------------------------------------------------------
+// The children of a drafted row are the T largest of logit + temp * Gumbel noise, best first: a draw of T
+// tokens without replacement, in order, from softmax(logits / temp).  One CTA per drafted row reads the
+// row's logits (left in memory by the head launch); a thread keeps the T best perturbed scores of its share
+// in registers together with a running (max, sum) of the raw logits, the lists are merged by a tournament
+// over their heads.  Reported log-probabilities are those of the raw logits.
+__global__ void __launch_bounds__(256)
+sx_gumbel_topk_kernel(int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp, int32_t *tok_out,
+                      float *logp_out) {
+  __shared__ unsigned long long s_best[2][8];
+  __shared__ float s_m[8], s_l[8];
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float *lg = logits + (size_t)sx_index(li, r) * ld;
+  const int row = smp.row0 + r;
+  const uint32_t sb = (uint32_t)(row / smp.P), sj = (uint32_t)(row % smp.P) + smp.slot_base;
+  unsigned long long v[SX_MAX_TOPK];
+#pragma unroll
+  for (int k = 0; k < SX_MAX_TOPK; ++k) v[k] = 0ull;
+  float m = -INFINITY, l = 0.f;
+  for (int a = tid * 4; a < V; a += 256 * 4) {
+    uint32_t w[4];
+    sx_philox4x32_10((uint32_t)(a >> 2), sj, sb, smp.offset, smp.k0, smp.k1, w);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = a + e;
+      if (i < V) {
+        const float x = lg[i];
+        const float mn = fmaxf(m, x);
+        l = l * expf(m - mn) + expf(x - mn);          // m = -inf at first: exp(-inf) = 0
+        m = mn;
+        const unsigned long long key = sx_pack(fmaf(smp.temp, sx_gumbel(w[e]), x), (uint32_t)i);
+        if (key > v[SX_MAX_TOPK - 1]) {
+          bool gt[SX_MAX_TOPK];
+#pragma unroll
+          for (int k = 0; k < SX_MAX_TOPK; ++k) gt[k] = v[k] > key;
+#pragma unroll
+          for (int k = SX_MAX_TOPK - 1; k >= 1; --k) v[k] = gt[k] ? v[k] : (gt[k - 1] ? key : v[k - 1]);
+          if (!gt[0]) v[0] = key;
+        }
+      }
+    }
+  }
+  // log-sum-exp of the raw logits over the block
+  float mm = sx_warp_max(m);
+  if (lane == 0) s_m[warp] = mm;
+  __syncthreads();
+  mm = s_m[0];
+  for (int w2 = 1; w2 < 8; ++w2) mm = fmaxf(mm, s_m[w2]);
+  float ll = sx_warp_sum(l > 0.f ? l * expf(m - mm) : 0.f);
+  if (lane == 0) s_l[warp] = ll;
+  __syncthreads();
+  float lsum = 0.f;
+  for (int w2 = 0; w2 < 8; ++w2) lsum += s_l[w2];
+  const float lse = mm + logf(lsum);
+  // tournament over the heads of the 256 sorted lists
+  for (int t = 0; t < T; ++t) {
+    unsigned long long best = v[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if (lane == 0) s_best[t & 1][warp] = best;
+    __syncthreads();
+    best = s_best[t & 1][0];
+    for (int w2 = 1; w2 < 8; ++w2) best = max(best, s_best[t & 1][w2]);
+    if (tid == 0) {
+      const int32_t id = (int32_t)sx_pack_index(best);
+      tok_out[(size_t)r * T + t] = (best != 0ull && id >= 0 && id < V) ? id : 0;
+      logp_out[(size_t)r * T + t] = (best != 0ull && id >= 0 && id < V) ? lg[id] - lse : -INFINITY;
+    }
+    if (best != 0ull && v[0] == best) {            // packed keys are unique (index inside): one winner
+#pragma unroll
+      for (int k = 0; k + 1 < SX_MAX_TOPK; ++k) v[k] = v[k + 1];
+      v[SX_MAX_TOPK - 1] = 0ull;
+    }
+  }
+}
+
+sx_status sx_launch_gumbel_topk(int R, int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp,
+                                int32_t *tok_out, float *logp_out, cudaStream_t st) {
+  return sx_rc(sx_launch(sx_gumbel_topk_kernel, dim3(R), dim3(256), 0, st, V, T, logits, ld, li, smp, tok_out, logp_out));
+}
+
+// Speculative sampling down a tree with sampled children.  One CTA per sequence walks from the root: at
+// the current slot p = softmax(target logits / temp) and q = softmax(logits of the drafted row that produced
+// the slot's children / temp) are held as unnormalised fp32 vectors with float64 sums; a kept child with
+// token x is accepted when u < min(1, p(x) / q(x)), a refusal replaces p by max(0, p - q) (renormalised
+// through its sum) and removes x from q; when nothing is accepted the slot's token is a Gumbel-max draw over
+// what is left of p.  pq holds 2 V floats per sequence.
+__device__ __forceinline__ double sx_block_sum_d(double v, double *red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];       // same order in every thread
+  return t;
+}
+
+__global__ void __launch_bounds__(1024)
+sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *target_logits, const float *draft_logits,
+                         const int32_t *cand_tok, const int32_t *parent, const int32_t *slot_row, SxSample smp,
+                         float *pq, int32_t *target_tok, int32_t *accept_len, int32_t *path, int32_t *recover,
+                         int32_t *status) {
+  __shared__ double red[32];
+  __shared__ double s_best[32];
+  __shared__ int s_besti[32];
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const float inv_tau = 1.0f / smp.temp;
+  float *Pv = pq + (size_t)b * 2 * V, *Qv = Pv + V;
+  const int32_t *ct = cand_tok + (size_t)b * P, *par = parent + (size_t)b * P, *srow = slot_row + (size_t)b * P;
+  int32_t *tt = target_tok + (size_t)b * P, *pa = path + (size_t)b * path_stride;
+  for (int s = tid; s < P; s += blockDim.x) tt[s] = -1;
+  if (tid == 0) pa[0] = 0;
+  int cur = 0, L = 0;
+  for (;;) {
+    const float *lp = target_logits + ((size_t)b * P + cur) * V;
+    const int row = srow[cur];
+    int nkids = 0;
+    for (int s = cur + 1; s < P; ++s) nkids += (par[s] == cur) ? 1 : 0;      // the same count in every thread
+    const bool has_q = nkids > 0 && row >= 0 && row < rows;
+    const float *lq = has_q ? draft_logits + ((size_t)b * rows + row) * V : nullptr;
+    // maxima, then the unnormalised vectors and their sums
+    float mp = -INFINITY, mq = -INFINITY;
+    for (int i = tid; i < V; i += blockDim.x) {
+      mp = fmaxf(mp, lp[i]);
+      if (lq) mq = fmaxf(mq, lq[i]);
+    }
+    mp = sx_block_max(mp, red);
+    mq = sx_block_max(mq, red);
+    double sp = 0.0, sq = 0.0;
+    for (int i = tid; i < V; i += blockDim.x) {
+      const float a = expf((lp[i] - mp) * inv_tau);
+      Pv[i] = a;
+      sp += (double)a;
+      if (lq) {
+        const float c = expf((lq[i] - mq) * inv_tau);
+        Qv[i] = c;
+        sq += (double)c;
+      }
+    }
+    sp = sx_block_sum_d(sp, red);
+    sq = sx_block_sum_d(sq, red);
+    int nxt = -1;
+    if (has_q) {
+      for (int s = cur + 1; s < P && nxt < 0; ++s) {
+        if (par[s] != cur) continue;
+        int x = ct[s];
+        if (x < 0 || x >= V) {
+          if (tid == 0) sx_set_status(status, SX_ERR_CAPACITY);
+          x = 0;
+        }
+        __syncthreads();                                                  // Pv / Qv of the last update are in place
+        const double px = (double)Pv[x] / sp, qx = (double)Qv[x] / sq;
+        const double ratio = qx > 0.0 ? fmin(1.0, px / qx) : 1.0;
+        uint32_t w[4];
+        sx_philox4x32_10(0u, 0x20000000u + (uint32_t)s, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+        const double u = ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
+        if (u < ratio) {                                                  // every thread takes the same decision
+          nxt = s;
+          break;
+        }
+        // refused: p <- max(0, p - q) with its new sum; x leaves q
+        const float fsp = (float)(1.0 / sp), fsq = (float)(1.0 / sq);
+        const double qx_un = (double)Qv[x];
+        __syncthreads();
+        double nsp = 0.0;
+        for (int i = tid; i < V; i += blockDim.x) {
+          const float rr = fmaxf(0.f, Pv[i] * fsp - Qv[i] * fsq);
+          Pv[i] = rr;
+          nsp += (double)rr;
+        }
+        if (tid == 0) Qv[x] = 0.f;
+        sp = sx_block_sum_d(nsp, red);
+        sq -= qx_un;
+      }
+    }
+    if (nxt >= 0) {
+      if (tid == 0) {
+        tt[cur] = ct[nxt];
+        if (L + 1 < path_stride) pa[L + 1] = nxt;
+      }
+      cur = nxt;
+      ++L;
+      __syncthreads();
+      continue;
+    }
+    // the slot's own draw: Gumbel-max over log(what is left of p), lower index among equals
+    __syncthreads();
+    double best = -INFINITY;
+    int besti = -1;
+    for (int a = tid * 4; a < V; a += blockDim.x * 4) {
+      uint32_t w[4];
+      sx_philox4x32_10((uint32_t)(a >> 2), (uint32_t)cur, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int i = a + e;
+        if (i < V && Pv[i] > 0.f) {
+          const float uu = (float)((w[e] >> 9) * 2u + 1u) * 5.9604644775390625e-8f;
+          const double sc = (double)(logf(Pv[i]) - logf(-logf(uu)));
+          if (sc > best) { best = sc; besti = i; }
+        }
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+      if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+    }
+    if ((tid & 31) == 0) { s_best[tid >> 5] = best; s_besti[tid >> 5] = besti; }
+    __syncthreads();
+    if (tid == 0) {
+      best = -INFINITY;
+      besti = -1;
+      for (int w2 = 0; w2 < (int)(blockDim.x >> 5); ++w2) {
+        const double ob = s_best[w2];
+        const int oi = s_besti[w2];
+        if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+      }
+      if (besti < 0) besti = 0;
+      tt[cur] = besti;
+      recover[b] = besti;
+      accept_len[b] = L;
+      for (int j = L + 1; j < path_stride; ++j) pa[j] = -1;
+    }
+    break;
+  }
+}
+
+size_t sx_tree_spec_ws_bytes(int B, int V) { return (size_t)B * 2 * V * sizeof(float); }
+
+sx_status sx_launch_tree_spec_walk(int B, int P, int V, int rows, int path_stride, const float *target_logits,
+                                   const float *draft_logits, const int32_t *cand_tok, const int32_t *parent,
+                                   const int32_t *slot_row, SxSample smp, void *pq_ws, int32_t *target_tok,
+                                   int32_t *accept_len, int32_t *path, int32_t *recover, int32_t *status,
+                                   cudaStream_t st) {
+  return sx_rc(sx_launch(sx_tree_spec_walk_kernel, dim3(B), dim3(1024), 0, st, P, V, rows, path_stride, target_logits,
+                         draft_logits, cand_tok, parent, slot_row, smp, (float *)pq_ws, target_tok, accept_len, path,
+                         recover, status));
+}

@@ -136,16 +136,17 @@ struct SxSample {
   int P, row0;
   uint32_t slot_base;            // added to the slot word (separates the draft stream from the verify stream)
 };
-// Optional copy of the head's logits: row r of the launch goes to out[r * ld + 0 .. V) (fp32).
+// Optional copy of the head's logits: row r of the launch goes to out[ri(r) * ld + 0 .. V) (fp32).
 struct SxLogitsOut {
   float *out;
   size_t ld;
+  SxIndex ri;
 };
 // head: per-CTA partial results out[cta][row]; returns the number of CTAs used in *G
 sx_status sx_launch_head(const bf16 *W, int Ntot, int V, int K, const bf16 *X, int R, int T, int lse,
                          SxHeadPartial *parts, int part_stride, int *G, float *z, int S, int sm_count,
                          int32_t *status, cudaStream_t st, const SxSample *smp = nullptr,
-                         SxLogitsOut lo = SxLogitsOut{nullptr, 0}, bool tiled = false);
+                         SxLogitsOut lo = SxLogitsOut{nullptr, 0, SxIndex{nullptr, 1, 0}}, bool tiled = false);
 
 // Speculative sampling with sampled drafts: writes the kept draft token or the residual draw of every
 // verify slot to target_tok [B, P].  target_logits [B * P, V], draft_logits [B, K, V] (K = P - 1), both
@@ -157,3 +158,14 @@ sx_status sx_launch_spec_sample(int B, int P, int V, const float *target_logits,
                            const int32_t *cand_tok, SxSample smp, void *parts_ws, int sm_count, int32_t *target_tok,
                            int32_t *status, cudaStream_t st);
 int sx_head_max_rows(int T, int lse);
+
+// Sampled children in a tree: the T best of logit + temp * Gumbel noise per drafted row (rows of `logits` are
+// addressed through li), and the speculative walk over the laid-out tree (pq_ws: sx_tree_spec_ws_bytes).
+sx_status sx_launch_gumbel_topk(int R, int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp,
+                                int32_t *tok_out, float *logp_out, cudaStream_t st);
+size_t sx_tree_spec_ws_bytes(int B, int V);
+sx_status sx_launch_tree_spec_walk(int B, int P, int V, int rows, int path_stride, const float *target_logits,
+                                   const float *draft_logits, const int32_t *cand_tok, const int32_t *parent,
+                                   const int32_t *slot_row, SxSample smp, void *pq_ws, int32_t *target_tok,
+                                   int32_t *accept_len, int32_t *path, int32_t *recover, int32_t *status,
+                                   cudaStream_t st);

@@ -201,14 +201,39 @@ def _set_sampling(sx: binding.SpecExit, sample) -> None:
         sx.sx_set_sampling(sample.temperature, sample.seed, sample.offset)
 
 
+def _tree_walk(rep: Report, model, th, d, sample, out: Dict[str, torch.Tensor]):
+    """Sampled children: the oracle's speculative walk, adopting the GPU's decision where the accept test is
+    within 1e-4 of its threshold or the two best scores of a draw within 1e-3 (recorded as exempt)."""
+    g_path = [[int(x) for x in row if int(x) >= 0] for row in out["path_d"].cpu()]
+    g_tt = out["target_tok_d"].cpu().to(torch.int64)
+
+    def decide(kind, key, default, margin):
+        b, s = key
+        got = (s in g_path[b]) if kind == "accept" else int(g_tt[b, s])
+        if got == default:
+            return default
+        if margin < (1e-4 if kind == "accept" else 1e-3):
+            return got
+        raise ParityError(f"tree walk {kind} b={b} slot={s}: gpu {got} vs {default} (margin {margin:.3e})")
+
+    w = orc.tree_speculative_walk(model, th, d, sample, decide=decide)
+    rep.exempt += w.exempt
+    if not torch.equal(g_tt, w.target_tok):
+        raise ParityError("tree walk: tokens of the visited slots differ")
+    return w
+
+
 def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, parent, slot_signal,
                   out: Dict[str, torch.Tensor], gstate: Dict[str, torch.Tensor], K: int, sample=None,
-                  draft_logits=None):
-    """verify + exit comparison, shared by chain and tree."""
+                  draft_logits=None, walk=None):
+    """verify + exit comparison, shared by chain and tree.  ``walk``: the verification result when it was not
+    a per-slot target token followed by the greedy walk (sampled children in a tree)."""
     B, P = cand_tok.shape
     sampling = sample is not None and sample.temperature > 0.0
     full_rule = sampling and sample.sample_drafts
-    if full_rule:
+    if walk is not None:
+        tt, gap = walk.target_tok, torch.ones(B, P, dtype=torch.float64)
+    elif full_rule:
         so = orc.speculative_sample(model, th, cand_tok, draft_logits, sample)
         tt = so.target_tok
         # a slot may fall the other way when the accept test is within 1e-4 of its threshold, or
@@ -227,7 +252,8 @@ def _compare_tail(rep: Report, model, cfg, state0: orc.ExitState, th, cand_tok, 
                 else:
                     raise ParityError(f"target token b={b} slot={j}: gpu {int(g_tt[b, j])} vs {int(tt[b, j])} "
                                       f"gap {float(gap[b, j]):.3e}")
-    v = orc.verify(model, th, cand_tok, parent, forced_target=forced, sample=sample, draft_logits=draft_logits)
+    v = walk if walk is not None else orc.verify(model, th, cand_tok, parent, forced_target=forced, sample=sample,
+                                                 draft_logits=draft_logits)
     g_L = out["accept_len_d"].cpu().to(torch.int64)
     g_path = out["path_d"].cpu().to(torch.int64)
     g_rec = out["recover_tok_d"].cpu().to(torch.int64)
@@ -465,10 +491,12 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
     cfg = cfg or harness.default_exit_cfg(wl)
     model = harness.oracle_model(case, act=act)
     T, D = wl.topk, wl.K
-    d0 = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes)
+    sampled_children = sample is not None and sample.sample_drafts and sample.temperature > 0.0
+    dsample = sample if sampled_children else None
+    d0 = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes, sample=dsample)
     th = harness.tree_target_hidden(case, d0)
     own = sx is None
-    sx = sx or make_gpu(case, act)
+    sx = sx or make_gpu(case, act, sample_drafts=sampled_children)
     out = sx.new_outputs(wl.B)
     gst = sx.new_state(wl.B)
     state0 = orc.ExitState.fresh(wl.B, wl.shape.S)
@@ -515,7 +543,7 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
         return torch.stack([g_hid[r.b, r.slot - lens[r.b]].to(torch.float64) for r in rows])
 
     d = orc.draft_tree(model, harness.oracle_kv(case), case.f0, case.t0, D, T, wl.max_nodes, chooser=chooser,
-                       before_round=before_round, head_input=head_input)
+                       before_round=before_round, head_input=head_input, sample=dsample)
     for b in range(wl.B):
         for c in d.cands[b]:
             if int(o["tree_cand_tok_d"][b, c.cid]) != c.tok or int(o["tree_cand_row_d"][b, c.cid]) != c.row:
@@ -531,8 +559,9 @@ def run_tree(case: harness.Case, cfg: orc.ExitCfg = None, act=(0, 0, 0), sx: bin
     _compare_signals(rep, o["slot_signal_d"], d.slot_signal)
     if sample is None:
         _free_tail(rep, model, cfg, state0, th, d0, d0.parent, out, wl.K, strict_free)
+    walk = _tree_walk(rep, model, th, d, sample, out) if sampled_children else None
     _compare_tail(rep, model, cfg, state0, th, d.cand_tok, d.parent, d.slot_signal, out,
-                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample)
+                  {k: v.cpu() for k, v in gst.items()}, wl.K, sample=sample, walk=walk)
     if own:
         sx.close()
     return rep

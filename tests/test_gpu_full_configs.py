@@ -86,3 +86,17 @@ def test_chain_config1_with_stochastic_acceptance(sample_drafts):
                            sample=orc.SampleCfg(1.0, 20250924, 3, sample_drafts))
     print(f"C1/tau=1/sampled drafts {sample_drafts}: accept_len {rep.accept_len} exempt {rep.exempt}")
     assert len(rep.exempt) <= 2
+
+
+def test_tree_config4_with_sampled_children():
+    """C4's shapes with the children of every drafted row drawn without replacement at temperature 1 and the
+    sequential accept / residual walk over the 151936-token vocabulary."""
+    from oracle import specexit_oracle as orc
+    wl = synth.workload("C4")
+    parity.TILED = True
+    try:
+        rep = parity.run_tree(harness.build_case(wl, poison_tail=True), sample=orc.SampleCfg(1.0, 20250924, 5, True))
+    finally:
+        parity.TILED = False
+    print(f"C4/tau=1/sampled children: accept_len {rep.accept_len} exempt {rep.exempt}")
+    assert len(rep.exempt) <= 2

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from oracle import specexit_oracle as orc
-from paper_2509_24248_b200 import synth
+from paper_2509_24248_b200 import binding, synth
 from tests import harness, parity
 
 pytestmark = pytest.mark.gpu
@@ -131,13 +131,44 @@ def test_sampled_drafts_on_an_odd_vocabulary_and_the_three_feature_layer():
     parity.run_chain(case, sample=orc.SampleCfg(0.8, 5, 3, True))
 
 
-def test_sampled_drafts_need_chain_mode_and_a_full_draft_vocabulary():
-    from paper_2509_24248_b200 import binding
-    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
-    wl = synth.Workload("sdt", sh, B=1, mode=synth.TREE, K=3, topk=2, max_nodes=5, len_lo=9, len_hi=9, seed=72)
-    with pytest.raises(binding.SxError):
-        parity.make_gpu(harness.build_case(wl), sample_drafts=True)
+def test_sampled_drafts_need_a_full_draft_vocabulary():
     sh2 = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16, Vd=100)
     wl2 = synth.Workload("sdv", sh2, B=1, mode=synth.CHAIN, K=3, len_lo=9, len_hi=9, seed=73)
     with pytest.raises(binding.SxError):
         parity.make_gpu(harness.build_case(wl2), sample_drafts=True)
+
+
+@pytest.mark.parametrize("topk,depth,nodes,tau", [(2, 3, 2 + 2 * 4, 1.0), (3, 3, 3 + 2 * 9, 0.7), (4, 3, 20, 1.5), (8, 2, 30, 1.0)])
+def test_tree_with_sampled_children(topk, depth, nodes, tau):
+    """Children drawn without replacement (the Gumbel-top-k of every drafted row) and the sequential accept /
+    residual walk over the laid-out tree: candidates, layout, the tokens of the visited slots, accepted
+    length, path, recover token and the exit decision against the oracle; the first two trees are unpruned."""
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
+    wl = synth.Workload("stc", sh, B=3, mode=synth.TREE, K=depth, topk=topk, max_nodes=nodes, len_lo=9, len_hi=60,
+                        seed=70 + topk, sigma_lo=0.0, sigma_hi=0.05)
+    case = harness.build_case(wl)
+    w = dict(case.weights)
+    w["head"] = (w["head"].to(torch.float32) * 20.0).to(torch.bfloat16)       # a peaked head: some children get accepted
+    case = dataclasses.replace(case, weights=w)
+    accepted = 0
+    for offset in (1, 2, 3):
+        rep = parity.run_tree(case, sample=orc.SampleCfg(tau, 4242, offset, True))
+        accepted += sum(rep.accept_len)
+        print("sampled children tau", tau, "offset", offset, "accept:", rep.accept_len, "exempt:", rep.exempt)
+        assert len(rep.exempt) <= 2
+    assert accepted > 0
+
+
+def test_sampled_children_need_the_full_vocabulary_and_a_positive_temperature_to_act():
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
+    wl = synth.Workload("stx", sh, B=2, mode=synth.TREE, K=3, topk=3, max_nodes=12, len_lo=9, len_hi=40, seed=75)
+    case = harness.build_case(wl)
+    # temperature 0 in a context created for sampled children: the deterministic tree and the greedy walk
+    sx = parity.make_gpu(case, sample_drafts=True)
+    parity.run_tree(case, sx=sx)
+    sx.close()
+    # a reduced draft vocabulary cannot be combined with sampled drafts
+    wl2 = dataclasses.replace(wl, shape=dataclasses.replace(sh, Vd=100))
+    case2 = harness.build_case(wl2)
+    with pytest.raises(binding.SxError, match="not supported"):
+        parity.make_gpu(case2, sample_drafts=True)
