@@ -425,6 +425,31 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
                   "commit_alone_ms": cms, "commit_weight_bytes": cbytes,
                   "commit_gbs": cbytes / (cms * 1e-3) / 1e9, "launches_per_loop_step": (la1 - la0) / n_loop}
 
+    # the same iteration captured once into a CUDA graph and replayed (what a serving loop would do: the
+    # library only enqueues kernels, so the capture needs nothing special); reported beside `value`
+    graph_rec = None
+    if args.temperature <= 0.0:
+        n_graph = max(3, min(steps, 300))
+        reset_state()
+        torch.cuda.synchronize()
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg):
+            reset_state()
+            sx.sx_spec_exit_iter(params, state, f0_d, t0_d, th_d, out)
+        for _ in range(3):
+            cg.replay()
+        torch.cuda.synchronize()
+        sx.check_status("graph warm-up")
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(n_graph):
+            cg.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        sx.check_status("graph replay")
+        graph_rec = {"ms_per_step": max_over_ranks(g0.elapsed_time(g1) / n_graph, dist, dev), "steps": n_graph}
+        del cg
+
     if timeline and rank == 0:
         write_timeline(timeline, step, wl.name)
 
@@ -489,6 +514,7 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
                      "frac_of_nominal": achieved / NOMINAL_HBM_GBS if achieved else None},
         "kernel_ms_per_step": {k: (v["ms"] / prof_steps) for k, v in prof.items()},
         "commit": commit,
+        "graph_replay": graph_rec,
         "clocks": clocks,
         "e2e": {"value": world * 1e3 / e2e_ms, "unit": "iterations/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},

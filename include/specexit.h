@@ -33,6 +33,10 @@
  *   - Matrices are bf16, row-major [out, in].  Activations handed between layers are
  *     bf16; accumulation, normalisation, softmax, rotary and signal math are fp32.
  *   - One sx_ctx per stream: a context is not thread-safe.
+ *   - The device entry points (all but sx_spec_exit_iter_host and the profiling calls) only enqueue
+ *     kernels, so a call - a whole sx_spec_exit_iter included - may be captured into a CUDA graph and
+ *     replayed; the replay reads the captured buffers, whatever they hold then.  sx_set_sampling takes
+ *     effect at enqueue time: a captured call keeps the temperature, seed and offset it was captured with.
  *   - With the environment variable SX_NVTX=1 the entry points open NVTX ranges ("sx spec exit iteration",
  *     "sx draft round k", "sx verify", "sx exit update", "sx commit") for timeline tools.
  */
