@@ -420,9 +420,10 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   if (c->round_sampled && c->dc.mode == SX_MODE_TREE) {
     // sampled children: the head above left the rows' logits in memory; the children are the T best of
     // logit + temperature * Gumbel noise (a draw without replacement), with their raw log-probabilities
-    SX_TRY(sx_launch_gumbel_topk(R, s.V, T, c->round_lo.out, c->round_lo.ld, c->round_lo.ri, c->round_smp, tok_out,
-                                 logp_out, st));
-    c->launches += 1;
+    SX_TRY(sx_launch_gumbel_topk(R, s.V, T, c->round_lo.out, c->round_lo.ld, c->round_lo.ri, c->round_smp,
+                                 (SxHeadPartial *)(ws + c->off_hparts), (size_t)c->head_G * c->head_rows, c->sm_count,
+                                 tok_out, logp_out, st));
+    c->launches += 2;
   }
   return SX_OK;
 }

@@ -1013,32 +1013,35 @@ sx_status sx_launch_spec_sample(int B, int P, int V, const float *target_logits,
 // Sampled children in a draft tree
 // ---------------------------------------------------------------------------------------
 // The children of a drafted row are the T largest of logit + temp * Gumbel noise, best first: a draw of T
-// tokens without replacement, in order, from softmax(logits / temp).  One CTA per drafted row reads the
-// row's logits (left in memory by the head launch); a thread keeps the T best perturbed scores of its share
-// in registers together with a running (max, sum) of the raw logits, the lists are merged by a tournament
-// over their heads.  Reported log-probabilities are those of the raw logits.
+// tokens without replacement, in order, from softmax(logits / temp).  The row's logits (left in memory by
+// the head launch) are cut into C chunks; CTA (chunk, row) keeps, per thread, the T best perturbed scores of
+// its share in registers together with a running (max, sum) of the raw logits, merges the lists by a
+// tournament over their heads and writes one partial result; a second kernel merges the C partial results
+// of a row the same way.  Keys are packed (score, index), so every merge order gives the same children.
+// Reported log-probabilities are those of the raw logits.
 __global__ void __launch_bounds__(256)
-sx_gumbel_topk_kernel(int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp, int32_t *tok_out,
-                      float *logp_out) {
+sx_gumbel_topk_kernel(int V, int T, int chunk, const float *logits, size_t ld, SxIndex li, SxSample smp,
+                      SxHeadPartial *parts) {
   __shared__ unsigned long long s_best[2][8];
   __shared__ float s_m[8], s_l[8];
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float *lg = logits + (size_t)sx_index(li, r) * ld;
   const int row = smp.row0 + r;
   const uint32_t sb = (uint32_t)(row / smp.P), sj = (uint32_t)(row % smp.P) + smp.slot_base;
+  const int i0 = blockIdx.x * chunk, i1 = min(V, i0 + chunk);           // chunk is a multiple of 4
   unsigned long long v[SX_MAX_TOPK];
 #pragma unroll
   for (int k = 0; k < SX_MAX_TOPK; ++k) v[k] = 0ull;
   float m = -INFINITY, l = 0.f;
-  for (int a = tid * 4; a < V; a += 256 * 4) {
+  for (int a = i0 + tid * 4; a < i1; a += 256 * 4) {
     uint32_t w[4];
     sx_philox4x32_10((uint32_t)(a >> 2), sj, sb, smp.offset, smp.k0, smp.k1, w);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int i = a + e;
-      if (i < V) {
+      if (i < i1) {
         const float x = lg[i];
         const float mn = fmaxf(m, x);
         l = l * expf(m - mn) + expf(x - mn);          // m = -inf at first: exp(-inf) = 0
@@ -1055,7 +1058,7 @@ sx_gumbel_topk_kernel(int V, int T, const float *logits, size_t ld, SxIndex li, 
       }
     }
   }
-  // log-sum-exp of the raw logits over the block
+  // (max, sum) of the raw logits over the chunk
   float mm = sx_warp_max(m);
   if (lane == 0) s_m[warp] = mm;
   __syncthreads();
@@ -1066,40 +1069,101 @@ sx_gumbel_topk_kernel(int V, int T, const float *logits, size_t ld, SxIndex li, 
   __syncthreads();
   float lsum = 0.f;
   for (int w2 = 0; w2 < 8; ++w2) lsum += s_l[w2];
-  const float lse = mm + logf(lsum);
+  SxHeadPartial *out = parts + (size_t)r * gridDim.x + blockIdx.x;
+  if (tid == 0) { out->m = mm; out->l = lsum; }
   // tournament over the heads of the 256 sorted lists
+  for (int t = 0; t < SX_MAX_TOPK; ++t) {
+    unsigned long long best = 0ull;
+    if (t < T) {
+      best = v[0];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+      if (lane == 0) s_best[t & 1][warp] = best;
+      __syncthreads();
+      best = s_best[t & 1][0];
+      for (int w2 = 1; w2 < 8; ++w2) best = max(best, s_best[t & 1][w2]);
+      if (best != 0ull && v[0] == best) {            // packed keys are unique (index inside): one winner
+#pragma unroll
+        for (int k = 0; k + 1 < SX_MAX_TOPK; ++k) v[k] = v[k + 1];
+        v[SX_MAX_TOPK - 1] = 0ull;
+      }
+    }
+    if (tid == 0) out->top[t] = best;
+  }
+}
+
+// merge of the C partial results of a row: one warp per row, lane c reads the lists of chunks c, c + 32, ...
+__global__ void __launch_bounds__(32)
+sx_gumbel_topk_merge_kernel(int V, int T, int C, const SxHeadPartial *parts, const float *logits, size_t ld, SxIndex li,
+                            int32_t *tok_out, float *logp_out) {
+  sx_pdl_launch_dependents();
+  sx_pdl_wait();
+  const int r = blockIdx.x, lane = threadIdx.x;
+  const SxHeadPartial *pr = parts + (size_t)r * C;
+  const float *lg = logits + (size_t)sx_index(li, r) * ld;
+  // log-sum-exp of the raw logits
+  float m = -INFINITY;
+  for (int c = lane; c < C; c += 32) m = fmaxf(m, pr[c].m);
+  m = sx_warp_max(m);
+  float l = 0.f;
+  for (int c = lane; c < C; c += 32) l += pr[c].l > 0.f ? pr[c].l * expf(pr[c].m - m) : 0.f;
+  l = sx_warp_sum(l);
+  const float lse = m + logf(l);
+  // every chunk's list is sorted: a lane walks its chunks' lists with one cursor per chunk (C <= 128: four)
+  int cur[4] = {0, 0, 0, 0};
   for (int t = 0; t < T; ++t) {
-    unsigned long long best = v[0];
+    unsigned long long mine = 0ull;
+    int which = -1;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = lane + 32 * j;
+      if (c < C && cur[j] < SX_MAX_TOPK) {
+        const unsigned long long k = pr[c].top[cur[j]];
+        if (k > mine) { mine = k; which = j; }
+      }
+    }
+    unsigned long long best = mine;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
-    if (lane == 0) s_best[t & 1][warp] = best;
-    __syncthreads();
-    best = s_best[t & 1][0];
-    for (int w2 = 1; w2 < 8; ++w2) best = max(best, s_best[t & 1][w2]);
-    if (tid == 0) {
-      const int32_t id = (int32_t)sx_pack_index(best);
-      tok_out[(size_t)r * T + t] = (best != 0ull && id >= 0 && id < V) ? id : 0;
-      logp_out[(size_t)r * T + t] = (best != 0ull && id >= 0 && id < V) ? lg[id] - lse : -INFINITY;
-    }
-    if (best != 0ull && v[0] == best) {            // packed keys are unique (index inside): one winner
+    if (best != 0ull && mine == best) {
 #pragma unroll
-      for (int k = 0; k + 1 < SX_MAX_TOPK; ++k) v[k] = v[k + 1];
-      v[SX_MAX_TOPK - 1] = 0ull;
+      for (int j = 0; j < 4; ++j)
+        if (j == which) ++cur[j];
+    }
+    if (lane == 0) {
+      const int32_t id = (int32_t)sx_pack_index(best);
+      const bool ok = best != 0ull && id >= 0 && id < V;
+      tok_out[(size_t)r * T + t] = ok ? id : 0;
+      logp_out[(size_t)r * T + t] = ok ? lg[id] - lse : -INFINITY;
     }
   }
 }
 
+// parts: room for `cap` partial results
 sx_status sx_launch_gumbel_topk(int R, int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp,
-                                int32_t *tok_out, float *logp_out, cudaStream_t st) {
-  return sx_rc(sx_launch(sx_gumbel_topk_kernel, dim3(R), dim3(256), 0, st, V, T, logits, ld, li, smp, tok_out, logp_out));
+                                SxHeadPartial *parts, size_t cap, int sm_count, int32_t *tok_out, float *logp_out,
+                                cudaStream_t st) {
+  if (R < 1 || T < 1 || T > SX_MAX_TOPK || (size_t)R > cap) return SX_ERR_UNSUPPORTED;
+  int C = (4 * sm_count + R - 1) / R;                 // about four CTAs per SM in all
+  if (C > 128) C = 128;
+  if ((size_t)R * C > cap) C = (int)(cap / R);
+  int chunk = (((V + C - 1) / C) + 1023) / 1024 * 1024;     // whole passes of the CTA: 256 threads x 4 indices
+  C = (V + chunk - 1) / chunk;
+  SX_TRY(sx_rc(sx_launch(sx_gumbel_topk_kernel, dim3(C, R), dim3(256), 0, st, V, T, chunk, logits, ld, li, smp, parts)));
+  return sx_rc(sx_launch(sx_gumbel_topk_merge_kernel, dim3(R), dim3(32), 0, st, V, T, C, (const SxHeadPartial *)parts, logits,
+                         ld, li, tok_out, logp_out));
 }
 
-// Speculative sampling down a tree with sampled children.  One CTA per sequence walks from the root: at
-// the current slot p = softmax(target logits / temp) and q = softmax(logits of the drafted row that produced
-// the slot's children / temp) are held as unnormalised fp32 vectors with float64 sums; a kept child with
-// token x is accepted when u < min(1, p(x) / q(x)), a refusal replaces p by max(0, p - q) (renormalised
-// through its sum) and removes x from q; when nothing is accepted the slot's token is a Gumbel-max draw over
-// what is left of p.  pq holds 2 V floats per sequence.
+// Speculative sampling down a tree with sampled children.  A cluster of SX_WALK_CTAS CTAs per sequence walks
+// from the root; CTA k of the cluster owns the k-th slice of the vocabulary.  At the current slot
+// p = softmax(target logits / temp) and q = softmax(logits of the drafted row that produced the slot's
+// children / temp) are held as unnormalised fp32 vectors (pq: 2 V floats per sequence) with float64 sums; a
+// kept child with token x is accepted when u < min(1, p(x) / q(x)), a refusal replaces p by max(0, p - q)
+// (renormalised through its sum) and removes x from q; when nothing is accepted the slot's token is a
+// Gumbel-max draw over what is left of p.  Sums, maxima and the draw are reduced per CTA, then over the
+// cluster through distributed shared memory in rank order, so every CTA holds the same values and takes the
+// same branches; the hardware cluster barrier is executed the same number of times by all of them.
+#define SX_WALK_CTAS 8
 __device__ __forceinline__ double sx_block_sum_d(double v, double *red) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -1111,6 +1175,50 @@ __device__ __forceinline__ double sx_block_sum_d(double v, double *red) {
   return t;
 }
 
+struct SxClusterSlot {
+  double a, b;
+  int i, pad;
+};
+__device__ __forceinline__ void sx_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ SxClusterSlot sx_cluster_read(const SxClusterSlot *local, uint32_t rank) {
+  const uint32_t la = (uint32_t)__cvta_generic_to_shared(local);
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
+  SxClusterSlot s;
+  asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(s.a) : "r"(ra) : "memory");
+  asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(s.b) : "r"(ra + 8u) : "memory");
+  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(s.i) : "r"(ra + 16u) : "memory");
+  s.pad = 0;
+  return s;
+}
+// Combines the CTAs' values (the same in every thread of a CTA) over the cluster, rank 0 first.
+// op 0: a and b are summed; 1: maxima; 2: (a, i) is the best score and its index, larger score first, then lower index.
+// slots alternate between two buffers: a CTA can only reach the write of the reduction after the next one once
+// every CTA has arrived at the next one's barrier, i.e. has finished reading this one.
+__device__ __forceinline__ void sx_cluster_reduce(SxClusterSlot *slots, SxClusterSlot *res, int &phase, int op, double &a,
+                                                  double &b, int &i) {
+  if (threadIdx.x == 0) {
+    slots[phase].a = a; slots[phase].b = b; slots[phase].i = i;
+  }
+  sx_cluster_sync();
+  if (threadIdx.x == 0) {
+    SxClusterSlot acc = sx_cluster_read(&slots[phase], 0u);
+    for (uint32_t r = 1; r < SX_WALK_CTAS; ++r) {
+      const SxClusterSlot o = sx_cluster_read(&slots[phase], r);
+      if (op == 0) { acc.a += o.a; acc.b += o.b; }
+      else if (op == 1) { acc.a = fmax(acc.a, o.a); acc.b = fmax(acc.b, o.b); }
+      else if (o.i >= 0 && (acc.i < 0 || o.a > acc.a || (o.a == acc.a && o.i < acc.i))) { acc.a = o.a; acc.i = o.i; }
+    }
+    *res = acc;
+  }
+  __syncthreads();
+  a = res->a; b = res->b; i = res->i;
+  __syncthreads();                       // res is rewritten by the next reduction
+  phase ^= 1;
+}
+
 __global__ void __launch_bounds__(1024)
 sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *target_logits, const float *draft_logits,
                          const int32_t *cand_tok, const int32_t *parent, const int32_t *slot_row, SxSample smp,
@@ -1119,16 +1227,22 @@ sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *t
   __shared__ double red[32];
   __shared__ double s_best[32];
   __shared__ int s_besti[32];
+  __shared__ SxClusterSlot slots[2], res;
   sx_pdl_launch_dependents();
   sx_pdl_wait();
-  const int b = blockIdx.x, tid = threadIdx.x;
+  const int b = blockIdx.x / SX_WALK_CTAS, rank = blockIdx.x % SX_WALK_CTAS, tid = threadIdx.x;
+  const bool lead = rank == 0 && tid == 0;
+  const int len = ((V + SX_WALK_CTAS - 1) / SX_WALK_CTAS + 3) / 4 * 4;    // slices start at multiples of 4
+  const int lo = min(V, rank * len), hi = min(V, lo + len);
   const float inv_tau = 1.0f / smp.temp;
   float *Pv = pq + (size_t)b * 2 * V, *Qv = Pv + V;
   const int32_t *ct = cand_tok + (size_t)b * P, *par = parent + (size_t)b * P, *srow = slot_row + (size_t)b * P;
   int32_t *tt = target_tok + (size_t)b * P, *pa = path + (size_t)b * path_stride;
-  for (int s = tid; s < P; s += blockDim.x) tt[s] = -1;
-  if (tid == 0) pa[0] = 0;
-  int cur = 0, L = 0;
+  if (rank == 0)
+    for (int s = tid; s < P; s += blockDim.x) tt[s] = -1;
+  if (lead) pa[0] = 0;
+  __syncthreads();
+  int cur = 0, L = 0, phase = 0, none = -1;
   for (;;) {
     const float *lp = target_logits + ((size_t)b * P + cur) * V;
     const int row = srow[cur];
@@ -1137,15 +1251,16 @@ sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *t
     const bool has_q = nkids > 0 && row >= 0 && row < rows;
     const float *lq = has_q ? draft_logits + ((size_t)b * rows + row) * V : nullptr;
     // maxima, then the unnormalised vectors and their sums
-    float mp = -INFINITY, mq = -INFINITY;
-    for (int i = tid; i < V; i += blockDim.x) {
-      mp = fmaxf(mp, lp[i]);
-      if (lq) mq = fmaxf(mq, lq[i]);
+    float mpf = -INFINITY, mqf = -INFINITY;
+    for (int i = lo + tid; i < hi; i += blockDim.x) {
+      mpf = fmaxf(mpf, lp[i]);
+      if (lq) mqf = fmaxf(mqf, lq[i]);
     }
-    mp = sx_block_max(mp, red);
-    mq = sx_block_max(mq, red);
+    double mpd = (double)sx_block_max(mpf, red), mqd = (double)sx_block_max(mqf, red);
+    sx_cluster_reduce(slots, &res, phase, 1, mpd, mqd, none);
+    const float mp = (float)mpd, mq = (float)mqd;
     double sp = 0.0, sq = 0.0;
-    for (int i = tid; i < V; i += blockDim.x) {
+    for (int i = lo + tid; i < hi; i += blockDim.x) {
       const float a = expf((lp[i] - mp) * inv_tau);
       Pv[i] = a;
       sp += (double)a;
@@ -1157,61 +1272,68 @@ sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *t
     }
     sp = sx_block_sum_d(sp, red);
     sq = sx_block_sum_d(sq, red);
+    sx_cluster_reduce(slots, &res, phase, 0, sp, sq, none);     // its barrier also publishes Pv / Qv to the cluster
     int nxt = -1;
     if (has_q) {
+      int refused[SX_MAX_TOPK], nref = 0;
       for (int s = cur + 1; s < P && nxt < 0; ++s) {
         if (par[s] != cur) continue;
         int x = ct[s];
         if (x < 0 || x >= V) {
-          if (tid == 0) sx_set_status(status, SX_ERR_CAPACITY);
+          if (lead) sx_set_status(status, SX_ERR_CAPACITY);
           x = 0;
         }
-        __syncthreads();                                                  // Pv / Qv of the last update are in place
-        const double px = (double)Pv[x] / sp, qx = (double)Qv[x] / sq;
+        // another CTA of the cluster may own x: read past this SM's L1.  A token refused before at this slot
+        // has left q; that is taken from the list, not from memory (its owner clears Qv[x] behind the barrier
+        // of the refusal, which orders nothing for the other CTAs), so that all CTAs see the same q(x).
+        bool gone = false;
+        for (int j = 0; j < nref; ++j) gone |= refused[j] == x;
+        const double px_un = (double)__ldcg(Pv + x), qx_un = gone ? 0.0 : (double)__ldcg(Qv + x);
+        const double px = px_un / sp, qx = qx_un / sq;
         const double ratio = qx > 0.0 ? fmin(1.0, px / qx) : 1.0;
         uint32_t w[4];
         sx_philox4x32_10(0u, 0x20000000u + (uint32_t)s, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
         const double u = ((double)(w[0] >> 9) + 0.5) * (1.0 / 8388608.0);
-        if (u < ratio) {                                                  // every thread takes the same decision
+        if (u < ratio) {                                                  // every thread of the cluster takes the same decision
           nxt = s;
           break;
         }
         // refused: p <- max(0, p - q) with its new sum; x leaves q
         const float fsp = (float)(1.0 / sp), fsq = (float)(1.0 / sq);
-        const double qx_un = (double)Qv[x];
-        __syncthreads();
-        double nsp = 0.0;
-        for (int i = tid; i < V; i += blockDim.x) {
+        double nsp = 0.0, zero = 0.0;
+        for (int i = lo + tid; i < hi; i += blockDim.x) {
           const float rr = fmaxf(0.f, Pv[i] * fsp - Qv[i] * fsq);
           Pv[i] = rr;
           nsp += (double)rr;
         }
-        if (tid == 0) Qv[x] = 0.f;
-        sp = sx_block_sum_d(nsp, red);
+        nsp = sx_block_sum_d(nsp, red);
+        sx_cluster_reduce(slots, &res, phase, 0, nsp, zero, none);        // everyone has read Qv[x] by now
+        if (tid == 0 && x >= lo && x < hi) Qv[x] = 0.f;
+        __syncthreads();
+        if (nref < SX_MAX_TOPK) refused[nref++] = x;
+        sp = nsp;
         sq -= qx_un;
       }
     }
     if (nxt >= 0) {
-      if (tid == 0) {
+      if (lead) {
         tt[cur] = ct[nxt];
         if (L + 1 < path_stride) pa[L + 1] = nxt;
       }
       cur = nxt;
       ++L;
-      __syncthreads();
       continue;
     }
     // the slot's own draw: Gumbel-max over log(what is left of p), lower index among equals
-    __syncthreads();
     double best = -INFINITY;
     int besti = -1;
-    for (int a = tid * 4; a < V; a += blockDim.x * 4) {
+    for (int a = lo + tid * 4; a < hi; a += blockDim.x * 4) {
       uint32_t w[4];
       sx_philox4x32_10((uint32_t)(a >> 2), (uint32_t)cur, (uint32_t)b, smp.offset, smp.k0, smp.k1, w);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int i = a + e;
-        if (i < V && Pv[i] > 0.f) {
+        if (i < hi && Pv[i] > 0.f) {
           const float uu = (float)((w[e] >> 9) * 2u + 1u) * 5.9604644775390625e-8f;
           const double sc = (double)(logf(Pv[i]) - logf(-logf(uu)));
           if (sc > best) { best = sc; besti = i; }
@@ -1226,14 +1348,16 @@ sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *t
     }
     if ((tid & 31) == 0) { s_best[tid >> 5] = best; s_besti[tid >> 5] = besti; }
     __syncthreads();
-    if (tid == 0) {
-      best = -INFINITY;
-      besti = -1;
-      for (int w2 = 0; w2 < (int)(blockDim.x >> 5); ++w2) {
-        const double ob = s_best[w2];
-        const int oi = s_besti[w2];
-        if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
-      }
+    best = -INFINITY;
+    besti = -1;
+    for (int w2 = 0; w2 < (int)(blockDim.x >> 5); ++w2) {                  // the same scan in every thread
+      const double ob = s_best[w2];
+      const int oi = s_besti[w2];
+      if (oi >= 0 && (besti < 0 || ob > best || (ob == best && oi < besti))) { best = ob; besti = oi; }
+    }
+    double unused = 0.0;
+    sx_cluster_reduce(slots, &res, phase, 2, best, unused, besti);
+    if (lead) {
       if (besti < 0) besti = 0;
       tt[cur] = besti;
       recover[b] = besti;
@@ -1242,6 +1366,7 @@ sx_tree_spec_walk_kernel(int P, int V, int rows, int path_stride, const float *t
     }
     break;
   }
+  sx_cluster_sync();                     // no CTA leaves while another may still read its shared memory
 }
 
 size_t sx_tree_spec_ws_bytes(int B, int V) { return (size_t)B * 2 * V * sizeof(float); }
@@ -1251,7 +1376,7 @@ sx_status sx_launch_tree_spec_walk(int B, int P, int V, int rows, int path_strid
                                    const int32_t *slot_row, SxSample smp, void *pq_ws, int32_t *target_tok,
                                    int32_t *accept_len, int32_t *path, int32_t *recover, int32_t *status,
                                    cudaStream_t st) {
-  return sx_rc(sx_launch(sx_tree_spec_walk_kernel, dim3(B), dim3(1024), 0, st, P, V, rows, path_stride, target_logits,
-                         draft_logits, cand_tok, parent, slot_row, smp, (float *)pq_ws, target_tok, accept_len, path,
-                         recover, status));
+  return sx_rc(sx_launch_cluster(sx_tree_spec_walk_kernel, dim3(B * SX_WALK_CTAS), dim3(1024), 0, SX_WALK_CTAS, st, P, V, rows,
+                                 path_stride, target_logits, draft_logits, cand_tok, parent, slot_row, smp, (float *)pq_ws,
+                                 target_tok, accept_len, path, recover, status));
 }

@@ -161,8 +161,10 @@ int sx_head_max_rows(int T, int lse);
 
 // Sampled children in a tree: the T best of logit + temp * Gumbel noise per drafted row (rows of `logits` are
 // addressed through li), and the speculative walk over the laid-out tree (pq_ws: sx_tree_spec_ws_bytes).
+// parts: scratch for `cap` partial results (the head launch's per-CTA results are no longer needed by then).
 sx_status sx_launch_gumbel_topk(int R, int V, int T, const float *logits, size_t ld, SxIndex li, SxSample smp,
-                                int32_t *tok_out, float *logp_out, cudaStream_t st);
+                                SxHeadPartial *parts, size_t cap, int sm_count, int32_t *tok_out, float *logp_out,
+                                cudaStream_t st);
 size_t sx_tree_spec_ws_bytes(int B, int V);
 sx_status sx_launch_tree_spec_walk(int B, int P, int V, int rows, int path_stride, const float *target_logits,
                                    const float *draft_logits, const int32_t *cand_tok, const int32_t *parent,
