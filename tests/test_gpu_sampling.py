@@ -159,6 +159,25 @@ def test_tree_with_sampled_children(topk, depth, nodes, tau):
     assert accepted > 0
 
 
+def test_sampled_children_on_an_odd_vocabulary_cut_into_several_chunks():
+    """V = 2501: the top-k pass cuts a row into three chunks (the last one ragged) and merges them; the walk's
+    eight vocabulary slices are 316 ids wide with a short last one.  Five sequences, a deep narrow tree."""
+    sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=2501, page=16)
+    wl = synth.Workload("stv", sh, B=5, mode=synth.TREE, K=5, topk=2, max_nodes=2 + 4 * 4, len_lo=9, len_hi=60,
+                        seed=91, sigma_lo=0.0, sigma_hi=0.05)
+    case = harness.build_case(wl)
+    w = dict(case.weights)
+    w["head"] = (w["head"].to(torch.float32) * 25.0).to(torch.bfloat16)
+    case = dataclasses.replace(case, weights=w)
+    accepted = 0
+    for offset in (1, 2):
+        rep = parity.run_tree(case, sample=orc.SampleCfg(0.8, 99, offset, True))
+        accepted += sum(rep.accept_len)
+        print("odd vocabulary, offset", offset, "accept:", rep.accept_len, "exempt:", rep.exempt)
+        assert len(rep.exempt) <= 2
+    assert accepted > 0
+
+
 def test_sampled_children_need_the_full_vocabulary_and_a_positive_temperature_to_act():
     sh = synth.ModelShape(H=64, n_q=4, n_kv=2, d=16, F=96, V=300, page=16)
     wl = synth.Workload("stx", sh, B=2, mode=synth.TREE, K=3, topk=3, max_nodes=12, len_lo=9, len_hi=40, seed=75)
