@@ -269,7 +269,8 @@ sx_status sx_tile_weight(const void *src_d, int32_t N, int32_t K, void *dst_d, v
  * blocks through tcgen05 tensor memory, which is faster on long caches but needs head_dim = 128, a page
  * size that is a multiple of 64 and at most 32 queries per (sequence, KV head) (group size * rows drafted
  * per sequence in the round).  SX_ATTN_AUTO (the state of a new context) takes SX_ATTN_TC where it is
- * supported and the cache capacity is at least four 128-key blocks per SM, else SX_ATTN_SPLIT.  Forcing
+ * supported, the round has more than four queries per (sequence, KV head) and the cache capacity is at least
+ * four 128-key blocks per SM, else SX_ATTN_SPLIT.  Forcing
  * SX_ATTN_TC makes a draft call return SX_ERR_UNSUPPORTED where the shape does not allow it.  Host-side
  * state, read when a call is issued. */
 enum { SX_ATTN_AUTO = 0, SX_ATTN_SPLIT = 1, SX_ATTN_TC = 2 };

@@ -387,19 +387,20 @@ static sx_status draft_round(sx_ctx *c, const sx_kv *kv, int round, int R, const
   SX_TRY(sx_launch_finish_qkv_rope(s, rm, part, sp, stride, q, *kv, status, st));
   const int B = kv->batch, nr = R / B;
   const int E = (c->dc.mode == SX_MODE_CHAIN) ? round : (round == 1 ? 1 : 1 + (round - 1) * c->dc.topk);
-  // Which attention kernel: the tensor-core one streams long caches faster; below a few blocks of keys per
-  // SM its set-up outweighs that and the split kernel is used (the host knows capacities, not lengths).
+  // Which attention kernel: the tensor-memory one for long caches with more than four queries per (sequence,
+  // KV head); below a few blocks of keys per SM its set-up outweighs its stream, and with up to four queries
+  // the split kernel's three small CTAs per SM keep more bytes in flight (the host knows capacities, not lengths).
   bool tc = sx_attn_tc_supported(s, nr, *kv);
   if (c->attn_kernel == SX_ATTN_SPLIT) tc = false;
   else if (c->attn_kernel == SX_ATTN_AUTO)
-    tc = tc && (long long)B * s.nkv * ((kv->max_pages * s.page + 127) / 128) >= 4ll * c->sm_count;
+    tc = tc && nr * (s.nq / s.nkv) > 4 && (long long)B * s.nkv * ((kv->max_pages * s.page + 127) / 128) >= 4ll * c->sm_count;
   else if (!tc) return SX_ERR_UNSUPPORTED;
   prof_mark(c, SX_PROF_ATTENTION, true, st);
   if (tc) {
     SX_TRY(sx_launch_attention_tc(s, rm, B, nr, E, q, *kv, (float *)(ws + c->off_attn), o, c->sm_count, status, st));
   } else {
     const int nsplit = sx_attn_splits(s, B, nr, kv->max_pages * s.page, c->sm_count);
-    SX_TRY(sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, status, st));
+    SX_TRY(sx_launch_attention(s, rm, B, nr, E, q, *kv, nsplit, (float *)(ws + c->off_attn), o, c->sm_count, status, st));
   }
   prof_mark(c, SX_PROF_ATTENTION, false, st);
   SX_TRY(gemm(c, SX_PROF_GEMM_O, c->w.wo_d, s.H, s.nq * s.d, o, R, ws, &sp, &stride, status, st));

@@ -58,7 +58,7 @@ sx_status sx_attn_init(int device);
 int sx_attn_splits(const SxShape &sh, int B, int nr, int n_cap, int sm_count);
 size_t sx_attn_ws_bytes(const SxShape &sh, int max_batch, int max_nr, int sm_count);
 sx_status sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int nr, int E, const bf16 *q,
-                         const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int32_t *status, cudaStream_t st);
+                         const sx_kv &kv, int nsplit, float *ws, bf16 *o_out, int sm_count, int32_t *status, cudaStream_t st);
 
 // The same attention on tcgen05 (sx_attention_tc.cu): head dimension 128, pages of a multiple of 64 slots,
 // at most 32 queries per (sequence, KV head).

@@ -16,9 +16,11 @@ __device__ __forceinline__ void sx_pdl_launch_dependents() {
 }
 __device__ __forceinline__ void sx_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// overlap = false launches in plain stream order (the kernel starts when its predecessor has completed; its
+// griddepcontrol instructions are then no-ops).
 template <typename... KArgs, typename... Args>
-inline cudaError_t sx_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                             Args &&...args) {
+inline cudaError_t sx_launch_opt(bool overlap, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, Args &&...args) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = grid;
@@ -29,8 +31,14 @@ inline cudaError_t sx_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = overlap ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t sx_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                             Args &&...args) {
+  return sx_launch_opt(true, kernel, grid, block, smem, st, std::forward<Args>(args)...);
 }
 
 // The same with a thread-block cluster of `cluster` CTAs along x (grid.x must be a multiple of it).
