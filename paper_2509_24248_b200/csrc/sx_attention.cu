@@ -56,12 +56,17 @@ __device__ __forceinline__ uint32_t sx_pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t *>(&v);
 }
 // 16-byte asynchronous copy global -> shared; reads nothing and writes zeros when !valid
+// The copies go past L1 (.cg).  With .ca they allocate L1 lines on their way, and the 192 KB a full SM has in
+// flight only fit when the kernel found the SM with a large L1: launched programmatically behind a GEMM the CTAs
+// inherit that kernel's shared-memory carve-out (the SM never idles, so it is not reconfigured), L1 stays at its
+// minimum and every CTA of a long launch ran a quarter slower (batch 32 x 2048-8192 cached tokens: 160 us against
+// 126 us in plain stream order; the same 160 us in plain order with the carve-out forced to its maximum).
 __device__ __forceinline__ void sx_cp_async16(uint32_t smem_dst, const void *gsrc, bool valid) {
   const uint32_t bytes = valid ? 16u : 0u;
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void sx_cp_async16_full(uint32_t smem_dst, const void *gsrc) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void sx_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -488,14 +493,10 @@ sx_status sx_launch_attention(const SxShape &sh, const SxRowMap &rm, int B, int 
   const size_t stage_bytes = (size_t)2 * 16 * sh.d * 2;       // 16 K rows and 16 V rows
   while (stages > 2 && gpc * stages * stage_bytes > SX_ATTN_SMEM_BUDGET) --stages;
   const size_t smem = (size_t)gpc * stages * stage_bytes;
-  // Programmatic dependent launch only while every CTA finds a place at once (three CTAs of four warps per SM).
-  // With more CTAs than places the same kernel runs a quarter slower when it was launched that way (measured on
-  // batch 32 x 2048-8192 cached tokens: 1536 CTAs, 160 us against 126 us per launch, every CTA slower by the same
-  // factor at the same number of resident CTAs), far more than the few microseconds of overlap are worth.
-  const bool overlap = (long long)grid.x * grid.y * grid.z * ((block.x + 127) / 128) <= 3ll * sm_count;
+  (void)sm_count;
   cudaError_t err = cudaSuccess;
 #define SX_ATTN_NT(DD, NN, QQ)                                                                                          \
-  err = sx_launch_opt(overlap, sx_attn_mma_kernel<DD, NN, QQ>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, \
+  err = sx_launch(sx_attn_mma_kernel<DD, NN, QQ>, grid, block, smem, st, sh.nq, sh.nkv, G, sh.page, page_shift, \
                       scale_log2, rm, nr, E, gpc, stages, q, kv, nsplit, ws_ml, ws_o, status)
 #define SX_ATTN(DD)                                  \
   switch (attn_qtiles(sh, nr)) {                     \
