@@ -352,12 +352,10 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
     launches0 = sx.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     accepted = torch.zeros(steps, wl.B, dtype=torch.int32, device=dev)
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
     ev0.record()
     for i in range(steps):
         step()
         accepted[i].copy_(out["accept_len_out_d"])
-        marks[i].record()          # one event per iteration: per-iteration percentiles
     ev1.record()
     torch.cuda.synchronize()
     sampler.mark_end()
@@ -365,6 +363,17 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
         dist.barrier()
     launches = sx.launch_count() - launches0
     sx.check_status("timed region")
+    # per-iteration percentiles: a second pass with one event per iteration (kept out of the timed region: an
+    # event record between two iterations costs microseconds and stops the first kernel of the next iteration
+    # from overlapping the last one of this)
+    n_marks = max(3, min(steps, 200))
+    mark0 = torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_marks)]
+    mark0.record()
+    for i in range(n_marks):
+        step()
+        marks[i].record()
+    torch.cuda.synchronize()
     # per-kernel durations: the same steps again with the library's per-launch CUDA events on (kept
     # out of the timed region above: an event record between back-to-back kernels costs microseconds)
     prof_steps = min(steps, 30)
@@ -374,7 +383,7 @@ def measure(args, wl, dev, dist, world, local, rank, steps, warmup, timeline=Non
     torch.cuda.synchronize()
     prof = sx.profile_end()
     clocks = sampler.stop()
-    per_step = sorted(a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks))
+    per_step = sorted(a.elapsed_time(b) for a, b in zip([mark0] + marks[:-1], marks))
     pct = lambda q: per_step[min(len(per_step) - 1, int(q * len(per_step)))]
     ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, dev)
     ms = ms_total / steps
